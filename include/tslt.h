@@ -1,0 +1,144 @@
+/*
+ * tslt.h — C ABI of libtslt: the data-parallel hot path of Truncated Sparse Logits
+ * Transmission (TSLT) for distributed speculative decoding, as hand-written CUDA kernels
+ * for sm_100a.
+ *
+ * Conventions shared by every entry point
+ *   - plain C ABI, no exceptions; every function returns an int status (TSLT_OK = 0,
+ *     negative on error).  Argument errors are found on the host before any launch and
+ *     leave the outputs untouched.
+ *   - the caller owns every buffer.  Pointers are DEVICE pointers unless marked HOST.  The
+ *     library never allocates or frees device memory: scratch comes from a caller-provided
+ *     workspace whose size is returned by the matching *_workspace_bytes query.  The
+ *     workspace must be 256-byte aligned and must not be shared by calls that can overlap
+ *     on the device.
+ *   - calls are asynchronous on the caller's stream (a cudaStream_t passed as void*; NULL
+ *     is the default stream) and return after enqueueing.
+ *   - logits are row-major [rows, V] in fp32 (TSLT_F32) or bf16 (TSLT_BF16); the base
+ *     pointer must be 16-byte aligned and row_stride_elems * sizeof(element) must be a
+ *     multiple of 16.  -inf logits are legal (probability 0, never selected).  NaN / +inf
+ *     logits give unspecified values but never an out-of-bounds access or a hang.
+ *   - uniforms are fp32 in [0,1); a value >= 1 is read as the largest float below 1.
+ *   - "sample" always means inverse CDF in ascending token index: the first index whose
+ *     cumulative mass exceeds u * total.
+ *   - device-side waits are bounded; a wait that ran out sets a status word in the
+ *     workspace, reported by tslt_workspace_status as TSLT_ERR_DEVICE_STATUS.
+ */
+#ifndef TSLT_H_
+#define TSLT_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TSLT_OK 0
+#define TSLT_ERR_INVALID_ARG (-1)
+#define TSLT_ERR_UNSUPPORTED (-2)
+#define TSLT_ERR_WORKSPACE (-3)
+#define TSLT_ERR_CUDA (-4)
+#define TSLT_ERR_DEVICE_STATUS (-5)
+
+#define TSLT_F32 0
+#define TSLT_BF16 1
+
+/* largest supported k (top-k size, or the candidate cap when top-p is on) */
+#define TSLT_MAX_K 1024
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+int tslt_version(void);
+
+/* Static string for a status code; never NULL. */
+const char* tslt_status_string(int status);
+
+/* Synchronous check of the device status word of a workspace used by earlier calls on
+ * `stream`: waits for the stream, copies the word back and stores it in *device_status
+ * (HOST, nullable).  Returns TSLT_OK if it is zero, TSLT_ERR_DEVICE_STATUS otherwise. */
+int tslt_workspace_status(const void* workspace, void* stream, int* device_status);
+
+/*
+ * Draft side: sparsify-then-sample (Section 3, Solution 1; sampling steps of Algorithms 2
+ * and 4).  For each of the B*gamma rows:
+ *   q   = softmax(logits / temperature) over the whole vocabulary;
+ *   S   = the first n tokens in the order (logit descending, index ascending), where
+ *         n = min(k, n*, number of finite logits) and n* is the smallest n whose
+ *         cumulative q reaches top_p (the crossing token is kept; top_p >= 1 disables it,
+ *         so (k, 1.0) is plain top-k and (cap, rho) is top-rho with a cap);
+ *   q~  = q restricted to S and renormalised (the truncation equation of Section 3.1);
+ *   num_samples tokens are drawn iid from q~, one uniform each (with replacement).
+ * Outputs: idx / logit hold the (token id, stored logit upcast to fp32) pairs of S in
+ * ASCENDING token id, padded with -1 / -inf up to k; count = n; token = the samples;
+ * lse (nullable) = ln sum exp(logits/temperature); mass (nullable) = sum_{S} q, the
+ * retained mass rho of Theorem 1.  A row with no finite logit gives count 0, token -1.
+ *
+ * Shapes: logits [B*gamma, V] with the given row stride; uniforms, token
+ * [B*gamma, num_samples]; idx, logit [B*gamma, k]; count, lse, mass [B*gamma].
+ * Requires 1 <= k <= min(V, TSLT_MAX_K), top_p > 0, temperature > 0, num_samples >= 0.
+ */
+int tslt_sparsify_workspace_bytes(int rows, int V, int k, int num_samples, size_t* bytes);
+int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
+                  long long row_stride_elems, int k, float top_p, float temperature,
+                  int num_samples, const float* uniforms, int* idx, float* logit, int* count,
+                  int* token, float* lse, float* mass, void* workspace, size_t workspace_bytes,
+                  void* stream);
+
+/*
+ * Verifier side, single candidate: speculative sampling against the sparse draft
+ * (Algorithm 3, with the acceptance ratio p/q~ as in Algorithm 5).  For each sequence b:
+ *   p_j = softmax(target_logits[b, j] / target_temperature), j = 0..gamma;
+ *   q~_j rebuilt from the received (idx, logit) pairs at draft_temperature;
+ *   position j is accepted iff u_accept[b, j] < min(1, p_j(x_j) / q~_j(x_j)), x_j =
+ *   draft_token[b, j]; accepted_len[b] = a = number of leading accepted positions;
+ *   a < gamma:  out_token[b] ~ norm(max(0, p_a - q~_a)) over the FULL vocabulary;
+ *   a = gamma:  out_token[b] ~ p_gamma (the bonus row); both use u_sample[b].
+ * Optional outputs (nullable): accept_prob[b, j] = min(1, p_j(x_j)/q~_j(x_j)),
+ * beta_hat[b, j] = sum_{S_j} min(p_j, q~_j) (the truncated acceptance rate of Section
+ * 3.2), lse_p[b, j] = ln sum exp(target row / target_temperature).
+ *
+ * Shapes: target_logits [B, gamma+1, V]; draft_idx, draft_logit [B, gamma, k] and
+ * draft_count [B, gamma] exactly as tslt_sparsify writes them; draft_token, u_accept
+ * [B, gamma]; u_sample, accepted_len, out_token [B].  Draft indices outside [0, V) are
+ * ignored (probability 0) rather than dereferenced.
+ */
+int tslt_verify_workspace_bytes(int B, int gamma, int V, int k, size_t* bytes);
+int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,
+                long long row_stride_elems, int k, const int* draft_idx,
+                const float* draft_logit, const int* draft_count, const int* draft_token,
+                float draft_temperature, float target_temperature, const float* u_accept,
+                const float* u_sample, int* accepted_len, int* out_token, float* accept_prob,
+                float* beta_hat, float* lse_p, void* workspace, size_t workspace_bytes,
+                void* stream);
+
+/*
+ * Verifier side, multi-candidate token tree (Algorithm 5 at every node met on the
+ * root-to-leaf search of Algorithm 8).  Node 0 is the root (the prefix); parent[i] < i;
+ * the children of a node, taken in ascending node id, are its candidates x^(1..k).
+ * target_logits[b, n] is the target distribution for the token AFTER node n, so the root
+ * row judges the root's children.  Starting at the root with p^(1) = p_node: child c is
+ * accepted iff u_accept[b, c] < min(1, p^(i)(x_c) / q~_node(x_c)); on acceptance the walk
+ * moves to c; on rejection p^(i+1) = norm(max(0, p^(i) - q~_node)) (after EVERY rejection,
+ * duplicates included).  The walk stops at a node whose children were all rejected, where
+ * out_token ~ p^(k+1), or at a leaf, where out_token ~ p_leaf; both use
+ * u_sample[b, stop node].  accepted_path[b, :] lists the accepted node ids (pad -1) and
+ * accepted_len[b] their number.
+ *
+ * parent and node_draft_row are HOST arrays [N]: node_draft_row[n] is the row (in [0, M))
+ * of node n's sparse draft in draft_idx / draft_logit [B, M, k] and draft_count [B, M], or
+ * -1 for a leaf.  A node is internal iff it has children iff node_draft_row[n] >= 0.
+ * node_token, u_accept, u_sample are [B, N] (entry 0 of node_token / u_accept unused).
+ * max_depth >= depth of the tree; accepted_path is [B, max_depth].  N <= 1024.
+ */
+int tslt_tree_verify_workspace_bytes(int B, int N, int V, int k, size_t* bytes);
+int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
+                     long long row_stride_elems, const int* parent, const int* node_draft_row,
+                     int M, int k, const int* node_token, const int* draft_idx,
+                     const float* draft_logit, const int* draft_count, float draft_temperature,
+                     float target_temperature, const float* u_accept, const float* u_sample,
+                     int max_depth, int* accepted_path, int* accepted_len, int* out_token,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSLT_H_ */

@@ -1,0 +1,691 @@
+// tslt_verify / tslt_tree_verify: verifier-side speculative sampling against a sparse draft
+// (Algorithm 3; Algorithm 5 along the walk of Algorithm 8) as one kernel each.
+//
+// Every target row is streamed from HBM exactly once through the bulk-copy ring.  The
+// streaming pass keeps nothing but one (max, sum) pair per 2 KB chunk of the row, written to
+// the workspace.  The CTA that finishes a sequence's last segment (found with a ticket
+// counter, no waiting) resolves the sequence: it turns the chunk partials into each row's
+// log-normaliser, rebuilds the sparse q~ in fp64, runs the acceptance tests, and samples the
+// correction token from the full-vocabulary residual.  Because q~ is sparse, the residual is
+// a multiple of p outside the draft set S and explicit values on S, so its CDF is the chunk
+// partials corrected by at most k entries; only the one chunk that holds the sampled token is
+// read a second time.
+#include <math.h>
+
+#include <vector>
+
+#include "tslt_common.cuh"
+#include "tslt_stream.cuh"
+
+namespace tslt {
+
+constexpr int kMaxChunks = 3072;   // chunk partials of one row must fit the resolver's shared memory
+constexpr int kMaxTreeNodes = 1024;
+
+struct VerifyParams {
+    const unsigned char* logits;
+    long long row_stride_bytes, row_bytes;
+    int V, B, rows_per_seq, k;
+    int nseg, tiles_per_seg, ntiles, nchunks;
+    ScaleC cp, cq;
+    const int* draft_idx;
+    const float* draft_logit;
+    const int* draft_count;
+    // sequence mode
+    int gamma;
+    const int* draft_token;
+    const float* u_accept;
+    const float* u_sample;
+    int* accepted_len;
+    int* out_token;
+    float* accept_prob;
+    float* beta_hat;
+    float* lse_p;
+    // tree mode
+    int N, M, max_depth;
+    const int* tree_meta;  // child_begin[N+1] | child_list[N-1] | node_draft_row[N]
+    const int* node_token;
+    int* accepted_path;
+    // workspace
+    int* status;
+    int* tickets;
+    float2* partials;  // [B * rows_per_seq, nchunks]
+};
+
+struct VerifyShared {
+    RingBars bars;
+    double scratch[16];
+    double slot_a, slot_q;
+    int slot_found;
+    int ticket;
+};
+
+// Resolver work arrays laid over the idle ring.
+struct ResolverArrays {
+    double* chunkR;  // kMaxChunks
+    int* s_idx;      // 1024
+    double* s_p;     // 1024
+    double* s_a;     // 1024
+    double* s_q;     // 1024
+    double* r;       // 1024
+};
+__device__ __forceinline__ ResolverArrays carve(unsigned char* ring) {
+    ResolverArrays a;
+    a.chunkR = reinterpret_cast<double*>(ring);
+    a.s_idx = reinterpret_cast<int*>(ring + 24576);
+    a.s_p = reinterpret_cast<double*>(ring + 28672);
+    a.s_a = reinterpret_cast<double*>(ring + 36864);
+    a.s_q = reinterpret_cast<double*>(ring + 45056);
+    a.r = reinterpret_cast<double*>(ring + 53248);
+    return a;
+}
+static_assert(53248 + 8192 <= kRingBytes, "resolver arrays must fit the ring");
+
+__device__ __forceinline__ double accept_probability(double p, double q) {
+    if (q > 0.0) {
+        const double ratio = p / q;
+        return ratio < 1.0 ? ratio : 1.0;
+    }
+    return p > 0.0 ? 1.0 : 0.0;
+}
+
+// base-2 log-normaliser of a row from its chunk partials: L2 = M + log2 sum S_c 2^(M_c - M)
+__device__ __forceinline__ double row_log2_norm(const float2* part, int nchunks, int tid, double* scratch) {
+    double mx = -INFINITY;
+    for (int c = tid; c < nchunks; c += kConsumerThreads) {
+        const float2 ms = __ldcg(&part[c]);
+        if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
+    }
+    mx = block_max(mx, tid, scratch);
+    double s = 0.0;
+    for (int c = tid; c < nchunks; c += kConsumerThreads) {
+        const float2 ms = __ldcg(&part[c]);
+        if (ms.y > 0.f) s += (double)ms.y * exp2((double)ms.x - mx);
+    }
+    s = block_sum(s, tid, scratch);
+    return s > 0.0 ? mx + log2(s) : -INFINITY;
+}
+
+template <typename T>
+__device__ __forceinline__ double token_prob(const unsigned char* rowp, int v, int V, double cd, double L2) {
+    if (v < 0 || v >= V || !(L2 > -INFINITY)) return 0.0;
+    const float z = Elt<T>::load(rowp, v);
+    if (!(fabsf(z) <= 3.4028234e38f)) return 0.0;  // non-finite logit: probability 0
+    return exp2((double)z * cd - L2);
+}
+
+// Rebuild q~ from the transmitted pairs of one draft row into s_idx / s_q; returns n.
+__device__ __forceinline__ int load_draft(const VerifyParams& p, size_t draft_row, const ResolverArrays& A,
+                                          int tid, double* scratch) {
+    int n = p.draft_count[draft_row];
+    n = n < 0 ? 0 : (n > p.k ? p.k : n);
+    const int* di = p.draft_idx + draft_row * (size_t)p.k;
+    const float* dl = p.draft_logit + draft_row * (size_t)p.k;
+    double mx = -INFINITY;
+    for (int i = tid; i < n; i += kConsumerThreads) {
+        A.s_idx[i] = di[i];
+        const float l = dl[i];
+        const bool fin = fabsf(l) <= 3.4028234e38f;
+        const double y = fin ? (double)l * p.cq.d : -INFINITY;
+        A.s_q[i] = y;
+        mx = fmax(mx, y);
+    }
+    mx = block_max(mx, tid, scratch);
+    double w = 0.0;
+    for (int i = tid; i < n; i += kConsumerThreads) {
+        const double y = A.s_q[i];
+        const double e = y > -INFINITY ? exp2(y - mx) : 0.0;
+        A.s_q[i] = e;
+        w += e;
+    }
+    const double W = block_sum(w, tid, scratch);
+    for (int i = tid; i < n; i += kConsumerThreads) A.s_q[i] = W > 0.0 ? A.s_q[i] / W : 0.0;
+    consumer_sync();
+    return n;
+}
+
+// Sample one token over the full vocabulary from the weights
+//   w(v) = c_out * p(v) for v outside S,   w(idx_i) = s_a[i] for the n entries of S,
+// by inverse CDF in ascending index with uniform u.  Returns -1 if the total is not positive.
+template <typename T>
+__device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const unsigned char* rowp,
+                                                 const float2* part, double L2, double c_out, int n,
+                                                 const ResolverArrays& A, float u_raw, int tid,
+                                                 VerifyShared* sh) {
+    constexpr int kChunkElems = kChunkBytes / Elt<T>::kBytes;
+    const int nch = p.nchunks;
+    for (int c = tid; c < nch; c += kConsumerThreads) {
+        const float2 ms = __ldcg(&part[c]);
+        A.chunkR[c] = (ms.y > 0.f && L2 > -INFINITY) ? c_out * (double)ms.y * exp2((double)ms.x - L2) : 0.0;
+    }
+    consumer_sync();
+    // entries of S replace c_out * p by their explicit value; one writer per chunk (S is ascending)
+    for (int i = tid; i < n; i += kConsumerThreads) {
+        const int v = A.s_idx[i];
+        if (v < 0 || v >= p.V) continue;
+        const int c = v / kChunkElems;
+        const int vp = i > 0 ? A.s_idx[i - 1] : -1;
+        const bool first = !(vp >= 0 && vp < p.V && vp / kChunkElems == c);
+        if (first) {
+            double acc = 0.0;
+            for (int j = i; j < n; ++j) {
+                const int vj = A.s_idx[j];
+                if (vj < 0 || vj >= p.V || vj / kChunkElems != c) break;
+                acc += A.s_a[j] - c_out * A.s_p[j];
+            }
+            const double val = A.chunkR[c] + acc;
+            A.chunkR[c] = val > 0.0 ? val : 0.0;
+        }
+    }
+    consumer_sync();
+    block_inclusive_scan(A.chunkR, nch, tid, sh->scratch);
+    const double Z = A.chunkR[nch - 1];
+    if (!(Z > 0.0)) {
+        consumer_sync();
+        return -1;
+    }
+    const double u = (double)clamp_uniform(u_raw);
+    const double target = u * Z;
+    int c = first_greater(A.chunkR, nch, target);
+    bool take_last = false;
+    if (c >= nch) {
+        // rounding left nothing above the target: last chunk with positive mass, its last positive item
+        c = nch - 1;
+        while (c > 0 && !(A.chunkR[c] - A.chunkR[c - 1] > 0.0)) --c;
+        take_last = true;
+    }
+    const double base = c > 0 ? A.chunkR[c - 1] : 0.0;
+    const double Rc = A.chunkR[c] - base;
+    const double frac = take_last ? 2.0 : (target - base) / Rc;
+    consumer_sync();
+    // second touch of one chunk: exact weights of its elements
+    const int v0 = c * kChunkElems;
+    const int ne = min(kChunkElems, p.V - v0);
+    for (int e = tid; e < ne; e += kConsumerThreads) A.r[e] = c_out * token_prob<T>(rowp, v0 + e, p.V, p.cp.d, L2);
+    consumer_sync();
+    for (int i = tid; i < n; i += kConsumerThreads) {
+        const int v = A.s_idx[i];
+        if (v >= v0 && v < v0 + ne) A.r[v - v0] = A.s_a[i] > 0.0 ? A.s_a[i] : 0.0;
+    }
+    consumer_sync();
+    // keep the plain weights for the "last positive" fallback, scan a copy in place of chunkR
+    double* cumr = A.chunkR;  // chunk table no longer needed
+    for (int e = tid; e < ne; e += kConsumerThreads) cumr[e] = A.r[e];
+    consumer_sync();
+    block_inclusive_scan(cumr, ne, tid, sh->scratch);
+    const double Rc2 = cumr[ne - 1];
+    int pos = frac < 1.5 ? first_greater(cumr, ne, frac * Rc2) : ne;
+    if (pos >= ne) {
+        pos = ne - 1;
+        while (pos > 0 && !(A.r[pos] > 0.0)) --pos;
+    }
+    consumer_sync();
+    return v0 + pos;
+}
+
+template <typename T>
+__device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ring, VerifyShared* sh, int tid) {
+    const ResolverArrays A = carve(ring);
+    const int gamma = p.gamma;
+    const size_t r0 = (size_t)b * (gamma + 1);
+    int a = 0;
+    bool running = true;
+    double L2_stop = -INFINITY;
+    for (int j = 0; j <= gamma; ++j) {
+        const float2* part = p.partials + (r0 + j) * (size_t)p.nchunks;
+        const double L2 = row_log2_norm(part, p.nchunks, tid, sh->scratch);
+        if (p.lse_p && tid == 0) p.lse_p[r0 + j] = (float)(L2 * 0.6931471805599453);
+        if (j == gamma) {
+            if (running) L2_stop = L2;
+            break;
+        }
+        if (!running && !p.accept_prob && !p.beta_hat) continue;  // only lse_p still wanted
+        const unsigned char* rowp = p.logits + (long long)(r0 + j) * p.row_stride_bytes;
+        const size_t dr = (size_t)b * gamma + j;
+        const int n = load_draft(p, dr, A, tid, sh->scratch);
+        const int x = p.draft_token[dr];
+        if (tid == 0) {
+            sh->slot_q = 0.0;
+        }
+        consumer_sync();
+        double bh = 0.0;
+        for (int i = tid; i < n; i += kConsumerThreads) {
+            const int v = A.s_idx[i];
+            if (v == x) sh->slot_q = A.s_q[i];
+            if (p.beta_hat) {
+                const double pv = token_prob<T>(rowp, v, p.V, p.cp.d, L2);
+                bh += fmin(pv, A.s_q[i]);
+            }
+        }
+        if (p.beta_hat) {
+            bh = block_sum(bh, tid, sh->scratch);
+            if (tid == 0) p.beta_hat[dr] = (float)bh;
+        } else {
+            consumer_sync();
+        }
+        const double px = token_prob<T>(rowp, x, p.V, p.cp.d, L2);
+        const double ap = accept_probability(px, sh->slot_q);
+        if (p.accept_prob && tid == 0) p.accept_prob[dr] = (float)ap;
+        if (running) {
+            const double r = (double)clamp_uniform(p.u_accept[dr]);
+            if (r < ap) {
+                ++a;
+            } else {
+                running = false;
+                L2_stop = L2;
+            }
+        }
+        consumer_sync();
+    }
+    // correction token: residual of the rejected position, or the bonus row
+    const unsigned char* rowp = p.logits + (long long)(r0 + a) * p.row_stride_bytes;
+    const float2* part = p.partials + (r0 + a) * (size_t)p.nchunks;
+    int n = 0;
+    if (a < gamma) {
+        n = load_draft(p, (size_t)b * gamma + a, A, tid, sh->scratch);
+        for (int i = tid; i < n; i += kConsumerThreads) {
+            const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2_stop);
+            A.s_p[i] = pv;
+            const double d = pv - A.s_q[i];
+            A.s_a[i] = d > 0.0 ? d : 0.0;
+        }
+        consumer_sync();
+    }
+    const float u = p.u_sample[b];
+    int tok = sample_full_vocab<T>(p, rowp, part, L2_stop, 1.0, n, A, u, tid, sh);
+    if (tok < 0 && n > 0) tok = sample_full_vocab<T>(p, rowp, part, L2_stop, 1.0, 0, A, u, tid, sh);  // degenerate residual
+    if (tid == 0) {
+        p.accepted_len[b] = a;
+        p.out_token[b] = tok;
+    }
+}
+
+template <typename T>
+__device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, VerifyShared* sh, int tid) {
+    const ResolverArrays A = carve(ring);
+    const int N = p.N;
+    const int* child_begin = p.tree_meta;
+    const int* child_list = p.tree_meta + (N + 1);
+    const int* node_draft_row = p.tree_meta + (N + 1) + (N - 1);
+    int* path = p.accepted_path + (size_t)b * p.max_depth;
+    for (int d = tid; d < p.max_depth; d += kConsumerThreads) path[d] = -1;
+    consumer_sync();
+    int node = 0, len = 0, tok = -1;
+    for (int depth = 0; depth <= p.max_depth; ++depth) {
+        const size_t r = (size_t)b * N + node;
+        const unsigned char* rowp = p.logits + (long long)r * p.row_stride_bytes;
+        const float2* part = p.partials + r * (size_t)p.nchunks;
+        const double L2 = row_log2_norm(part, p.nchunks, tid, sh->scratch);
+        const int dr = node_draft_row[node];
+        const float u = p.u_sample[r];
+        if (dr < 0) {
+            tok = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);  // leaf: bonus from its own row
+            break;
+        }
+        const int n = load_draft(p, (size_t)b * p.M + dr, A, tid, sh->scratch);
+        double ps = 0.0;
+        for (int i = tid; i < n; i += kConsumerThreads) {
+            const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2);
+            A.s_p[i] = pv;
+            A.s_a[i] = pv;
+            ps += pv;
+        }
+        const double PS = block_sum(ps, tid, sh->scratch);
+        const double out_mass = 1.0 - PS > 0.0 ? 1.0 - PS : 0.0;  // mass of p outside S
+        double c_out = 1.0;
+        bool accepted = false;
+        for (int ci = child_begin[node]; ci < child_begin[node + 1]; ++ci) {
+            const int c = child_list[ci];
+            const int x = p.node_token[(size_t)b * N + c];
+            if (tid == 0) sh->slot_found = 0;
+            consumer_sync();
+            for (int i = tid; i < n; i += kConsumerThreads)
+                if (A.s_idx[i] == x) {
+                    sh->slot_a = A.s_a[i];
+                    sh->slot_q = A.s_q[i];
+                    sh->slot_found = 1;
+                }
+            consumer_sync();
+            double pa, qx;
+            if (sh->slot_found) {
+                pa = sh->slot_a;
+                qx = sh->slot_q;
+            } else {
+                pa = c_out * token_prob<T>(rowp, x, p.V, p.cp.d, L2);
+                qx = 0.0;
+            }
+            const double ap = accept_probability(pa, qx);
+            const double rr = (double)clamp_uniform(p.u_accept[(size_t)b * N + c]);
+            if (rr < ap) {
+                if (len < p.max_depth && tid == 0) path[len] = c;
+                ++len;
+                node = c;
+                accepted = true;
+                consumer_sync();
+                break;
+            }
+            // rejected: p^(i+1) = norm(max(0, p^(i) - q~)), on S explicitly, elsewhere by the scalar
+            double zs = 0.0;
+            for (int i = tid; i < n; i += kConsumerThreads) {
+                const double d = A.s_a[i] - A.s_q[i];
+                zs += d > 0.0 ? d : 0.0;
+            }
+            const double Z = block_sum(zs, tid, sh->scratch) + c_out * out_mass;
+            if (Z > 0.0) {
+                for (int i = tid; i < n; i += kConsumerThreads) {
+                    const double d = A.s_a[i] - A.s_q[i];
+                    A.s_a[i] = d > 0.0 ? d / Z : 0.0;
+                }
+                c_out /= Z;
+            }
+            consumer_sync();
+        }
+        if (!accepted) {
+            tok = sample_full_vocab<T>(p, rowp, part, L2, c_out, n, A, u, tid, sh);
+            if (tok < 0) tok = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);
+            break;
+        }
+    }
+    if (tid == 0) {
+        p.accepted_len[b] = len;
+        p.out_token[b] = tok;
+    }
+}
+
+template <typename T, bool kTree>
+__global__ void __launch_bounds__(kBlockThreads) verify_kernel(const VerifyParams p) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>(((size_t)smem_raw + 127) & ~(size_t)127);
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(ring + kRingBytes);
+
+    const int tid = threadIdx.x;
+    const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
+    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
+    const int tile_begin = seg * p.tiles_per_seg;
+    const int tile_end = min(p.ntiles, tile_begin + p.tiles_per_seg);
+
+    ring_init(&sh->bars, tid);
+    __syncthreads();
+    if (tid >= kConsumerThreads) {
+        producer_loop<T>(rowp, p.row_bytes, tile_begin, tile_end, ring, &sh->bars, p.status);
+        return;
+    }
+    const int lane = tid & 31, warp = tid >> 5;
+    const float chi = p.cp.hi, clo = p.cp.lo;
+    float2* part = p.partials + (size_t)row * p.nchunks;
+    bool aborted = false;
+
+    for (int t = tile_begin; t < tile_end; ++t) {
+        const int it = t - tile_begin, s = it % kStages;
+        if (!mbar_wait(&sh->bars.full[s], (uint32_t)((it / kStages) & 1), &sh->bars.abort)) {
+            raise_abort(&sh->bars, p.status);
+            aborted = true;
+            break;
+        }
+        const uint32_t padded = tile_padded_bytes(p.row_bytes, t);
+        const unsigned char* tile = ring + s * kTileBytes;
+        float zmax = -INFINITY, M = -3.0e38f, negM = 3.0e38f;
+        float acc[kPer];
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int j = 0; j < kVecsPerLane; ++j) {
+            const uint32_t off = warp * kChunkBytes + (j * 32 + lane) * kVecBytes;
+            if (off < padded) {
+                float z[kPer];
+                unpack_vec<T>(lds_vec(tile + off), z);
+                float vmax = z[0];
+#pragma unroll
+                for (int e = 1; e < kPer; ++e) vmax = fmaxf(vmax, z[e]);
+                if (vmax > zmax) {
+                    zmax = vmax;
+                    const float Mn = fmaf(vmax, chi, vmax * clo);
+                    const float sc = ex2_approx(M - Mn);
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e) acc[e] *= sc;
+                    M = Mn;
+                    negM = -Mn;
+                }
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) acc[e] += ex2_approx(fmaf(z[e], chi, fmaf(z[e], clo, negM)));
+            }
+        }
+        // the warp's chunk of this tile is done: release the slot, then fold the 32 lane partials
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->bars.empty[s]);
+        if ((uint32_t)(warp * kChunkBytes) < padded) {
+            float sl = 0.f;
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) sl += acc[e];
+            const float Mw = warp_max(M);
+            sl *= ex2_approx(M - Mw);
+            const float Sw = warp_sum(sl);
+            if (lane == 0) part[t * kConsumerWarps + warp] = make_float2(Mw, Sw);
+        }
+    }
+    // collective decision on abort (a wait that ran out): nobody resolves, status word is set
+    int any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"((int)aborted), "n"(kConsumerBarrier), "n"(kConsumerThreads)
+        : "memory");
+    if (any) return;
+
+    // ---- ticket: the CTA that completes the sequence resolves it ---------------------------------
+    __threadfence();
+    consumer_sync();
+    const int b = row / p.rows_per_seq;
+    if (tid == 0) sh->ticket = atomicAdd(&p.tickets[b], 1);
+    consumer_sync();
+    if (sh->ticket != p.rows_per_seq * p.nseg - 1) return;
+    __threadfence();
+    if (kTree) resolve_tree<T>(p, b, ring, sh, tid);
+    else resolve_sequence<T>(p, b, ring, sh, tid);
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+struct VerifyPlan {
+    int nseg, tiles_per_seg, ntiles, nchunks;
+    size_t smem;
+    size_t ws_tickets_off, ws_meta_off, ws_partials_off, ws_bytes;
+};
+
+static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+static int sm_count_v() {
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        sms = v;
+    }
+    return sms;
+}
+
+static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes, int meta_ints) {
+    VerifyPlan pl;
+    const long long row_bytes = (long long)V * elt_bytes;
+    pl.ntiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
+    pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
+    const long long rows = (long long)B * rows_per_seq;
+    const int sms = sm_count_v();
+    int nseg = 1;
+    while (nseg < 16 && rows * nseg < 4LL * sms && pl.ntiles / (nseg * 2) >= 2) nseg *= 2;
+    pl.tiles_per_seg = (pl.ntiles + nseg - 1) / nseg;
+    pl.nseg = (pl.ntiles + pl.tiles_per_seg - 1) / pl.tiles_per_seg;
+    if (pl.nseg < 1) pl.nseg = 1;
+    pl.smem = kRingBytes + sizeof(VerifyShared) + 256;
+    size_t off = kWsHeaderBytes;
+    pl.ws_tickets_off = off;
+    off = up256(off + (size_t)B * sizeof(int));
+    pl.ws_meta_off = off;
+    off = up256(off + (size_t)meta_ints * sizeof(int));
+    pl.ws_partials_off = off;
+    off = up256(off + (size_t)rows * pl.nchunks * sizeof(float2));
+    pl.ws_bytes = off;
+    return pl;
+}
+
+ScaleC make_scale(float temperature);  // defined with the sparsify launcher
+
+static int check_common(const void* logits, int dtype, int V, long long row_stride_elems, int k,
+                        float tq, float tp, const void* workspace) {
+    if (dtype != TSLT_F32 && dtype != TSLT_BF16) return TSLT_ERR_UNSUPPORTED;
+    const int eb = dtype == TSLT_F32 ? 4 : 2;
+    if (V <= 0 || k <= 0 || k > V || !(tq > 0.f) || !(tp > 0.f) || !isfinite(tq) || !isfinite(tp))
+        return TSLT_ERR_INVALID_ARG;
+    if (k > TSLT_MAX_K) return TSLT_ERR_UNSUPPORTED;
+    if ((long long)V * eb > (long long)kMaxChunks * kChunkBytes) return TSLT_ERR_UNSUPPORTED;
+    if (!logits || !workspace) return TSLT_ERR_INVALID_ARG;
+    if (row_stride_elems < V || ((uintptr_t)logits & 15) || ((row_stride_elems * eb) & 15) ||
+        ((uintptr_t)workspace & 255))
+        return TSLT_ERR_INVALID_ARG;
+    return TSLT_OK;
+}
+
+template <bool kTree>
+static int launch_verify(VerifyParams& p, const VerifyPlan& pl, int dtype, cudaStream_t st) {
+    auto kern = dtype == TSLT_F32 ? verify_kernel<float, kTree> : verify_kernel<bf16_t, kTree>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
+        return TSLT_ERR_CUDA;
+    const long long grid = (long long)p.B * p.rows_per_seq * pl.nseg;
+    kern<<<(unsigned)grid, kBlockThreads, pl.smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+}
+
+}  // namespace tslt
+
+using namespace tslt;
+
+extern "C" int tslt_verify_workspace_bytes(int B, int gamma, int V, int k, size_t* bytes) {
+    if (!bytes || B < 0 || gamma < 0 || V <= 0 || k <= 0 || k > V || k > TSLT_MAX_K) return TSLT_ERR_INVALID_ARG;
+    VerifyPlan a = make_verify_plan(B, gamma + 1, V, 2, 0), b = make_verify_plan(B, gamma + 1, V, 4, 0);
+    *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
+    return TSLT_OK;
+}
+
+extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,
+                           long long row_stride_elems, int k, const int* draft_idx, const float* draft_logit,
+                           const int* draft_count, const int* draft_token, float draft_temperature,
+                           float target_temperature, const float* u_accept, const float* u_sample,
+                           int* accepted_len, int* out_token, float* accept_prob, float* beta_hat,
+                           float* lse_p, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || gamma < 0) return TSLT_ERR_INVALID_ARG;
+    if (B == 0) return TSLT_OK;
+    int rc = check_common(target_logits, dtype, V, row_stride_elems, k, draft_temperature, target_temperature,
+                          workspace);
+    if (rc != TSLT_OK) return rc;
+    if (!u_sample || !accepted_len || !out_token ||
+        (gamma > 0 && (!draft_idx || !draft_logit || !draft_count || !draft_token || !u_accept)))
+        return TSLT_ERR_INVALID_ARG;
+    if ((long long)B * (gamma + 1) > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    const int eb = dtype == TSLT_F32 ? 4 : 2;
+    VerifyPlan pl = make_verify_plan(B, gamma + 1, V, eb, 0);
+    if (workspace_bytes < pl.ws_bytes) return TSLT_ERR_WORKSPACE;
+    VerifyParams p = {};
+    p.logits = (const unsigned char*)target_logits;
+    p.row_stride_bytes = row_stride_elems * eb;
+    p.row_bytes = (long long)V * eb;
+    p.V = V; p.B = B; p.rows_per_seq = gamma + 1; p.k = k;
+    p.nseg = pl.nseg; p.tiles_per_seg = pl.tiles_per_seg; p.ntiles = pl.ntiles; p.nchunks = pl.nchunks;
+    p.cp = make_scale(target_temperature);
+    p.cq = make_scale(draft_temperature);
+    p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
+    p.gamma = gamma; p.draft_token = draft_token; p.u_accept = u_accept; p.u_sample = u_sample;
+    p.accepted_len = accepted_len; p.out_token = out_token;
+    p.accept_prob = accept_prob; p.beta_hat = beta_hat; p.lse_p = lse_p;
+    unsigned char* ws = (unsigned char*)workspace;
+    p.status = (int*)ws;
+    p.tickets = (int*)(ws + pl.ws_tickets_off);
+    p.partials = (float2*)(ws + pl.ws_partials_off);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, pl.ws_meta_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
+    return launch_verify<false>(p, pl, dtype, st);
+}
+
+extern "C" int tslt_tree_verify_workspace_bytes(int B, int N, int V, int k, size_t* bytes) {
+    if (!bytes || B < 0 || N <= 0 || N > kMaxTreeNodes || V <= 0 || k <= 0 || k > V || k > TSLT_MAX_K)
+        return TSLT_ERR_INVALID_ARG;
+    VerifyPlan a = make_verify_plan(B, N, V, 2, 3 * N), b = make_verify_plan(B, N, V, 4, 3 * N);
+    *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
+    return TSLT_OK;
+}
+
+extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
+                                long long row_stride_elems, const int* parent, const int* node_draft_row,
+                                int M, int k, const int* node_token, const int* draft_idx,
+                                const float* draft_logit, const int* draft_count, float draft_temperature,
+                                float target_temperature, const float* u_accept, const float* u_sample,
+                                int max_depth, int* accepted_path, int* accepted_len, int* out_token,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || N <= 0 || M < 0 || max_depth < 0 || !parent || !node_draft_row) return TSLT_ERR_INVALID_ARG;
+    if (N > kMaxTreeNodes) return TSLT_ERR_UNSUPPORTED;
+    // ---- tree structure, checked on the host ----------------------------------------------------
+    if (parent[0] != -1) return TSLT_ERR_INVALID_ARG;
+    std::vector<int> nchild(N, 0), depth(N, 0);
+    int maxd = 0;
+    for (int n = 1; n < N; ++n) {
+        if (parent[n] < 0 || parent[n] >= n) return TSLT_ERR_INVALID_ARG;
+        nchild[parent[n]]++;
+        depth[n] = depth[parent[n]] + 1;
+        if (depth[n] > maxd) maxd = depth[n];
+    }
+    if (maxd > max_depth) return TSLT_ERR_INVALID_ARG;
+    for (int n = 0; n < N; ++n) {
+        const bool internal = nchild[n] > 0;
+        if (internal != (node_draft_row[n] >= 0)) return TSLT_ERR_INVALID_ARG;
+        if (node_draft_row[n] >= M) return TSLT_ERR_INVALID_ARG;
+    }
+    if (B == 0) return TSLT_OK;
+    int rc = check_common(target_logits, dtype, V, row_stride_elems, k, draft_temperature, target_temperature,
+                          workspace);
+    if (rc != TSLT_OK) return rc;
+    if (!u_sample || !accepted_len || !out_token || (max_depth > 0 && !accepted_path) ||
+        (N > 1 && (!node_token || !u_accept)) || (M > 0 && (!draft_idx || !draft_logit || !draft_count)))
+        return TSLT_ERR_INVALID_ARG;
+    if ((long long)B * N > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    const int eb = dtype == TSLT_F32 ? 4 : 2;
+    VerifyPlan pl = make_verify_plan(B, N, V, eb, 3 * N);
+    if (workspace_bytes < pl.ws_bytes) return TSLT_ERR_WORKSPACE;
+    // children of every node in ascending id: child_begin[N+1] | child_list[N-1] | node_draft_row[N]
+    std::vector<int> meta(3 * N, 0);
+    int* child_begin = meta.data();
+    int* child_list = meta.data() + (N + 1);
+    int* ndr = meta.data() + (N + 1) + (N - 1);
+    child_begin[0] = 0;
+    for (int n = 0; n < N; ++n) child_begin[n + 1] = child_begin[n] + nchild[n];
+    std::vector<int> fill(child_begin, child_begin + N);
+    for (int n = 1; n < N; ++n) child_list[fill[parent[n]]++] = n;
+    for (int n = 0; n < N; ++n) ndr[n] = node_draft_row[n];
+
+    VerifyParams p = {};
+    p.logits = (const unsigned char*)target_logits;
+    p.row_stride_bytes = row_stride_elems * eb;
+    p.row_bytes = (long long)V * eb;
+    p.V = V; p.B = B; p.rows_per_seq = N; p.k = k;
+    p.nseg = pl.nseg; p.tiles_per_seg = pl.tiles_per_seg; p.ntiles = pl.ntiles; p.nchunks = pl.nchunks;
+    p.cp = make_scale(target_temperature);
+    p.cq = make_scale(draft_temperature);
+    p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
+    p.u_accept = u_accept; p.u_sample = u_sample;
+    p.accepted_len = accepted_len; p.out_token = out_token;
+    p.N = N; p.M = M; p.max_depth = max_depth;
+    p.node_token = node_token; p.accepted_path = accepted_path;
+    unsigned char* ws = (unsigned char*)workspace;
+    p.status = (int*)ws;
+    p.tickets = (int*)(ws + pl.ws_tickets_off);
+    p.tree_meta = (const int*)(ws + pl.ws_meta_off);
+    p.partials = (float2*)(ws + pl.ws_partials_off);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, pl.ws_meta_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
+    // pageable source: the runtime stages it before returning, so `meta` may go out of scope
+    if (cudaMemcpyAsync(ws + pl.ws_meta_off, meta.data(), meta.size() * sizeof(int), cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return TSLT_ERR_CUDA;
+    return launch_verify<true>(p, pl, dtype, st);
+}

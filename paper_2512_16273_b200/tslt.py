@@ -1,0 +1,314 @@
+"""Thin Python binding of libtslt (include/tslt.h): argument marshalling only.
+
+Every step of the hot path runs in the CUDA kernels of libtslt.so; this module checks
+shapes, hands raw device pointers and the current CUDA stream to the C ABI, and uses torch
+only to own device memory.  There is no CPU fallback: importing the binding without the
+built library, or calling it with CPU tensors, raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libtslt.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_STATUS = 0, -1, -2, -3, -4, -5
+F32, BF16 = 0, 1
+MAX_K = 1024
+
+EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status",
+           "tslt_sparsify_workspace_bytes", "tslt_sparsify",
+           "tslt_verify_workspace_bytes", "tslt_verify",
+           "tslt_tree_verify_workspace_bytes", "tslt_tree_verify"]
+
+
+class TsltError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtslt.so (built in-tree by paper_2512_16273_b200/build.py).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("libtslt.so is not built: run `python -m paper_2512_16273_b200.build` "
+                          "(nvcc, sm_100a).  There is no fallback path.")
+    L = ctypes.CDLL(_LIB_PATH)
+    i, ll, f, p, sz = ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+    psz = ctypes.POINTER(ctypes.c_size_t)
+    L.tslt_version.restype = i
+    L.tslt_version.argtypes = []
+    L.tslt_status_string.restype = ctypes.c_char_p
+    L.tslt_status_string.argtypes = [i]
+    L.tslt_workspace_status.restype = i
+    L.tslt_workspace_status.argtypes = [p, p, ctypes.POINTER(i)]
+    L.tslt_sparsify_workspace_bytes.restype = i
+    L.tslt_sparsify_workspace_bytes.argtypes = [i, i, i, i, psz]
+    L.tslt_sparsify.restype = i
+    L.tslt_sparsify.argtypes = [p, i, i, i, i, ll, i, f, f, i, p, p, p, p, p, p, p, p, sz, p]
+    L.tslt_verify_workspace_bytes.restype = i
+    L.tslt_verify_workspace_bytes.argtypes = [i, i, i, i, psz]
+    L.tslt_verify.restype = i
+    L.tslt_verify.argtypes = [p, i, i, i, i, ll, i, p, p, p, p, f, f, p, p, p, p, p, p, p, p, sz, p]
+    L.tslt_tree_verify_workspace_bytes.restype = i
+    L.tslt_tree_verify_workspace_bytes.argtypes = [i, i, i, i, psz]
+    L.tslt_tree_verify.restype = i
+    L.tslt_tree_verify.argtypes = [p, i, i, i, i, ll, p, p, i, i, p, p, p, p, f, f, p, p, i, p, p, p,
+                                   p, sz, p]
+    _lib = L
+    return L
+
+
+def version() -> int:
+    return lib().tslt_version()
+
+
+def status_string(status: int) -> str:
+    return lib().tslt_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise TsltError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TsltError(ERR_UNSUPPORTED, "dtype %s" % t.dtype)
+
+
+def _cuda(t: Optional[torch.Tensor], name: str, dtype=None) -> Optional[torch.Tensor]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (libtslt has no CPU path)" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("%s must have dtype %s" % (name, dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return t
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _row_layout(logits: torch.Tensor):
+    """(rows, V, row stride in elements) of a tensor [..., V] whose leading dimensions flatten
+    to equally spaced rows (a contiguous tensor, or a [:, ..., :V] view of a padded one)."""
+    if logits.dim() < 1 or (logits.shape[-1] > 1 and logits.stride(-1) != 1):
+        raise ValueError("logits must be contiguous along the vocabulary")
+    V = logits.shape[-1]
+    rows = logits.numel() // V if V else 0
+    if logits.dim() == 1:
+        return rows, V, V
+    stride = logits.stride(-2)
+    for d in range(logits.dim() - 2):
+        if logits.shape[d] > 1 and logits.stride(d) != logits.stride(d + 1) * logits.shape[d + 1]:
+            raise ValueError("rows of logits must be equally spaced in memory")
+    if rows <= 1 or logits.shape[-2] == 1:
+        # a single row per block: take the spacing from the next dimension that has one
+        stride = V
+        for d in range(logits.dim() - 2, -1, -1):
+            if logits.shape[d] > 1:
+                stride = logits.stride(d)
+                break
+    return rows, V, max(int(stride), V)
+
+
+_ws_cache: Dict[tuple, torch.Tensor] = {}
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """A cached device buffer of at least nbytes (torch's allocator returns >= 512-byte aligned)."""
+    key = (str(device), torch.cuda.current_stream(device).cuda_stream)
+    ws = _ws_cache.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(max(int(nbytes), 4096), dtype=torch.uint8, device=device)
+        _ws_cache[key] = ws
+    return ws
+
+
+def sparsify_workspace_bytes(rows: int, V: int, k: int, num_samples: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().tslt_sparsify_workspace_bytes(rows, V, k, num_samples, ctypes.byref(n)),
+           "tslt_sparsify_workspace_bytes")
+    return int(n.value)
+
+
+def verify_workspace_bytes(B: int, gamma: int, V: int, k: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().tslt_verify_workspace_bytes(B, gamma, V, k, ctypes.byref(n)), "tslt_verify_workspace_bytes")
+    return int(n.value)
+
+
+def tree_verify_workspace_bytes(B: int, N: int, V: int, k: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().tslt_tree_verify_workspace_bytes(B, N, V, k, ctypes.byref(n)),
+           "tslt_tree_verify_workspace_bytes")
+    return int(n.value)
+
+
+def workspace_status(ws: torch.Tensor) -> int:
+    """Synchronous: device status word of a workspace (0 = every device-side wait completed)."""
+    word = ctypes.c_int(0)
+    rc = lib().tslt_workspace_status(_ptr(ws), _stream(), ctypes.byref(word))
+    if rc not in (OK, ERR_DEVICE_STATUS):
+        raise TsltError(rc, "tslt_workspace_status")
+    return int(word.value)
+
+
+def sparsify(logits: torch.Tensor, k: int, top_p: float = 1.0, temperature: float = 1.0,
+             uniforms: Optional[torch.Tensor] = None, *, want_stats: bool = True,
+             out: Optional[dict] = None, ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_sparsify on logits [..., V] (fp32 / bf16, CUDA).  uniforms [rows, num_samples] fp32.
+
+    Returns dict(idx [rows,k] int32, logit [rows,k] fp32, count [rows] int32,
+    token [rows,num_samples] int32, lse [rows] fp32, mass [rows] fp32, workspace)."""
+    if not logits.is_cuda:
+        raise ValueError("logits must be a CUDA tensor (libtslt has no CPU path)")
+    rows, V, stride = _row_layout(logits)
+    flat = logits
+    dev = logits.device
+    ns = 0
+    if uniforms is not None:
+        _cuda(uniforms, "uniforms", torch.float32)
+        if rows and uniforms.numel() % rows:
+            raise ValueError("uniforms must be [rows, num_samples]")
+        ns = uniforms.numel() // rows if rows else 0
+    o = out if out is not None else {}
+    if "idx" not in o:
+        o["idx"] = torch.empty(rows, k, dtype=torch.int32, device=dev)
+        o["logit"] = torch.empty(rows, k, dtype=torch.float32, device=dev)
+        o["count"] = torch.empty(rows, dtype=torch.int32, device=dev)
+        o["token"] = torch.empty(rows, ns, dtype=torch.int32, device=dev)
+        if want_stats:
+            o["lse"] = torch.empty(rows, dtype=torch.float32, device=dev)
+            o["mass"] = torch.empty(rows, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(sparsify_workspace_bytes(rows, V, k, ns), dev)
+    rc = lib().tslt_sparsify(_ptr(flat), _dtype_code(logits), rows, 1, V, stride, k, top_p, temperature,
+                             ns, _ptr(uniforms), _ptr(o["idx"]), _ptr(o["logit"]), _ptr(o["count"]),
+                             _ptr(o["token"]), _ptr(o.get("lse")), _ptr(o.get("mass")), _ptr(ws),
+                             ws.numel(), _stream())
+    _check(rc, "tslt_sparsify")
+    o["workspace"] = ws
+    return o
+
+
+def verify(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_logit: torch.Tensor,
+           draft_count: torch.Tensor, draft_token: torch.Tensor, draft_temperature: float,
+           target_temperature: float, u_accept: torch.Tensor, u_sample: torch.Tensor, *,
+           want_diag: bool = True, out: Optional[dict] = None,
+           ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_verify.  target_logits [B, gamma+1, V]; drafts [B, gamma, k] as written by sparsify.
+
+    Returns dict(accepted_len [B], out_token [B], and with want_diag accept_prob, beta_hat
+    [B, gamma], lse_p [B, gamma+1], workspace)."""
+    if not target_logits.is_cuda:
+        raise ValueError("target_logits must be a CUDA tensor (libtslt has no CPU path)")
+    if target_logits.dim() != 3:
+        raise ValueError("target_logits must be [B, gamma+1, V]")
+    B, g1, V = target_logits.shape
+    _, _, stride = _row_layout(target_logits)
+    gamma = g1 - 1
+    k = draft_idx.shape[-1] if gamma > 0 else 1
+    dev = target_logits.device
+    _cuda(draft_idx, "draft_idx", torch.int32)
+    _cuda(draft_logit, "draft_logit", torch.float32)
+    _cuda(draft_count, "draft_count", torch.int32)
+    _cuda(draft_token, "draft_token", torch.int32)
+    _cuda(u_accept, "u_accept", torch.float32)
+    _cuda(u_sample, "u_sample", torch.float32)
+    if draft_idx.numel() != B * gamma * k or draft_logit.numel() != B * gamma * k or \
+            draft_count.numel() != B * gamma or draft_token.numel() != B * gamma or \
+            u_accept.numel() != B * gamma or u_sample.numel() != B:
+        raise ValueError("draft / uniform shapes do not match target_logits")
+    o = out if out is not None else {}
+    if "accepted_len" not in o:
+        o["accepted_len"] = torch.empty(B, dtype=torch.int32, device=dev)
+        o["out_token"] = torch.empty(B, dtype=torch.int32, device=dev)
+        if want_diag:
+            o["accept_prob"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
+            o["beta_hat"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
+            o["lse_p"] = torch.empty(B, gamma + 1, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(verify_workspace_bytes(B, gamma, V, k), dev)
+    rc = lib().tslt_verify(_ptr(target_logits), _dtype_code(target_logits), B, gamma, V, stride, k,
+                           _ptr(draft_idx), _ptr(draft_logit), _ptr(draft_count), _ptr(draft_token),
+                           draft_temperature, target_temperature, _ptr(u_accept), _ptr(u_sample),
+                           _ptr(o["accepted_len"]), _ptr(o["out_token"]), _ptr(o.get("accept_prob")),
+                           _ptr(o.get("beta_hat")), _ptr(o.get("lse_p")), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "tslt_verify")
+    o["workspace"] = ws
+    return o
+
+
+def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_row: Sequence[int],
+                node_token: torch.Tensor, draft_idx: torch.Tensor, draft_logit: torch.Tensor,
+                draft_count: torch.Tensor, draft_temperature: float, target_temperature: float,
+                u_accept: torch.Tensor, u_sample: torch.Tensor, max_depth: int, *,
+                out: Optional[dict] = None, ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_tree_verify.  target_logits [B, N, V]; parent / node_draft_row are host sequences [N];
+    drafts [B, M, k].  Returns dict(accepted_path [B, max_depth], accepted_len [B], out_token [B])."""
+    if not target_logits.is_cuda:
+        raise ValueError("target_logits must be a CUDA tensor (libtslt has no CPU path)")
+    if target_logits.dim() != 3:
+        raise ValueError("target_logits must be [B, N, V]")
+    B, N, V = target_logits.shape
+    _, _, stride = _row_layout(target_logits)
+    par = np.ascontiguousarray(np.asarray(parent, dtype=np.int32))
+    ndr = np.ascontiguousarray(np.asarray(node_draft_row, dtype=np.int32))
+    if par.shape != (N,) or ndr.shape != (N,):
+        raise ValueError("parent and node_draft_row must have N entries")
+    M = int((ndr >= 0).sum())
+    k = draft_idx.shape[-1] if M > 0 else 1
+    dev = target_logits.device
+    for name, t, dt in (("node_token", node_token, torch.int32), ("draft_idx", draft_idx, torch.int32),
+                        ("draft_logit", draft_logit, torch.float32), ("draft_count", draft_count, torch.int32),
+                        ("u_accept", u_accept, torch.float32), ("u_sample", u_sample, torch.float32)):
+        _cuda(t, name, dt)
+    if node_token.numel() != B * N or u_accept.numel() != B * N or u_sample.numel() != B * N or \
+            draft_idx.numel() != B * M * k or draft_logit.numel() != B * M * k or draft_count.numel() != B * M:
+        raise ValueError("tree tensors do not match target_logits / the tree shape")
+    o = out if out is not None else {}
+    if "accepted_len" not in o:
+        o["accepted_path"] = torch.empty(B, max_depth, dtype=torch.int32, device=dev)
+        o["accepted_len"] = torch.empty(B, dtype=torch.int32, device=dev)
+        o["out_token"] = torch.empty(B, dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(tree_verify_workspace_bytes(B, N, V, k), dev)
+    rc = lib().tslt_tree_verify(_ptr(target_logits), _dtype_code(target_logits), B, N, V, stride,
+                                par.ctypes.data_as(ctypes.c_void_p), ndr.ctypes.data_as(ctypes.c_void_p),
+                                M, k, _ptr(node_token), _ptr(draft_idx), _ptr(draft_logit), _ptr(draft_count),
+                                draft_temperature, target_temperature, _ptr(u_accept), _ptr(u_sample),
+                                max_depth, _ptr(o["accepted_path"]), _ptr(o["accepted_len"]),
+                                _ptr(o["out_token"]), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "tslt_tree_verify")
+    o["workspace"] = ws
+    return o
+
+
+def payload_bits(count: int, V: int, b_prob: int = 32) -> int:
+    """Uplink payload of one sparse distribution, the per-distribution data volume of Section
+    2.2 with the vocabulary size replaced by the retained count: count * (b_prob + ceil(log2 V))."""
+    return int(count) * (int(b_prob) + math.ceil(math.log2(V)))

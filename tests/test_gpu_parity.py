@@ -1,0 +1,298 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Sizes span several tiles, ragged tails and split rows."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_16273_b200 import synth, tslt
+from parity_utils import (compare_sparsify, compare_tree, compare_verify, run_sequence_case, to_gpu_rows,
+                          to_np)
+
+pytestmark = pytest.mark.gpu
+
+
+def small_logits(B, gamma, V, dtype, seed, sigma_t=0.5):
+    return synth.sequence_logits(B, gamma, V, dtype, sigma_t, seed, "cpu")
+
+
+@pytest.mark.parametrize("V", [8, 16, 100, 1000, 1001, 4099, 8192, 8200, 20011, 70001])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_sequence_small_vocab_sweep(V, dtype):
+    """Tiny to mid vocabularies: single tile, ragged tails (V not a multiple of the vector
+    width), several tiles, split rows."""
+    B, gamma = 3, 2
+    zq, zp = small_logits(B, gamma, V, dtype, seed=V)
+    for k, top_p, T, ns in [(1, 1.0, 1.0, 1), (min(V, 5), 1.0, 0.7, 2), (min(V, 64), 0.9, 1.0, 1),
+                            (min(V, 300), 0.95, 0.5, 3), (min(V, 1024), 1.0, 1.3, 1)]:
+        run_sequence_case(zq, zp, k, top_p, T, seed=7 * V + k, num_samples=ns,
+                          what="V=%d %s k=%d p=%g T=%g" % (V, dtype, k, top_p, T))
+
+
+def test_k_equals_V_small():
+    for V in (8, 16, 33, 1024):
+        zq, zp = small_logits(2, 3, V, torch.float32, seed=100 + V)
+        run_sequence_case(zq, zp, V, 1.0, 1.0, seed=V, what="k=V=%d" % V)
+        run_sequence_case(zq, zp, V, 0.7, 0.8, seed=V + 1, what="k=V=%d top-p" % V)
+
+
+@pytest.mark.parametrize("cfg_id", [0, 1, 2])
+def test_config_full_size(cfg_id):
+    """Benchmark configs 0-2 at full size, every row and sequence compared."""
+    cfg = synth.CONFIGS[cfg_id]
+    dt = synth.torch_dtype(cfg["dtype"])
+    flagged = total = 0
+    for seed in (0, 1):
+        zq, zp = synth.sequence_logits(cfg["B"], cfg["gamma"], cfg["V"], dt, cfg["sigma_t"], seed, "cpu")
+        f1, f2, _, _ = run_sequence_case(zq, zp, cfg["k"], cfg["top_p"], cfg["temperature"], seed,
+                                         what=cfg["name"])
+        flagged += f1[0] + f2[0]
+        total += f1[1] + f2[1]
+    assert flagged <= 0.25 * total  # the exemption is the exception, not the rule
+
+
+def test_top_p_below_cap_and_second_temperature():
+    """Low temperature so the nucleus cut lands below the cap (both branches of n = min(k, n*))."""
+    zq, zp = small_logits(4, 4, 32000, torch.bfloat16, seed=77)
+    _, _, ref_s, _ = run_sequence_case(zq, zp, 256, 0.9, 0.5, seed=5, what="top-p T=0.5")
+    assert (ref_s["count"] < 256).any()
+    _, _, ref_s, _ = run_sequence_case(zq, zp, 32, 0.9, 1.0, seed=6, what="top-p cap binds")
+    assert (ref_s["count"] == 32).any()
+
+
+def adversarial_rows(V, dtype):
+    rows = []
+    asc = torch.linspace(-8, 8, V)
+    rows.append(asc)                                   # ascending: every element beats the threshold
+    rows.append(asc.flip(0))                           # descending
+    rows.append(torch.zeros(V))                        # all equal: ties everywhere
+    t = torch.zeros(V); t[::7] = 1.0; rows.append(t)   # two values, heavy ties at the cut
+    g = torch.Generator().manual_seed(3)
+    r = torch.randn(V, generator=g); r[torch.rand(V, generator=g) < 0.3] = -float("inf"); rows.append(r)
+    rows.append(torch.full((V,), -float("inf")))       # no finite logit at all
+    r2 = torch.full((V,), -float("inf")); r2[V // 2] = 1.5; r2[5] = 0.5; rows.append(r2)  # fewer finite than k
+    r3 = torch.randn(V, generator=g) * 30; rows.append(r3)  # wide dynamic range
+    r4 = torch.randn(V, generator=g); r4[::3] = -0.0; r4[1::3] = 0.0; rows.append(r4)   # signed zeros
+    return torch.stack(rows).to(dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V", [1000, 40000])
+def test_sparsify_adversarial_rows(V, dtype):
+    z = adversarial_rows(V, dtype)
+    rows = z.shape[0]
+    for k, top_p in [(1, 1.0), (7, 1.0), (64, 1.0), (257, 1.0), (1000, 1.0), (128, 0.9)]:
+        u = synth.uniforms((rows, 2), k, synth.TID_U_DRAFT)
+        ref = oracle.sparsify(z, k, top_p, 1.0, u.numpy())
+        gpu = tslt.sparsify(z.cuda(), k, top_p, 1.0, u.cuda())
+        torch.cuda.synchronize()
+        assert tslt.workspace_status(gpu["workspace"]) == 0
+        compare_sparsify(gpu, ref, "adversarial V=%d k=%d p=%g" % (V, k, top_p))
+
+
+def test_verify_edge_tokens_and_uniforms():
+    """u = 0, u just below 1 and u >= 1 (clamped) for every decision; draft token outside the
+    transmitted set; target row with -inf at the drafted token."""
+    B, gamma, V, k = 6, 3, 5000, 16
+    zq, zp = small_logits(B, gamma, V, torch.bfloat16, seed=9)
+    ud = synth.uniforms((B * gamma, 1), 1, synth.TID_U_DRAFT)
+    ref_s = oracle.sparsify(zq.reshape(-1, V), k, 1.0, 1.0, ud.numpy())
+    tok = ref_s["token"][:, 0].reshape(B, gamma).copy()
+    tok[1, 0] = int(np.setdiff1d(np.arange(V), ref_s["idx"][gamma * 1])[0])  # not in S
+    zp = zp.clone()
+    zp[2, 0, tok[2, 0]] = -float("inf")                                      # p(x) = 0: never accepted
+    one_m = float(np.nextafter(np.float32(1), np.float32(0)))
+    ua = torch.tensor([[0.0] * gamma, [0.5] * gamma, [0.0] * gamma, [one_m] * gamma, [1.0] * gamma,
+                       [0.0, 0.0, 3.0]], dtype=torch.float32)
+    for us_val in (0.0, one_m, 1.0, 0.37):
+        us = torch.full((B,), us_val, dtype=torch.float32)
+        ref = oracle.verify(zp, ref_s["idx"].reshape(B, gamma, k), ref_s["logit"].reshape(B, gamma, k),
+                            ref_s["count"].reshape(B, gamma), tok, 1.0, 1.0, ua.numpy(), us.numpy())
+        gpu = tslt.verify(zp.cuda(), torch.from_numpy(ref_s["idx"]).cuda().view(B, gamma, k),
+                          torch.from_numpy(ref_s["logit"]).cuda().view(B, gamma, k),
+                          torch.from_numpy(ref_s["count"]).cuda().view(B, gamma),
+                          torch.from_numpy(tok).cuda(), 1.0, 1.0, ua.cuda(), us.cuda())
+        torch.cuda.synchronize()
+        compare_verify(gpu, ref, "edge us=%g" % us_val)
+    assert ref["accepted_len"][2] == 0 and ref["accept_prob"][2, 0] == 0.0
+
+
+def test_identical_models_accept_everything():
+    B, gamma, V = 4, 5, 30000
+    zq, _ = small_logits(B, gamma, V, torch.bfloat16, seed=12)
+    zp = torch.cat([zq, zq[:, :1]], dim=1).contiguous()
+    _, _, _, ref_v = run_sequence_case(zq, zp, 1024, 1.0, 1.0, seed=3, what="identical")
+    # with k < V the truncated q~ exceeds p on S, so acceptance is p/q~ = rho < 1: not all accepted,
+    # but beta^ equals the retained mass
+    zq2, _ = small_logits(2, 2, 512, torch.float32, seed=13)
+    zp2 = torch.cat([zq2, zq2[:, :1]], dim=1).contiguous()
+    _, _, ref_s, ref_v = run_sequence_case(zq2, zp2, 512, 1.0, 1.0, seed=4, what="identical k=V")
+    assert (ref_v["accepted_len"] == 2).all()
+
+
+def test_strided_rows_and_zero_rows():
+    V, k = 3000, 32
+    stride = 3008  # multiple of 8 elements: rows stay 16-byte aligned
+    buf = torch.randn(5, stride).to(torch.bfloat16)
+    z = buf[:, :V]
+    u = synth.uniforms((5, 1), 2, synth.TID_U_DRAFT)
+    ref = oracle.sparsify(z.contiguous(), k, 1.0, 1.0, u.numpy())
+    gpu = tslt.sparsify(buf.cuda()[:, :V], k, 1.0, 1.0, u.cuda())
+    torch.cuda.synchronize()
+    compare_sparsify(gpu, ref, "strided")
+    empty = tslt.sparsify(torch.empty(0, V, dtype=torch.bfloat16, device="cuda"), k, 1.0, 1.0,
+                          torch.empty(0, 1, device="cuda"))
+    assert empty["idx"].shape == (0, k)
+
+
+def test_determinism_and_canaries():
+    """Same inputs twice give identical bytes; nothing is written outside the output buffers."""
+    cfg = synth.CONFIGS[1]
+    zq, zp = synth.sequence_logits(cfg["B"], cfg["gamma"], cfg["V"], torch.bfloat16, 0.5, 3, "cpu")
+    B, gamma, V, k = cfg["B"], cfg["gamma"], cfg["V"], cfg["k"]
+    rows = B * gamma
+    u = synth.uniforms((rows, 2), 3, synth.TID_U_DRAFT).cuda()
+    zq_d = zq.cuda()
+    pad = 64
+    CAN_I, CAN_F = -123456789, -1234.5
+
+    def padded(n, dtype, val):
+        t = torch.full((n + 2 * pad,), val, dtype=dtype, device="cuda")
+        return t, t[pad:pad + n]
+
+    outs = []
+    for _ in range(2):
+        bufs = {}
+        o = {}
+        for name, n, dt, val in (("idx", rows * k, torch.int32, CAN_I), ("logit", rows * k, torch.float32, CAN_F),
+                                 ("count", rows, torch.int32, CAN_I), ("token", rows * 2, torch.int32, CAN_I),
+                                 ("lse", rows, torch.float32, CAN_F), ("mass", rows, torch.float32, CAN_F)):
+            bufs[name], o[name] = padded(n, dt, val)
+        o["idx"] = o["idx"].view(rows, k); o["logit"] = o["logit"].view(rows, k); o["token"] = o["token"].view(rows, 2)
+        tslt.sparsify(zq_d, k, cfg["top_p"], cfg["temperature"], u, out=o)
+        torch.cuda.synchronize()
+        for name, full in bufs.items():
+            val = CAN_I if full.dtype == torch.int32 else CAN_F
+            assert (full[:pad] == val).all() and (full[-pad:] == val).all(), name
+        outs.append({n: to_np(o[n]).copy() for n in ("idx", "logit", "count", "token", "lse", "mass")})
+    for n in outs[0]:
+        assert outs[0][n].tobytes() == outs[1][n].tobytes(), n
+
+
+def run_tree_case(B, expansion, V, dtype, k, T, seed, sigma_t=0.5, what=""):
+    parent, ndr, M, depth = synth.complete_tree(expansion)
+    N = len(parent)
+    zq, zp = synth.tree_logits(B, parent, ndr, V, dtype, sigma_t, seed, "cpu")
+    kmax = max(expansion)
+    ud = synth.uniforms((B * M, kmax), seed, synth.TID_U_DRAFT)
+    ref_s = oracle.sparsify(zq.reshape(B * M, V), k, 1.0, T, ud.numpy())
+    gpu_s = tslt.sparsify(to_gpu_rows(zq), k, 1.0, T, ud.cuda())
+    torch.cuda.synchronize()
+    compare_sparsify(gpu_s, ref_s, what + " tree sparsify")
+    toks = np.zeros((B, N), np.int32)
+    for n in range(N):
+        if ndr[n] >= 0:
+            ch = [c for c in range(N) if parent[c] == n]
+            for b in range(B):
+                toks[b, ch] = ref_s["token"][b * M + ndr[n], :len(ch)]
+    ua = synth.uniforms((B, N), seed, synth.TID_U_ACCEPT)
+    us = synth.uniforms((B, N), seed, synth.TID_U_SAMPLE)
+    ref = oracle.tree_verify(zp, parent, ndr, toks, ref_s["idx"].reshape(B, M, k), ref_s["logit"].reshape(B, M, k),
+                             ref_s["count"].reshape(B, M), T, T, ua.numpy(), us.numpy(), depth)
+    gpu = tslt.tree_verify(to_gpu_rows(zp), parent, ndr, torch.from_numpy(toks).cuda(),
+                           torch.from_numpy(ref_s["idx"]).cuda().view(B, M, k),
+                           torch.from_numpy(ref_s["logit"]).cuda().view(B, M, k),
+                           torch.from_numpy(ref_s["count"]).cuda().view(B, M), T, T, ua.cuda(), us.cuda(), depth)
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(gpu["workspace"]) == 0
+    return compare_tree(gpu, ref, what), ref
+
+
+@pytest.mark.parametrize("expansion,V,dtype,k", [((2, 2, 2), 32000, torch.bfloat16, 64),
+                                                  ((3,), 1000, torch.float32, 8),
+                                                  ((1, 1, 1, 1), 5000, torch.bfloat16, 16),
+                                                  ((4, 2), 20011, torch.float32, 300),
+                                                  ((2, 3), 16, torch.float32, 4)])
+def test_tree_small(expansion, V, dtype, k):
+    lens = []
+    for seed in range(3):
+        _, ref = run_tree_case(6, expansion, V, dtype, k, 1.0, seed, what="tree %s V=%d" % (expansion, V))
+        lens.append(ref["accepted_len"])
+    assert np.concatenate(lens).max() >= 1  # some child is accepted somewhere
+
+
+def test_tree_config3_reduced_batch():
+    cfg = synth.CONFIGS[3]
+    (flagged, total), ref = run_tree_case(4, cfg["expansion"], cfg["V"], torch.bfloat16, cfg["k"], 1.0, 0,
+                                          what=cfg["name"])
+    assert flagged <= total // 2
+
+
+def test_tree_duplicate_children_and_single_node():
+    """Identical sibling tokens (drawn with replacement) and the degenerate root-only tree."""
+    V, k, B = 2000, 4, 5
+    parent, ndr, M, depth = synth.complete_tree((3,))
+    N = len(parent)
+    zq, zp = synth.tree_logits(B, parent, ndr, V, torch.float32, 0.5, 4, "cpu")
+    ref_s = oracle.sparsify(zq.reshape(B * M, V), k, 1.0, 1.0, np.zeros((B * M, 1), np.float32))
+    toks = np.zeros((B, N), np.int32)
+    toks[:, 1:] = ref_s["token"][:, :1]  # all three children carry the same token
+    one_m = float(np.nextafter(np.float32(1), np.float32(0)))
+    ua = torch.full((B, N), one_m)
+    us = synth.uniforms((B, N), 4, synth.TID_U_SAMPLE)
+    ref = oracle.tree_verify(zp, parent, ndr, toks, ref_s["idx"].reshape(B, M, k), ref_s["logit"].reshape(B, M, k),
+                             ref_s["count"].reshape(B, M), 1.0, 1.0, ua.numpy(), us.numpy(), depth)
+    gpu = tslt.tree_verify(zp.cuda(), parent, ndr, torch.from_numpy(toks).cuda(),
+                           torch.from_numpy(ref_s["idx"]).cuda().view(B, M, k),
+                           torch.from_numpy(ref_s["logit"]).cuda().view(B, M, k),
+                           torch.from_numpy(ref_s["count"]).cuda().view(B, M), 1.0, 1.0, ua.cuda(), us.cuda(), depth)
+    torch.cuda.synchronize()
+    compare_tree(gpu, ref, "duplicates")
+    # root only: the "tree" is a leaf, the token is a plain sample of the root row
+    z1 = zp[:, :1].contiguous()
+    ref = oracle.tree_verify(z1, [-1], [-1], np.zeros((B, 1), np.int32), np.zeros((B, 0, 1), np.int32),
+                             np.zeros((B, 0, 1), np.float32), np.zeros((B, 0), np.int32), 1.0, 1.0,
+                             np.zeros((B, 1), np.float32), us[:, :1].numpy(), 0)
+    e_i = torch.empty(0, dtype=torch.int32, device="cuda")
+    gpu = tslt.tree_verify(z1.cuda(), [-1], [-1], torch.zeros(B, 1, dtype=torch.int32, device="cuda"), e_i,
+                           torch.empty(0, device="cuda"), e_i, 1.0, 1.0, torch.zeros(B, 1, device="cuda"),
+                           us[:, :1].contiguous().cuda(), 0)
+    torch.cuda.synchronize()
+    assert (to_np(gpu["accepted_len"]) == 0).all()
+    bad = (to_np(gpu["out_token"]) != ref["out_token"]) & ((ref["flags"] & oracle.FLAG_RES) == 0)
+    assert not bad.any()
+
+
+def test_argument_errors_leave_outputs_untouched():
+    V, k = 1000, 8
+    z = torch.randn(2, V, device="cuda")
+    u = torch.rand(2, 1, device="cuda")
+    out = tslt.sparsify(z, k, 1.0, 1.0, u)
+    torch.cuda.synchronize()
+    snapshot = out["idx"].clone()
+    for kwargs in (dict(k=0), dict(k=V + 1), dict(top_p=0.0), dict(temperature=0.0), dict(temperature=float("nan")),
+                   dict(k=2000)):
+        args = dict(k=k, top_p=1.0, temperature=1.0)
+        args.update(kwargs)
+        o2 = {n: out[n] for n in ("idx", "logit", "count", "token", "lse", "mass")}
+        if args["k"] != k:
+            o2 = None
+        with pytest.raises((tslt.TsltError, ValueError, RuntimeError)):
+            tslt.sparsify(z if args["k"] <= V + 1 else torch.randn(2, 4000, device="cuda"), args["k"], args["top_p"],
+                          args["temperature"], u, out=o2)
+    torch.cuda.synchronize()
+    assert torch.equal(out["idx"], snapshot)
+    # misaligned base pointer
+    zb = torch.randn(2 * V + 8, device="cuda")[1:1 + 2 * V].view(2, V)
+    with pytest.raises(tslt.TsltError):
+        tslt.sparsify(zb, k, 1.0, 1.0, u)
+    # workspace too small
+    with pytest.raises(tslt.TsltError):
+        tslt.sparsify(z, k, 1.0, 1.0, u, ws=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    # bad tree: parent not before child
+    with pytest.raises(tslt.TsltError):
+        tslt.tree_verify(torch.randn(1, 3, V, device="cuda"), [-1, 2, 0], [0, 1, -1],
+                         torch.zeros(1, 3, dtype=torch.int32, device="cuda"),
+                         torch.zeros(1, 2, k, dtype=torch.int32, device="cuda"), torch.zeros(1, 2, k, device="cuda"),
+                         torch.zeros(1, 2, dtype=torch.int32, device="cuda"), 1.0, 1.0,
+                         torch.zeros(1, 3, device="cuda"), torch.zeros(1, 3, device="cuda"), 2)
