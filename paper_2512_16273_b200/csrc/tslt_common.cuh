@@ -19,7 +19,7 @@ constexpr int kTileBytes = 16384;
 constexpr int kChunkBytes = kTileBytes / kConsumerWarps;  // 2048 B: the unit of per-chunk partial sums
 constexpr int kVecBytes = 16;
 constexpr int kVecsPerLane = kChunkBytes / (32 * kVecBytes);  // 4
-constexpr int kStages = 4;
+constexpr int kStages = 3;
 constexpr int kRingBytes = kStages * kTileBytes;
 
 // Named barrier for the consumer warps (barrier 0 is left to __syncthreads before the roles split).
@@ -227,6 +227,10 @@ template <> struct Elt<bf16_t> {
         return __uint_as_float(b << 16);
     }
 };
+
+__device__ __forceinline__ uint4 lds_vec(const unsigned char* p) {
+    return *reinterpret_cast<const uint4*>(p);
+}
 
 // Unpack one 16-byte vector into fp32 values.
 template <typename T> __device__ __forceinline__ void unpack_vec(const uint4& v, float* z);

@@ -89,54 +89,68 @@ struct Candidates {
     int* count;         // shared counter
 };
 
-// Trim the buffer to its exact top-k under (key descending, idx ascending).  All 256 consumer
-// threads call it with the same arguments after a barrier.  On return *count <= k and every
-// thread gets the k-th key (or 0 if fewer than k entries were present: nothing trimmed) in
-// *kth_key; the return value tells whether k entries are present.
+// Exact top-k, under the order (key descending, idx ascending), of a virtual sequence of n
+// items; item i is a member iff src.valid(i) and has src.key(i), src.idx(i) (indices are
+// distinct).  The winners replace the contents of the candidate buffer (the source may read the
+// buffer: winners are staged in tmp first).  All 256 consumer threads call it with the same
+// arguments after a barrier.  Returns true iff at least k members exist, in which case
+// *kth_key is the k-th key; *cb.count is set to min(k, members).
 // kKeyHiOnly: keys come from bf16 values, so only the two high bytes vary (the low 16 bits
 // follow from the sign).  idx_hi_byte: highest byte of an index that can be non-zero.
-template <bool kKeyHiOnly>
-__device__ __forceinline__ bool trim_to_topk(Candidates cb, int k, int idx_hi_byte, SelectScratch* sc,
-                                             int tid, uint32_t* kth_key) {
-    const int n = *cb.count;
-    consumer_sync();
-    if (n < k) {
-        *kth_key = 0;
-        return false;
-    }
-    int n_gt;
-    auto all = [&](int) { return true; };
-    auto getk = [&](int i) { return cb.key[i]; };
-    uint32_t kth;
-    if (kKeyHiOnly) {
-        kth = radix_select<true>(n, k, 3, 2, 0u, getk, all, sc, tid, &n_gt);
-        // low half of a key made from a bf16 value: 0x0000 for non-negative, 0xffff for negative
-        kth = (kth & 0xffff0000u) | ((kth & 0x80000000u) ? 0u : 0xffffu);
-    } else {
-        kth = radix_select<true>(n, k, 3, 0, 0u, getk, all, sc, tid, &n_gt);
+template <bool kKeyHiOnly, typename Src>
+__device__ __forceinline__ bool select_topk(const Src& src, int n, int k, int idx_hi_byte, Candidates cb,
+                                            SelectScratch* sc, int tid, uint32_t* kth_key) {
+    int* iscr = reinterpret_cast<int*>(sc->hist);
+    int my = 0;
+    for (int i = tid; i < n; i += kConsumerThreads) my += src.valid(i) ? 1 : 0;
+    const int members = block_sum_int(my, tid, iscr);
+    uint32_t kth = 0, idx_cut = 0xffffffffu;
+    const bool full = members >= k;
+    if (members > k) {
+        int n_gt;
+        auto valid = [&](int i) { return src.valid(i); };
+        auto getk = [&](int i) { return src.key(i); };
+        if (kKeyHiOnly) {
+            kth = radix_select<true>(n, k, 3, 2, 0u, getk, valid, sc, tid, &n_gt);
+            // low half of a key made from a bf16 value: 0x0000 for non-negative, 0xffff for negative
+            kth = (kth & 0xffff0000u) | ((kth & 0x80000000u) ? 0u : 0xffffu);
+        } else {
+            kth = radix_select<true>(n, k, 3, 0, 0u, getk, valid, sc, tid, &n_gt);
+        }
+        const int need = k - n_gt;  // ties to keep, >= 1
+        int eq = 0;
+        for (int i = tid; i < n; i += kConsumerThreads) eq += (src.valid(i) && src.key(i) == kth) ? 1 : 0;
+        const int n_eq = block_sum_int(eq, tid, iscr);
+        if (n_eq > need) {
+            int dummy;
+            auto tie = [&](int i) { return src.valid(i) && src.key(i) == kth; };
+            auto geti = [&](int i) { return (uint32_t)src.idx(i); };
+            idx_cut = radix_select<false>(n, need, idx_hi_byte, 0, 0u, geti, tie, sc, tid, &dummy);
+        }
+    } else if (members == k) {
+        // the k-th key is the smallest member
+        uint32_t mn = 0xffffffffu;
+        for (int i = tid; i < n; i += kConsumerThreads)
+            if (src.valid(i)) mn = min(mn, src.key(i));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        if ((tid & 31) == 0) sc->hist[tid >> 5] = mn;
+        consumer_sync();
+        mn = sc->hist[0];
+#pragma unroll
+        for (int w = 1; w < kConsumerWarps; ++w) mn = min(mn, sc->hist[w]);
+        consumer_sync();
+        kth = mn;
     }
     *kth_key = kth;
-    if (n == k) return true;
-    const int need = k - n_gt;  // ties to keep, >= 1
-    // number of ties
-    int my = 0;
-    for (int i = tid; i < n; i += kConsumerThreads) my += (cb.key[i] == kth);
-    int* iscr = reinterpret_cast<int*>(sc->hist);
-    const int n_eq = block_sum_int(my, tid, iscr);
-    uint32_t idx_cut = 0xffffffffu;
-    if (n_eq > need) {
-        int dummy;
-        auto tie = [&](int i) { return cb.key[i] == kth; };
-        auto geti = [&](int i) { return (uint32_t)cb.idx[i]; };
-        idx_cut = radix_select<false>(n, need, idx_hi_byte, 0, 0u, geti, tie, sc, tid, &dummy);
-    }
     if (tid == 0) sc->counter = 0;
     consumer_sync();
     for (int i = tid; i < n; i += kConsumerThreads) {
-        uint32_t key = cb.key[i];
-        int id = cb.idx[i];
+        if (!src.valid(i)) continue;
+        const uint32_t key = src.key(i);
+        const int id = src.idx(i);
         if (key > kth || (key == kth && (uint32_t)id <= idx_cut)) {
-            int pos = atomicAdd(&sc->counter, 1);
+            const int pos = atomicAdd(&sc->counter, 1);
             if (pos < k) {
                 cb.tmp_key[pos] = key;
                 cb.tmp_idx[pos] = id;
@@ -144,13 +158,15 @@ __device__ __forceinline__ bool trim_to_topk(Candidates cb, int k, int idx_hi_by
         }
     }
     consumer_sync();
-    for (int i = tid; i < k; i += kConsumerThreads) {
+    const int kept = min(sc->counter, k);
+    for (int i = tid; i < kept; i += kConsumerThreads) {
         cb.key[i] = cb.tmp_key[i];
         cb.idx[i] = cb.tmp_idx[i];
     }
-    if (tid == 0) *cb.count = k;
     consumer_sync();
-    return true;
+    if (tid == 0) *cb.count = kept;
+    consumer_sync();
+    return full;
 }
 
 // Bitonic sort of a[0..P) (P a power of two, shared memory), descending if kDescending.

@@ -12,6 +12,7 @@
 #include <math.h>
 
 #include "tslt_common.cuh"
+#include "tslt_rowmath.cuh"
 #include "tslt_select.cuh"
 #include "tslt_stream.cuh"
 
@@ -64,16 +65,68 @@ __host__ __device__ inline size_t sparsify_smem_bytes(int cap, int k) {
     return kRingBytes + (size_t)cap * 8 + (size_t)k * 8 + align_up(sizeof(SparsifyShared), 16) + 256;
 }
 
-template <typename T, bool kKeyHiOnly>
+// Sources for select_topk: the candidate buffer, one ring tile, or both.
+struct BufferSrc {
+    const uint32_t* k_;
+    const int* i_;
+    __device__ __forceinline__ bool valid(int) const { return true; }
+    __device__ __forceinline__ uint32_t key(int i) const { return k_[i]; }
+    __device__ __forceinline__ int idx(int i) const { return i_[i]; }
+};
+template <typename T> struct TileSrc {
+    const unsigned char* tile;
+    int elem0;
+    __device__ __forceinline__ bool valid(int i) const { return tile_elem<T>(tile, i) > -INFINITY; }
+    __device__ __forceinline__ uint32_t key(int i) const { return float_to_key(tile_elem<T>(tile, i)); }
+    __device__ __forceinline__ int idx(int i) const { return elem0 + i; }
+};
+// entries of the buffer that precede the tile, followed by every logit of the tile above tau
+template <typename T> struct UnionSrc {
+    const uint32_t* k_;
+    const int* i_;
+    int nb;
+    const unsigned char* tile;
+    int elem0;
+    float tau;
+    __device__ __forceinline__ bool valid(int i) const {
+        return i < nb ? i_[i] < elem0 : tile_elem<T>(tile, i - nb) > tau;
+    }
+    __device__ __forceinline__ uint32_t key(int i) const {
+        return i < nb ? k_[i] : float_to_key(tile_elem<T>(tile, i - nb));
+    }
+    __device__ __forceinline__ int idx(int i) const { return i < nb ? i_[i] : elem0 + (i - nb); }
+};
+
+__device__ __forceinline__ int barrier_or(bool pred) {
+    int any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"((int)pred), "n"(kConsumerBarrier), "n"(kConsumerThreads)
+        : "memory");
+    return any;
+}
+
+// Trim the candidate buffer to its exact top-k and raise tau to the k-th logit once k exist.
+template <bool kKeyHiOnly>
 __device__ __forceinline__ void rebuild(Candidates cb, int k, int idx_hi_byte, SparsifyShared* sh, int tid) {
+    const int n = min(*cb.count, 1 << 30);
+    consumer_sync();
+    if (n <= k) return;  // nothing to trim; tau unchanged (uniform: n is the same for every thread)
     uint32_t kth;
-    bool full = trim_to_topk<kKeyHiOnly>(cb, k, idx_hi_byte, &sh->sel, tid, &kth);
+    BufferSrc src{cb.key, cb.idx};
+    const bool full = select_topk<kKeyHiOnly>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
     if (full && tid == 0) sh->tau = key_to_float(kth);
     consumer_sync();
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kBlockThreads) sparsify_kernel(const SparsifyParams p) {
+__device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
+                                          unsigned char* ring, double Mrow, double Srow, int tid);
+
+template <typename T>
+__global__ void __launch_bounds__(kBlockThreads, 3) sparsify_kernel(const SparsifyParams p) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     constexpr int kPer = Elt<T>::kPerVec;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -109,10 +162,8 @@ __global__ void __launch_bounds__(kBlockThreads) sparsify_kernel(const SparsifyP
     const float chi = p.c.hi, clo = p.c.lo;
 
     // ---- streaming pass ----------------------------------------------------------------
-    float zmax = -INFINITY, M = -3.0e38f, negM = 3.0e38f;
-    float acc[kPer];
-#pragma unroll
-    for (int j = 0; j < kPer; ++j) acc[j] = 0.f;
+    LaneSum ls;
+    ls.reset();
     bool live = true;
 
     for (int t = tile_begin; t < tile_end; ++t) {
@@ -122,142 +173,68 @@ __global__ void __launch_bounds__(kBlockThreads) sparsify_kernel(const SparsifyP
         const unsigned char* tile = ring + s * kTileBytes;
         const float tau = sh->tau;
         const int tile_elem0 = t * (kTileBytes / Elt<T>::kBytes);
-        bool want_action = !arrived;
+        // the first tile of a segment is not filtered: its exact top-k is selected in place below
+        bool want_action = !arrived || it == 0;
+        if (arrived) {
+            LaneTile<T> lt;
+            lt.load(tile, warp, lane, padded);
+            const float lm = lt.lane_max();
+            if (lm > ls.zmax) ls.raise(lm, chi, clo);
+            lt.accumulate(ls, chi, clo);
+            if (it != 0 && lm > tau) {
 #pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j) {
-            const uint32_t off = warp * kChunkBytes + (j * 32 + lane) * kVecBytes;
-            if (arrived && off < padded) {
-                float z[kPer];
-                unpack_vec<T>(lds_vec(tile + off), z);
-                float vmax = z[0];
+                for (int j = 0; j < kVecsPerLane; ++j) {
+                    if (lt.vec_max(j) > tau) {
+                        const int e0 = tile_elem0 + (warp * kChunkBytes + (j * 32 + lane) * kVecBytes) / Elt<T>::kBytes;
 #pragma unroll
-                for (int e = 1; e < kPer; ++e) vmax = fmaxf(vmax, z[e]);
-                if (vmax > zmax) {
-                    zmax = vmax;
-                    const float Mn = fmaf(vmax, chi, vmax * clo);
-                    const float sc = ex2_approx(M - Mn);
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e) acc[e] *= sc;
-                    M = Mn;
-                    negM = -Mn;
-                }
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) acc[e] += ex2_approx(fmaf(z[e], chi, fmaf(z[e], clo, negM)));
-                if (vmax > tau) {
-                    const int e0 = tile_elem0 + (int)(off / Elt<T>::kBytes);
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e) {
-                        if (z[e] > tau) {
-                            const int pos = atomicAdd(&sh->cand_count, 1);
-                            if (pos < cap) {
-                                cand_key[pos] = float_to_key(z[e]);
-                                cand_idx[pos] = e0 + e;
-                            } else {
-                                sh->overflow = 1;
+                        for (int e = 0; e < kPer; ++e) {
+                            const float z = lt.elem(j, e);
+                            if (z > tau) {
+                                const int pos = atomicAdd(&sh->cand_count, 1);
+                                if (pos < cap) {
+                                    cand_key[pos] = float_to_key(z);
+                                    cand_idx[pos] = e0 + e;
+                                } else {
+                                    sh->overflow = 1;
+                                }
+                                if (pos + 1 > high) want_action = true;
                             }
-                            if (pos + 1 > high) want_action = true;
                         }
                     }
                 }
             }
         }
         // one barrier per tile: it also tells everyone whether the buffer needs attention
-        int any;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
-            "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
-            : "=r"(any)
-            : "r"((int)want_action), "n"(kConsumerBarrier), "n"(kConsumerThreads)
-            : "memory");
-        if (any) {
+        if (barrier_or(want_action)) {
             // a wait that ran out is decided collectively, so that nobody is left at a barrier
-            int gave_up;
-            asm volatile(
-                "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
-                "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
-                : "=r"(gave_up)
-                : "r"((int)!arrived), "n"(kConsumerBarrier), "n"(kConsumerThreads)
-                : "memory");
-            if (gave_up) {
+            if (barrier_or(!arrived)) {
                 if (!arrived) raise_abort(&sh->bars, p.status);
                 live = false;
                 break;
             }
-            const int ovf = sh->overflow;
-            consumer_sync();
-            if (!ovf) {
-                rebuild<T, kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
+            const int tile_elems = (int)(padded / Elt<T>::kBytes);
+            uint32_t kth;
+            bool full;
+            if (it == 0) {
+                TileSrc<T> src{tile, tile_elem0};
+                full = select_topk<kHiOnly>(src, tile_elems, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
             } else {
-                // This tile alone brought more candidates than fit.  Drop what it appended and
-                // feed it again in pieces that are guaranteed to fit, trimming in between.
-                // (The count before the tile was at most `high`; everything above it is this tile's.)
-                const int tile_elems = (int)(padded / Elt<T>::kBytes);
-                const int piece = cap - k;
-                if (tid == 0) {
-                    sh->overflow = 0;
-                }
-                // entries of earlier tiles are exactly those whose index lies below this tile
+                const int ovf = sh->overflow;
+                const int nb = min(sh->cand_count, cap);
                 consumer_sync();
-                {
-                    // compact away this tile's entries (their indices are >= tile_elem0)
-                    const int n_all = min(sh->cand_count, cap);
-                    consumer_sync();
-                    if (tid == 0) sh->sel.counter = 0;
-                    consumer_sync();
-                    // earlier entries number at most `high` <= cap - piece... keep them via tmp-free in-place pass:
-                    // process in rounds of 256 so that reads of a round precede its writes
-                    for (int base = 0; base < n_all; base += kConsumerThreads) {
-                        const int i = base + tid;
-                        uint32_t key = 0;
-                        int id = -1;
-                        bool keep = false;
-                        if (i < n_all) {
-                            key = cand_key[i];
-                            id = cand_idx[i];
-                            keep = id < tile_elem0;
-                        }
-                        consumer_sync();
-                        if (keep) {
-                            const int pos = atomicAdd(&sh->sel.counter, 1);  // pos <= i: never overtakes unread entries
-                            cand_key[pos] = key;
-                            cand_idx[pos] = id;
-                        }
-                        consumer_sync();
-                    }
-                    if (tid == 0) sh->cand_count = sh->sel.counter;
-                    consumer_sync();
-                }
-                for (int e_begin = 0; e_begin < tile_elems; e_begin += piece) {
-                    if (sh->cand_count + piece > cap) {
-                        consumer_sync();
-                        rebuild<T, kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
-                    } else {
-                        consumer_sync();
-                    }
-                    const float tau2 = sh->tau;
-                    const int e_end = min(tile_elems, e_begin + piece);
-                    for (int e = e_begin + tid; e < e_end; e += kConsumerThreads) {
-                        float z;
-                        if (Elt<T>::kBytes == 4) {
-                            z = reinterpret_cast<const float*>(tile)[e];
-                        } else {
-                            z = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(tile)[e] << 16);
-                        }
-                        if (z > tau2) {
-                            const int pos = atomicAdd(&sh->cand_count, 1);
-                            cand_key[pos] = float_to_key(z);
-                            cand_idx[pos] = tile_elem0 + e;
-                        }
-                    }
-                    consumer_sync();
-                }
-                if (sh->cand_count > high) {
-                    consumer_sync();
-                    rebuild<T, kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
+                if (!ovf) {
+                    BufferSrc src{cand_key, cand_idx};
+                    full = select_topk<kHiOnly>(src, nb, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
                 } else {
-                    consumer_sync();
+                    // this tile brought more candidates than fit: redo it from shared memory, selecting
+                    // over the earlier entries of the buffer and every logit of the tile above tau
+                    if (tid == 0) sh->overflow = 0;
+                    UnionSrc<T> src{cand_key, cand_idx, nb, tile, tile_elem0, tau};
+                    full = select_topk<kHiOnly>(src, nb + tile_elems, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
                 }
             }
+            if (full && tid == 0) sh->tau = key_to_float(kth);
+            consumer_sync();
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->bars.empty[s]);
@@ -266,20 +243,17 @@ __global__ void __launch_bounds__(kBlockThreads) sparsify_kernel(const SparsifyP
     consumer_sync();
 
     // ---- row statistics ------------------------------------------------------------------
-    float Mrow_f = warp_max(M);
+    float Mrow_f = warp_max(ls.M);
     if (lane == 0) sh->scratch[warp] = (double)Mrow_f;
     consumer_sync();
     double Mrow = sh->scratch[0];
     for (int w = 1; w < kConsumerWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
     consumer_sync();
-    double s_thread = 0.0;
-#pragma unroll
-    for (int e = 0; e < kPer; ++e) s_thread += (double)acc[e];
-    double Srow = block_sum(s_thread * exp2((double)M - Mrow), tid, sh->scratch);
+    double Srow = block_sum(ls.total_f64() * exp2((double)ls.M - Mrow), tid, sh->scratch);
 
     // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
     if (p.nseg > 1) {
-        rebuild<T, kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);  // <= k entries per segment
+        rebuild<kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);  // <= k entries per segment
         const int n = sh->cand_count;
         uint2* my_entries = p.seg_entries + ((size_t)row * p.nseg + seg) * (size_t)k;
         for (int i = tid; i < n; i += kConsumerThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
@@ -326,8 +300,18 @@ __global__ void __launch_bounds__(kBlockThreads) sparsify_kernel(const SparsifyP
         Srow = Sall;
     }
 
-    // ---- exact top-k of the row --------------------------------------------------------------
-    rebuild<T, kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
+    finalize_row<T>(p, row, cb, sh, ring, Mrow, Srow, tid);
+}
+
+// Exact top-k of the row, nucleus cut, renormalisation, sampling and the ascending-index payload.
+template <typename T>
+__device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
+                                          unsigned char* ring, double Mrow, double Srow, int tid) {
+    constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
+    const int k = p.k;
+    uint32_t* cand_key = cb.key;
+    int* cand_idx = cb.idx;
+    rebuild<kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
     const int n0 = min(sh->cand_count, k);
     const double L2 = Mrow + log2(Srow);  // base-2 log of the softmax normaliser
     const double cd = p.c.d;

@@ -106,8 +106,4 @@ __device__ __forceinline__ uint32_t tile_padded_bytes(long long row_bytes, int t
     return (bytes + 15u) & ~15u;
 }
 
-__device__ __forceinline__ uint4 lds_vec(const unsigned char* p) {
-    return *reinterpret_cast<const uint4*>(p);
-}
-
 }  // namespace tslt

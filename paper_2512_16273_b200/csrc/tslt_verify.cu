@@ -15,11 +15,12 @@
 #include <vector>
 
 #include "tslt_common.cuh"
+#include "tslt_rowmath.cuh"
 #include "tslt_stream.cuh"
 
 namespace tslt {
 
-constexpr int kMaxChunks = 3072;   // chunk partials of one row must fit the resolver's shared memory
+constexpr int kMaxChunks = 2048;   // chunk partials of one row must fit the resolver's shared memory
 constexpr int kMaxTreeNodes = 1024;
 
 struct VerifyParams {
@@ -60,7 +61,7 @@ struct VerifyShared {
     int ticket;
 };
 
-// Resolver work arrays laid over the idle ring.
+// Resolver work arrays, laid over the idle ring (and a little beyond it).
 struct ResolverArrays {
     double* chunkR;  // kMaxChunks
     int* s_idx;      // 1024
@@ -69,17 +70,18 @@ struct ResolverArrays {
     double* s_q;     // 1024
     double* r;       // 1024
 };
-__device__ __forceinline__ ResolverArrays carve(unsigned char* ring) {
+constexpr int kResolverBytes = kMaxChunks * 8 + 1024 * 4 + 4 * 1024 * 8;
+constexpr int kVerifyArena = kResolverBytes > kRingBytes ? kResolverBytes : kRingBytes;
+__device__ __forceinline__ ResolverArrays carve(unsigned char* arena) {
     ResolverArrays a;
-    a.chunkR = reinterpret_cast<double*>(ring);
-    a.s_idx = reinterpret_cast<int*>(ring + 24576);
-    a.s_p = reinterpret_cast<double*>(ring + 28672);
-    a.s_a = reinterpret_cast<double*>(ring + 36864);
-    a.s_q = reinterpret_cast<double*>(ring + 45056);
-    a.r = reinterpret_cast<double*>(ring + 53248);
+    a.chunkR = reinterpret_cast<double*>(arena);
+    a.s_idx = reinterpret_cast<int*>(arena + kMaxChunks * 8);
+    a.s_p = reinterpret_cast<double*>(arena + kMaxChunks * 8 + 4096);
+    a.s_a = a.s_p + 1024;
+    a.s_q = a.s_a + 1024;
+    a.r = a.s_q + 1024;
     return a;
 }
-static_assert(53248 + 8192 <= kRingBytes, "resolver arrays must fit the ring");
 
 __device__ __forceinline__ double accept_probability(double p, double q) {
     if (q > 0.0) {
@@ -393,11 +395,10 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, 
 }
 
 template <typename T, bool kTree>
-__global__ void __launch_bounds__(kBlockThreads) verify_kernel(const VerifyParams p) {
-    constexpr int kPer = Elt<T>::kPerVec;
+__global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>(((size_t)smem_raw + 127) & ~(size_t)127);
-    VerifyShared* sh = reinterpret_cast<VerifyShared*>(ring + kRingBytes);
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(ring + kVerifyArena);
 
     const int tid = threadIdx.x;
     const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
@@ -425,42 +426,20 @@ __global__ void __launch_bounds__(kBlockThreads) verify_kernel(const VerifyParam
         }
         const uint32_t padded = tile_padded_bytes(p.row_bytes, t);
         const unsigned char* tile = ring + s * kTileBytes;
-        float zmax = -INFINITY, M = -3.0e38f, negM = 3.0e38f;
-        float acc[kPer];
-#pragma unroll
-        for (int e = 0; e < kPer; ++e) acc[e] = 0.f;
-#pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j) {
-            const uint32_t off = warp * kChunkBytes + (j * 32 + lane) * kVecBytes;
-            if (off < padded) {
-                float z[kPer];
-                unpack_vec<T>(lds_vec(tile + off), z);
-                float vmax = z[0];
-#pragma unroll
-                for (int e = 1; e < kPer; ++e) vmax = fmaxf(vmax, z[e]);
-                if (vmax > zmax) {
-                    zmax = vmax;
-                    const float Mn = fmaf(vmax, chi, vmax * clo);
-                    const float sc = ex2_approx(M - Mn);
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e) acc[e] *= sc;
-                    M = Mn;
-                    negM = -Mn;
-                }
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) acc[e] += ex2_approx(fmaf(z[e], chi, fmaf(z[e], clo, negM)));
-            }
-        }
-        // the warp's chunk of this tile is done: release the slot, then fold the 32 lane partials
+        LaneTile<T> lt;
+        lt.load(tile, warp, lane, padded);
+        // the warp's chunk of this tile is in registers: release the slot
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->bars.empty[s]);
         if ((uint32_t)(warp * kChunkBytes) < padded) {
-            float sl = 0.f;
-#pragma unroll
-            for (int e = 0; e < kPer; ++e) sl += acc[e];
-            const float Mw = warp_max(M);
-            sl *= ex2_approx(M - Mw);
-            const float Sw = warp_sum(sl);
+            LaneSum ls;
+            ls.reset();
+            const float lm = lt.lane_max();
+            if (lm > -INFINITY) ls.raise(lm, chi, clo);
+            lt.accumulate(ls, chi, clo);
+            // fold the 32 lane partials into the chunk's (max, sum)
+            const float Mw = warp_max(ls.M);
+            const float Sw = warp_sum(ls.total() * ex2_approx(ls.M - Mw));
             if (lane == 0) part[t * kConsumerWarps + warp] = make_float2(Mw, Sw);
         }
     }
@@ -519,7 +498,7 @@ static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes
     pl.tiles_per_seg = (pl.ntiles + nseg - 1) / nseg;
     pl.nseg = (pl.ntiles + pl.tiles_per_seg - 1) / pl.tiles_per_seg;
     if (pl.nseg < 1) pl.nseg = 1;
-    pl.smem = kRingBytes + sizeof(VerifyShared) + 256;
+    pl.smem = kVerifyArena + sizeof(VerifyShared) + 256;
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
     off = up256(off + (size_t)B * sizeof(int));
