@@ -1,5 +1,5 @@
-// Shared device helpers of libtslt: layout constants, mbarrier / bulk-copy (TMA) wrappers
-// with bounded waits, block-level scans and reductions, and the order-preserving key map.
+// Shared device helpers of libtslt: layout constants, block-level scans and reductions, the
+// order-preserving key map and the element accessors.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -10,27 +10,23 @@
 namespace tslt {
 
 // ---- CTA shape ---------------------------------------------------------------------------
-// 8 consumer warps do the arithmetic; one extra producer warp drives the bulk-copy ring.
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kBlockThreads = kConsumerThreads + 32;
-// A tile is what one bulk copy brings in; each consumer warp owns one contiguous chunk of it.
-constexpr int kTileBytes = 16384;
-constexpr int kChunkBytes = kTileBytes / kConsumerWarps;  // 2048 B: the unit of per-chunk partial sums
+// 8 warps per CTA.  A chunk is the 2 KB a warp reads in one step (four 16-byte vectors per lane,
+// vector j of lane l at byte offset (j * 32 + l) * 16, so that every load instruction of the warp
+// covers 512 contiguous bytes); it is also the unit of the verifier's per-chunk partial sums.
+constexpr int kWarps = 8;
+constexpr int kBlockThreads = kWarps * 32;
+constexpr int kConsumerWarps = kWarps;
+constexpr int kConsumerThreads = kBlockThreads;
+constexpr int kChunkBytes = 2048;
 constexpr int kVecBytes = 16;
 constexpr int kVecsPerLane = kChunkBytes / (32 * kVecBytes);  // 4
-constexpr int kStages = 3;
-constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kVecsPerChunk = kChunkBytes / kVecBytes;        // 128
 
-// Named barrier for the consumer warps (barrier 0 is left to __syncthreads before the roles split).
+// Named barrier used by the block-level helpers (all 256 threads take part).
 constexpr int kConsumerBarrier = 1;
 
 // Workspace header: word 0 is the device status (0 = fine).
 constexpr int kWsHeaderBytes = 256;
-constexpr int kStatusWaitTimeout = 1;
-
-// Spin limits for device-side waits (each probe suspends for a while in hardware first).
-constexpr uint32_t kSpinLimit = 1u << 22;
 
 __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync %0, %1;" ::"n"(kConsumerBarrier), "n"(kConsumerThreads) : "memory");
@@ -38,58 +34,6 @@ __device__ __forceinline__ void consumer_sync() {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-// ---- mbarrier ----------------------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_fence_init() {
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: returns false when the limit ran out or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    return false;
-}
-
-// ---- bulk asynchronous copy (TMA, untiled): global -> this CTA's shared memory ------------
-// dst, src 16-byte aligned, bytes a non-zero multiple of 16; completion is signalled on `bar`.
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar,
-                                              uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
 }
 
 // ---- small math --------------------------------------------------------------------------
@@ -136,7 +80,7 @@ __device__ __forceinline__ float clamp_uniform(float u) {
     return u;
 }
 
-// ---- block-level helpers for the 256 consumer threads ------------------------------------
+// ---- block-level helpers for the 256 threads of a CTA ------------------------------------
 // All take `tid` in [0, 256) and a scratch array of >= 8 elements in shared memory, and end
 // with a consumer_sync() so the scratch can be reused right away.
 __device__ __forceinline__ double block_sum(double v, int tid, double* scratch) {
@@ -228,9 +172,8 @@ template <> struct Elt<bf16_t> {
     }
 };
 
-__device__ __forceinline__ uint4 lds_vec(const unsigned char* p) {
-    return *reinterpret_cast<const uint4*>(p);
-}
+// 16-byte streaming load of logits: read once, so marked evict-first.
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) { return __ldcs(p); }
 
 // Unpack one 16-byte vector into fp32 values.
 template <typename T> __device__ __forceinline__ void unpack_vec(const uint4& v, float* z);
@@ -245,11 +188,13 @@ template <> __device__ __forceinline__ void unpack_vec<bf16_t>(const uint4& v, f
     z[6] = __uint_as_float(v.w << 16); z[7] = __uint_as_float(v.w & 0xffff0000u);
 }
 
-// The scale that turns a stored logit into the base-2 exponent z * log2(e) / T, split in
-// two floats so that the product is accurate to ~1e-15 relative: hi <= c, lo > 0.
+// The scale c = log2(e) / T that turns a stored logit into a base-2 exponent.  The streaming
+// pass uses its fp32 rounding `f` in one fused multiply-add per logit, y = z * f - M, where M is
+// the fp32 exponent of a running maximum; `d` is the value all fp64 code uses.  |f/d - 1| <=
+// 2^-25 moves a row's log-normaliser by less than 1e-7 relative.
 struct ScaleC {
-    float hi, lo;
-    double d;  // hi + lo as a double: the value all fp64 code uses
+    float f;
+    double d;
 };
 
 }  // namespace tslt

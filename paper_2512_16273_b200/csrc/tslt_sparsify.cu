@@ -1,22 +1,42 @@
 // tslt_sparsify: draft-side sparsify-then-sample (Section 3, Solution 1; the sampling steps
 // of Algorithms 2 and 4) as one kernel.
 //
-// One CTA streams one segment of one logits row through the bulk-copy ring exactly once.
-// While streaming, each consumer thread keeps an online (max, sum) for the softmax
-// normaliser and pushes every logit above a running threshold tau into a shared candidate
-// buffer.  tau is the exact k-th largest logit seen so far (radix select with ties broken
-// toward the lower index), so the buffer always contains the row's top-k.  The CTA that
-// holds the whole row (the only one, or the last of the row's segments to finish) then
-// trims to the exact top-k, applies the top-rho cut, renormalises in fp64, draws the samples
-// by inverse CDF and writes the (index, logit) pairs in ascending index.
+// One CTA reads one segment of one logits row from HBM exactly once, with 16-byte loads that go
+// straight to registers (each warp instruction covers 512 contiguous bytes).  Warps run freely:
+// there is no barrier in the steady state.  Each lane keeps an online (max, sum) for the softmax
+// normaliser and copies every 16-byte vector that holds a logit at or above a running threshold
+// into a shared staging buffer (the test is on the vector's packed maximum, so a lane tile
+// without a candidate costs a handful of instructions and nothing is searched inside a vector
+// while streaming).  The threshold comes from a 4096-bin histogram of the order-preserving keys
+// (top 12 bits) of the staged vectors' maxima: the highest bin above which at least k distinct
+// logits have been seen is a lower bound on the row's k-th largest logit, so no member of the
+// top-k is ever skipped, whatever the order in which the warps run.  The warps take turns
+// rescanning the histogram, which tightens the threshold as the row streams by.  Staged vectors
+// are later expanded into (key, index) candidates, again filtered against the threshold.  The CTA that holds the whole row (the only
+// one, or the last of the row's segments to finish) then finds the bin that holds the k-th
+// largest logit, keeps everything above it, breaks the tie inside it exactly (logit descending,
+// index ascending), applies the top-rho cut, renormalises in fp64, draws the samples by inverse
+// CDF and writes the (index, logit) pairs in ascending index.
+//
+// Rare paths: a staging buffer that fills up is expanded early by all warps together (and the
+// candidate list compacted to the current threshold); a buffer that overflows before they can meet (adversarial
+// rows: sorted ascending, all equal) is abandoned and the segment's exact top-k is selected
+// again from global memory with a radix select.
 #include <math.h>
 
 #include "tslt_common.cuh"
 #include "tslt_rowmath.cuh"
 #include "tslt_select.cuh"
-#include "tslt_stream.cuh"
 
 namespace tslt {
+
+constexpr int kHistBins = 4096;   // fine bins: key >> 20 (sign, exponent and three mantissa bits)
+constexpr int kHistShift = 20;
+constexpr int kCoarseBins = 128;  // coarse bin = fine bin >> 5: lets a scan find the right 32 fine bins in one step
+constexpr int kLowestFiniteBin = 0x00800000u >> kHistShift;  // bin of -FLT_MAX: every finite logit passes
+constexpr int kBoundaryCap = 960;   // entries of the k-th logit's bin that the direct tie-break handles
+constexpr int kArenaBytes = 24576;  // histograms (16.5 KB) + boundary list (7.5 KB); fp64 work arrays afterwards
+constexpr int kRankSortMax = 256;   // up to this many entries are ordered by counting, more by a bitonic sort
 
 struct SegStat {
     double S;  // sum of 2^(y - M) over the segment
@@ -27,7 +47,6 @@ struct SegStat {
 struct SparsifyParams {
     const unsigned char* logits;
     long long row_stride_bytes;
-    long long row_bytes;
     int V, rows, k;
     float top_p;
     ScaleC c;
@@ -39,33 +58,47 @@ struct SparsifyParams {
     int* token;
     float* lse;
     float* mass;
-    int nseg, tiles_per_seg, ntiles;
-    int cap, high;
+    int nseg, chunks_per_seg, nchunks;
+    int cap, high;      // candidate (key, index) list: capacity and compaction mark
+    int vcap, vhigh;    // staged vectors: capacity and early-expansion mark
     int idx_hi_byte;
     int* status;
     int* tickets;
     SegStat* seg_stats;
-    uint2* seg_entries;  // [rows, nseg, k] (key, idx)
+    uint2* seg_entries;  // [rows, nseg, seg_cap] (key, idx)
+    int seg_cap;
 };
 
 struct SparsifyShared {
-    RingBars bars;
-    SelectScratch sel;
-    double scratch[16];
-    float tau;
-    int cand_count;
-    int overflow;
+    // ---- read by push_vector through its shared-memory address -------------------------------------
+    int vec_count;   // staged vectors
+    int overflow;    // a buffer was found full: its contents are no longer complete
+    int trim_request;
+    int vcap, vhigh;
+    uint32_t vdata_addr, vidx_addr, hist_addr, coarse_addr;  // shared-space addresses of the arrays
+    // --------------------------------------------------------------------------------------------
+    int cand_count;  // expanded (key, index) candidates
+    int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
     int ticket;
+    int sel_bin, sel_above;  // bin of the k-th largest logit and the number of logits in higher bins
+    int n_win, n_bnd;
+    int warp_tot[kWarps];
+    double scratch[16];
+    SelectScratch sel;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// shared-memory carve-up (dynamic): ring | cand_key | cand_idx | tmp_key | tmp_idx | SparsifyShared
-__host__ __device__ inline size_t sparsify_smem_bytes(int cap, int k) {
-    return kRingBytes + (size_t)cap * 8 + (size_t)k * 8 + align_up(sizeof(SparsifyShared), 16) + 256;
+// shared-memory carve-up (dynamic):
+//   arena | vec_data[vcap] | vec_idx[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k] | SparsifyShared
+__host__ __device__ inline size_t sparsify_shared_off(int cap, int vcap, int k) {
+    return align_up((size_t)kArenaBytes + (size_t)vcap * 20 + (size_t)cap * 8 + (size_t)k * 8, 16);
+}
+__host__ __device__ inline size_t sparsify_smem_bytes(int cap, int vcap, int k) {
+    return sparsify_shared_off(cap, vcap, k) + align_up(sizeof(SparsifyShared), 16);
 }
 
-// Sources for select_topk: the candidate buffer, one ring tile, or both.
+// Sources for select_topk: the candidate buffer, or a run of logits in global memory.
 struct BufferSrc {
     const uint32_t* k_;
     const int* i_;
@@ -73,190 +106,442 @@ struct BufferSrc {
     __device__ __forceinline__ uint32_t key(int i) const { return k_[i]; }
     __device__ __forceinline__ int idx(int i) const { return i_[i]; }
 };
-template <typename T> struct TileSrc {
-    const unsigned char* tile;
+template <typename T> struct GlobalSrc {
+    const unsigned char* row;
     int elem0;
-    __device__ __forceinline__ bool valid(int i) const { return tile_elem<T>(tile, i) > -INFINITY; }
-    __device__ __forceinline__ uint32_t key(int i) const { return float_to_key(tile_elem<T>(tile, i)); }
+    __device__ __forceinline__ bool valid(int i) const { return Elt<T>::load(row, elem0 + i) > -INFINITY; }
+    __device__ __forceinline__ uint32_t key(int i) const { return float_to_key(Elt<T>::load(row, elem0 + i)); }
     __device__ __forceinline__ int idx(int i) const { return elem0 + i; }
 };
-// entries of the buffer that precede the tile, followed by every logit of the tile above tau
-template <typename T> struct UnionSrc {
-    const uint32_t* k_;
-    const int* i_;
-    int nb;
-    const unsigned char* tile;
-    int elem0;
-    float tau;
-    __device__ __forceinline__ bool valid(int i) const {
-        return i < nb ? i_[i] < elem0 : tile_elem<T>(tile, i - nb) > tau;
-    }
-    __device__ __forceinline__ uint32_t key(int i) const {
-        return i < nb ? k_[i] : float_to_key(tile_elem<T>(tile, i - nb));
-    }
-    __device__ __forceinline__ int idx(int i) const { return i < nb ? i_[i] : elem0 + (i - nb); }
-};
 
-__device__ __forceinline__ int barrier_or(bool pred) {
-    int any;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
-        : "=r"(any)
-        : "r"((int)pred), "n"(kConsumerBarrier), "n"(kConsumerThreads)
-        : "memory");
-    return any;
+__device__ __forceinline__ float bin_lower_edge(int bin) { return key_to_float((uint32_t)bin << kHistShift); }
+
+// ---- shared memory by address: one out-of-line copy of the rare paths, still shared-space code ----
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
+    asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t atoms_add(uint32_t addr, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void reds_add(uint32_t addr, uint32_t v) {
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// Trim the candidate buffer to its exact top-k and raise tau to the k-th logit once k exist.
-template <bool kKeyHiOnly>
-__device__ __forceinline__ void rebuild(Candidates cb, int k, int idx_hi_byte, SparsifyShared* sh, int tid) {
-    const int n = min(*cb.count, 1 << 30);
+// Count one logit in both histogram levels (fine first: a scan that sees the coarse count also
+// finds the fine one).
+__device__ __forceinline__ void hist_count(uint32_t hist_addr, uint32_t coarse_addr, int bin, uint32_t delta) {
+    reds_add(hist_addr + 4u * (uint32_t)bin, delta);
+    reds_add(coarse_addr + 4u * (uint32_t)(bin >> 5), delta);
+}
+
+__device__ __forceinline__ void sts_v4(uint32_t addr, const uint4& v) {
+    asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax, and count
+// that logit.  Out of line on purpose: it is rare, and inlined copies of it in the streaming
+// loop would not fit the instruction cache.
+__device__ __noinline__ void push_vector(uint32_t sh_addr, uint4 data, int vec_index, float vmax) {
+    const uint32_t pos = atoms_add(sh_addr + offsetof(SparsifyShared, vec_count), 1u);
+    if (pos < lds_u32(sh_addr + offsetof(SparsifyShared, vcap))) {
+        sts_v4(lds_u32(sh_addr + offsetof(SparsifyShared, vdata_addr)) + 16u * pos, data);
+        sts_u32(lds_u32(sh_addr + offsetof(SparsifyShared, vidx_addr)) + 4u * pos, (uint32_t)vec_index);
+    } else {
+        sts_u32(sh_addr + offsetof(SparsifyShared, overflow), 1u);
+    }
+    if (pos + 1u == lds_u32(sh_addr + offsetof(SparsifyShared, vhigh)))
+        sts_u32(sh_addr + offsetof(SparsifyShared, trim_request), 1u);
+    hist_count(lds_u32(sh_addr + offsetof(SparsifyShared, hist_addr)),
+               lds_u32(sh_addr + offsetof(SparsifyShared, coarse_addr)), (int)(float_to_key(vmax) >> kHistShift), 1u);
+}
+
+// One warp: the highest fine bin b with (number of counted logits in bins >= b) >= k, or -1 if
+// fewer than k are counted; *above gets the count in the bins above b (the total if none).
+// Two steps whatever the values: the 128 coarse counts, then the 32 fine bins of the coarse bin
+// in which the running count crosses k.
+__device__ __noinline__ int scan_boundary(uint32_t hist_addr, uint32_t coarse_addr, int k, uint32_t* above_out) {
+    const int lane = threadIdx.x & 31;
+    // lane l owns coarse bins 127-4l .. 124-4l (descending)
+    uint32_t c[4], tot = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        c[i] = lds_u32(coarse_addr + 4u * (uint32_t)(127 - 4 * lane - i));
+        tot += c[i];
+    }
+    uint32_t incl = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, incl >= (uint32_t)k);
+    if (!hit) {
+        *above_out = __shfl_sync(0xffffffffu, incl, 31);
+        return -1;
+    }
+    const int l = __ffs(hit) - 1;
+    uint32_t run = incl - tot;  // counted above this lane's bins
+    int cbin = 0;
+    bool done = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (!done) {
+            if (run + c[i] >= (uint32_t)k) {
+                cbin = 127 - 4 * lane - i;
+                done = true;
+            } else {
+                run += c[i];
+            }
+        }
+    }
+    cbin = __shfl_sync(0xffffffffu, cbin, l);
+    const uint32_t above_c = __shfl_sync(0xffffffffu, run, l);
+    // fine bins of that coarse bin, lane 0 the highest
+    const int fb = cbin * 32 + 31 - lane;
+    const uint32_t f = lds_u32(hist_addr + 4u * (uint32_t)fb);
+    uint32_t fincl = f;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, fincl, o);
+        if (lane >= o) fincl += t;
+    }
+    const unsigned fhit = __ballot_sync(0xffffffffu, above_c + fincl >= (uint32_t)k);
+    if (!fhit) {  // the fine counts lag the coarse one (another warp is mid-push): nothing to report yet
+        *above_out = 0;
+        return -2;
+    }
+    const int fl = __ffs(fhit) - 1;
+    *above_out = above_c + __shfl_sync(0xffffffffu, fincl - f, fl);
+    return cbin * 32 + 31 - fl;
+}
+
+// One warp: raise thr_bin to the bin scan_boundary finds.  Counts that other warps are still adding
+// can only be missed, never invented, so the result is always a valid lower bound.
+__device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
+    uint32_t above;
+    const int found = scan_boundary(sh->hist_addr, sh->coarse_addr, k, &above);
+    if ((threadIdx.x & 31) == 0 && found > *(volatile int*)&sh->thr_bin) atomicMax(&sh->thr_bin, found);
+}
+
+// The running threshold in the form the lane-tile test wants.  A logit is a candidate iff its
+// key bin is >= thr_bin, i.e. iff it is >= the bin's lower edge.
+//   fp32 rows: the edge itself, compared as floats.
+//   bf16 rows: P = the largest bf16 value below the edge, in both halves of a word; a packed
+//              word w holds a candidate iff max.bf16x2(w, P) != P (NaN halves never differ).
+template <typename T> struct Threshold;
+template <> struct Threshold<float> {
+    float edge;
+    __device__ __forceinline__ explicit Threshold(int bin) : edge(bin_lower_edge(bin)) {}
+};
+template <> struct Threshold<bf16_t> {
+    uint32_t P2;
+    __device__ __forceinline__ explicit Threshold(int bin) {
+        uint32_t k16 = ((uint32_t)bin << (kHistShift - 16)) - 1u;  // key of the value just below the edge
+        if (k16 == 0x7fffu) k16 = 0x7ffeu;                         // -0 shares +0's key: step past it
+        const uint32_t b16 = (k16 & 0x8000u) ? (k16 & 0x7fffu) : (~k16 & 0xffffu);
+        P2 = b16 | (b16 << 16);
+    }
+};
+
+// Stage the vectors of a lane tile that hold a candidate (reduce_max() already called): a test on
+// the lane's packed maximum, then one per vector.
+__device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, int lane_vec0,
+                                            uint32_t sh_addr) {
+    const uint32_t P2 = th.P2;
+    if (bf16x2_max(lt.lane_max2(), P2) != P2) {
+#pragma unroll
+        for (int j = 0; j < kVecsPerLane; ++j)
+            if (bf16x2_max(lt.vm[j], P2) != P2)
+                push_vector(sh_addr, make_uint4(lt.w[4 * j], lt.w[4 * j + 1], lt.w[4 * j + 2], lt.w[4 * j + 3]),
+                            lane_vec0 + j * 32, lt.vec_max(j));
+    }
+}
+__device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, int lane_vec0,
+                                            uint32_t sh_addr) {
+    const float thr = th.edge;
+    if (fmaxf(fmaxf(lt.vm[0], lt.vm[1]), fmaxf(lt.vm[2], lt.vm[3])) >= thr) {
+#pragma unroll
+        for (int j = 0; j < kVecsPerLane; ++j)
+            if (lt.vm[j] >= thr)
+                push_vector(sh_addr,
+                            make_uint4(__float_as_uint(lt.z[4 * j]), __float_as_uint(lt.z[4 * j + 1]),
+                                       __float_as_uint(lt.z[4 * j + 2]), __float_as_uint(lt.z[4 * j + 3])),
+                            lane_vec0 + j * 32, lt.vm[j]);
+    }
+}
+
+// All threads: turn the staged vectors into (key, index) candidates, keeping the logits whose bin
+// is >= bin, and empty the staging buffer.  A full candidate list raises the overflow flag.
+template <typename T>
+__device__ __noinline__ void expand_staged(const uint4* vdata, const int* vidx, Candidates cb, int cap, int bin, int V,
+                                           SparsifyShared* sh, int tid) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    const int nv = min(sh->vec_count, sh->vcap);
+    const uint32_t min_key = (uint32_t)bin << kHistShift;
+    for (int i = tid; i < nv; i += kBlockThreads) {
+        const uint4 d = vdata[i];
+        const int e0 = vidx[i] * kPer;
+        float z[kPer];
+        unpack_vec<T>(d, z);
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            if (z[e] >= -3.4028234e38f && e0 + e < V) {
+                const uint32_t kk = float_to_key(z[e]);
+                if (kk >= min_key) {
+                    const int pos = atomicAdd(cb.count, 1);
+                    if (pos < cap) {
+                        cb.key[pos] = kk;
+                        cb.idx[pos] = e0 + e;
+                    } else {
+                        sh->overflow = 1;
+                    }
+                }
+            }
+        }
+    }
     consumer_sync();
-    if (n <= k) return;  // nothing to trim; tau unchanged (uniform: n is the same for every thread)
-    uint32_t kth;
-    BufferSrc src{cb.key, cb.idx};
-    const bool full = select_topk<kKeyHiOnly>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
-    if (full && tid == 0) sh->tau = key_to_float(kth);
+    if (tid == 0) {
+        sh->vec_count = 0;
+        if (*cb.count > cap) *cb.count = cap;
+    }
+    consumer_sync();
+}
+
+// All threads: drop the buffer entries whose bin is below `bin` (entries are held in registers
+// between the read and the write phase, so the compaction is in place).
+__device__ __noinline__ void compact_buffer(Candidates cb, int bin, SparsifyShared* sh, int tid) {
+    constexpr int E = 16;  // cap <= 4096 = 16 * 256
+    const int n = min(*cb.count, E * kBlockThreads);
+    uint32_t ek[E];
+    int ei[E];
+    unsigned keep = 0;
+    int cnt = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int i = tid * E + e;
+        ek[e] = 0u;
+        ei[e] = 0;
+        if (i < n) {
+            ek[e] = cb.key[i];
+            ei[e] = cb.idx[i];
+            if ((int)(ek[e] >> kHistShift) >= bin) {
+                keep |= 1u << e;
+                ++cnt;
+            }
+        }
+    }
+    const int lane = tid & 31, warp = tid >> 5;
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) sh->warp_tot[warp] = incl;
+    consumer_sync();  // every entry has been read, warp totals are in place
+    int off = incl - cnt, total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        const int t = sh->warp_tot[w];
+        if (w < warp) off += t;
+        total += t;
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (keep & (1u << e)) {
+            cb.key[off] = ek[e];
+            cb.idx[off] = ei[e];
+            ++off;
+        }
+    consumer_sync();
+    if (tid == 0) *cb.count = total;
     consumer_sync();
 }
 
 template <typename T>
 __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* ring, double Mrow, double Srow, int tid);
+                                          unsigned char* arena, double Mrow, double Srow, bool hist_valid, int tid);
+
+// Radix-select fallbacks, out of line (one copy each).
+template <typename T>
+__device__ __noinline__ void reselect_from_global(const unsigned char* rowp, int e0, int n, int k, int idx_hi_byte,
+                                                  Candidates cb, SparsifyShared* sh, int tid) {
+    uint32_t kth;
+    GlobalSrc<T> src{rowp, e0};
+    select_topk<(Elt<T>::kBytes == 2)>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
+}
+template <bool kKeyHiOnly>
+__device__ __noinline__ void reselect_from_buffer(int n, int k, int idx_hi_byte, Candidates cb, SparsifyShared* sh,
+                                                  int tid) {
+    uint32_t kth;
+    BufferSrc src{cb.key, cb.idx};
+    select_topk<kKeyHiOnly>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
+}
 
 template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, 3) sparsify_kernel(const SparsifyParams p) {
+__global__ void __launch_bounds__(kBlockThreads, 4) sparsify_kernel(const SparsifyParams p) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     constexpr int kPer = Elt<T>::kPerVec;
+    constexpr int kChunkElems = kChunkBytes / Elt<T>::kBytes;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* ring = reinterpret_cast<unsigned char*>(align_up((size_t)smem_raw, 128));
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(ring + kRingBytes);
+    // every pointer below is derived from smem_raw by plain offsets, so that the compiler keeps
+    // them in the shared address space (shared-memory atomics and loads, not generic ones)
+    unsigned char* arena = smem_raw;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
+    uint32_t* coarse = hist + kHistBins;
+    uint4* vec_data = reinterpret_cast<uint4*>(arena + kArenaBytes);
+    int* vec_idx = reinterpret_cast<int*>(vec_data + p.vcap);
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(vec_idx + p.vcap);
     int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
     uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
-    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(align_up((size_t)(tmp_idx + p.k), 16));
+    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, p.vcap, p.k));
+    const uint32_t sh_addr = smem_u32(sh);
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const int tile_begin = seg * p.tiles_per_seg;
-    const int tile_end = min(p.ntiles, tile_begin + p.tiles_per_seg);
+    const int chunk_begin = seg * p.chunks_per_seg;
+    const int chunk_end = min(p.nchunks, chunk_begin + p.chunks_per_seg);
+    const RowExtent ext = row_extent<T>(p.V);
+    const int k = p.k;
+    const float c = p.c.f;
 
-    ring_init(&sh->bars, tid);
+    for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
     if (tid == 0) {
-        sh->tau = -INFINITY;
+        sh->thr_bin = kLowestFiniteBin;
         sh->cand_count = 0;
+        sh->vec_count = 0;
         sh->overflow = 0;
+        sh->trim_request = 0;
+        sh->vcap = p.vcap;
+        sh->vhigh = p.vhigh;
+        sh->vdata_addr = smem_u32(vec_data);
+        sh->vidx_addr = smem_u32(vec_idx);
+        sh->hist_addr = smem_u32(hist);
+        sh->coarse_addr = smem_u32(coarse);
     }
     __syncthreads();
-
-    if (tid >= kConsumerThreads) {
-        producer_loop<T>(rowp, p.row_bytes, tile_begin, tile_end, ring, &sh->bars, p.status);
-        return;
-    }
-
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
-    const int lane = tid & 31, warp = tid >> 5;
-    const int cap = p.cap, high = p.high, k = p.k;
-    const float chi = p.c.hi, clo = p.c.lo;
 
-    // ---- streaming pass ----------------------------------------------------------------
-    LaneSum ls;
-    ls.reset();
-    bool live = true;
-
-    for (int t = tile_begin; t < tile_end; ++t) {
-        const int it = t - tile_begin, s = it % kStages;
-        const bool arrived = mbar_wait(&sh->bars.full[s], (uint32_t)((it / kStages) & 1), &sh->bars.abort);
-        const uint32_t padded = tile_padded_bytes(p.row_bytes, t);
-        const unsigned char* tile = ring + s * kTileBytes;
-        const float tau = sh->tau;
-        const int tile_elem0 = t * (kTileBytes / Elt<T>::kBytes);
-        // the first tile of a segment is not filtered: its exact top-k is selected in place below
-        bool want_action = !arrived || it == 0;
-        if (arrived) {
+    // ---- first threshold, from the segment's first chunks (one per warp) ---------------------------
+    // For k <= 256 the histogram takes only the maxima of the 1024 16-byte vectors of these chunks:
+    // the k-th largest of them is a lower bound on the k-th largest logit, and close to it while k
+    // is small against 1024.  Larger k counts every logit of the chunks.  The counts are wiped
+    // afterwards: the streaming loop below starts again at the first chunk (an L2 hit) and counts
+    // what it pushes.
+    {
+        const int ch0 = chunk_begin + warp;
+        if (ch0 < chunk_end) {
             LaneTile<T> lt;
-            lt.load(tile, warp, lane, padded);
-            const float lm = lt.lane_max();
-            if (lm > ls.zmax) ls.raise(lm, chi, clo);
-            lt.accumulate(ls, chi, clo);
-            if (it != 0 && lm > tau) {
+            lt.load(rowp, (long long)ch0 * kVecsPerChunk, lane, ext);
+            lt.reduce_max();
+            if (k <= 256) {
 #pragma unroll
                 for (int j = 0; j < kVecsPerLane; ++j) {
-                    if (lt.vec_max(j) > tau) {
-                        const int e0 = tile_elem0 + (warp * kChunkBytes + (j * 32 + lane) * kVecBytes) / Elt<T>::kBytes;
-#pragma unroll
-                        for (int e = 0; e < kPer; ++e) {
-                            const float z = lt.elem(j, e);
-                            if (z > tau) {
-                                const int pos = atomicAdd(&sh->cand_count, 1);
-                                if (pos < cap) {
-                                    cand_key[pos] = float_to_key(z);
-                                    cand_idx[pos] = e0 + e;
-                                } else {
-                                    sh->overflow = 1;
-                                }
-                                if (pos + 1 > high) want_action = true;
-                            }
-                        }
-                    }
+                    const float z = lt.vec_max(j);
+                    if (z >= -3.4028234e38f) hist_count(sh->hist_addr, sh->coarse_addr, (int)(float_to_key(z) >> kHistShift), 1u);
                 }
-            }
-        }
-        // one barrier per tile: it also tells everyone whether the buffer needs attention
-        if (barrier_or(want_action)) {
-            // a wait that ran out is decided collectively, so that nobody is left at a barrier
-            if (barrier_or(!arrived)) {
-                if (!arrived) raise_abort(&sh->bars, p.status);
-                live = false;
-                break;
-            }
-            const int tile_elems = (int)(padded / Elt<T>::kBytes);
-            uint32_t kth;
-            bool full;
-            if (it == 0) {
-                TileSrc<T> src{tile, tile_elem0};
-                full = select_topk<kHiOnly>(src, tile_elems, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
             } else {
-                const int ovf = sh->overflow;
-                const int nb = min(sh->cand_count, cap);
-                consumer_sync();
-                if (!ovf) {
-                    BufferSrc src{cand_key, cand_idx};
-                    full = select_topk<kHiOnly>(src, nb, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
-                } else {
-                    // this tile brought more candidates than fit: redo it from shared memory, selecting
-                    // over the earlier entries of the buffer and every logit of the tile above tau
-                    if (tid == 0) sh->overflow = 0;
-                    UnionSrc<T> src{cand_key, cand_idx, nb, tile, tile_elem0, tau};
-                    full = select_topk<kHiOnly>(src, nb + tile_elems, k, p.idx_hi_byte, cb, &sh->sel, tid, &kth);
+#pragma unroll 4
+                for (int e = 0; e < kVecsPerLane * kPer; ++e) {
+                    const float z = lt.elem(e / kPer, e % kPer);
+                    if (z >= -3.4028234e38f) hist_count(sh->hist_addr, sh->coarse_addr, (int)(float_to_key(z) >> kHistShift), 1u);
                 }
             }
-            if (full && tid == 0) sh->tau = key_to_float(kth);
-            consumer_sync();
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh->bars.empty[s]);
+        __syncthreads();
+        if (warp == 0) raise_threshold(sh, k);
+        __syncthreads();
+        for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+        __syncthreads();
     }
-    if (!live) return;  // status word already set; outputs left untouched
-    consumer_sync();
+
+    // ---- streaming: no barriers; warp w rescans the histogram on its turn --------------------------
+    LaneSum ls;
+    ls.reset();
+    int ch = chunk_begin + warp, step = 0;
+    for (;;) {
+        while (ch < chunk_end) {
+            __syncwarp();
+            if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
+            LaneTile<T> lt;
+            lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+            const float lm = lt.reduce_max();
+            if (lm > ls.zmax) ls.raise(lm, c);
+            lt.accumulate(ls, c);
+            const Threshold<T> th(*(volatile int*)&sh->thr_bin);
+            filter_push(lt, th, ch * kVecsPerChunk + lane, sh_addr);
+            if ((step & (kWarps - 1)) == warp) {
+                __syncwarp();
+                raise_threshold(sh, k);
+            }
+            ch += kWarps;
+            ++step;
+        }
+        const int all_done = __syncthreads_and(ch >= chunk_end);
+        const int want_trim = sh->trim_request;
+        __syncthreads();
+        if (all_done) break;
+        if (want_trim) {
+            if (!sh->overflow) {
+                if (warp == 0) raise_threshold(sh, k);
+                consumer_sync();
+                const int bin = sh->thr_bin;
+                expand_staged<T>(vec_data, vec_idx, cb, p.cap, bin, p.V, sh, tid);
+                if (sh->cand_count > p.high) compact_buffer(cb, bin, sh, tid);
+            }
+            if (tid == 0) sh->trim_request = 0;
+            __syncthreads();
+        }
+    }
+
+    // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
+    if (!sh->overflow) {
+        if (warp == 0) raise_threshold(sh, k);
+        consumer_sync();
+        expand_staged<T>(vec_data, vec_idx, cb, p.cap, sh->thr_bin, p.V, sh, tid);
+    }
+    bool hist_valid = false;  // the streaming histogram counted vector maxima only
+    if (sh->overflow) {
+        const int e0 = chunk_begin * kChunkElems;
+        const int n = min(p.V, chunk_end * kChunkElems) - e0;
+        reselect_from_global<T>(rowp, e0, n, k, p.idx_hi_byte, cb, sh, tid);
+        if (tid == 0) sh->overflow = 0;
+        consumer_sync();
+    }
 
     // ---- row statistics ------------------------------------------------------------------
     float Mrow_f = warp_max(ls.M);
     if (lane == 0) sh->scratch[warp] = (double)Mrow_f;
     consumer_sync();
     double Mrow = sh->scratch[0];
-    for (int w = 1; w < kConsumerWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
+    for (int w = 1; w < kWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
     consumer_sync();
     double Srow = block_sum(ls.total_f64() * exp2((double)ls.M - Mrow), tid, sh->scratch);
 
     // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
     if (p.nseg > 1) {
-        rebuild<kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);  // <= k entries per segment
-        const int n = sh->cand_count;
-        uint2* my_entries = p.seg_entries + ((size_t)row * p.nseg + seg) * (size_t)k;
-        for (int i = tid; i < n; i += kConsumerThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
+        // hand over the candidates (all at or above this segment's final threshold)
+        int n = sh->cand_count;
+        if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
+            compact_buffer(cb, sh->thr_bin, sh, tid);
+            n = sh->cand_count;
+        }
+        if (n > p.seg_cap) {  // heavy ties at the boundary: hand over the exact k
+            reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
+            n = sh->cand_count;
+        }
+        uint2* my_entries = p.seg_entries + ((size_t)row * p.nseg + seg) * (size_t)p.seg_cap;
+        for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
         if (tid == 0) {
             SegStat st;
             st.S = Srow;
@@ -285,9 +570,9 @@ __global__ void __launch_bounds__(kBlockThreads, 3) sparsify_kernel(const Sparsi
             const double Mg = (double)__ldcg(&st->M);
             Sall += Sg * exp2(Mg - Mall);
             const int ng = __ldcg(&st->n);
-            const uint2* ent = p.seg_entries + ((size_t)row * p.nseg + g) * (size_t)k;
+            const uint2* ent = p.seg_entries + ((size_t)row * p.nseg + g) * (size_t)p.seg_cap;
             const int base = sh->cand_count;
-            for (int i = tid; i < ng; i += kConsumerThreads) {
+            for (int i = tid; i < ng; i += kBlockThreads) {
                 uint2 e2 = __ldcg(&ent[i]);
                 cand_key[base + i] = e2.x;
                 cand_idx[base + i] = (int)e2.y;
@@ -298,37 +583,136 @@ __global__ void __launch_bounds__(kBlockThreads, 3) sparsify_kernel(const Sparsi
         }
         Mrow = Mall;
         Srow = Sall;
+        hist_valid = false;
     }
 
-    finalize_row<T>(p, row, cb, sh, ring, Mrow, Srow, tid);
+    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, hist_valid, tid);
+}
+
+// Position of entry (key, idx) of the buffer in the order (key descending, idx ascending) /
+// (idx ascending), by counting the entries that precede it.
+__device__ __forceinline__ int rank_by_key(const uint32_t* key, const int* idx, int n, uint32_t my_key, int my_idx) {
+    int r = 0;
+    for (int j = 0; j < n; ++j) {
+        const uint32_t kj = key[j];
+        const int ij = idx[j];
+        r += (kj > my_key || (kj == my_key && ij < my_idx)) ? 1 : 0;
+    }
+    return r;
+}
+__device__ __forceinline__ int rank_by_idx(const int* idx, int n, int my_idx) {
+    int r = 0;
+    for (int j = 0; j < n; ++j) r += idx[j] < my_idx ? 1 : 0;
+    return r;
 }
 
 // Exact top-k of the row, nucleus cut, renormalisation, sampling and the ascending-index payload.
 template <typename T>
 __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* ring, double Mrow, double Srow, int tid) {
+                                          unsigned char* arena, double Mrow, double Srow, bool hist_valid, int tid) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     const int k = p.k;
+    const int lane = tid & 31, warp = tid >> 5;
     uint32_t* cand_key = cb.key;
     int* cand_idx = cb.idx;
-    rebuild<kHiOnly>(cb, k, p.idx_hi_byte, sh, tid);
-    const int n0 = min(sh->cand_count, k);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
+    uint2* bnd = reinterpret_cast<uint2*>(arena + (kHistBins + kCoarseBins) * 4);
+    const int nc = sh->cand_count;
+
+    // ---- the bin of the k-th largest logit ------------------------------------------------------
+    if (!hist_valid) {
+        for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+        consumer_sync();
+        for (int i = tid; i < nc; i += kBlockThreads)
+            hist_count(sh->hist_addr, sh->coarse_addr, (int)(cand_key[i] >> kHistShift), 1u);
+        consumer_sync();
+    }
+    if (warp == 0) {
+        uint32_t above;
+        const int b = scan_boundary(sh->hist_addr, sh->coarse_addr, k, &above);
+        if (lane == 0) {
+            sh->sel_bin = b;  // -1: fewer than k candidates exist, all of them are kept
+            sh->sel_above = (int)above;
+            sh->n_win = 0;
+            sh->n_bnd = 0;
+        }
+    }
+    consumer_sync();
+    const int sel_bin = sh->sel_bin;
+    // ---- everything above that bin is in; the bin itself goes to the boundary list ---------------
+    for (int i = tid; i < nc; i += kBlockThreads) {
+        const uint32_t kk = cand_key[i];
+        const int bin = (int)(kk >> kHistShift);
+        if (bin > sel_bin) {
+            const int pos = atomicAdd(&sh->n_win, 1);
+            if (pos < k) {
+                cb.tmp_key[pos] = kk;
+                cb.tmp_idx[pos] = cand_idx[i];
+            }
+        } else if (bin == sel_bin) {
+            const int pos = atomicAdd(&sh->n_bnd, 1);
+            if (pos < kBoundaryCap) bnd[pos] = make_uint2(kk, (uint32_t)cand_idx[i]);
+        }
+    }
+    consumer_sync();
+    const int n_above = min(sh->n_win, k), nb = sh->n_bnd;
+    int n0;
+    if (nb > kBoundaryCap) {
+        // heavy ties: radix select over the whole buffer (leaves its winners at the front of the buffer)
+        reselect_from_buffer<kHiOnly>(nc, k, p.idx_hi_byte, cb, sh, tid);
+        n0 = min(sh->cand_count, k);
+    } else {
+        const int need = min(k - n_above, nb);
+        for (int t = tid; t < nb; t += kBlockThreads) {
+            const uint2 me = bnd[t];
+            int r = t;
+            if (nb > need) {
+                r = 0;
+                for (int j = 0; j < nb; ++j) {
+                    const uint2 o = bnd[j];
+                    r += (o.x > me.x || (o.x == me.x && (int)o.y < (int)me.y)) ? 1 : 0;
+                }
+            }
+            if (r < need) {
+                cb.tmp_key[n_above + r] = me.x;
+                cb.tmp_idx[n_above + r] = (int)me.y;
+            }
+        }
+        consumer_sync();
+        n0 = n_above + need;
+        for (int i = tid; i < n0; i += kBlockThreads) {
+            cand_key[i] = cb.tmp_key[i];
+            cand_idx[i] = cb.tmp_idx[i];
+        }
+        consumer_sync();
+    }
+
     const double L2 = Mrow + log2(Srow);  // base-2 log of the softmax normaliser
     const double cd = p.c.d;
-    // the ring is idle now: reuse it for the fp64 work arrays
-    unsigned long long* comp = reinterpret_cast<unsigned long long*>(ring);           // 1024 * 8
-    double* wv = reinterpret_cast<double*>(ring + 8192);                              // 1024 * 8
-    double* cum = reinterpret_cast<double*>(ring + 16384);                            // 1024 * 8
+    // the histogram and the boundary list are no longer needed: their arena holds the fp64 work arrays
+    unsigned long long* comp = reinterpret_cast<unsigned long long*>(arena);          // 1024 * 8
+    double* wv = reinterpret_cast<double*>(arena + 8192);                             // 1024 * 8
+    double* cum = reinterpret_cast<double*>(arena + 16384);                           // 1024 * 8
     int n = n0;
     double mass = 0.0;
     if (n0 > 0 && p.top_p < 1.0f) {
         // order the candidates by (logit descending, index ascending) and cut at the nucleus
-        const int P = next_pow2(n0);
-        for (int i = tid; i < P; i += kConsumerThreads)
-            comp[i] = i < n0 ? (((unsigned long long)cand_key[i] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)cand_idx[i])) : 0ull;
-        consumer_sync();
-        bitonic_sort<true>(comp, P, tid);
-        for (int i = tid; i < n0; i += kConsumerThreads) {
+        if (n0 <= kRankSortMax) {
+            if (tid < n0) {
+                const uint32_t kk = cand_key[tid];
+                const int ii = cand_idx[tid];
+                const int r = rank_by_key(cand_key, cand_idx, n0, kk, ii);
+                comp[r] = ((unsigned long long)kk << 32) | (unsigned long long)(0xffffffffu - (uint32_t)ii);
+            }
+            consumer_sync();
+        } else {
+            const int P = next_pow2(n0);
+            for (int i = tid; i < P; i += kBlockThreads)
+                comp[i] = i < n0 ? (((unsigned long long)cand_key[i] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)cand_idx[i])) : 0ull;
+            consumer_sync();
+            bitonic_sort<true>(comp, P, tid);
+        }
+        for (int i = tid; i < n0; i += kBlockThreads) {
             const float z = key_to_float((uint32_t)(comp[i] >> 32));
             cum[i] = exp2((double)z * cd - L2);
         }
@@ -344,7 +728,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
         n = lo < n0 ? lo + 1 : n0;
         mass = cum[n - 1];
         consumer_sync();
-        for (int i = tid; i < n; i += kConsumerThreads) {
+        for (int i = tid; i < n; i += kBlockThreads) {
             cand_key[i] = (uint32_t)(comp[i] >> 32);
             cand_idx[i] = (int)(0xffffffffu - (uint32_t)(comp[i] & 0xffffffffull));
         }
@@ -352,15 +736,23 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     }
     // ascending index order
     if (n > 0) {
-        const int P = next_pow2(n);
-        for (int i = tid; i < P; i += kConsumerThreads)
-            comp[i] = i < n ? (((unsigned long long)(uint32_t)cand_idx[i] << 32) | (unsigned long long)cand_key[i]) : ~0ull;
-        consumer_sync();
-        bitonic_sort<false>(comp, P, tid);
+        if (n <= kRankSortMax) {
+            if (tid < n) {
+                const int ii = cand_idx[tid];
+                comp[rank_by_idx(cand_idx, n, ii)] = ((unsigned long long)(uint32_t)ii << 32) | (unsigned long long)cand_key[tid];
+            }
+            consumer_sync();
+        } else {
+            const int P = next_pow2(n);
+            for (int i = tid; i < P; i += kBlockThreads)
+                comp[i] = i < n ? (((unsigned long long)(uint32_t)cand_idx[i] << 32) | (unsigned long long)cand_key[i]) : ~0ull;
+            consumer_sync();
+            bitonic_sort<false>(comp, P, tid);
+        }
     }
     // renormalised truncated distribution in fp64: w_i = 2^(y_i - m_S), CDF by inclusive scan
     double my_max = -INFINITY;
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         const float z = key_to_float((uint32_t)(comp[i] & 0xffffffffull));
         const double y = (double)z * cd;
         wv[i] = y;
@@ -368,7 +760,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     }
     const double mS = block_max(my_max, tid, sh->scratch);
     double my_mass = 0.0;
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         const double y = wv[i];
         if (!(p.top_p < 1.0f)) my_mass += exp2(y - L2);
         const double w = exp2(y - mS);
@@ -382,7 +774,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     // ---- outputs ------------------------------------------------------------------------------
     int* o_idx = p.idx + (size_t)row * k;
     float* o_logit = p.logit + (size_t)row * k;
-    for (int i = tid; i < k; i += kConsumerThreads) {
+    for (int i = tid; i < k; i += kBlockThreads) {
         if (i < n) {
             o_idx[i] = (int)(comp[i] >> 32);
             o_logit[i] = key_to_float((uint32_t)(comp[i] & 0xffffffffull));
@@ -397,7 +789,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
         if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
     }
     const double W = n > 0 ? cum[n - 1] : 0.0;
-    for (int sidx = tid; sidx < p.num_samples; sidx += kConsumerThreads) {
+    for (int sidx = tid; sidx < p.num_samples; sidx += kBlockThreads) {
         int tok = -1;
         if (n > 0) {
             const float u = clamp_uniform(p.uniforms[(size_t)row * p.num_samples + sidx]);
@@ -415,7 +807,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
-    int nseg, tiles_per_seg, ntiles, cap, high;
+    int nseg, chunks_per_seg, nchunks, cap, high, vcap, vhigh, seg_cap;
     size_t smem;
     size_t ws_tickets_off, ws_stats_off, ws_entries_off, ws_bytes;
 };
@@ -435,29 +827,34 @@ static int sm_count_cached() {
 static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     SparsifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
-    pl.ntiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
-    pl.cap = 4 * k;
-    if (pl.cap < 2048) pl.cap = 2048;
+    pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
+    pl.cap = 16 * k;
+    if (pl.cap < 1024) pl.cap = 1024;
     if (pl.cap > 4096) pl.cap = 4096;
     pl.high = pl.cap - pl.cap / 4;
-    // Split a row over several CTAs when there are too few rows to fill the machine.
+    pl.vcap = k <= 128 ? 1024 : 2048;
+    pl.vhigh = pl.vcap - pl.vcap / 4;
+    pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above)
+    // Split a row over several CTAs when there are too few rows to fill the machine; a segment
+    // keeps at least two chunks per warp and the segments' winners must fit one buffer.
     const int sms = sm_count_cached();
     int nseg = 1;
-    const int max_seg_by_cap = pl.cap / k;
+    const int max_seg_by_cap = pl.cap / pl.seg_cap;
     while (nseg < 16 && nseg * 2 <= max_seg_by_cap && (long long)rows * nseg < 4LL * sms &&
-           pl.ntiles / (nseg * 2) >= 2)
+           pl.nchunks / (nseg * 2) >= 2 * kWarps)
         nseg *= 2;
-    pl.tiles_per_seg = (pl.ntiles + nseg - 1) / nseg;
-    pl.nseg = (pl.ntiles + pl.tiles_per_seg - 1) / pl.tiles_per_seg;
+    pl.chunks_per_seg = (pl.nchunks + nseg - 1) / nseg;
+    pl.chunks_per_seg = (pl.chunks_per_seg + kWarps - 1) / kWarps * kWarps;
+    pl.nseg = (pl.nchunks + pl.chunks_per_seg - 1) / pl.chunks_per_seg;
     if (pl.nseg < 1) pl.nseg = 1;
-    pl.smem = sparsify_smem_bytes(pl.cap, k);
+    pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
     off = align_up(off + (size_t)rows * sizeof(int), 256);
     pl.ws_stats_off = off;
     off = align_up(off + (size_t)rows * pl.nseg * sizeof(SegStat), 256);
     pl.ws_entries_off = off;
-    off = align_up(off + (pl.nseg > 1 ? (size_t)rows * pl.nseg * k * sizeof(uint2) : 0), 256);
+    off = align_up(off + (pl.nseg > 1 ? (size_t)rows * pl.nseg * pl.seg_cap * sizeof(uint2) : 0), 256);
     pl.ws_bytes = off;
     return pl;
 }
@@ -465,13 +862,8 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
 ScaleC make_scale(float temperature) {
     const double c = 1.4426950408889634 / (double)temperature;
     ScaleC s;
-    float hi = (float)c;
-    if ((double)hi > c) hi = nextafterf(hi, 0.0f);
-    float lo = (float)(c - (double)hi);
-    if (!(lo > 0.0f)) lo = 1e-30f;
-    s.hi = hi;
-    s.lo = lo;
-    s.d = (double)hi + (double)lo;
+    s.f = (float)c;
+    s.d = c;
     return s;
 }
 
@@ -513,15 +905,14 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     SparsifyParams p;
     p.logits = (const unsigned char*)logits;
     p.row_stride_bytes = row_stride_elems * eb;
-    p.row_bytes = (long long)V * eb;
     p.V = V; p.rows = rows; p.k = k;
     p.top_p = top_p;
     p.c = make_scale(temperature);
     p.num_samples = num_samples;
     p.uniforms = uniforms;
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
-    p.nseg = pl.nseg; p.tiles_per_seg = pl.tiles_per_seg; p.ntiles = pl.ntiles;
-    p.cap = pl.cap; p.high = pl.high;
+    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
+    p.cap = pl.cap; p.high = pl.high; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
     p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
@@ -533,7 +924,8 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     // status word and tickets start at zero
     if (cudaMemsetAsync(ws, 0, pl.ws_stats_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
     auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sparsify_smem_bytes(4096, 2048, TSLT_MAX_K)) != cudaSuccess)
         return TSLT_ERR_CUDA;
     kern<<<rows * pl.nseg, kBlockThreads, pl.smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;

@@ -1,9 +1,10 @@
 // tslt_verify / tslt_tree_verify: verifier-side speculative sampling against a sparse draft
 // (Algorithm 3; Algorithm 5 along the walk of Algorithm 8) as one kernel each.
 //
-// Every target row is streamed from HBM exactly once through the bulk-copy ring.  The
-// streaming pass keeps nothing but one (max, sum) pair per 2 KB chunk of the row, written to
-// the workspace.  The CTA that finishes a sequence's last segment (found with a ticket
+// Every target row is read from HBM exactly once, with 16-byte loads that go straight to
+// registers (each warp instruction covers 512 contiguous bytes); warps run freely, one 2 KB
+// chunk per step.  The streaming pass keeps nothing but one (max, sum) pair per chunk of the
+// row, written to the workspace.  The CTA that finishes a sequence's last segment (found with a ticket
 // counter, no waiting) resolves the sequence: it turns the chunk partials into each row's
 // log-normaliser, rebuilds the sparse q~ in fp64, runs the acceptance tests, and samples the
 // correction token from the full-vocabulary residual.  Because q~ is sparse, the residual is
@@ -16,7 +17,6 @@
 
 #include "tslt_common.cuh"
 #include "tslt_rowmath.cuh"
-#include "tslt_stream.cuh"
 
 namespace tslt {
 
@@ -25,9 +25,9 @@ constexpr int kMaxTreeNodes = 1024;
 
 struct VerifyParams {
     const unsigned char* logits;
-    long long row_stride_bytes, row_bytes;
+    long long row_stride_bytes;
     int V, B, rows_per_seq, k;
-    int nseg, tiles_per_seg, ntiles, nchunks;
+    int nseg, chunks_per_seg, nchunks;
     ScaleC cp, cq;
     const int* draft_idx;
     const float* draft_logit;
@@ -54,14 +54,13 @@ struct VerifyParams {
 };
 
 struct VerifyShared {
-    RingBars bars;
     double scratch[16];
     double slot_a, slot_q;
     int slot_found;
     int ticket;
 };
 
-// Resolver work arrays, laid over the idle ring (and a little beyond it).
+// Resolver work arrays (dynamic shared memory; only the CTA that resolves a sequence uses them).
 struct ResolverArrays {
     double* chunkR;  // kMaxChunks
     int* s_idx;      // 1024
@@ -71,7 +70,7 @@ struct ResolverArrays {
     double* r;       // 1024
 };
 constexpr int kResolverBytes = kMaxChunks * 8 + 1024 * 4 + 4 * 1024 * 8;
-constexpr int kVerifyArena = kResolverBytes > kRingBytes ? kResolverBytes : kRingBytes;
+constexpr int kVerifyArena = kResolverBytes;
 __device__ __forceinline__ ResolverArrays carve(unsigned char* arena) {
     ResolverArrays a;
     a.chunkR = reinterpret_cast<double*>(arena);
@@ -94,13 +93,13 @@ __device__ __forceinline__ double accept_probability(double p, double q) {
 // base-2 log-normaliser of a row from its chunk partials: L2 = M + log2 sum S_c 2^(M_c - M)
 __device__ __forceinline__ double row_log2_norm(const float2* part, int nchunks, int tid, double* scratch) {
     double mx = -INFINITY;
-    for (int c = tid; c < nchunks; c += kConsumerThreads) {
+    for (int c = tid; c < nchunks; c += kBlockThreads) {
         const float2 ms = __ldcg(&part[c]);
         if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
     }
     mx = block_max(mx, tid, scratch);
     double s = 0.0;
-    for (int c = tid; c < nchunks; c += kConsumerThreads) {
+    for (int c = tid; c < nchunks; c += kBlockThreads) {
         const float2 ms = __ldcg(&part[c]);
         if (ms.y > 0.f) s += (double)ms.y * exp2((double)ms.x - mx);
     }
@@ -124,7 +123,7 @@ __device__ __forceinline__ int load_draft(const VerifyParams& p, size_t draft_ro
     const int* di = p.draft_idx + draft_row * (size_t)p.k;
     const float* dl = p.draft_logit + draft_row * (size_t)p.k;
     double mx = -INFINITY;
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         A.s_idx[i] = di[i];
         const float l = dl[i];
         const bool fin = fabsf(l) <= 3.4028234e38f;
@@ -134,14 +133,14 @@ __device__ __forceinline__ int load_draft(const VerifyParams& p, size_t draft_ro
     }
     mx = block_max(mx, tid, scratch);
     double w = 0.0;
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         const double y = A.s_q[i];
         const double e = y > -INFINITY ? exp2(y - mx) : 0.0;
         A.s_q[i] = e;
         w += e;
     }
     const double W = block_sum(w, tid, scratch);
-    for (int i = tid; i < n; i += kConsumerThreads) A.s_q[i] = W > 0.0 ? A.s_q[i] / W : 0.0;
+    for (int i = tid; i < n; i += kBlockThreads) A.s_q[i] = W > 0.0 ? A.s_q[i] / W : 0.0;
     consumer_sync();
     return n;
 }
@@ -156,13 +155,13 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
                                                  VerifyShared* sh) {
     constexpr int kChunkElems = kChunkBytes / Elt<T>::kBytes;
     const int nch = p.nchunks;
-    for (int c = tid; c < nch; c += kConsumerThreads) {
+    for (int c = tid; c < nch; c += kBlockThreads) {
         const float2 ms = __ldcg(&part[c]);
         A.chunkR[c] = (ms.y > 0.f && L2 > -INFINITY) ? c_out * (double)ms.y * exp2((double)ms.x - L2) : 0.0;
     }
     consumer_sync();
     // entries of S replace c_out * p by their explicit value; one writer per chunk (S is ascending)
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         const int v = A.s_idx[i];
         if (v < 0 || v >= p.V) continue;
         const int c = v / kChunkElems;
@@ -203,16 +202,16 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
     // second touch of one chunk: exact weights of its elements
     const int v0 = c * kChunkElems;
     const int ne = min(kChunkElems, p.V - v0);
-    for (int e = tid; e < ne; e += kConsumerThreads) A.r[e] = c_out * token_prob<T>(rowp, v0 + e, p.V, p.cp.d, L2);
+    for (int e = tid; e < ne; e += kBlockThreads) A.r[e] = c_out * token_prob<T>(rowp, v0 + e, p.V, p.cp.d, L2);
     consumer_sync();
-    for (int i = tid; i < n; i += kConsumerThreads) {
+    for (int i = tid; i < n; i += kBlockThreads) {
         const int v = A.s_idx[i];
         if (v >= v0 && v < v0 + ne) A.r[v - v0] = A.s_a[i] > 0.0 ? A.s_a[i] : 0.0;
     }
     consumer_sync();
     // keep the plain weights for the "last positive" fallback, scan a copy in place of chunkR
     double* cumr = A.chunkR;  // chunk table no longer needed
-    for (int e = tid; e < ne; e += kConsumerThreads) cumr[e] = A.r[e];
+    for (int e = tid; e < ne; e += kBlockThreads) cumr[e] = A.r[e];
     consumer_sync();
     block_inclusive_scan(cumr, ne, tid, sh->scratch);
     const double Rc2 = cumr[ne - 1];
@@ -226,8 +225,8 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
 }
 
 template <typename T>
-__device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ring, VerifyShared* sh, int tid) {
-    const ResolverArrays A = carve(ring);
+__device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* arena, VerifyShared* sh, int tid) {
+    const ResolverArrays A = carve(arena);
     const int gamma = p.gamma;
     const size_t r0 = (size_t)b * (gamma + 1);
     int a = 0;
@@ -251,7 +250,7 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ri
         }
         consumer_sync();
         double bh = 0.0;
-        for (int i = tid; i < n; i += kConsumerThreads) {
+        for (int i = tid; i < n; i += kBlockThreads) {
             const int v = A.s_idx[i];
             if (v == x) sh->slot_q = A.s_q[i];
             if (p.beta_hat) {
@@ -285,7 +284,7 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ri
     int n = 0;
     if (a < gamma) {
         n = load_draft(p, (size_t)b * gamma + a, A, tid, sh->scratch);
-        for (int i = tid; i < n; i += kConsumerThreads) {
+        for (int i = tid; i < n; i += kBlockThreads) {
             const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2_stop);
             A.s_p[i] = pv;
             const double d = pv - A.s_q[i];
@@ -303,14 +302,14 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ri
 }
 
 template <typename T>
-__device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, VerifyShared* sh, int tid) {
-    const ResolverArrays A = carve(ring);
+__device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* arena, VerifyShared* sh, int tid) {
+    const ResolverArrays A = carve(arena);
     const int N = p.N;
     const int* child_begin = p.tree_meta;
     const int* child_list = p.tree_meta + (N + 1);
     const int* node_draft_row = p.tree_meta + (N + 1) + (N - 1);
     int* path = p.accepted_path + (size_t)b * p.max_depth;
-    for (int d = tid; d < p.max_depth; d += kConsumerThreads) path[d] = -1;
+    for (int d = tid; d < p.max_depth; d += kBlockThreads) path[d] = -1;
     consumer_sync();
     int node = 0, len = 0, tok = -1;
     for (int depth = 0; depth <= p.max_depth; ++depth) {
@@ -326,7 +325,7 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, 
         }
         const int n = load_draft(p, (size_t)b * p.M + dr, A, tid, sh->scratch);
         double ps = 0.0;
-        for (int i = tid; i < n; i += kConsumerThreads) {
+        for (int i = tid; i < n; i += kBlockThreads) {
             const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2);
             A.s_p[i] = pv;
             A.s_a[i] = pv;
@@ -341,7 +340,7 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, 
             const int x = p.node_token[(size_t)b * N + c];
             if (tid == 0) sh->slot_found = 0;
             consumer_sync();
-            for (int i = tid; i < n; i += kConsumerThreads)
+            for (int i = tid; i < n; i += kBlockThreads)
                 if (A.s_idx[i] == x) {
                     sh->slot_a = A.s_a[i];
                     sh->slot_q = A.s_q[i];
@@ -368,13 +367,13 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, 
             }
             // rejected: p^(i+1) = norm(max(0, p^(i) - q~)), on S explicitly, elsewhere by the scalar
             double zs = 0.0;
-            for (int i = tid; i < n; i += kConsumerThreads) {
+            for (int i = tid; i < n; i += kBlockThreads) {
                 const double d = A.s_a[i] - A.s_q[i];
                 zs += d > 0.0 ? d : 0.0;
             }
             const double Z = block_sum(zs, tid, sh->scratch) + c_out * out_mass;
             if (Z > 0.0) {
-                for (int i = tid; i < n; i += kConsumerThreads) {
+                for (int i = tid; i < n; i += kBlockThreads) {
                     const double d = A.s_a[i] - A.s_q[i];
                     A.s_a[i] = d > 0.0 ? d / Z : 0.0;
                 }
@@ -397,78 +396,50 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* ring, 
 template <typename T, bool kTree>
 __global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* ring = reinterpret_cast<unsigned char*>(((size_t)smem_raw + 127) & ~(size_t)127);
-    VerifyShared* sh = reinterpret_cast<VerifyShared*>(ring + kVerifyArena);
+    unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const int tile_begin = seg * p.tiles_per_seg;
-    const int tile_end = min(p.ntiles, tile_begin + p.tiles_per_seg);
-
-    ring_init(&sh->bars, tid);
-    __syncthreads();
-    if (tid >= kConsumerThreads) {
-        producer_loop<T>(rowp, p.row_bytes, tile_begin, tile_end, ring, &sh->bars, p.status);
-        return;
-    }
-    const int lane = tid & 31, warp = tid >> 5;
-    const float chi = p.cp.hi, clo = p.cp.lo;
+    const int chunk_begin = seg * p.chunks_per_seg;
+    const int chunk_end = min(p.nchunks, chunk_begin + p.chunks_per_seg);
+    const RowExtent ext = row_extent<T>(p.V);
+    const float c = p.cp.f;
     float2* part = p.partials + (size_t)row * p.nchunks;
-    bool aborted = false;
 
-    for (int t = tile_begin; t < tile_end; ++t) {
-        const int it = t - tile_begin, s = it % kStages;
-        if (!mbar_wait(&sh->bars.full[s], (uint32_t)((it / kStages) & 1), &sh->bars.abort)) {
-            raise_abort(&sh->bars, p.status);
-            aborted = true;
-            break;
-        }
-        const uint32_t padded = tile_padded_bytes(p.row_bytes, t);
-        const unsigned char* tile = ring + s * kTileBytes;
+    // ---- streaming pass: (max, sum) of every chunk, the chunk's own maximum as the reference ----
+    for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
         LaneTile<T> lt;
-        lt.load(tile, warp, lane, padded);
-        // the warp's chunk of this tile is in registers: release the slot
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh->bars.empty[s]);
-        if ((uint32_t)(warp * kChunkBytes) < padded) {
-            LaneSum ls;
-            ls.reset();
-            const float lm = lt.lane_max();
-            if (lm > -INFINITY) ls.raise(lm, chi, clo);
-            lt.accumulate(ls, chi, clo);
-            // fold the 32 lane partials into the chunk's (max, sum)
-            const float Mw = warp_max(ls.M);
-            const float Sw = warp_sum(ls.total() * ex2_approx(ls.M - Mw));
-            if (lane == 0) part[t * kConsumerWarps + warp] = make_float2(Mw, Sw);
+        lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+        const float wm = warp_max(lt.reduce_max());
+        LaneSum ls;
+        ls.reset();
+        if (wm > -INFINITY) {
+            ls.zmax = wm;
+            ls.M = wm * c;
         }
+        lt.accumulate(ls, c);
+        const float Sw = warp_sum(ls.total());
+        if (lane == 0) part[ch] = make_float2(ls.M, Sw);
     }
-    // collective decision on abort (a wait that ran out): nobody resolves, status word is set
-    int any;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, %2, %3, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
-        : "=r"(any)
-        : "r"((int)aborted), "n"(kConsumerBarrier), "n"(kConsumerThreads)
-        : "memory");
-    if (any) return;
 
     // ---- ticket: the CTA that completes the sequence resolves it ---------------------------------
     __threadfence();
-    consumer_sync();
+    __syncthreads();
     const int b = row / p.rows_per_seq;
     if (tid == 0) sh->ticket = atomicAdd(&p.tickets[b], 1);
-    consumer_sync();
+    __syncthreads();
     if (sh->ticket != p.rows_per_seq * p.nseg - 1) return;
     __threadfence();
-    if (kTree) resolve_tree<T>(p, b, ring, sh, tid);
-    else resolve_sequence<T>(p, b, ring, sh, tid);
+    if (kTree) resolve_tree<T>(p, b, arena, sh, tid);
+    else resolve_sequence<T>(p, b, arena, sh, tid);
 }
 
 // ---- host side -------------------------------------------------------------------------------
 
 struct VerifyPlan {
-    int nseg, tiles_per_seg, ntiles, nchunks;
+    int nseg, chunks_per_seg, nchunks;
     size_t smem;
     size_t ws_tickets_off, ws_meta_off, ws_partials_off, ws_bytes;
 };
@@ -489,14 +460,15 @@ static int sm_count_v() {
 static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes, int meta_ints) {
     VerifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
-    pl.ntiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
     pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
     const long long rows = (long long)B * rows_per_seq;
     const int sms = sm_count_v();
-    int nseg = 1;
-    while (nseg < 16 && rows * nseg < 4LL * sms && pl.ntiles / (nseg * 2) >= 2) nseg *= 2;
-    pl.tiles_per_seg = (pl.ntiles + nseg - 1) / nseg;
-    pl.nseg = (pl.ntiles + pl.tiles_per_seg - 1) / pl.tiles_per_seg;
+    // One CTA per row segment.  Segments are 8 chunks per warp (128 KB) when that still gives
+    // the machine sixteen CTAs per SM to balance over, and shrink down to one chunk per warp otherwise.
+    int cps = 8 * kWarps;
+    while (cps > kWarps && rows * ((pl.nchunks + cps - 1) / cps) < 16LL * sms) cps /= 2;
+    pl.chunks_per_seg = cps;
+    pl.nseg = (pl.nchunks + cps - 1) / cps;
     if (pl.nseg < 1) pl.nseg = 1;
     pl.smem = kVerifyArena + sizeof(VerifyShared) + 256;
     size_t off = kWsHeaderBytes;
@@ -569,9 +541,8 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     VerifyParams p = {};
     p.logits = (const unsigned char*)target_logits;
     p.row_stride_bytes = row_stride_elems * eb;
-    p.row_bytes = (long long)V * eb;
     p.V = V; p.B = B; p.rows_per_seq = gamma + 1; p.k = k;
-    p.nseg = pl.nseg; p.tiles_per_seg = pl.tiles_per_seg; p.ntiles = pl.ntiles; p.nchunks = pl.nchunks;
+    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
@@ -645,9 +616,8 @@ extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int
     VerifyParams p = {};
     p.logits = (const unsigned char*)target_logits;
     p.row_stride_bytes = row_stride_elems * eb;
-    p.row_bytes = (long long)V * eb;
     p.V = V; p.B = B; p.rows_per_seq = N; p.k = k;
-    p.nseg = pl.nseg; p.tiles_per_seg = pl.tiles_per_seg; p.ntiles = pl.ntiles; p.nchunks = pl.nchunks;
+    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
