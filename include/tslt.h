@@ -21,8 +21,10 @@
  *   - uniforms are fp32 in [0,1); a value >= 1 is read as the largest float below 1.
  *   - "sample" always means inverse CDF in ascending token index: the first index whose
  *     cumulative mass exceeds u * total.
- *   - device-side waits are bounded; a wait that ran out sets a status word in the
- *     workspace, reported by tslt_workspace_status as TSLT_ERR_DEVICE_STATUS.
+ *   - no kernel waits on another CTA: CTAs that share a row or a sequence meet through a
+ *     ticket counter in the workspace and the last one to arrive carries on.  The first word
+ *     of the workspace is a device status word (0 = fine) that tslt_workspace_status reads
+ *     back; a non-zero word is reported as TSLT_ERR_DEVICE_STATUS.
  */
 #ifndef TSLT_H_
 #define TSLT_H_
@@ -99,7 +101,8 @@ int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
  * Shapes: target_logits [B, gamma+1, V]; draft_idx, draft_logit [B, gamma, k] and
  * draft_count [B, gamma] exactly as tslt_sparsify writes them; draft_token, u_accept
  * [B, gamma]; u_sample, accepted_len, out_token [B].  Draft indices outside [0, V) are
- * ignored (probability 0) rather than dereferenced.
+ * ignored (probability 0) rather than dereferenced.  Requires gamma < 1024 and
+ * V * sizeof(element) <= 4 MiB (TSLT_ERR_UNSUPPORTED otherwise).
  */
 int tslt_verify_workspace_bytes(int B, int gamma, int V, int k, size_t* bytes);
 int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,

@@ -224,60 +224,96 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
     return v0 + pos;
 }
 
+// One warp: base-2 log-normaliser of a row from its chunk partials (warp shuffles only).
+__device__ __forceinline__ double row_log2_norm_warp(const float2* part, int nchunks, int lane) {
+    double mx = -INFINITY;
+    for (int c = lane; c < nchunks; c += 32) {
+        const float2 ms = __ldcg(&part[c]);
+        if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
+    }
+    mx = warp_max(mx);
+    double s = 0.0;
+    for (int c = lane; c < nchunks; c += 32) {
+        const float2 ms = __ldcg(&part[c]);
+        if (ms.y > 0.f) s += (double)ms.y * exp2((double)ms.x - mx);
+    }
+    s = warp_sum(s);
+    return s > 0.0 ? mx + log2(s) : -INFINITY;
+}
+
+// One warp: acceptance probability min(1, p(x) / q~(x)) of one position, and (if wanted) the
+// truncated acceptance rate sum_S min(p, q~).  q~ is rebuilt from the transmitted pairs in
+// passes over global memory (at most 8 KB, cache resident); nothing is staged.
+template <typename T>
+__device__ __forceinline__ double position_accept_prob(const VerifyParams& p, size_t draft_row, const unsigned char* rowp,
+                                                       double L2, int lane, double* beta_hat_out) {
+    int n = p.draft_count[draft_row];
+    n = n < 0 ? 0 : (n > p.k ? p.k : n);
+    const int* di = p.draft_idx + draft_row * (size_t)p.k;
+    const float* dl = p.draft_logit + draft_row * (size_t)p.k;
+    const int x = p.draft_token[draft_row];
+    double mx = -INFINITY;
+    for (int i = lane; i < n; i += 32) {
+        const float l = dl[i];
+        if (fabsf(l) <= 3.4028234e38f) mx = fmax(mx, (double)l * p.cq.d);
+    }
+    mx = warp_max(mx);
+    double w = 0.0, ex = 0.0;
+    for (int i = lane; i < n; i += 32) {
+        const float l = dl[i];
+        const double e = fabsf(l) <= 3.4028234e38f ? exp2((double)l * p.cq.d - mx) : 0.0;
+        w += e;
+        if (di[i] == x) ex = e;
+    }
+    const double W = warp_sum(w);
+    ex = warp_max(ex);  // the pairs are distinct: at most one lane found x
+    const double qx = W > 0.0 ? ex / W : 0.0;
+    if (beta_hat_out) {
+        double bh = 0.0;
+        for (int i = lane; i < n; i += 32) {
+            const float l = dl[i];
+            const double e = fabsf(l) <= 3.4028234e38f ? exp2((double)l * p.cq.d - mx) : 0.0;
+            bh += fmin(token_prob<T>(rowp, di[i], p.V, p.cp.d, L2), W > 0.0 ? e / W : 0.0);
+        }
+        *beta_hat_out = warp_sum(bh);
+    }
+    return accept_probability(token_prob<T>(rowp, x, p.V, p.cp.d, L2), qx);
+}
+
 template <typename T>
 __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* arena, VerifyShared* sh, int tid) {
     const ResolverArrays A = carve(arena);
     const int gamma = p.gamma;
+    const int lane = tid & 31, warp = tid >> 5;
     const size_t r0 = (size_t)b * (gamma + 1);
-    int a = 0;
-    bool running = true;
-    double L2_stop = -INFINITY;
-    for (int j = 0; j <= gamma; ++j) {
+    // ---- every position on its own warp: log-normaliser of its target row, then its acceptance test
+    double* L2s = A.chunkR;               // gamma + 1 entries (gamma < 1024, checked on the host)
+    double* aps = A.chunkR + (gamma + 1);  // gamma entries
+    for (int j = warp; j <= gamma; j += kWarps) {
         const float2* part = p.partials + (r0 + j) * (size_t)p.nchunks;
-        const double L2 = row_log2_norm(part, p.nchunks, tid, sh->scratch);
-        if (p.lse_p && tid == 0) p.lse_p[r0 + j] = (float)(L2 * 0.6931471805599453);
-        if (j == gamma) {
-            if (running) L2_stop = L2;
-            break;
+        const double L2 = row_log2_norm_warp(part, p.nchunks, lane);
+        if (lane == 0) {
+            L2s[j] = L2;
+            if (p.lse_p) p.lse_p[r0 + j] = (float)(L2 * 0.6931471805599453);
         }
-        if (!running && !p.accept_prob && !p.beta_hat) continue;  // only lse_p still wanted
-        const unsigned char* rowp = p.logits + (long long)(r0 + j) * p.row_stride_bytes;
-        const size_t dr = (size_t)b * gamma + j;
-        const int n = load_draft(p, dr, A, tid, sh->scratch);
-        const int x = p.draft_token[dr];
-        if (tid == 0) {
-            sh->slot_q = 0.0;
-        }
-        consumer_sync();
-        double bh = 0.0;
-        for (int i = tid; i < n; i += kBlockThreads) {
-            const int v = A.s_idx[i];
-            if (v == x) sh->slot_q = A.s_q[i];
-            if (p.beta_hat) {
-                const double pv = token_prob<T>(rowp, v, p.V, p.cp.d, L2);
-                bh += fmin(pv, A.s_q[i]);
+        if (j < gamma) {
+            const unsigned char* rowp = p.logits + (long long)(r0 + j) * p.row_stride_bytes;
+            const size_t dr = (size_t)b * gamma + j;
+            double bh = 0.0;
+            const double ap = position_accept_prob<T>(p, dr, rowp, L2, lane, p.beta_hat ? &bh : nullptr);
+            if (lane == 0) {
+                aps[j] = ap;
+                if (p.accept_prob) p.accept_prob[dr] = (float)ap;
+                if (p.beta_hat) p.beta_hat[dr] = (float)bh;
             }
         }
-        if (p.beta_hat) {
-            bh = block_sum(bh, tid, sh->scratch);
-            if (tid == 0) p.beta_hat[dr] = (float)bh;
-        } else {
-            consumer_sync();
-        }
-        const double px = token_prob<T>(rowp, x, p.V, p.cp.d, L2);
-        const double ap = accept_probability(px, sh->slot_q);
-        if (p.accept_prob && tid == 0) p.accept_prob[dr] = (float)ap;
-        if (running) {
-            const double r = (double)clamp_uniform(p.u_accept[dr]);
-            if (r < ap) {
-                ++a;
-            } else {
-                running = false;
-                L2_stop = L2;
-            }
-        }
-        consumer_sync();
     }
+    consumer_sync();
+    // ---- the leading run of accepted positions (strict <) ---------------------------------------
+    int a = 0;
+    while (a < gamma && (double)clamp_uniform(p.u_accept[(size_t)b * gamma + a]) < aps[a]) ++a;
+    const double L2_stop = L2s[a];
+    consumer_sync();  // chunkR is reused below
     // correction token: residual of the rejected position, or the bonus row
     const unsigned char* rowp = p.logits + (long long)(r0 + a) * p.row_stride_bytes;
     const float2* part = p.partials + (r0 + a) * (size_t)p.nchunks;
@@ -425,10 +461,13 @@ __global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyPa
     }
 
     // ---- ticket: the CTA that completes the sequence resolves it ---------------------------------
-    __threadfence();
+    // (the barrier orders every warp's partials before thread 0's fence, which publishes them)
     __syncthreads();
     const int b = row / p.rows_per_seq;
-    if (tid == 0) sh->ticket = atomicAdd(&p.tickets[b], 1);
+    if (tid == 0) {
+        __threadfence();
+        sh->ticket = atomicAdd(&p.tickets[b], 1);
+    }
     __syncthreads();
     if (sh->ticket != p.rows_per_seq * p.nseg - 1) return;
     __threadfence();
@@ -534,7 +573,7 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     if (!u_sample || !accepted_len || !out_token ||
         (gamma > 0 && (!draft_idx || !draft_logit || !draft_count || !draft_token || !u_accept)))
         return TSLT_ERR_INVALID_ARG;
-    if ((long long)B * (gamma + 1) > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    if ((long long)B * (gamma + 1) > 0x7fffffffLL / 16 || gamma >= 1024) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
     VerifyPlan pl = make_verify_plan(B, gamma + 1, V, eb, 0);
     if (workspace_bytes < pl.ws_bytes) return TSLT_ERR_WORKSPACE;
