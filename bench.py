@@ -44,7 +44,7 @@ UNIT = "rows/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
 # under profiles/ (None until a capture exists for that kernel).
-NCU_TRAFFIC_BYTES = {"sparsify_kernel": None, "verify_kernel": None}
+NCU_TRAFFIC_BYTES = {"sparsify_kernel": 1092.2e6, "verify_kernel": 1197.1e6}
 
 
 def measured_peak_gbs():
@@ -105,7 +105,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -315,7 +315,7 @@ def run_e2e(tslt, zq, zp, ud, ua, us, k, top_p, T, steps, warmup):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", action="store_true", help="also time the k / top-p sweep and the other configs")
