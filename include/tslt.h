@@ -41,12 +41,16 @@ extern "C" {
 #define TSLT_ERR_WORKSPACE (-3)
 #define TSLT_ERR_CUDA (-4)
 #define TSLT_ERR_DEVICE_STATUS (-5)
+#define TSLT_ERR_STATIC_SCRATCH (-6)
 
 #define TSLT_F32 0
 #define TSLT_BF16 1
 
 /* largest supported k (top-k size, or the candidate cap when top-p is on) */
 #define TSLT_MAX_K 1024
+
+/* size of the scratch array built into the library for tslt_verify_static */
+#define TSLT_STATIC_SCRATCH_BYTES (8u << 20)
 
 /* Library version as major * 10000 + minor * 100 + patch. */
 int tslt_version(void);
@@ -112,6 +116,40 @@ int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,
                 const float* u_sample, int* accepted_len, int* out_token, float* accept_prob,
                 float* beta_hat, float* lse_p, void* workspace, size_t workspace_bytes,
                 void* stream);
+
+/*
+ * tslt_verify without a workspace argument, for callers that must not allocate device memory.
+ * (The paper has no counterpart of this call; it exists for the sake of such callers only.)
+ *
+ * Who these callers are: a decoding loop inside a serving process that handed every byte of HBM
+ * to its own pool at start-up (weights, KV cache) and forbids cudaMalloc afterwards, because
+ * cudaMalloc synchronises the whole device and can fail once memory is fragmented or full; or
+ * a plug-in written in C whose host framework owns the allocator and gives the plug-in no handle
+ * on it.  Such a caller still owns its inputs and outputs and passes them exactly as to
+ * tslt_verify; only the scratch (ticket counters and one (max, sum) pair per 2 KB of every target
+ * row) comes from the library: a fixed array of TSLT_STATIC_SCRATCH_BYTES (8 MiB) in device
+ * memory that every GPU holds from the moment the library is loaded until the process exits.
+ *
+ *   - Limit: the call is refused with TSLT_ERR_STATIC_SCRATCH, before anything touches the
+ *     device, when the scratch tslt_verify would need for these sizes and this dtype exceeds
+ *     that size (about B * (gamma + 1) * V * sizeof(element) / 256 bytes; B = 256, gamma = 8,
+ *     V = 256000 in bf16 needs 4.6 MiB).  Use tslt_verify with your own workspace for larger
+ *     problems.
+ *   - The first call on each device looks up the array's device address (the device that is
+ *     current at the call); make that first call before any stream capture begins.
+ *   - The call itself allocates and frees nothing, on the host or on the device.
+ *   - All calls on a device share the one array, which still holds what the previous call wrote;
+ *     each call clears the words that must start at zero on its stream before its kernel runs.
+ *     Two calls that can overlap on the GPU (different streams, no dependency) race on the array
+ *     and give wrong results: serialise them.
+ * Arguments, results and every other rule are those of tslt_verify.
+ */
+int tslt_verify_static(const void* target_logits, int dtype, int B, int gamma, int V,
+                       long long row_stride_elems, int k, const int* draft_idx,
+                       const float* draft_logit, const int* draft_count, const int* draft_token,
+                       float draft_temperature, float target_temperature, const float* u_accept,
+                       const float* u_sample, int* accepted_len, int* out_token, float* accept_prob,
+                       float* beta_hat, float* lse_p, void* stream);
 
 /*
  * Verifier side, multi-candidate token tree (Algorithm 5 at every node met on the

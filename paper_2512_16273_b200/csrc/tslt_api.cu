@@ -13,6 +13,7 @@ extern "C" const char* tslt_status_string(int status) {
         case TSLT_ERR_WORKSPACE: return "workspace too small";
         case TSLT_ERR_CUDA: return "CUDA runtime error";
         case TSLT_ERR_DEVICE_STATUS: return "the device status word of the workspace is not zero; outputs of that call are invalid";
+        case TSLT_ERR_STATIC_SCRATCH: return "problem needs more scratch than the array built into the library holds";
         default: return "unknown status";
     }
 }

@@ -13,6 +13,7 @@
 // read a second time.
 #include <math.h>
 
+#include <mutex>
 #include <vector>
 
 #include "tslt_common.cuh"
@@ -595,6 +596,54 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, pl.ws_meta_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
     return launch_verify<false>(p, pl, dtype, st);
+}
+
+// ---- tslt_verify_static: the same verification with the scratch memory built into the library ----
+// Scratch of the no-allocation entry point: ticket counters and per-chunk partial sums.  Every
+// GPU that loads the library carries this array until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[TSLT_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel could use, so the address is asked for once
+// per device (with that device current) and remembered.
+static int static_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static void* cache[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TSLT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return TSLT_ERR_CUDA;
+        cache[dev] = ptr;
+    }
+    *out = cache[dev];
+    return TSLT_OK;
+}
+
+extern "C" int tslt_verify_static(const void* target_logits, int dtype, int B, int gamma, int V,
+                                  long long row_stride_elems, int k, const int* draft_idx,
+                                  const float* draft_logit, const int* draft_count, const int* draft_token,
+                                  float draft_temperature, float target_temperature, const float* u_accept,
+                                  const float* u_sample, int* accepted_len, int* out_token, float* accept_prob,
+                                  float* beta_hat, float* lse_p, void* stream) {
+    // the size the ordinary entry point would ask a workspace for; too much is refused before
+    // anything touches the device
+    if (dtype != TSLT_F32 && dtype != TSLT_BF16) return TSLT_ERR_UNSUPPORTED;
+    if (B < 0 || gamma < 0 || V <= 0 || k <= 0 || k > V) return TSLT_ERR_INVALID_ARG;
+    if (k > TSLT_MAX_K || (long long)B * (gamma + 1) > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    const size_t need = make_verify_plan(B, gamma + 1, V, dtype == TSLT_F32 ? 4 : 2, 0).ws_bytes;
+    if (need > (size_t)TSLT_STATIC_SCRATCH_BYTES) return TSLT_ERR_STATIC_SCRATCH;
+    if (B == 0) return TSLT_OK;
+    void* scratch = nullptr;
+    const int rs = static_scratch_address(&scratch);
+    if (rs != TSLT_OK) return rs;
+    // tslt_verify zeroes the status word and the ticket counters on the stream before its kernel,
+    // so whatever the previous call left in the array does no harm
+    return tslt_verify(target_logits, dtype, B, gamma, V, row_stride_elems, k, draft_idx, draft_logit, draft_count,
+                       draft_token, draft_temperature, target_temperature, u_accept, u_sample, accepted_len,
+                       out_token, accept_prob, beta_hat, lse_p, scratch, (size_t)TSLT_STATIC_SCRATCH_BYTES, stream);
 }
 
 extern "C" int tslt_tree_verify_workspace_bytes(int B, int N, int V, int k, size_t* bytes) {

@@ -19,12 +19,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libtslt.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_STATUS = 0, -1, -2, -3, -4, -5
+ERR_STATIC_SCRATCH = -6
+STATIC_SCRATCH_BYTES = 8 << 20
 F32, BF16 = 0, 1
 MAX_K = 1024
 
 EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status",
            "tslt_sparsify_workspace_bytes", "tslt_sparsify",
-           "tslt_verify_workspace_bytes", "tslt_verify",
+           "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify"]
 
 
@@ -62,6 +64,8 @@ def lib() -> ctypes.CDLL:
     L.tslt_verify_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_verify.restype = i
     L.tslt_verify.argtypes = [p, i, i, i, i, ll, i, p, p, p, p, f, f, p, p, p, p, p, p, p, p, sz, p]
+    L.tslt_verify_static.restype = i
+    L.tslt_verify_static.argtypes = [p, i, i, i, i, ll, i, p, p, p, p, f, f, p, p, p, p, p, p, p, p]
     L.tslt_tree_verify_workspace_bytes.restype = i
     L.tslt_tree_verify_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_tree_verify.restype = i
@@ -261,6 +265,40 @@ def verify(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_logit: to
     _check(rc, "tslt_verify")
     o["workspace"] = ws
     return o
+
+
+def verify_static(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_logit: torch.Tensor,
+                  draft_count: torch.Tensor, draft_token: torch.Tensor, draft_temperature: float,
+                  target_temperature: float, u_accept: torch.Tensor, u_sample: torch.Tensor, out: dict) -> dict:
+    """tslt_verify_static: tslt_verify for callers that may not allocate device memory.  The scratch
+    is an 8 MiB array built into the library (shared by all calls on the device, so calls must not
+    overlap), and this wrapper allocates nothing either: `out` must already hold the output tensors
+    accepted_len [B] and out_token [B] (int32) and may hold accept_prob, beta_hat [B, gamma] and
+    lse_p [B, gamma+1] (fp32).  Raises TsltError(ERR_STATIC_SCRATCH) when the problem needs more
+    scratch than the array holds."""
+    if not target_logits.is_cuda or target_logits.dim() != 3:
+        raise ValueError("target_logits must be a CUDA tensor [B, gamma+1, V]")
+    B, g1, V = target_logits.shape
+    _, _, stride = _row_layout(target_logits)
+    gamma = g1 - 1
+    k = draft_idx.shape[-1] if gamma > 0 else 1
+    for name, t, dt in (("draft_idx", draft_idx, torch.int32), ("draft_logit", draft_logit, torch.float32),
+                        ("draft_count", draft_count, torch.int32), ("draft_token", draft_token, torch.int32),
+                        ("u_accept", u_accept, torch.float32), ("u_sample", u_sample, torch.float32),
+                        ("accepted_len", out["accepted_len"], torch.int32), ("out_token", out["out_token"], torch.int32)):
+        _cuda(t, name, dt)
+    if draft_idx.numel() != B * gamma * k or draft_logit.numel() != B * gamma * k or \
+            draft_count.numel() != B * gamma or draft_token.numel() != B * gamma or \
+            u_accept.numel() != B * gamma or u_sample.numel() != B or \
+            out["accepted_len"].numel() != B or out["out_token"].numel() != B:
+        raise ValueError("draft / uniform / output shapes do not match target_logits")
+    rc = lib().tslt_verify_static(_ptr(target_logits), _dtype_code(target_logits), B, gamma, V, stride, k,
+                                  _ptr(draft_idx), _ptr(draft_logit), _ptr(draft_count), _ptr(draft_token),
+                                  draft_temperature, target_temperature, _ptr(u_accept), _ptr(u_sample),
+                                  _ptr(out["accepted_len"]), _ptr(out["out_token"]), _ptr(out.get("accept_prob")),
+                                  _ptr(out.get("beta_hat")), _ptr(out.get("lse_p")), _stream())
+    _check(rc, "tslt_verify_static")
+    return out
 
 
 def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_row: Sequence[int],
