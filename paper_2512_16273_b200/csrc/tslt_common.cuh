@@ -25,6 +25,51 @@ constexpr int kVecsPerChunk = kChunkBytes / kVecBytes;        // 128
 // Named barrier used by the block-level helpers (all 256 threads take part).
 constexpr int kConsumerBarrier = 1;
 
+// How the rows of a call map to CTAs: every row is cut into nseg segments of cps chunks (the last
+// may be shorter), one CTA per segment, block = row * nseg + seg.
+struct RowSplit {
+    int rows, nseg, cps, grid;
+};
+struct RowWork {
+    int row, seg, nseg, chunk_begin, chunk_end;
+};
+__host__ __device__ inline RowWork locate_work(const RowSplit& sp, int block, int nchunks) {
+    RowWork w;
+    w.row = block / sp.nseg;
+    w.seg = block - w.row * sp.nseg;
+    w.nseg = sp.nseg;
+    w.chunk_begin = w.seg * sp.cps;
+    w.chunk_end = w.chunk_begin + sp.cps < nchunks ? w.chunk_begin + sp.cps : nchunks;
+    return w;
+}
+// slots = CTAs the machine holds at once; max_seg = most segments a row may be cut into;
+// big_cps = segment length (chunks) to use when there are at least `slots` rows (0: whole rows).
+// With fewer rows than slots, rows are cut so that about two CTAs per slot exist, a segment
+// keeping at least two chunks per warp.
+inline RowSplit make_row_split(long long rows, int nchunks, int slots, int max_seg, int big_cps) {
+    RowSplit sp;
+    sp.rows = (int)rows;
+    if (nchunks < 1) nchunks = 1;
+    int by_len = nchunks / 16;
+    if (by_len < 1) by_len = 1;
+    if (max_seg > by_len) max_seg = by_len;
+    if (max_seg < 1) max_seg = 1;
+    int nseg = 1;
+    if (rows >= slots) {
+        if (big_cps > 0) nseg = (nchunks + big_cps - 1) / big_cps;
+    } else if (rows > 0) {
+        nseg = (int)((2LL * slots + rows - 1) / rows);
+    }
+    if (nseg > max_seg) nseg = max_seg;
+    if (nseg < 1) nseg = 1;
+    int cps = (nchunks + nseg - 1) / nseg;
+    cps = (cps + 7) / 8 * 8;
+    sp.nseg = (nchunks + cps - 1) / cps;
+    sp.cps = cps;
+    sp.grid = sp.rows * sp.nseg;
+    return sp;
+}
+
 // Workspace header: word 0 is the device status (0 = fine).
 constexpr int kWsHeaderBytes = 256;
 

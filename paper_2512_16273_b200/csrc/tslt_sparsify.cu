@@ -36,6 +36,7 @@ constexpr int kCoarseBins = 128;  // coarse bin = fine bin >> 5: lets a scan fin
 constexpr int kLowestFiniteBin = 0x00800000u >> kHistShift;  // bin of -FLT_MAX: every finite logit passes
 constexpr int kBoundaryCap = 960;   // entries of the k-th logit's bin that the direct tie-break handles
 constexpr int kArenaBytes = 24576;  // histograms (16.5 KB) + boundary list (7.5 KB); fp64 work arrays afterwards
+constexpr int kSparsifyCtasPerSm = 4;  // 64 registers per thread
 constexpr int kRankSortMax = 256;   // up to this many entries are ordered by counting, more by a bitonic sort
 
 struct SegStat {
@@ -58,7 +59,8 @@ struct SparsifyParams {
     int* token;
     float* lse;
     float* mass;
-    int nseg, chunks_per_seg, nchunks;
+    int nchunks;
+    RowSplit split;
     int cap, high;      // candidate (key, index) list: capacity and compaction mark
     int vcap, vhigh;    // staged vectors: capacity and early-expansion mark
     int idx_hi_byte;
@@ -387,7 +389,7 @@ __device__ __noinline__ void reselect_from_buffer(int n, int k, int idx_hi_byte,
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, 4) sparsify_kernel(const SparsifyParams p) {
+__global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_kernel(const SparsifyParams p) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr int kChunkElems = kChunkBytes / Elt<T>::kBytes;
@@ -407,10 +409,9 @@ __global__ void __launch_bounds__(kBlockThreads, 4) sparsify_kernel(const Sparsi
     const uint32_t sh_addr = smem_u32(sh);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
+    const int row = wk.row, chunk_begin = wk.chunk_begin, chunk_end = wk.chunk_end;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const int chunk_begin = seg * p.chunks_per_seg;
-    const int chunk_end = min(p.nchunks, chunk_begin + p.chunks_per_seg);
     const RowExtent ext = row_extent<T>(p.V);
     const int k = p.k;
     const float c = p.c.f;
@@ -529,7 +530,8 @@ __global__ void __launch_bounds__(kBlockThreads, 4) sparsify_kernel(const Sparsi
     double Srow = block_sum(ls.total_f64() * exp2((double)ls.M - Mrow), tid, sh->scratch);
 
     // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
-    if (p.nseg > 1) {
+    if (wk.nseg > 1) {
+        const size_t slot0 = (size_t)row * wk.nseg;  // this row's first segment slot
         // hand over the candidates (all at or above this segment's final threshold)
         int n = sh->cand_count;
         if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
@@ -540,37 +542,37 @@ __global__ void __launch_bounds__(kBlockThreads, 4) sparsify_kernel(const Sparsi
             reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
             n = sh->cand_count;
         }
-        uint2* my_entries = p.seg_entries + ((size_t)row * p.nseg + seg) * (size_t)p.seg_cap;
+        uint2* my_entries = p.seg_entries + (slot0 + wk.seg) * (size_t)p.seg_cap;
         for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
         if (tid == 0) {
             SegStat st;
             st.S = Srow;
             st.M = (float)Mrow;
             st.n = n;
-            p.seg_stats[(size_t)row * p.nseg + seg] = st;
+            p.seg_stats[slot0 + wk.seg] = st;
         }
         __threadfence();
         consumer_sync();
         if (tid == 0) sh->ticket = atomicAdd(&p.tickets[row], 1);
         consumer_sync();
-        if (sh->ticket != p.nseg - 1) return;
+        if (sh->ticket != wk.nseg - 1) return;
         __threadfence();
         // gather every segment's candidates and statistics
         if (tid == 0) sh->cand_count = 0;
         consumer_sync();
         double Mall = -INFINITY;
-        for (int g = 0; g < p.nseg; ++g) {
-            const SegStat* st = &p.seg_stats[(size_t)row * p.nseg + g];
+        for (int g = 0; g < wk.nseg; ++g) {
+            const SegStat* st = &p.seg_stats[slot0 + g];
             Mall = fmax(Mall, (double)__ldcg(&st->M));
         }
         double Sall = 0.0;
-        for (int g = 0; g < p.nseg; ++g) {
-            const SegStat* st = &p.seg_stats[(size_t)row * p.nseg + g];
+        for (int g = 0; g < wk.nseg; ++g) {
+            const SegStat* st = &p.seg_stats[slot0 + g];
             const double Sg = __ldcg(&st->S);
             const double Mg = (double)__ldcg(&st->M);
             Sall += Sg * exp2(Mg - Mall);
             const int ng = __ldcg(&st->n);
-            const uint2* ent = p.seg_entries + ((size_t)row * p.nseg + g) * (size_t)p.seg_cap;
+            const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
             const int base = sh->cand_count;
             for (int i = tid; i < ng; i += kBlockThreads) {
                 uint2 e2 = __ldcg(&ent[i]);
@@ -807,7 +809,8 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
-    int nseg, chunks_per_seg, nchunks, cap, high, vcap, vhigh, seg_cap;
+    int nchunks, cap, high, vcap, vhigh, seg_cap;
+    RowSplit split;
     size_t smem;
     size_t ws_tickets_off, ws_stats_off, ws_entries_off, ws_bytes;
 };
@@ -824,6 +827,8 @@ static int sm_count_cached() {
     return sms;
 }
 
+constexpr int kSmemPerSm = 227 * 1024;
+
 static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     SparsifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
@@ -835,26 +840,22 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.vcap = k <= 128 ? 1024 : 2048;
     pl.vhigh = pl.vcap - pl.vcap / 4;
     pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above)
-    // Split a row over several CTAs when there are too few rows to fill the machine; a segment
-    // keeps at least two chunks per warp and the segments' winners must fit one buffer.
-    const int sms = sm_count_cached();
-    int nseg = 1;
-    const int max_seg_by_cap = pl.cap / pl.seg_cap;
-    while (nseg < 16 && nseg * 2 <= max_seg_by_cap && (long long)rows * nseg < 4LL * sms &&
-           pl.nchunks / (nseg * 2) >= 2 * kWarps)
-        nseg *= 2;
-    pl.chunks_per_seg = (pl.nchunks + nseg - 1) / nseg;
-    pl.chunks_per_seg = (pl.chunks_per_seg + kWarps - 1) / kWarps * kWarps;
-    pl.nseg = (pl.nchunks + pl.chunks_per_seg - 1) / pl.chunks_per_seg;
-    if (pl.nseg < 1) pl.nseg = 1;
     pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
+    // CTAs the machine holds at once: launch bounds and the shared-memory footprint decide
+    int per_sm = (int)(kSmemPerSm / (pl.smem + 1024));
+    if (per_sm > kSparsifyCtasPerSm) per_sm = kSparsifyCtasPerSm;
+    if (per_sm < 1) per_sm = 1;
+    // a split row's segments must fit the candidate list of the CTA that merges them
+    const int max_seg = pl.cap / pl.seg_cap < 16 ? pl.cap / pl.seg_cap : 16;
+    pl.split = make_row_split(rows, pl.nchunks, per_sm * sm_count_cached(), max_seg, 0);
+    const size_t split_rows = pl.split.nseg > 1 ? (size_t)rows : 0;
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
     off = align_up(off + (size_t)rows * sizeof(int), 256);
     pl.ws_stats_off = off;
-    off = align_up(off + (size_t)rows * pl.nseg * sizeof(SegStat), 256);
+    off = align_up(off + split_rows * pl.split.nseg * sizeof(SegStat), 256);
     pl.ws_entries_off = off;
-    off = align_up(off + (pl.nseg > 1 ? (size_t)rows * pl.nseg * pl.seg_cap * sizeof(uint2) : 0), 256);
+    off = align_up(off + split_rows * pl.split.nseg * pl.seg_cap * sizeof(uint2), 256);
     pl.ws_bytes = off;
     return pl;
 }
@@ -911,7 +912,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.num_samples = num_samples;
     p.uniforms = uniforms;
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
-    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
+    p.nchunks = pl.nchunks; p.split = pl.split;
     p.cap = pl.cap; p.high = pl.high; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
     p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
     unsigned char* ws = (unsigned char*)workspace;
@@ -927,6 +928,6 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sparsify_smem_bytes(4096, 2048, TSLT_MAX_K)) != cudaSuccess)
         return TSLT_ERR_CUDA;
-    kern<<<rows * pl.nseg, kBlockThreads, pl.smem, st>>>(p);
+    kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
 }

@@ -28,7 +28,8 @@ struct VerifyParams {
     const unsigned char* logits;
     long long row_stride_bytes;
     int V, B, rows_per_seq, k;
-    int nseg, chunks_per_seg, nchunks;
+    int nchunks;
+    RowSplit split;
     ScaleC cp, cq;
     const int* draft_idx;
     const float* draft_logit;
@@ -430,23 +431,15 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* arena,
     }
 }
 
-template <typename T, bool kTree>
-__global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyParams p) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
-    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int row = blockIdx.x / p.nseg, seg = blockIdx.x % p.nseg;
-    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const int chunk_begin = seg * p.chunks_per_seg;
-    const int chunk_end = min(p.nchunks, chunk_begin + p.chunks_per_seg);
+// Streaming pass over chunks [chunk_begin, chunk_end) of one row: (max, sum) of every chunk, the
+// chunk's own maximum as the reference exponent.
+template <typename T>
+__device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWork& wk, int lane, int warp) {
+    const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
     const RowExtent ext = row_extent<T>(p.V);
     const float c = p.cp.f;
-    float2* part = p.partials + (size_t)row * p.nchunks;
-
-    // ---- streaming pass: (max, sum) of every chunk, the chunk's own maximum as the reference ----
-    for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
+    float2* part = p.partials + (size_t)wk.row * p.nchunks;
+    for (int ch = wk.chunk_begin + warp; ch < wk.chunk_end; ch += kWarps) {
         LaneTile<T> lt;
         lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
         const float wm = warp_max(lt.reduce_max());
@@ -460,26 +453,55 @@ __global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyPa
         const float Sw = warp_sum(ls.total());
         if (lane == 0) part[ch] = make_float2(ls.M, Sw);
     }
+}
 
+// Small problems, one launch: stream, then the CTA that completes a sequence resolves it.
+template <typename T, bool kTree>
+__global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyParams p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
+    const int tid = threadIdx.x;
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
+    stream_chunks<T>(p, wk, tid & 31, tid >> 5);
     // ---- ticket: the CTA that completes the sequence resolves it ---------------------------------
     // (the barrier orders every warp's partials before thread 0's fence, which publishes them)
     __syncthreads();
-    const int b = row / p.rows_per_seq;
+    const int b = wk.row / p.rows_per_seq;
     if (tid == 0) {
         __threadfence();
         sh->ticket = atomicAdd(&p.tickets[b], 1);
     }
     __syncthreads();
-    if (sh->ticket != p.rows_per_seq * p.nseg - 1) return;
+    if (sh->ticket != p.rows_per_seq * p.split.nseg - 1) return;
     __threadfence();
     if (kTree) resolve_tree<T>(p, b, arena, sh, tid);
     else resolve_sequence<T>(p, b, arena, sh, tid);
 }
 
+// Large problems, two launches on the stream: the streaming pass alone (no shared memory, no
+// ticket, no fence: the kernel boundary publishes the partials) ...
+template <typename T>
+__global__ void __launch_bounds__(kBlockThreads, 4) verify_stream_kernel(const VerifyParams p) {
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
+    stream_chunks<T>(p, wk, threadIdx.x & 31, threadIdx.x >> 5);
+}
+// ... then one CTA per sequence resolves it.
+template <typename T, bool kTree>
+__global__ void __launch_bounds__(kBlockThreads, 4) verify_resolve_kernel(const VerifyParams p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* arena = smem_raw;
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
+    if (kTree) resolve_tree<T>(p, blockIdx.x, arena, sh, threadIdx.x);
+    else resolve_sequence<T>(p, blockIdx.x, arena, sh, threadIdx.x);
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 struct VerifyPlan {
-    int nseg, chunks_per_seg, nchunks;
+    int nchunks;
+    bool two_launches;  // enough rows to fill the machine: stream kernel + resolve kernel
+    RowSplit split;
     size_t smem;
     size_t ws_tickets_off, ws_meta_off, ws_partials_off, ws_bytes;
 };
@@ -497,19 +519,16 @@ static int sm_count_v() {
     return sms;
 }
 
+constexpr int kVerifyCtasPerSm = 4;  // what the launch bounds and the shared-memory footprint allow
+
 static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes, int meta_ints) {
     VerifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
     pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
     const long long rows = (long long)B * rows_per_seq;
-    const int sms = sm_count_v();
-    // One CTA per row segment.  Segments are 8 chunks per warp (128 KB) when that still gives
-    // the machine sixteen CTAs per SM to balance over, and shrink down to one chunk per warp otherwise.
-    int cps = 8 * kWarps;
-    while (cps > kWarps && rows * ((pl.nchunks + cps - 1) / cps) < 16LL * sms) cps /= 2;
-    pl.chunks_per_seg = cps;
-    pl.nseg = (pl.nchunks + cps - 1) / cps;
-    if (pl.nseg < 1) pl.nseg = 1;
+    const int slots = kVerifyCtasPerSm * sm_count_v();
+    pl.two_launches = rows >= slots;
+    pl.split = make_row_split(rows, pl.nchunks, slots, 16, 64);
     pl.smem = kVerifyArena + sizeof(VerifyShared) + 256;
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
@@ -544,8 +563,17 @@ static int launch_verify(VerifyParams& p, const VerifyPlan& pl, int dtype, cudaS
     auto kern = dtype == TSLT_F32 ? verify_kernel<float, kTree> : verify_kernel<bf16_t, kTree>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
         return TSLT_ERR_CUDA;
-    const long long grid = (long long)p.B * p.rows_per_seq * pl.nseg;
-    kern<<<(unsigned)grid, kBlockThreads, pl.smem, st>>>(p);
+    if (!pl.two_launches) {
+        kern<<<(unsigned)pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
+        return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+    }
+    auto resolve = dtype == TSLT_F32 ? verify_resolve_kernel<float, kTree> : verify_resolve_kernel<bf16_t, kTree>;
+    if (cudaFuncSetAttribute(resolve, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
+        return TSLT_ERR_CUDA;
+    if (dtype == TSLT_F32) verify_stream_kernel<float><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
+    else verify_stream_kernel<bf16_t><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+    resolve<<<(unsigned)p.B, kBlockThreads, pl.smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
 }
 
@@ -582,7 +610,7 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     p.logits = (const unsigned char*)target_logits;
     p.row_stride_bytes = row_stride_elems * eb;
     p.V = V; p.B = B; p.rows_per_seq = gamma + 1; p.k = k;
-    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
+    p.nchunks = pl.nchunks; p.split = pl.split;
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
@@ -705,7 +733,7 @@ extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int
     p.logits = (const unsigned char*)target_logits;
     p.row_stride_bytes = row_stride_elems * eb;
     p.V = V; p.B = B; p.rows_per_seq = N; p.k = k;
-    p.nseg = pl.nseg; p.chunks_per_seg = pl.chunks_per_seg; p.nchunks = pl.nchunks;
+    p.nchunks = pl.nchunks; p.split = pl.split;
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;

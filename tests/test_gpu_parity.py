@@ -60,6 +60,16 @@ def test_top_p_below_cap_and_second_temperature():
     assert (ref_s["count"] == 32).any()
 
 
+def test_many_rows_take_the_two_launch_verifier():
+    """At least 592 target rows (one per CTA slot of the machine): the verifier runs as a streaming
+    kernel followed by a resolve kernel instead of one fused launch."""
+    zq, zp = small_logits(100, 6, 4099, torch.bfloat16, seed=21)          # 700 target rows
+    run_sequence_case(zq, zp, 32, 1.0, 1.0, seed=21, what="two-launch verify")
+    run_sequence_case(zq, zp, 64, 0.9, 0.7, seed=22, num_samples=2, what="two-launch verify top-p")
+    _, ref = run_tree_case(20, (3, 3, 3), 5000, torch.float32, 16, 1.0, 23, what="two-launch tree")  # 800 rows
+    assert ref["accepted_len"].max() >= 1
+
+
 def adversarial_rows(V, dtype):
     rows = []
     asc = torch.linspace(-8, 8, V)
