@@ -217,6 +217,12 @@ template <> struct Elt<bf16_t> {
     }
 };
 
+// Ask the copy engine to bring `bytes` (a non-zero multiple of 16) at the 16-byte aligned global
+// address p into L2; nothing is written anywhere else and nothing has to be waited for.
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // 16-byte streaming load of logits: read once, so marked evict-first.
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) { return __ldcs(p); }
 

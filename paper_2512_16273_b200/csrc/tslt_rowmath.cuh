@@ -29,6 +29,18 @@ template <typename T> __host__ __device__ inline RowExtent row_extent(int V) {
     return e;
 }
 
+// One lane of the warp asks for chunk `ch` of the row (clipped to the row's whole vectors) to be
+// brought into L2, so that the warp's loads of it, one step later, are L2 hits.
+__device__ __forceinline__ void prefetch_chunk(const unsigned char* row, int ch, int chunk_end, int lane,
+                                               const RowExtent& ext) {
+    if (lane == 0 && ch < chunk_end) {
+        const long long v0 = (long long)ch * kVecsPerChunk;
+        long long nv = ext.nvec_full - v0;
+        if (nv > kVecsPerChunk) nv = kVecsPerChunk;
+        if (nv > 0) prefetch_l2(row + v0 * kVecBytes, (uint32_t)nv * kVecBytes);
+    }
+}
+
 // Online softmax state of one lane: sum of 2^(z * c - M) in four packed accumulators.
 struct LaneSum {
     float2 acc[4];

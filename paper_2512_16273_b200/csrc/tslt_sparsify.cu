@@ -37,6 +37,7 @@ constexpr int kLowestFiniteBin = 0x00800000u >> kHistShift;  // bin of -FLT_MAX:
 constexpr int kBoundaryCap = 960;   // entries of the k-th logit's bin that the direct tie-break handles
 constexpr int kArenaBytes = 24576;  // histograms (16.5 KB) + boundary list (7.5 KB); fp64 work arrays afterwards
 constexpr int kSparsifyCtasPerSm = 4;  // 64 registers per thread
+constexpr int kPrefetchSteps = 1;      // how many of its own steps ahead a warp asks L2 for its chunk
 constexpr int kRankSortMax = 256;   // up to this many entries are ordered by counting, more by a bitonic sort
 
 struct SegStat {
@@ -476,6 +477,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
             LaneTile<T> lt;
             lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+            prefetch_chunk(rowp, ch + kPrefetchSteps * kWarps, chunk_end, lane, ext);
             const float lm = lt.reduce_max();
             if (lm > ls.zmax) ls.raise(lm, c);
             lt.accumulate(ls, c);

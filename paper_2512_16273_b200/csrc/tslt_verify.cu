@@ -442,6 +442,7 @@ __device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWo
     for (int ch = wk.chunk_begin + warp; ch < wk.chunk_end; ch += kWarps) {
         LaneTile<T> lt;
         lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+        prefetch_chunk(rowp, ch + kWarps, wk.chunk_end, lane, ext);
         const float wm = warp_max(lt.reduce_max());
         LaneSum ls;
         ls.reset();
@@ -479,10 +480,12 @@ __global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyPa
     else resolve_sequence<T>(p, b, arena, sh, tid);
 }
 
+constexpr int kStreamCtasPerSm = 6;  // streaming-only kernel: 42 registers per thread, no shared memory
+
 // Large problems, two launches on the stream: the streaming pass alone (no shared memory, no
 // ticket, no fence: the kernel boundary publishes the partials) ...
 template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, 4) verify_stream_kernel(const VerifyParams p) {
+__global__ void __launch_bounds__(kBlockThreads, kStreamCtasPerSm) verify_stream_kernel(const VerifyParams p) {
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
     stream_chunks<T>(p, wk, threadIdx.x & 31, threadIdx.x >> 5);
 }
@@ -519,7 +522,7 @@ static int sm_count_v() {
     return sms;
 }
 
-constexpr int kVerifyCtasPerSm = 4;  // what the launch bounds and the shared-memory footprint allow
+constexpr int kVerifyCtasPerSm = 4;  // fused kernel: what the launch bounds and the shared-memory footprint allow
 
 static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes, int meta_ints) {
     VerifyPlan pl;
@@ -528,7 +531,7 @@ static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes
     const long long rows = (long long)B * rows_per_seq;
     const int slots = kVerifyCtasPerSm * sm_count_v();
     pl.two_launches = rows >= slots;
-    pl.split = make_row_split(rows, pl.nchunks, slots, 16, 64);
+    pl.split = make_row_split(rows, pl.nchunks, slots, pl.two_launches ? 64 : 16, 32);
     pl.smem = kVerifyArena + sizeof(VerifyShared) + 256;
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
