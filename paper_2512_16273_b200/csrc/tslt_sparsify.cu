@@ -389,7 +389,38 @@ __device__ __noinline__ void reselect_from_buffer(int n, int k, int idx_hi_byte,
     select_topk<kKeyHiOnly>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
 }
 
-template <typename T>
+// All threads: bring every segment's candidates and statistics of a row into the candidate list.
+__device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row, int nseg, Candidates cb,
+                                                SparsifyShared* sh, int tid, double* Mrow, double* Srow) {
+    const size_t slot0 = (size_t)row * nseg;
+    if (tid == 0) sh->cand_count = 0;
+    consumer_sync();
+    double Mall = -INFINITY;
+    for (int g = 0; g < nseg; ++g) Mall = fmax(Mall, (double)__ldcg(&p.seg_stats[slot0 + g].M));
+    double Sall = 0.0;
+    for (int g = 0; g < nseg; ++g) {
+        const SegStat* st = &p.seg_stats[slot0 + g];
+        Sall += __ldcg(&st->S) * exp2((double)__ldcg(&st->M) - Mall);
+        const int ng = __ldcg(&st->n);
+        const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
+        const int base = sh->cand_count;
+        for (int i = tid; i < ng; i += kBlockThreads) {
+            const uint2 e2 = __ldcg(&ent[i]);
+            cb.key[base + i] = e2.x;
+            cb.idx[base + i] = (int)e2.y;
+        }
+        consumer_sync();
+        if (tid == 0) sh->cand_count = base + ng;
+        consumer_sync();
+    }
+    *Mrow = Mall;
+    *Srow = Sall;
+}
+
+// kHandOff = false: one launch does everything; the segments of a split row meet through a ticket.
+// kHandOff = true: every segment hands its candidates and statistics over and the CTA ends; the
+// rows are finished by sparsify_finish_kernel, launched next on the stream.
+template <typename T, bool kHandOff>
 __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_kernel(const SparsifyParams p) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     constexpr int kPer = Elt<T>::kPerVec;
@@ -532,7 +563,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     double Srow = block_sum(ls.total_f64() * exp2((double)ls.M - Mrow), tid, sh->scratch);
 
     // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
-    if (wk.nseg > 1) {
+    if (kHandOff || wk.nseg > 1) {
         const size_t slot0 = (size_t)row * wk.nseg;  // this row's first segment slot
         // hand over the candidates (all at or above this segment's final threshold)
         int n = sh->cand_count;
@@ -553,44 +584,44 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             st.n = n;
             p.seg_stats[slot0 + wk.seg] = st;
         }
-        __threadfence();
+        if (kHandOff) return;  // the kernel boundary publishes the hand-over
         consumer_sync();
-        if (tid == 0) sh->ticket = atomicAdd(&p.tickets[row], 1);
+        if (tid == 0) {
+            __threadfence();
+            sh->ticket = atomicAdd(&p.tickets[row], 1);
+        }
         consumer_sync();
         if (sh->ticket != wk.nseg - 1) return;
         __threadfence();
-        // gather every segment's candidates and statistics
-        if (tid == 0) sh->cand_count = 0;
-        consumer_sync();
-        double Mall = -INFINITY;
-        for (int g = 0; g < wk.nseg; ++g) {
-            const SegStat* st = &p.seg_stats[slot0 + g];
-            Mall = fmax(Mall, (double)__ldcg(&st->M));
-        }
-        double Sall = 0.0;
-        for (int g = 0; g < wk.nseg; ++g) {
-            const SegStat* st = &p.seg_stats[slot0 + g];
-            const double Sg = __ldcg(&st->S);
-            const double Mg = (double)__ldcg(&st->M);
-            Sall += Sg * exp2(Mg - Mall);
-            const int ng = __ldcg(&st->n);
-            const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
-            const int base = sh->cand_count;
-            for (int i = tid; i < ng; i += kBlockThreads) {
-                uint2 e2 = __ldcg(&ent[i]);
-                cand_key[base + i] = e2.x;
-                cand_idx[base + i] = (int)e2.y;
-            }
-            consumer_sync();
-            if (tid == 0) sh->cand_count = base + ng;
-            consumer_sync();
-        }
-        Mrow = Mall;
-        Srow = Sall;
+        gather_segments(p, row, wk.nseg, cb, sh, tid, &Mrow, &Srow);
         hist_valid = false;
     }
 
     finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, hist_valid, tid);
+}
+
+// Second launch of the two-launch form: one CTA per row merges the row's segments and finishes it.
+// Same shared-memory carve-up as the streaming kernel, with no staging buffer (vcap = 0).
+template <typename T>
+__global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const SparsifyParams p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* arena = smem_raw;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(arena + kArenaBytes);
+    int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
+    uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
+    int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
+    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, 0, p.k));
+    const int tid = threadIdx.x, row = blockIdx.x;
+    if (tid == 0) {
+        sh->hist_addr = smem_u32(hist);
+        sh->coarse_addr = smem_u32(hist + kHistBins);
+        sh->overflow = 0;
+    }
+    Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
+    double Mrow, Srow;
+    gather_segments(p, row, p.split.nseg, cb, sh, tid, &Mrow, &Srow);
+    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, false, tid);
 }
 
 // Position of entry (key, idx) of the buffer in the order (key descending, idx ascending) /
@@ -811,6 +842,7 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
+    bool two_launches;  // enough rows to fill the machine: streaming kernel + finish kernel
     int nchunks, cap, high, vcap, vhigh, seg_cap;
     RowSplit split;
     size_t smem;
@@ -849,8 +881,9 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (per_sm < 1) per_sm = 1;
     // a split row's segments must fit the candidate list of the CTA that merges them
     const int max_seg = pl.cap / pl.seg_cap < 16 ? pl.cap / pl.seg_cap : 16;
+    pl.two_launches = rows >= per_sm * sm_count_cached();
     pl.split = make_row_split(rows, pl.nchunks, per_sm * sm_count_cached(), max_seg, 0);
-    const size_t split_rows = pl.split.nseg > 1 ? (size_t)rows : 0;
+    const size_t split_rows = (pl.two_launches || pl.split.nseg > 1) ? (size_t)rows : 0;
     size_t off = kWsHeaderBytes;
     pl.ws_tickets_off = off;
     off = align_up(off + (size_t)rows * sizeof(int), 256);
@@ -926,10 +959,20 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     cudaStream_t st = (cudaStream_t)stream;
     // status word and tickets start at zero
     if (cudaMemsetAsync(ws, 0, pl.ws_stats_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
-    auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
+    auto kern = dtype == TSLT_F32 ? (pl.two_launches ? sparsify_kernel<float, true> : sparsify_kernel<float, false>)
+                                  : (pl.two_launches ? sparsify_kernel<bf16_t, true> : sparsify_kernel<bf16_t, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sparsify_smem_bytes(4096, 2048, TSLT_MAX_K)) != cudaSuccess)
         return TSLT_ERR_CUDA;
     kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+    if (pl.two_launches) {
+        auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
+        if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
+            return TSLT_ERR_CUDA;
+        fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+    }
+    return TSLT_OK;
 }

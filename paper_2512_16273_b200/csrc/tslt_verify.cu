@@ -442,7 +442,6 @@ __device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWo
     for (int ch = wk.chunk_begin + warp; ch < wk.chunk_end; ch += kWarps) {
         LaneTile<T> lt;
         lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
-        prefetch_chunk(rowp, ch + kWarps, wk.chunk_end, lane, ext);
         const float wm = warp_max(lt.reduce_max());
         LaneSum ls;
         ls.reset();
