@@ -41,9 +41,10 @@ constexpr int kPrefetchSteps = 1;      // how many of its own steps ahead a warp
 constexpr int kRankSortMax = 256;   // up to this many entries are ordered by counting, more by a bitonic sort
 
 struct SegStat {
-    double S;  // sum of 2^(y - M) over the segment
-    float M;   // reference exponent (base 2)
-    int n;     // candidates written for the segment
+    double S[kWarps];  // per warp: sum of 2^(y - M) over the warp's chunks of the segment
+    float M[kWarps];   // per warp: reference exponent (base 2)
+    int n;             // candidates written for the segment
+    int pad;
 };
 
 struct SparsifyParams {
@@ -393,14 +394,54 @@ __device__ __noinline__ void reselect_from_buffer(int n, int k, int idx_hi_byte,
 __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row, int nseg, Candidates cb,
                                                 SparsifyShared* sh, int tid, double* Mrow, double* Srow) {
     const size_t slot0 = (size_t)row * nseg;
+    if (nseg == 1 && p.seg_cap <= 8 * kBlockThreads) {
+        // one segment: every load is issued before anything is used, so the row costs one trip to memory
+        const SegStat* st = &p.seg_stats[slot0];
+        const uint2* ent = p.seg_entries + slot0 * (size_t)p.seg_cap;
+        uint2 e[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = tid + j * kBlockThreads;
+            e[j] = i < p.seg_cap ? __ldcg(&ent[i]) : make_uint2(0u, 0u);
+        }
+        const int n = __ldcg(&st->n);
+        double Mall = -INFINITY, Sall = 0.0, Sw[kWarps], Mw[kWarps];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            Sw[w] = __ldcg(&st->S[w]);
+            Mw[w] = (double)__ldcg(&st->M[w]);
+        }
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) Mall = fmax(Mall, Mw[w]);
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w)
+            if (Sw[w] > 0.0) Sall += Sw[w] * exp2(Mw[w] - Mall);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = tid + j * kBlockThreads;
+            if (i < n) {
+                cb.key[i] = e[j].x;
+                cb.idx[i] = (int)e[j].y;
+            }
+        }
+        if (tid == 0) sh->cand_count = n;
+        consumer_sync();
+        *Mrow = Mall;
+        *Srow = Sall;
+        return;
+    }
     if (tid == 0) sh->cand_count = 0;
     consumer_sync();
     double Mall = -INFINITY;
-    for (int g = 0; g < nseg; ++g) Mall = fmax(Mall, (double)__ldcg(&p.seg_stats[slot0 + g].M));
+    for (int g = 0; g < nseg; ++g)
+        for (int w = 0; w < kWarps; ++w) Mall = fmax(Mall, (double)__ldcg(&p.seg_stats[slot0 + g].M[w]));
     double Sall = 0.0;
     for (int g = 0; g < nseg; ++g) {
         const SegStat* st = &p.seg_stats[slot0 + g];
-        Sall += __ldcg(&st->S) * exp2((double)__ldcg(&st->M) - Mall);
+        for (int w = 0; w < kWarps; ++w) {
+            const double Sw = __ldcg(&st->S[w]);
+            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st->M[w]) - Mall);
+        }
         const int ng = __ldcg(&st->n);
         const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
         const int base = sh->cand_count;
@@ -553,14 +594,22 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         consumer_sync();
     }
 
-    // ---- row statistics ------------------------------------------------------------------
-    float Mrow_f = warp_max(ls.M);
-    if (lane == 0) sh->scratch[warp] = (double)Mrow_f;
-    consumer_sync();
-    double Mrow = sh->scratch[0];
-    for (int w = 1; w < kWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
-    consumer_sync();
-    double Srow = block_sum(ls.total_f64() * exp2((double)ls.M - Mrow), tid, sh->scratch);
+    // ---- statistics: one (M, S) pair per warp; combined here only if this CTA finishes the row ----
+    const float Mw = warp_max(ls.M);
+    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
+    double Mrow = 0.0, Srow = 0.0;
+    if (!kHandOff && wk.nseg == 1) {
+        if (lane == 0) {
+            sh->scratch[warp] = (double)Mw;
+            sh->scratch[kWarps + warp] = Sw;
+        }
+        consumer_sync();
+        Mrow = sh->scratch[0];
+        for (int w = 1; w < kWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
+        for (int w = 0; w < kWarps; ++w)
+            if (sh->scratch[kWarps + w] > 0.0) Srow += sh->scratch[kWarps + w] * exp2(sh->scratch[w] - Mrow);
+        consumer_sync();
+    }
 
     // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
     if (kHandOff || wk.nseg > 1) {
@@ -577,13 +626,12 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         }
         uint2* my_entries = p.seg_entries + (slot0 + wk.seg) * (size_t)p.seg_cap;
         for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
-        if (tid == 0) {
-            SegStat st;
-            st.S = Srow;
-            st.M = (float)Mrow;
-            st.n = n;
-            p.seg_stats[slot0 + wk.seg] = st;
+        SegStat* st = &p.seg_stats[slot0 + wk.seg];
+        if (lane == 0) {
+            st->S[warp] = Sw;
+            st->M[warp] = Mw;
         }
+        if (tid == 0) st->n = n;
         if (kHandOff) return;  // the kernel boundary publishes the hand-over
         consumer_sync();
         if (tid == 0) {
@@ -613,6 +661,8 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
     SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, 0, p.k));
     const int tid = threadIdx.x, row = blockIdx.x;
+    // the uniforms are needed last: ask for their cache line now
+    if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) {
         sh->hist_addr = smem_u32(hist);
         sh->coarse_addr = smem_u32(hist + kHistBins);
@@ -839,6 +889,175 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     }
 }
 
+// ---- finish kernel for small k --------------------------------------------------------------------
+// Rows whose hand-over is at most 256 candidates in one segment (k <= 128) are finished by a CTA of
+// 128 threads with 6 KB of shared memory, so that every row of a large batch is resident at once:
+// finishing a row is a chain of a dozen dependent steps (one trip to memory, rank counting, two
+// scans), and what it costs machine-wide is the length of that chain times the number of waves.
+constexpr int kSmallThreads = 128;
+constexpr int kSmallCand = 256;
+
+struct SmallShared {
+    uint32_t key[kSmallCand];
+    int idx[kSmallCand];
+    uint32_t wkey[kSmallThreads];  // winners in (key descending, index ascending) order, then in ascending index
+    int widx[kSmallThreads];
+    uint32_t okey[kSmallThreads];
+    int oidx[kSmallThreads];
+    double cum[kSmallThreads];
+    double wv[kSmallThreads];
+    double red[8];
+    int n_cut;
+};
+
+__device__ __forceinline__ void small_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kSmallThreads) : "memory"); }
+
+// inclusive scan of one value per thread over the 128 threads; returns this thread's inclusive sum
+__device__ __forceinline__ double small_scan(double v, int tid, double* red, double* total) {
+    const int lane = tid & 31, warp = tid >> 5;
+    double incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) red[warp] = incl;
+    small_sync();
+    double base = 0.0, tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kSmallThreads / 32; ++w) {
+        const double t = red[w];
+        if (w < warp) base += t;
+        tot += t;
+    }
+    small_sync();
+    *total = tot;
+    return base + incl;
+}
+__device__ __forceinline__ double small_max(double v, int tid, double* red) {
+    v = warp_max(v);
+    if ((tid & 31) == 0) red[tid >> 5] = v;
+    small_sync();
+    double m = red[0];
+#pragma unroll
+    for (int w = 1; w < kSmallThreads / 32; ++w) m = fmax(m, red[w]);
+    small_sync();
+    return m;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kernel(const SparsifyParams p) {
+    __shared__ SmallShared sm;
+    const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
+    // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
+    const SegStat* st = &p.seg_stats[row];
+    const uint2* ent = p.seg_entries + (size_t)row * p.seg_cap;
+    uint2 e0 = make_uint2(0u, 0u), e1 = make_uint2(0u, 0u);
+    if (tid < p.seg_cap) e0 = __ldcg(&ent[tid]);
+    if (tid + kSmallThreads < p.seg_cap) e1 = __ldcg(&ent[tid + kSmallThreads]);
+    int nc = __ldcg(&st->n);
+    float u_raw = 0.f;
+    if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];
+    double Mrow = -INFINITY, Srow = 0.0, Sw[kWarps], Mw[kWarps];
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        Sw[w] = __ldcg(&st->S[w]);
+        Mw[w] = (double)__ldcg(&st->M[w]);
+    }
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) Mrow = fmax(Mrow, Mw[w]);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w)
+        if (Sw[w] > 0.0) Srow += Sw[w] * exp2(Mw[w] - Mrow);
+    nc = nc < 0 ? 0 : (nc > kSmallCand ? kSmallCand : nc);
+    if (tid < nc) { sm.key[tid] = e0.x; sm.idx[tid] = (int)e0.y; }
+    if (tid + kSmallThreads < nc) { sm.key[tid + kSmallThreads] = e1.x; sm.idx[tid + kSmallThreads] = (int)e1.y; }
+    small_sync();
+    // ---- exact top-k by counting ranks under (key descending, index ascending) -------------------
+    {
+        int r0 = 0, r1 = 0;
+        const int i1 = tid + kSmallThreads;
+        for (int j = 0; j < nc; ++j) {
+            const uint32_t kj = sm.key[j];
+            const int ij = sm.idx[j];
+            r0 += (kj > e0.x || (kj == e0.x && ij < (int)e0.y)) ? 1 : 0;
+            r1 += (kj > e1.x || (kj == e1.x && ij < (int)e1.y)) ? 1 : 0;
+        }
+        if (tid < nc && r0 < k) { sm.wkey[r0] = e0.x; sm.widx[r0] = (int)e0.y; }
+        if (i1 < nc && r1 < k) { sm.wkey[r1] = e1.x; sm.widx[r1] = (int)e1.y; }
+    }
+    small_sync();
+    const int n0 = nc < k ? nc : k;
+    const double L2 = Mrow + log2(Srow);
+    const double cd = p.c.d;
+    // ---- nucleus cut on the cumulative q in that order ---------------------------------------------
+    int n = n0;
+    double mass = 0.0;
+    {
+        double q = 0.0;
+        if (tid < n0) q = exp2((double)key_to_float(sm.wkey[tid]) * cd - L2);
+        double tot;
+        const double c_incl = small_scan(q, tid, sm.red, &tot);
+        if (p.top_p < 1.0f) {
+            if (tid == 0) sm.n_cut = n0;
+            if (tid < n0) sm.cum[tid] = c_incl;
+            small_sync();
+            const double tp = (double)p.top_p;
+            // first crossing of the cumulative: exactly one thread, if any
+            if (tid < n0 && c_incl >= tp && (tid == 0 || sm.cum[tid - 1] < tp)) sm.n_cut = tid + 1;
+            small_sync();
+            n = sm.n_cut;
+            mass = n > 0 ? sm.cum[n - 1] : 0.0;
+            small_sync();
+        } else {
+            mass = tot;
+        }
+    }
+    // ---- ascending index order -----------------------------------------------------------------------
+    if (tid < n) {
+        const int mine = sm.widx[tid];
+        int r = 0;
+        for (int j = 0; j < n; ++j) r += sm.widx[j] < mine ? 1 : 0;
+        sm.oidx[r] = mine;
+        sm.okey[r] = sm.wkey[tid];
+    }
+    small_sync();
+    // ---- renormalised truncated distribution and its CDF in fp64 -------------------------------------
+    double y = -INFINITY;
+    if (tid < n) y = (double)key_to_float(sm.okey[tid]) * cd;
+    const double mS = small_max(y, tid, sm.red);
+    const double w = tid < n ? exp2(y - mS) : 0.0;
+    double W;
+    const double cw = small_scan(w, tid, sm.red, &W);
+    if (tid < n) { sm.cum[tid] = cw; sm.wv[tid] = w; }
+    small_sync();
+    // ---- outputs ----------------------------------------------------------------------------------------
+    int* o_idx = p.idx + (size_t)row * k;
+    float* o_logit = p.logit + (size_t)row * k;
+    if (tid < k) {
+        o_idx[tid] = tid < n ? sm.oidx[tid] : -1;
+        o_logit[tid] = tid < n ? key_to_float(sm.okey[tid]) : -INFINITY;
+    }
+    if (tid == 0) {
+        p.count[row] = n;
+        if (p.lse) p.lse[row] = n0 > 0 ? (float)(L2 * 0.6931471805599453) : -INFINITY;
+        if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
+    }
+    for (int sidx = tid; sidx < p.num_samples; sidx += kSmallThreads) {
+        int tok = -1;
+        if (n > 0) {
+            const float u = clamp_uniform(sidx == tid ? u_raw : p.uniforms[(size_t)row * p.num_samples + sidx]);
+            int pos = first_greater(sm.cum, n, (double)u * W);
+            if (pos >= n) {
+                pos = n - 1;
+                while (pos > 0 && !(sm.wv[pos] > 0.0)) --pos;
+            }
+            tok = sm.oidx[pos];
+        }
+        p.token[(size_t)row * p.num_samples + sidx] = tok;
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
@@ -873,7 +1092,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.high = pl.cap - pl.cap / 4;
     pl.vcap = k <= 128 ? 1024 : 2048;
     pl.vhigh = pl.vcap - pl.vcap / 4;
-    pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above)
+    pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above); see below
     pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
     // CTAs the machine holds at once: launch bounds and the shared-memory footprint decide
     int per_sm = (int)(kSmemPerSm / (pl.smem + 1024));
@@ -971,7 +1190,12 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
         if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
             return TSLT_ERR_CUDA;
-        fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
+        if (pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallThreads) {
+            if (dtype == TSLT_F32) sparsify_finish_small_kernel<float><<<rows, kSmallThreads, 0, st>>>(p);
+            else sparsify_finish_small_kernel<bf16_t><<<rows, kSmallThreads, 0, st>>>(p);
+        } else {
+            fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
+        }
         if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     }
     return TSLT_OK;
