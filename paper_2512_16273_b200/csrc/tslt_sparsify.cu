@@ -374,6 +374,50 @@ template <typename T>
 __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
                                           unsigned char* arena, double Mrow, double Srow, bool hist_valid, int tid);
 
+// All threads: second pass over a segment whose buffers overflowed.  The histogram went on counting,
+// so the final threshold is as tight as ever: read the segment again and append every logit whose
+// bin is >= bin straight to the (emptied) candidate list.  A list that fills up again (a huge tie)
+// leaves the overflow flag set for the radix select.
+template <typename T>
+__device__ __noinline__ void recollect_from_global(const unsigned char* rowp, int chunk_begin, int chunk_end, int bin,
+                                                   const RowExtent ext, Candidates cb, int cap, SparsifyShared* sh,
+                                                   int tid) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    const int lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        *cb.count = 0;
+        sh->overflow = 0;
+    }
+    consumer_sync();
+    const float edge = bin_lower_edge(bin);
+    for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
+        LaneTile<T> lt;
+        lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+        if (lt.reduce_max() >= edge) {
+#pragma unroll 1
+            for (int j = 0; j < kVecsPerLane; ++j) {
+                if (!(lt.vec_max(j) >= edge)) continue;
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    const float z = lt.elem(j, e);
+                    if (z >= edge) {
+                        const int pos = atomicAdd(cb.count, 1);
+                        if (pos < cap) {
+                            cb.key[pos] = float_to_key(z);
+                            cb.idx[pos] = (ch * kVecsPerChunk + j * 32 + lane) * kPer + e;
+                        } else {
+                            sh->overflow = 1;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    consumer_sync();
+    if (tid == 0 && *cb.count > cap) *cb.count = cap;
+    consumer_sync();
+}
+
 // Radix-select fallbacks, out of line (one copy each).
 template <typename T>
 __device__ __noinline__ void reselect_from_global(const unsigned char* rowp, int e0, int n, int k, int idx_hi_byte,
@@ -586,6 +630,11 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         expand_staged<T>(vec_data, vec_idx, cb, p.cap, sh->thr_bin, p.V, sh, tid);
     }
     bool hist_valid = false;  // the streaming histogram counted vector maxima only
+    if (sh->overflow) {
+        if (warp == 0) raise_threshold(sh, k);
+        consumer_sync();
+        recollect_from_global<T>(rowp, chunk_begin, chunk_end, sh->thr_bin, ext, cb, p.cap, sh, tid);
+    }
     if (sh->overflow) {
         const int e0 = chunk_begin * kChunkElems;
         const int n = min(p.V, chunk_end * kChunkElems) - e0;
@@ -1091,7 +1140,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (pl.cap > 4096) pl.cap = 4096;
     pl.high = pl.cap - pl.cap / 4;
     pl.vcap = k <= 128 ? 1024 : 2048;
-    pl.vhigh = pl.vcap - pl.vcap / 4;
+    pl.vhigh = k <= 256 ? pl.vcap - pl.vcap / 4 : pl.vcap / 2;  // large k stages most vectors: leave room to react
     pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above); see below
     pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
     // CTAs the machine holds at once: launch bounds and the shared-memory footprint decide
