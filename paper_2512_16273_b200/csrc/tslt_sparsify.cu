@@ -74,12 +74,11 @@ struct SparsifyParams {
 };
 
 struct SparsifyShared {
-    // ---- read by push_vector through its shared-memory address -------------------------------------
+    // ---- written by push_vector through their shared-space addresses ---------------------------------
     int vec_count;   // staged vectors
     int overflow;    // a buffer was found full: its contents are no longer complete
     int trim_request;
-    int vcap, vhigh;
-    uint32_t vdata_addr, vidx_addr, hist_addr, coarse_addr;  // shared-space addresses of the arrays
+    uint32_t hist_addr, coarse_addr;  // shared-space addresses of the two histogram levels
     // --------------------------------------------------------------------------------------------
     int cand_count;  // expanded (key, index) candidates
     int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
@@ -150,21 +149,30 @@ __device__ __forceinline__ void sts_v4(uint32_t addr, const uint4& v) {
                  : "memory");
 }
 
+// Where the staging buffer and the histograms of this CTA are, as the out-of-line push wants it:
+// everything sits at fixed offsets of the CTA's dynamic shared memory.
+struct StageRef {
+    uint32_t smem;     // shared-space address of the dynamic shared memory (the fine histogram)
+    uint32_t sh_addr;  // shared-space address of the SparsifyShared block
+    uint32_t caps;     // vcap | vhigh << 16
+};
+
 // Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax, and count
 // that logit.  Out of line on purpose: it is rare, and inlined copies of it in the streaming
-// loop would not fit the instruction cache.
-__device__ __noinline__ void push_vector(uint32_t sh_addr, uint4 data, int vec_index, float vmax) {
+// loop would not fit the instruction cache.  All its operands arrive in registers.
+__device__ __noinline__ void push_vector(uint32_t smem, uint32_t sh_addr, uint32_t caps, uint4 data, int vec_index,
+                                         float vmax) {
+    const uint32_t vcap = caps & 0xffffu, vhigh = caps >> 16;
     const uint32_t pos = atoms_add(sh_addr + offsetof(SparsifyShared, vec_count), 1u);
-    if (pos < lds_u32(sh_addr + offsetof(SparsifyShared, vcap))) {
-        sts_v4(lds_u32(sh_addr + offsetof(SparsifyShared, vdata_addr)) + 16u * pos, data);
-        sts_u32(lds_u32(sh_addr + offsetof(SparsifyShared, vidx_addr)) + 4u * pos, (uint32_t)vec_index);
+    hist_count(smem, smem + 4u * kHistBins, (int)(float_to_key(vmax) >> kHistShift), 1u);
+    const uint32_t vdata = smem + kArenaBytes;
+    if (pos < vcap) {
+        sts_v4(vdata + 16u * pos, data);
+        sts_u32(vdata + 16u * vcap + 4u * pos, (uint32_t)vec_index);
     } else {
         sts_u32(sh_addr + offsetof(SparsifyShared, overflow), 1u);
     }
-    if (pos + 1u == lds_u32(sh_addr + offsetof(SparsifyShared, vhigh)))
-        sts_u32(sh_addr + offsetof(SparsifyShared, trim_request), 1u);
-    hist_count(lds_u32(sh_addr + offsetof(SparsifyShared, hist_addr)),
-               lds_u32(sh_addr + offsetof(SparsifyShared, coarse_addr)), (int)(float_to_key(vmax) >> kHistShift), 1u);
+    if (pos + 1u == vhigh) sts_u32(sh_addr + offsetof(SparsifyShared, trim_request), 1u);
 }
 
 // One warp: the highest fine bin b with (number of counted logits in bins >= b) >= k, or -1 if
@@ -255,40 +263,58 @@ template <> struct Threshold<bf16_t> {
     }
 };
 
-// Stage the vectors of a lane tile that hold a candidate (reduce_max() already called): a test on
-// the lane's packed maximum, then one per vector.
+// Stage the vectors of a lane tile that hold a candidate (reduce_max() already called).  One test
+// on the lane's packed maximum; lanes that pass mark which of their four vectors hold a candidate,
+// and then all of them stage their next marked vector together, whichever of the four it is, so
+// that the push runs once per round for the whole warp (almost always a single round).
 __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, int lane_vec0,
-                                            uint32_t sh_addr) {
+                                            const StageRef& st) {
     const uint32_t P2 = th.P2;
     if (bf16x2_max(lt.lane_max2(), P2) != P2) {
+        uint32_t mask = 0;
 #pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j)
-            if (bf16x2_max(lt.vm[j], P2) != P2)
-                push_vector(sh_addr, make_uint4(lt.w[4 * j], lt.w[4 * j + 1], lt.w[4 * j + 2], lt.w[4 * j + 3]),
-                            lane_vec0 + j * 32, lt.vec_max(j));
+        for (int j = 0; j < kVecsPerLane; ++j) mask |= (bf16x2_max(lt.vm[j], P2) != P2) ? (1u << j) : 0u;
+        while (mask) {
+            const int j = __ffs(mask) - 1;
+            mask &= mask - 1;
+            uint4 v = make_uint4(lt.w[0], lt.w[1], lt.w[2], lt.w[3]);
+            uint32_t m2 = lt.vm[0];
+            if (j == 1) { v = make_uint4(lt.w[4], lt.w[5], lt.w[6], lt.w[7]); m2 = lt.vm[1]; }
+            if (j == 2) { v = make_uint4(lt.w[8], lt.w[9], lt.w[10], lt.w[11]); m2 = lt.vm[2]; }
+            if (j == 3) { v = make_uint4(lt.w[12], lt.w[13], lt.w[14], lt.w[15]); m2 = lt.vm[3]; }
+            push_vector(st.smem, st.sh_addr, st.caps, v, lane_vec0 + j * 32,
+                        fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
+        }
     }
 }
 __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, int lane_vec0,
-                                            uint32_t sh_addr) {
+                                            const StageRef& st) {
     const float thr = th.edge;
     if (fmaxf(fmaxf(lt.vm[0], lt.vm[1]), fmaxf(lt.vm[2], lt.vm[3])) >= thr) {
+        uint32_t mask = 0;
 #pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j)
-            if (lt.vm[j] >= thr)
-                push_vector(sh_addr,
-                            make_uint4(__float_as_uint(lt.z[4 * j]), __float_as_uint(lt.z[4 * j + 1]),
-                                       __float_as_uint(lt.z[4 * j + 2]), __float_as_uint(lt.z[4 * j + 3])),
-                            lane_vec0 + j * 32, lt.vm[j]);
+        for (int j = 0; j < kVecsPerLane; ++j) mask |= (lt.vm[j] >= thr) ? (1u << j) : 0u;
+        while (mask) {
+            const int j = __ffs(mask) - 1;
+            mask &= mask - 1;
+            float a = lt.z[0], b = lt.z[1], c = lt.z[2], d = lt.z[3], m = lt.vm[0];
+            if (j == 1) { a = lt.z[4]; b = lt.z[5]; c = lt.z[6]; d = lt.z[7]; m = lt.vm[1]; }
+            if (j == 2) { a = lt.z[8]; b = lt.z[9]; c = lt.z[10]; d = lt.z[11]; m = lt.vm[2]; }
+            if (j == 3) { a = lt.z[12]; b = lt.z[13]; c = lt.z[14]; d = lt.z[15]; m = lt.vm[3]; }
+            push_vector(st.smem, st.sh_addr, st.caps,
+                        make_uint4(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d)),
+                        lane_vec0 + j * 32, m);
+        }
     }
 }
 
 // All threads: turn the staged vectors into (key, index) candidates, keeping the logits whose bin
 // is >= bin, and empty the staging buffer.  A full candidate list raises the overflow flag.
 template <typename T>
-__device__ __noinline__ void expand_staged(const uint4* vdata, const int* vidx, Candidates cb, int cap, int bin, int V,
-                                           SparsifyShared* sh, int tid) {
+__device__ __noinline__ void expand_staged(const uint4* vdata, const int* vidx, int vcap, Candidates cb, int cap,
+                                           int bin, int V, SparsifyShared* sh, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
-    const int nv = min(sh->vec_count, sh->vcap);
+    const int nv = min(sh->vec_count, vcap);
     const uint32_t min_key = (uint32_t)bin << kHistShift;
     for (int i = tid; i < nv; i += kBlockThreads) {
         const uint4 d = vdata[i];
@@ -523,7 +549,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
     SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, p.vcap, p.k));
-    const uint32_t sh_addr = smem_u32(sh);
+    const StageRef stage{smem_u32(smem_raw), smem_u32(sh), (uint32_t)p.vcap | ((uint32_t)p.vhigh << 16)};
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
@@ -540,10 +566,6 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         sh->vec_count = 0;
         sh->overflow = 0;
         sh->trim_request = 0;
-        sh->vcap = p.vcap;
-        sh->vhigh = p.vhigh;
-        sh->vdata_addr = smem_u32(vec_data);
-        sh->vidx_addr = smem_u32(vec_idx);
         sh->hist_addr = smem_u32(hist);
         sh->coarse_addr = smem_u32(coarse);
     }
@@ -598,7 +620,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             if (lm > ls.zmax) ls.raise(lm, c);
             lt.accumulate(ls, c);
             const Threshold<T> th(*(volatile int*)&sh->thr_bin);
-            filter_push(lt, th, ch * kVecsPerChunk + lane, sh_addr);
+            filter_push(lt, th, ch * kVecsPerChunk + lane, stage);
             if ((step & (kWarps - 1)) == warp) {
                 __syncwarp();
                 raise_threshold(sh, k);
@@ -615,7 +637,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
                 if (warp == 0) raise_threshold(sh, k);
                 consumer_sync();
                 const int bin = sh->thr_bin;
-                expand_staged<T>(vec_data, vec_idx, cb, p.cap, bin, p.V, sh, tid);
+                expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, bin, p.V, sh, tid);
                 if (sh->cand_count > p.high) compact_buffer(cb, bin, sh, tid);
             }
             if (tid == 0) sh->trim_request = 0;
@@ -627,7 +649,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     if (!sh->overflow) {
         if (warp == 0) raise_threshold(sh, k);
         consumer_sync();
-        expand_staged<T>(vec_data, vec_idx, cb, p.cap, sh->thr_bin, p.V, sh, tid);
+        expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, sh->thr_bin, p.V, sh, tid);
     }
     bool hist_valid = false;  // the streaming histogram counted vector maxima only
     if (sh->overflow) {
