@@ -646,11 +646,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     }
 
     // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
-    if (!sh->overflow) {
-        if (warp == 0) raise_threshold(sh, k);
-        consumer_sync();
-        expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, sh->thr_bin, p.V, sh, tid);
-    }
+    if (!sh->overflow) expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, sh->thr_bin, p.V, sh, tid);
     bool hist_valid = false;  // the streaming histogram counted vector maxima only
     if (sh->overflow) {
         if (warp == 0) raise_threshold(sh, k);
