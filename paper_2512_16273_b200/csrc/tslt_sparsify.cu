@@ -475,17 +475,18 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
             e[j] = i < p.seg_cap ? __ldcg(&ent[i]) : make_uint2(0u, 0u);
         }
         const int n = __ldcg(&st->n);
-        double Mall = -INFINITY, Sall = 0.0, Sw[kWarps], Mw[kWarps];
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            Sw[w] = __ldcg(&st->S[w]);
-            Mw[w] = (double)__ldcg(&st->M[w]);
+        // fp64 is scarce (two warp instructions per clock per SM): one warp combines the eight
+        // per-warp pairs, one pair per lane, and leaves (M, S) in shared memory for the others
+        if (tid < 32) {
+            const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
+            const double Mw = tid < kWarps ? (double)__ldcg(&st->M[tid]) : -INFINITY;
+            const double Mall = warp_max(Sw > 0.0 ? Mw : -INFINITY);
+            const double Sall = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mall) : 0.0);
+            if (tid == 0) {
+                sh->scratch[0] = Mall;
+                sh->scratch[1] = Sall;
+            }
         }
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) Mall = fmax(Mall, Mw[w]);
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w)
-            if (Sw[w] > 0.0) Sall += Sw[w] * exp2(Mw[w] - Mall);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int i = tid + j * kBlockThreads;
@@ -496,22 +497,34 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
         }
         if (tid == 0) sh->cand_count = n;
         consumer_sync();
-        *Mrow = Mall;
-        *Srow = Sall;
+        *Mrow = sh->scratch[0];
+        *Srow = sh->scratch[1];
+        consumer_sync();
         return;
     }
     if (tid == 0) sh->cand_count = 0;
     consumer_sync();
-    double Mall = -INFINITY;
-    for (int g = 0; g < nseg; ++g)
-        for (int w = 0; w < kWarps; ++w) Mall = fmax(Mall, (double)__ldcg(&p.seg_stats[slot0 + g].M[w]));
-    double Sall = 0.0;
+    if (tid < 32) {  // one warp combines the nseg * 8 per-warp pairs (fp64 is scarce)
+        double Mall = -INFINITY;
+        for (int i = tid; i < nseg * kWarps; i += 32) {
+            const SegStat* st = &p.seg_stats[slot0 + i / kWarps];
+            if (__ldcg(&st->S[i % kWarps]) > 0.0) Mall = fmax(Mall, (double)__ldcg(&st->M[i % kWarps]));
+        }
+        Mall = warp_max(Mall);
+        double Sall = 0.0;
+        for (int i = tid; i < nseg * kWarps; i += 32) {
+            const SegStat* st = &p.seg_stats[slot0 + i / kWarps];
+            const double Sw = __ldcg(&st->S[i % kWarps]);
+            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st->M[i % kWarps]) - Mall);
+        }
+        Sall = warp_sum(Sall);
+        if (tid == 0) {
+            sh->scratch[0] = Mall;
+            sh->scratch[1] = Sall;
+        }
+    }
     for (int g = 0; g < nseg; ++g) {
         const SegStat* st = &p.seg_stats[slot0 + g];
-        for (int w = 0; w < kWarps; ++w) {
-            const double Sw = __ldcg(&st->S[w]);
-            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st->M[w]) - Mall);
-        }
         const int ng = __ldcg(&st->n);
         const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
         const int base = sh->cand_count;
@@ -524,8 +537,9 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
         if (tid == 0) sh->cand_count = base + ng;
         consumer_sync();
     }
-    *Mrow = Mall;
-    *Srow = Sall;
+    *Mrow = sh->scratch[0];
+    *Srow = sh->scratch[1];
+    consumer_sync();
 }
 
 // kHandOff = false: one launch does everything; the segments of a split row meet through a ticket.
@@ -671,10 +685,20 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             sh->scratch[kWarps + warp] = Sw;
         }
         consumer_sync();
+        if (tid < 32) {  // one warp combines the eight pairs (fp64 is scarce)
+            const double Sx = tid < kWarps ? sh->scratch[kWarps + tid] : 0.0;
+            const double Mx = tid < kWarps ? sh->scratch[tid] : -INFINITY;
+            const double Mall = warp_max(Sx > 0.0 ? Mx : -INFINITY);
+            const double Sall = warp_sum(Sx > 0.0 ? Sx * exp2(Mx - Mall) : 0.0);
+            __syncwarp();
+            if (tid == 0) {
+                sh->scratch[0] = Mall;
+                sh->scratch[1] = Sall;
+            }
+        }
+        consumer_sync();
         Mrow = sh->scratch[0];
-        for (int w = 1; w < kWarps; ++w) Mrow = fmax(Mrow, sh->scratch[w]);
-        for (int w = 0; w < kWarps; ++w)
-            if (sh->scratch[kWarps + w] > 0.0) Srow += sh->scratch[kWarps + w] * exp2(sh->scratch[w] - Mrow);
+        Srow = sh->scratch[1];
         consumer_sync();
     }
 
@@ -839,7 +863,9 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
         consumer_sync();
     }
 
-    const double L2 = Mrow + log2(Srow);  // base-2 log of the softmax normaliser
+    if (tid == 0) sh->scratch[2] = Mrow + log2(Srow);  // base-2 log of the softmax normaliser (once: fp64 is scarce)
+    consumer_sync();
+    const double L2 = sh->scratch[2];
     const double cd = p.c.d;
     // the histogram and the boundary list are no longer needed: their arena holds the fp64 work arrays
     unsigned long long* comp = reinterpret_cast<unsigned long long*>(arena);          // 1024 * 8
@@ -1025,17 +1051,14 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     int nc = __ldcg(&st->n);
     float u_raw = 0.f;
     if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];
-    double Mrow = -INFINITY, Srow = 0.0, Sw[kWarps], Mw[kWarps];
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        Sw[w] = __ldcg(&st->S[w]);
-        Mw[w] = (double)__ldcg(&st->M[w]);
+    // the log-normaliser once, by one warp (fp64 is scarce): one per-warp pair per lane
+    if (tid < 32) {
+        const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
+        const double Mw = tid < kWarps ? (double)__ldcg(&st->M[tid]) : -INFINITY;
+        const double Mrow = warp_max(Sw > 0.0 ? Mw : -INFINITY);
+        const double Srow = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mrow) : 0.0);
+        if (tid == 0) sm.red[7] = Mrow + log2(Srow);
     }
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) Mrow = fmax(Mrow, Mw[w]);
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w)
-        if (Sw[w] > 0.0) Srow += Sw[w] * exp2(Mw[w] - Mrow);
     nc = nc < 0 ? 0 : (nc > kSmallCand ? kSmallCand : nc);
     if (tid < nc) { sm.key[tid] = e0.x; sm.idx[tid] = (int)e0.y; }
     if (tid + kSmallThreads < nc) { sm.key[tid + kSmallThreads] = e1.x; sm.idx[tid + kSmallThreads] = (int)e1.y; }
@@ -1055,7 +1078,7 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     }
     small_sync();
     const int n0 = nc < k ? nc : k;
-    const double L2 = Mrow + log2(Srow);
+    const double L2 = sm.red[7];  // written before the barriers above; red[0..3] serve the scans
     const double cd = p.c.d;
     // ---- nucleus cut on the cumulative q in that order ---------------------------------------------
     int n = n0;
