@@ -42,9 +42,11 @@ WORKLOAD = synth.CONFIGS[4]
 METRIC = "TSLT sparsify+verify rows/s and achieved HBM GB/s as fraction of B200 peak"
 UNIT = "rows/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
-# under profiles/ (None until a capture exists for that kernel).
-NCU_TRAFFIC_BYTES = {"sparsify_kernel": 1092.2e6, "verify_kernel": 1197.1e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each entry point's streaming kernel
+# (sparsify_kernel, verify_stream_kernel) from the ncu captures summarised under profiles/.  Each
+# entry point is two kernels on this workload (streaming, then finish / resolve: 4 launches per
+# step); the event-timed duration of an entry point covers both.
+NCU_TRAFFIC_BYTES = {"sparsify_kernel": 1098.5e6, "verify_kernel": 1189.7e6}
 
 
 def measured_peak_gbs():
@@ -395,7 +397,7 @@ def main():
                 "warmup": max(args.warmup, 3), "ms_per_step": secs_max * 1e3 / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32 (bf16 logits upcast; fp64 on the <=k candidate set)",
                 "data": "synthetic", "config": workload_config(B), "clocks": clocks, "roofline": roofline,
-                "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": 2 * args.steps}
+                "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": 4 * args.steps}
         if extras:
             line["sweep"] = extras
         print(json.dumps(line))
