@@ -234,13 +234,18 @@ __device__ __forceinline__ double row_log2_norm_warp(const float2* part, int nch
         if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
     }
     mx = warp_max(mx);
+    // fp64 is scarce (two warp instructions per clock per SM): the per-chunk factors 2^(M_c - M)
+    // are taken in fp32 (the exponents are differences of nearby chunk maxima, so the 1-ulp factor
+    // errors are ~1e-7 with random sign over hundreds of chunks); the sum is kept in fp64
     double s = 0.0;
     for (int c = lane; c < nchunks; c += 32) {
         const float2 ms = __ldcg(&part[c]);
-        if (ms.y > 0.f) s += (double)ms.y * exp2((double)ms.x - mx);
+        if (ms.y > 0.f) s += (double)(ms.y * exp2f((float)((double)ms.x - mx)));
     }
     s = warp_sum(s);
-    return s > 0.0 ? mx + log2(s) : -INFINITY;
+    double L2 = -INFINITY;
+    if (lane == 0 && s > 0.0) L2 = mx + log2(s);  // one lane: a double log2 is ~60 fp64 instructions
+    return __shfl_sync(0xffffffffu, L2, 0);
 }
 
 // One warp: acceptance probability min(1, p(x) / q~(x)) of one position, and (if wanted) the
@@ -291,8 +296,25 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
     // ---- every position on its own warp: log-normaliser of its target row, then its acceptance test
     double* L2s = A.chunkR;               // gamma + 1 entries (gamma < 1024, checked on the host)
     double* aps = A.chunkR + (gamma + 1);  // gamma entries
-    for (int j = warp; j <= gamma; j += kWarps) {
+    // (the bonus row's log-normaliser is only needed if every position is accepted or lse_p is wanted)
+    const int j_end = p.lse_p ? gamma + 1 : gamma;
+    for (int j = warp; j < j_end; j += kWarps) {
         const float2* part = p.partials + (r0 + j) * (size_t)p.nchunks;
+        if (j < gamma) {
+            // what the acceptance test will read after the log-normaliser is asked for now: the
+            // position's transmitted pairs and the target logit of its drafted token
+            const size_t dr = (size_t)b * gamma + j;
+            for (int o = lane * 32; o < p.k; o += 32 * 32) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_logit + dr * (size_t)p.k + o));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_idx + dr * (size_t)p.k + o));
+            }
+            if (lane == 0) {
+                const int x = p.draft_token[dr];
+                if (x >= 0 && x < p.V)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.logits + (long long)(r0 + j) * p.row_stride_bytes +
+                                                                   (size_t)x * Elt<T>::kBytes));
+            }
+        }
         const double L2 = row_log2_norm_warp(part, p.nchunks, lane);
         if (lane == 0) {
             L2s[j] = L2;
@@ -314,6 +336,11 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
     // ---- the leading run of accepted positions (strict <) ---------------------------------------
     int a = 0;
     while (a < gamma && (double)clamp_uniform(p.u_accept[(size_t)b * gamma + a]) < aps[a]) ++a;
+    if (a == gamma && !p.lse_p) {  // all accepted: now the bonus row is needed (uniform branch)
+        const double L2 = row_log2_norm_warp(p.partials + (r0 + gamma) * (size_t)p.nchunks, p.nchunks, lane);
+        if (tid == 0) L2s[gamma] = L2;
+        consumer_sync();
+    }
     const double L2_stop = L2s[a];
     consumer_sync();  // chunkR is reused below
     // correction token: residual of the rejected position, or the bonus row
