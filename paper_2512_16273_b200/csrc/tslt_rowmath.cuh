@@ -18,8 +18,8 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
 
 // Where a row's data ends: whole 16-byte vectors, then `rem` elements of one ragged vector.
 struct RowExtent {
-    long long nvec_full;  // number of whole vectors
-    int rem;              // elements of the ragged last vector (0 if none)
+    int nvec_full;  // number of whole vectors
+    int rem;        // elements of the ragged last vector (0 if none)
 };
 template <typename T> __host__ __device__ inline RowExtent row_extent(int V) {
     constexpr int per = 16 / Elt<T>::kBytes;
@@ -34,24 +34,30 @@ template <typename T> __host__ __device__ inline RowExtent row_extent(int V) {
 __device__ __forceinline__ void prefetch_chunk(const unsigned char* row, int ch, int chunk_end, int lane,
                                                const RowExtent& ext) {
     if (lane == 0 && ch < chunk_end) {
-        const long long v0 = (long long)ch * kVecsPerChunk;
-        long long nv = ext.nvec_full - v0;
+        const int v0 = ch * kVecsPerChunk;
+        int nv = ext.nvec_full - v0;
         if (nv > kVecsPerChunk) nv = kVecsPerChunk;
-        if (nv > 0) prefetch_l2(row + v0 * kVecBytes, (uint32_t)nv * kVecBytes);
+        if (nv > 0) prefetch_l2(row + (size_t)v0 * kVecBytes, (uint32_t)nv * kVecBytes);
     }
 }
 
-// Online softmax state of one lane: sum of 2^(z * c - M) in four packed accumulators.
+// Online softmax state of one lane: sum of 2^(z * c - M) in four packed accumulators.  The
+// reference M is raised only when a logit's exponent would exceed it by more than kRaiseSlack:
+// terms up to 2^32 are as exact in fp32 as terms below 1, and a reference that follows every new
+// maximum would be rescaled by some lane of the warp on most steps.
+constexpr float kRaiseSlack = 32.0f;
 struct LaneSum {
     float2 acc[4];
     float M;     // reference exponent (base 2), -3e38 while the lane has seen nothing finite
-    float zmax;  // largest logit seen
+    float zmax;  // logit the reference was last set from
     __device__ __forceinline__ void reset() {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] = make_float2(0.f, 0.f);
         M = -3.0e38f;
         zmax = -INFINITY;
     }
+    // does a lane tile whose largest logit is lm need a new reference first?
+    __device__ __forceinline__ bool needs_raise(float lm, float c) const { return fmaf(lm, c, -M) > kRaiseSlack; }
     // raise the reference to the exponent of a new maximum
     __device__ __forceinline__ void raise(float new_max, float c) {
         zmax = new_max;
@@ -82,7 +88,7 @@ template <> struct LaneTile<bf16_t> {
 
     // Chunk whose first vector is number vec0 of the row at `row`; vectors past the row's end read
     // as -inf, the ragged last vector is fetched element by element.
-    __device__ __forceinline__ void load(const unsigned char* row, long long vec0, int lane, const RowExtent& ext) {
+    __device__ __forceinline__ void load(const unsigned char* row, int vec0, int lane, const RowExtent& ext) {
         const uint4* base = reinterpret_cast<const uint4*>(row) + vec0 + lane;
         if (vec0 + kVecsPerChunk <= ext.nvec_full) {
 #pragma unroll
@@ -93,7 +99,7 @@ template <> struct LaneTile<bf16_t> {
         } else {
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j) {
-                const long long vi = vec0 + j * 32 + lane;
+                const int vi = vec0 + j * 32 + lane;
                 uint4 v = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf
                 if (vi < ext.nvec_full) {
                     v = ldg_stream(base + j * 32);
@@ -143,7 +149,7 @@ template <> struct LaneTile<float> {
     float z[16];
     float vm[4];  // maximum of vector j (set by reduce_max)
 
-    __device__ __forceinline__ void load(const unsigned char* row, long long vec0, int lane, const RowExtent& ext) {
+    __device__ __forceinline__ void load(const unsigned char* row, int vec0, int lane, const RowExtent& ext) {
         const uint4* base = reinterpret_cast<const uint4*>(row) + vec0 + lane;
         if (vec0 + kVecsPerChunk <= ext.nvec_full) {
 #pragma unroll
@@ -155,7 +161,7 @@ template <> struct LaneTile<float> {
         } else {
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j) {
-                const long long vi = vec0 + j * 32 + lane;
+                const int vi = vec0 + j * 32 + lane;
                 uint4 v = make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);  // -inf
                 if (vi < ext.nvec_full) {
                     v = ldg_stream(base + j * 32);

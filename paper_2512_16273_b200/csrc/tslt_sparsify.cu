@@ -418,7 +418,7 @@ __device__ __noinline__ void recollect_from_global(const unsigned char* rowp, in
     const float edge = bin_lower_edge(bin);
     for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
         LaneTile<T> lt;
-        lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+        lt.load(rowp, ch * kVecsPerChunk, lane, ext);
         if (lt.reduce_max() >= edge) {
 #pragma unroll 1
             for (int j = 0; j < kVecsPerLane; ++j) {
@@ -596,7 +596,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         const int ch0 = chunk_begin + warp;
         if (ch0 < chunk_end) {
             LaneTile<T> lt;
-            lt.load(rowp, (long long)ch0 * kVecsPerChunk, lane, ext);
+            lt.load(rowp, ch0 * kVecsPerChunk, lane, ext);
             lt.reduce_max();
             if (k <= 256) {
 #pragma unroll
@@ -628,10 +628,10 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             __syncwarp();
             if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
             LaneTile<T> lt;
-            lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+            lt.load(rowp, ch * kVecsPerChunk, lane, ext);
             prefetch_chunk(rowp, ch + kPrefetchSteps * kWarps, chunk_end, lane, ext);
             const float lm = lt.reduce_max();
-            if (lm > ls.zmax) ls.raise(lm, c);
+            if (ls.needs_raise(lm, c)) ls.raise(lm, c);
             lt.accumulate(ls, c);
             const Threshold<T> th(*(volatile int*)&sh->thr_bin);
             filter_push(lt, th, ch * kVecsPerChunk + lane, stage);

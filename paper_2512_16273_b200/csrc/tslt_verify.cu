@@ -468,7 +468,7 @@ __device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWo
     float2* part = p.partials + (size_t)wk.row * p.nchunks;
     for (int ch = wk.chunk_begin + warp; ch < wk.chunk_end; ch += kWarps) {
         LaneTile<T> lt;
-        lt.load(rowp, (long long)ch * kVecsPerChunk, lane, ext);
+        lt.load(rowp, ch * kVecsPerChunk, lane, ext);
         const float wm = warp_max(lt.reduce_max());
         LaneSum ls;
         ls.reset();

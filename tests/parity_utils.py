@@ -24,7 +24,8 @@ def close(a, b, rtol=RTOL, atol=0.0):
     a = np.asarray(a, np.float64)
     b = np.asarray(b, np.float64)
     both_inf = np.isinf(a) & np.isinf(b) & (np.sign(a) == np.sign(b))
-    ok = both_inf | (np.abs(a - b) <= atol + rtol * np.abs(b))
+    with np.errstate(invalid="ignore"):  # inf - inf where both are infinite: covered by both_inf
+        ok = both_inf | (np.abs(a - b) <= atol + rtol * np.abs(b))
     return ok
 
 

@@ -70,6 +70,67 @@ def test_many_rows_take_the_two_launch_verifier():
     assert ref["accepted_len"].max() >= 1
 
 
+def test_config4_full_size_sampled_against_oracle():
+    """The benchmark workload at full size (B = 256, gamma = 8, V = 256000, bf16: 2048 draft rows and
+    2304 target rows drawn on the GPU), in the launch configuration bench.py times (two kernels
+    per entry point).  The oracle checks a sample: every 64th draft row and every 32nd sequence."""
+    cfg = synth.CONFIGS[4]
+    B, gamma, V, k, T = cfg["B"], cfg["gamma"], cfg["V"], cfg["k"], cfg["temperature"]
+    zq, zp = synth.sequence_logits(B, gamma, V, torch.bfloat16, cfg["sigma_t"], 0, "cuda")
+    ud = synth.uniforms((B * gamma, 1), 0, synth.TID_U_DRAFT, "cuda")
+    ua = synth.uniforms((B, gamma), 0, synth.TID_U_ACCEPT, "cuda")
+    us = synth.uniforms((B,), 0, synth.TID_U_SAMPLE, "cuda")
+    for kk, top_p in ((k, 1.0), (1024, 0.95)):
+        gs = tslt.sparsify(zq, kk, top_p, T, ud)
+        gv = tslt.verify(zp, gs["idx"].view(B, gamma, kk), gs["logit"].view(B, gamma, kk), gs["count"].view(B, gamma),
+                         gs["token"].view(B, gamma), T, T, ua, us)
+        torch.cuda.synchronize()
+        assert tslt.workspace_status(gs["workspace"]) == 0 and tslt.workspace_status(gv["workspace"]) == 0
+        rows = torch.arange(0, B * gamma, 64)
+        ref_s = oracle.sparsify(zq.view(-1, V)[rows.cuda()].cpu(), kk, top_p, T, ud[rows.cuda()].cpu().numpy())
+        sub = {n: gs[n][rows.cuda()] for n in ("idx", "logit", "count", "token", "lse", "mass")}
+        compare_sparsify(sub, ref_s, "config 4 sampled rows k=%d" % kk)
+        seqs = torch.arange(0, B, 32).cuda()
+        take = lambda t: t[seqs].cpu()
+        ref_v = oracle.verify(take(zp), take(gs["idx"].view(B, gamma, kk)).numpy(), take(gs["logit"].view(B, gamma, kk)).numpy(),
+                              take(gs["count"].view(B, gamma)).numpy(), take(gs["token"].view(B, gamma)).numpy(), T, T,
+                              take(ua).numpy(), take(us).numpy())
+        subv = {n: gv[n][seqs] for n in ("accepted_len", "out_token", "accept_prob", "beta_hat", "lse_p")}
+        compare_verify(subv, ref_v, "config 4 sampled sequences k=%d" % kk)
+
+
+def test_tree_config3_full_batch_sampled():
+    """Config 3 at full size (B = 16, 640 target rows: the two-launch verifier), four sequences checked."""
+    cfg = synth.CONFIGS[3]
+    B, V, k = cfg["B"], cfg["V"], cfg["k"]
+    parent, ndr, M, depth = synth.complete_tree(cfg["expansion"])
+    N = len(parent)
+    zq, zp = synth.tree_logits(B, parent, ndr, V, torch.bfloat16, cfg["sigma_t"], 5, "cuda")
+    ud = synth.uniforms((B * M, 3), 5, synth.TID_U_DRAFT, "cuda")
+    gs = tslt.sparsify(zq, k, 1.0, 1.0, ud)
+    st = gs["token"].view(B, M, 3)
+    toks = torch.zeros(B, N, dtype=torch.int32, device="cuda")
+    for n in range(N):
+        if ndr[n] >= 0:
+            ch = [c for c in range(N) if parent[c] == n]
+            toks[:, ch] = st[:, ndr[n], :len(ch)]
+    ua = synth.uniforms((B, N), 5, synth.TID_U_ACCEPT, "cuda")
+    us = synth.uniforms((B, N), 5, synth.TID_U_SAMPLE, "cuda")
+    gt = tslt.tree_verify(zp, parent, ndr, toks, gs["idx"].view(B, M, k), gs["logit"].view(B, M, k),
+                          gs["count"].view(B, M), 1.0, 1.0, ua, us, depth)
+    torch.cuda.synchronize()
+    seqs = torch.tensor([0, 5, 10, 15]).cuda()
+    take = lambda t: t[seqs].cpu()
+    ref_s = oracle.sparsify(take(zq).reshape(-1, V), k, 1.0, 1.0, take(ud.view(B, M, 3)).reshape(-1, 3).numpy())
+    compare_sparsify({n: gs[n].view(B, M, -1)[seqs].reshape(4 * M, -1).squeeze(-1) if gs[n].dim() == 1 else
+                      gs[n].view(B, M, -1)[seqs].reshape(4 * M, -1) for n in ("idx", "logit", "count", "token", "lse", "mass")},
+                     ref_s, "config 3 sampled drafts")
+    ref_t = oracle.tree_verify(take(zp), parent, ndr, take(toks).numpy(), take(gs["idx"].view(B, M, k)).numpy(),
+                               take(gs["logit"].view(B, M, k)).numpy(), take(gs["count"].view(B, M)).numpy(), 1.0, 1.0,
+                               take(ua).numpy(), take(us).numpy(), depth)
+    compare_tree({n: gt[n][seqs] for n in ("accepted_path", "accepted_len", "out_token")}, ref_t, "config 3 sampled trees")
+
+
 def adversarial_rows(V, dtype):
     rows = []
     asc = torch.linspace(-8, 8, V)
