@@ -67,7 +67,6 @@ struct SparsifyParams {
     int vcap, vhigh;    // staged vectors: capacity and early-expansion mark
     int idx_hi_byte;
     int* status;
-    int* tickets;
     SegStat* seg_stats;
     uint2* seg_entries;  // [rows, nseg, seg_cap] (key, idx)
     int seg_cap;
@@ -82,7 +81,6 @@ struct SparsifyShared {
     // --------------------------------------------------------------------------------------------
     int cand_count;  // expanded (key, index) candidates
     int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
-    int ticket;
     int sel_bin, sel_above;  // bin of the k-th largest logit and the number of logits in higher bins
     int n_win, n_bnd;
     int warp_tot[kWarps];
@@ -542,10 +540,9 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
     consumer_sync();
 }
 
-// kHandOff = false: one launch does everything; the segments of a split row meet through a ticket.
-// kHandOff = true: every segment hands its candidates and statistics over and the CTA ends; the
+// First launch: every segment streams, hands its candidates and statistics over and ends; the
 // rows are finished by sparsify_finish_kernel, launched next on the stream.
-template <typename T, bool kHandOff>
+template <typename T>
 __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_kernel(const SparsifyParams p) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     constexpr int kPer = Elt<T>::kPerVec;
@@ -661,7 +658,6 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
 
     // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
     if (!sh->overflow) expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, sh->thr_bin, p.V, sh, tid);
-    bool hist_valid = false;  // the streaming histogram counted vector maxima only
     if (sh->overflow) {
         if (warp == 0) raise_threshold(sh, k);
         consumer_sync();
@@ -675,71 +671,31 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         consumer_sync();
     }
 
-    // ---- statistics: one (M, S) pair per warp; combined here only if this CTA finishes the row ----
+    // ---- hand-over: candidates (all at or above this segment's final threshold) and one (M, S) pair
+    // per warp; the kernel boundary publishes them to the finish kernel
     const float Mw = warp_max(ls.M);
     const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
-    double Mrow = 0.0, Srow = 0.0;
-    if (!kHandOff && wk.nseg == 1) {
-        if (lane == 0) {
-            sh->scratch[warp] = (double)Mw;
-            sh->scratch[kWarps + warp] = Sw;
-        }
-        consumer_sync();
-        if (tid < 32) {  // one warp combines the eight pairs (fp64 is scarce)
-            const double Sx = tid < kWarps ? sh->scratch[kWarps + tid] : 0.0;
-            const double Mx = tid < kWarps ? sh->scratch[tid] : -INFINITY;
-            const double Mall = warp_max(Sx > 0.0 ? Mx : -INFINITY);
-            const double Sall = warp_sum(Sx > 0.0 ? Sx * exp2(Mx - Mall) : 0.0);
-            __syncwarp();
-            if (tid == 0) {
-                sh->scratch[0] = Mall;
-                sh->scratch[1] = Sall;
-            }
-        }
-        consumer_sync();
-        Mrow = sh->scratch[0];
-        Srow = sh->scratch[1];
-        consumer_sync();
+    int n = sh->cand_count;
+    if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
+        compact_buffer(cb, sh->thr_bin, sh, tid);
+        n = sh->cand_count;
     }
-
-    // ---- segments of a split row meet through the workspace; the last to arrive goes on ------
-    if (kHandOff || wk.nseg > 1) {
-        const size_t slot0 = (size_t)row * wk.nseg;  // this row's first segment slot
-        // hand over the candidates (all at or above this segment's final threshold)
-        int n = sh->cand_count;
-        if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
-            compact_buffer(cb, sh->thr_bin, sh, tid);
-            n = sh->cand_count;
-        }
-        if (n > p.seg_cap) {  // heavy ties at the boundary: hand over the exact k
-            reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
-            n = sh->cand_count;
-        }
-        uint2* my_entries = p.seg_entries + (slot0 + wk.seg) * (size_t)p.seg_cap;
-        for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
-        SegStat* st = &p.seg_stats[slot0 + wk.seg];
-        if (lane == 0) {
-            st->S[warp] = Sw;
-            st->M[warp] = Mw;
-        }
-        if (tid == 0) st->n = n;
-        if (kHandOff) return;  // the kernel boundary publishes the hand-over
-        consumer_sync();
-        if (tid == 0) {
-            __threadfence();
-            sh->ticket = atomicAdd(&p.tickets[row], 1);
-        }
-        consumer_sync();
-        if (sh->ticket != wk.nseg - 1) return;
-        __threadfence();
-        gather_segments(p, row, wk.nseg, cb, sh, tid, &Mrow, &Srow);
-        hist_valid = false;
+    if (n > p.seg_cap) {  // heavy ties at the boundary: hand over the exact k
+        reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
+        n = sh->cand_count;
     }
-
-    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, hist_valid, tid);
+    const size_t slot = (size_t)row * wk.nseg + wk.seg;
+    uint2* my_entries = p.seg_entries + slot * (size_t)p.seg_cap;
+    for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
+    SegStat* st = &p.seg_stats[slot];
+    if (lane == 0) {
+        st->S[warp] = Sw;
+        st->M[warp] = Mw;
+    }
+    if (tid == 0) st->n = n;
 }
 
-// Second launch of the two-launch form: one CTA per row merges the row's segments and finishes it.
+// Second launch: one CTA per row merges the row's segments and finishes it.
 // Same shared-memory carve-up as the streaming kernel, with no staging buffer (vcap = 0).
 template <typename T>
 __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const SparsifyParams p) {
@@ -752,6 +708,7 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
     SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, 0, p.k));
     const int tid = threadIdx.x, row = blockIdx.x;
+    if (row == 0 && tid == 0) *p.status = 0;
     // the uniforms are needed last: ask for their cache line now
     if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) {
@@ -1042,6 +999,7 @@ template <typename T>
 __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kernel(const SparsifyParams p) {
     __shared__ SmallShared sm;
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
+    if (row == 0 && tid == 0) *p.status = 0;
     // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
     const SegStat* st = &p.seg_stats[row];
     const uint2* ent = p.seg_entries + (size_t)row * p.seg_cap;
@@ -1151,11 +1109,10 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
-    bool two_launches;  // enough rows to fill the machine: streaming kernel + finish kernel
     int nchunks, cap, high, vcap, vhigh, seg_cap;
     RowSplit split;
     size_t smem;
-    size_t ws_tickets_off, ws_stats_off, ws_entries_off, ws_bytes;
+    size_t ws_stats_off, ws_entries_off, ws_bytes;
 };
 
 static int sm_count_cached() {
@@ -1190,12 +1147,27 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (per_sm < 1) per_sm = 1;
     // a split row's segments must fit the candidate list of the CTA that merges them
     const int max_seg = pl.cap / pl.seg_cap < 16 ? pl.cap / pl.seg_cap : 16;
-    pl.two_launches = rows >= per_sm * sm_count_cached();
-    pl.split = make_row_split(rows, pl.nchunks, per_sm * sm_count_cached(), max_seg, 0);
-    const size_t split_rows = (pl.two_launches || pl.split.nseg > 1) ? (size_t)rows : 0;
+    // One CTA per row.  Only when there are fewer rows than half the SMs and the rows are long is a
+    // row cut into segments (of at least 32 chunks): every segment pays the first threshold and the
+    // hand-over, which on the benchmark's small configurations costs more than it gains.
+    (void)per_sm;
+    pl.split.rows = rows;
+    int nseg = 1;
+    if (rows > 0 && 2 * rows < sm_count_cached()) {
+        nseg = sm_count_cached() / rows;
+        if (nseg > pl.nchunks / 32) nseg = pl.nchunks / 32;
+        if (nseg > max_seg) nseg = max_seg;
+        if (nseg < 1) nseg = 1;
+    }
+    int cps = (pl.nchunks + nseg - 1) / nseg;
+    cps = (cps + kWarps - 1) / kWarps * kWarps;
+    if (cps < kWarps) cps = kWarps;
+    pl.split.nseg = (pl.nchunks + cps - 1) / cps;
+    if (pl.split.nseg < 1) pl.split.nseg = 1;
+    pl.split.cps = cps;
+    pl.split.grid = rows * pl.split.nseg;
+    const size_t split_rows = (size_t)rows;
     size_t off = kWsHeaderBytes;
-    pl.ws_tickets_off = off;
-    off = align_up(off + (size_t)rows * sizeof(int), 256);
     pl.ws_stats_off = off;
     off = align_up(off + split_rows * pl.split.nseg * sizeof(SegStat), 256);
     pl.ws_entries_off = off;
@@ -1261,32 +1233,26 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
-    p.tickets = (int*)(ws + pl.ws_tickets_off);
     p.seg_stats = (SegStat*)(ws + pl.ws_stats_off);
     p.seg_entries = (uint2*)(ws + pl.ws_entries_off);
 
     cudaStream_t st = (cudaStream_t)stream;
-    // status word and tickets start at zero
-    if (cudaMemsetAsync(ws, 0, pl.ws_stats_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
-    auto kern = dtype == TSLT_F32 ? (pl.two_launches ? sparsify_kernel<float, true> : sparsify_kernel<float, false>)
-                                  : (pl.two_launches ? sparsify_kernel<bf16_t, true> : sparsify_kernel<bf16_t, false>);
+    auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sparsify_smem_bytes(4096, 2048, TSLT_MAX_K)) != cudaSuccess)
         return TSLT_ERR_CUDA;
     kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
-    if (pl.two_launches) {
+    if (pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallThreads) {
+        if (dtype == TSLT_F32) sparsify_finish_small_kernel<float><<<rows, kSmallThreads, 0, st>>>(p);
+        else sparsify_finish_small_kernel<bf16_t><<<rows, kSmallThreads, 0, st>>>(p);
+    } else {
         auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
         if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
             return TSLT_ERR_CUDA;
-        if (pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallThreads) {
-            if (dtype == TSLT_F32) sparsify_finish_small_kernel<float><<<rows, kSmallThreads, 0, st>>>(p);
-            else sparsify_finish_small_kernel<bf16_t><<<rows, kSmallThreads, 0, st>>>(p);
-        } else {
-            fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
-        }
-        if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+        fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
     }
+    if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }
