@@ -1022,17 +1022,20 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     if (tid + kSmallThreads < nc) { sm.key[tid + kSmallThreads] = e1.x; sm.idx[tid + kSmallThreads] = (int)e1.y; }
     small_sync();
     // ---- exact top-k by counting ranks under (key descending, index ascending) -------------------
-    {
-        int r0 = 0, r1 = 0;
-        const int i1 = tid + kSmallThreads;
-        for (int j = 0; j < nc; ++j) {
-            const uint32_t kj = sm.key[j];
-            const int ij = sm.idx[j];
-            r0 += (kj > e0.x || (kj == e0.x && ij < (int)e0.y)) ? 1 : 0;
-            r1 += (kj > e1.x || (kj == e1.x && ij < (int)e1.y)) ? 1 : 0;
-        }
-        if (tid < nc && r0 < k) { sm.wkey[r0] = e0.x; sm.widx[r0] = (int)e0.y; }
-        if (i1 < nc && r1 < k) { sm.wkey[r1] = e1.x; sm.widx[r1] = (int)e1.y; }
+    // (only the threads that hold a candidate count; the 64-bit composite makes it one compare per entry)
+    if (tid < nc) {
+        const unsigned long long mine = ((unsigned long long)e0.x << 32) | (unsigned long long)(0xffffffffu - e0.y);
+        int r0 = 0;
+        for (int j = 0; j < nc; ++j)
+            r0 += ((((unsigned long long)sm.key[j] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)sm.idx[j])) > mine) ? 1 : 0;
+        if (r0 < k) { sm.wkey[r0] = e0.x; sm.widx[r0] = (int)e0.y; }
+    }
+    if (tid + kSmallThreads < nc) {
+        const unsigned long long mine = ((unsigned long long)e1.x << 32) | (unsigned long long)(0xffffffffu - e1.y);
+        int r1 = 0;
+        for (int j = 0; j < nc; ++j)
+            r1 += ((((unsigned long long)sm.key[j] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)sm.idx[j])) > mine) ? 1 : 0;
+        if (r1 < k) { sm.wkey[r1] = e1.x; sm.widx[r1] = (int)e1.y; }
     }
     small_sync();
     const int n0 = nc < k ? nc : k;
