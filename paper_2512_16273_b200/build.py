@@ -12,7 +12,7 @@ LIB = os.path.join(HERE, "libtslt.so")
 SOURCES = ["tslt_api.cu", "tslt_sparsify.cu", "tslt_verify.cu"]
 HEADERS = ["tslt_common.cuh", "tslt_rowmath.cuh", "tslt_select.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared", "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC", "-shared"]
 
 
 def _nvcc() -> str:
@@ -35,7 +35,7 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = list(NVCC_FLAGS)
     if verbose:
         flags += ["-Xptxas", "-v"]
     tmp = LIB + ".tmp%d" % os.getpid()

@@ -396,7 +396,7 @@ __device__ __noinline__ void compact_buffer(Candidates cb, int bin, SparsifyShar
 
 template <typename T>
 __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* arena, double Mrow, double Srow, bool hist_valid, int tid);
+                                          unsigned char* arena, double Mrow, double Srow, int tid);
 
 // All threads: second pass over a segment whose buffers overflowed.  The histogram went on counting,
 // so the final threshold is as tight as ever: read the segment again and append every logit whose
@@ -719,7 +719,7 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
     double Mrow, Srow;
     gather_segments(p, row, p.split.nseg, cb, sh, tid, &Mrow, &Srow);
-    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, false, tid);
+    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, tid);
 }
 
 // Position of entry (key, idx) of the buffer in the order (key descending, idx ascending) /
@@ -742,7 +742,7 @@ __device__ __forceinline__ int rank_by_idx(const int* idx, int n, int my_idx) {
 // Exact top-k of the row, nucleus cut, renormalisation, sampling and the ascending-index payload.
 template <typename T>
 __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* arena, double Mrow, double Srow, bool hist_valid, int tid) {
+                                          unsigned char* arena, double Mrow, double Srow, int tid) {
     constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
     const int k = p.k;
     const int lane = tid & 31, warp = tid >> 5;
@@ -753,13 +753,12 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     const int nc = sh->cand_count;
 
     // ---- the bin of the k-th largest logit ------------------------------------------------------
-    if (!hist_valid) {
-        for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
-        consumer_sync();
-        for (int i = tid; i < nc; i += kBlockThreads)
-            hist_count(sh->hist_addr, sh->coarse_addr, (int)(cand_key[i] >> kHistShift), 1u);
-        consumer_sync();
-    }
+    // exact counts of the candidates (the streaming histogram only counted vector maxima)
+    for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+    consumer_sync();
+    for (int i = tid; i < nc; i += kBlockThreads)
+        hist_count(sh->hist_addr, sh->coarse_addr, (int)(cand_key[i] >> kHistShift), 1u);
+    consumer_sync();
     if (warp == 0) {
         uint32_t above;
         const int b = scan_boundary(sh->hist_addr, sh->coarse_addr, k, &above);
