@@ -81,6 +81,31 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// An entry point is a streaming kernel followed by a finish / resolve kernel on the same stream.
+// The second kernel is launched with programmatic stream serialization: its CTAs may be placed on
+// SMs that the first kernel's last wave leaves free, and wait at their very first instruction
+// until the first kernel has completed and its writes are visible.  The first kernel allows that
+// as soon as it starts.  (Launched without the attribute, both instructions do nothing.)
+__device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_primary_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename Params>
+inline cudaError_t launch_dependent(void (*kernel)(const Params), unsigned grid, unsigned block, size_t smem,
+                                    cudaStream_t st, const Params& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 // ---- small math --------------------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

@@ -570,6 +570,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     const int k = p.k;
     const float c = p.c.f;
 
+    allow_dependent_launch();
     for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
     if (tid == 0) {
         sh->thr_bin = kLowestFiniteBin;
@@ -708,7 +709,6 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
     SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, 0, p.k));
     const int tid = threadIdx.x, row = blockIdx.x;
-    if (row == 0 && tid == 0) *p.status = 0;
     // the uniforms are needed last: ask for their cache line now
     if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) {
@@ -716,6 +716,8 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
         sh->coarse_addr = smem_u32(hist + kHistBins);
         sh->overflow = 0;
     }
+    wait_for_primary_kernel();  // nothing the streaming kernel wrote is read before this point
+    if (row == 0 && tid == 0) *p.status = 0;
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
     double Mrow, Srow;
     gather_segments(p, row, p.split.nseg, cb, sh, tid, &Mrow, &Srow);
@@ -998,6 +1000,9 @@ template <typename T>
 __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kernel(const SparsifyParams p) {
     __shared__ SmallShared sm;
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
+    float u_raw = 0.f;
+    if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];  // an input: may be read early
+    wait_for_primary_kernel();  // nothing the streaming kernel wrote is read before this point
     if (row == 0 && tid == 0) *p.status = 0;
     // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
     const SegStat* st = &p.seg_stats[row];
@@ -1006,8 +1011,6 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     if (tid < p.seg_cap) e0 = __ldcg(&ent[tid]);
     if (tid + kSmallThreads < p.seg_cap) e1 = __ldcg(&ent[tid + kSmallThreads]);
     int nc = __ldcg(&st->n);
-    float u_raw = 0.f;
-    if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];
     // the log-normaliser once, by one warp (fp64 is scarce): one per-warp pair per lane
     if (tid < 32) {
         const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
@@ -1246,14 +1249,15 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     if (pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallThreads) {
-        if (dtype == TSLT_F32) sparsify_finish_small_kernel<float><<<rows, kSmallThreads, 0, st>>>(p);
-        else sparsify_finish_small_kernel<bf16_t><<<rows, kSmallThreads, 0, st>>>(p);
+        auto fin = dtype == TSLT_F32 ? sparsify_finish_small_kernel<float> : sparsify_finish_small_kernel<bf16_t>;
+        if (launch_dependent(fin, rows, kSmallThreads, 0, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     } else {
         auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
         if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
             return TSLT_ERR_CUDA;
-        fin<<<rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st>>>(p);
+        if (launch_dependent(fin, rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st, p) != cudaSuccess)
+            return TSLT_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;

@@ -512,6 +512,7 @@ constexpr int kStreamCtasPerSm = 6;  // streaming-only kernel: 42 registers per 
 // ticket, no fence: the kernel boundary publishes the partials) ...
 template <typename T>
 __global__ void __launch_bounds__(kBlockThreads, kStreamCtasPerSm) verify_stream_kernel(const VerifyParams p) {
+    allow_dependent_launch();
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
     stream_chunks<T>(p, wk, threadIdx.x & 31, threadIdx.x >> 5);
 }
@@ -521,6 +522,7 @@ __global__ void __launch_bounds__(kBlockThreads, 4) verify_resolve_kernel(const 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* arena = smem_raw;
     VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
+    wait_for_primary_kernel();  // the partials come from the streaming kernel
     if (kTree) resolve_tree<T>(p, blockIdx.x, arena, sh, threadIdx.x);
     else resolve_sequence<T>(p, blockIdx.x, arena, sh, threadIdx.x);
 }
@@ -602,8 +604,7 @@ static int launch_verify(VerifyParams& p, const VerifyPlan& pl, int dtype, cudaS
     if (dtype == TSLT_F32) verify_stream_kernel<float><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     else verify_stream_kernel<bf16_t><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
-    resolve<<<(unsigned)p.B, kBlockThreads, pl.smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+    return launch_dependent(resolve, (unsigned)p.B, kBlockThreads, pl.smem, st, p) == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
 }
 
 }  // namespace tslt
