@@ -73,7 +73,7 @@ struct SparsifyParams {
 };
 
 struct SparsifyShared {
-    // ---- written by push_vector through their shared-space addresses ---------------------------------
+    // ---- written by stage_vector through their shared-space addresses --------------------------------
     int vec_count;   // staged vectors
     int overflow;    // a buffer was found full: its contents are no longer complete
     int trim_request;
@@ -91,9 +91,9 @@ struct SparsifyShared {
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // shared-memory carve-up (dynamic):
-//   arena | vec_data[vcap] | vec_idx[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k] | SparsifyShared
+//   arena | staged[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k] | SparsifyShared
 __host__ __device__ inline size_t sparsify_shared_off(int cap, int vcap, int k) {
-    return align_up((size_t)kArenaBytes + (size_t)vcap * 20 + (size_t)cap * 8 + (size_t)k * 8, 16);
+    return align_up((size_t)kArenaBytes + (size_t)vcap * 8 + (size_t)cap * 8 + (size_t)k * 8, 16);
 }
 __host__ __device__ inline size_t sparsify_smem_bytes(int cap, int vcap, int k) {
     return sparsify_shared_off(cap, vcap, k) + align_up(sizeof(SparsifyShared), 16);
@@ -142,35 +142,30 @@ __device__ __forceinline__ void hist_count(uint32_t hist_addr, uint32_t coarse_a
     reds_add(coarse_addr + 4u * (uint32_t)(bin >> 5), delta);
 }
 
-__device__ __forceinline__ void sts_v4(uint32_t addr, const uint4& v) {
-    asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
+__device__ __forceinline__ void sts_v2(uint32_t addr, uint32_t x, uint32_t y) {
+    asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
 }
 
-// Where the staging buffer and the histograms of this CTA are, as the out-of-line push wants it:
-// everything sits at fixed offsets of the CTA's dynamic shared memory.
+// Where the staging buffer and the histograms of this CTA are: everything sits at fixed offsets of
+// the CTA's dynamic shared memory, addressed in the shared space.
 struct StageRef {
     uint32_t smem;     // shared-space address of the dynamic shared memory (the fine histogram)
     uint32_t sh_addr;  // shared-space address of the SparsifyShared block
     uint32_t caps;     // vcap | vhigh << 16
 };
 
-// Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax, and count
-// that logit.  Out of line on purpose: it is rare, and inlined copies of it in the streaming
-// loop would not fit the instruction cache.  All its operands arrive in registers.
-__device__ __noinline__ void push_vector(uint32_t smem, uint32_t sh_addr, uint32_t caps, uint4 data, int vec_index,
-                                         float vmax) {
-    const uint32_t vcap = caps & 0xffffu, vhigh = caps >> 16;
-    const uint32_t pos = atoms_add(sh_addr + offsetof(SparsifyShared, vec_count), 1u);
-    hist_count(smem, smem + 4u * kHistBins, (int)(float_to_key(vmax) >> kHistShift), 1u);
-    const uint32_t vdata = smem + kArenaBytes;
-    if (pos < vcap) {
-        sts_v4(vdata + 16u * pos, data);
-        sts_u32(vdata + 16u * vcap + 4u * pos, (uint32_t)vec_index);
-    } else {
-        sts_u32(sh_addr + offsetof(SparsifyShared, overflow), 1u);
-    }
-    if (pos + 1u == vhigh) sts_u32(sh_addr + offsetof(SparsifyShared, trim_request), 1u);
+// Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax: only its
+// number and the key of that logit are kept (8 bytes), and the logit is counted.  The vector's
+// data is read again from global memory when the staged vectors are expanded, and only if its
+// largest logit still passes the threshold of that moment: a fraction of the staged vectors.
+__device__ __forceinline__ void stage_vector(const StageRef& st, int vec_index, float vmax) {
+    const uint32_t vcap = st.caps & 0xffffu, vhigh = st.caps >> 16;
+    const uint32_t pos = atoms_add(st.sh_addr + offsetof(SparsifyShared, vec_count), 1u);
+    const uint32_t key = float_to_key(vmax);
+    hist_count(st.smem, st.smem + 4u * kHistBins, (int)(key >> kHistShift), 1u);
+    if (pos < vcap) sts_v2(st.smem + kArenaBytes + 8u * pos, (uint32_t)vec_index, key);
+    else sts_u32(st.sh_addr + offsetof(SparsifyShared, overflow), 1u);
+    if (pos + 1u == vhigh) sts_u32(st.sh_addr + offsetof(SparsifyShared, trim_request), 1u);
 }
 
 // One warp: the highest fine bin b with (number of counted logits in bins >= b) >= k, or -1 if
@@ -264,7 +259,7 @@ template <> struct Threshold<bf16_t> {
 // Stage the vectors of a lane tile that hold a candidate (reduce_max() already called).  One test
 // on the lane's packed maximum; lanes that pass mark which of their four vectors hold a candidate,
 // and then all of them stage their next marked vector together, whichever of the four it is, so
-// that the push runs once per round for the whole warp (almost always a single round).
+// that the staging code runs once per round for the whole warp (almost always a single round).
 __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, int lane_vec0,
                                             const StageRef& st) {
     const uint32_t P2 = th.P2;
@@ -275,13 +270,11 @@ __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Th
         while (mask) {
             const int j = __ffs(mask) - 1;
             mask &= mask - 1;
-            uint4 v = make_uint4(lt.w[0], lt.w[1], lt.w[2], lt.w[3]);
             uint32_t m2 = lt.vm[0];
-            if (j == 1) { v = make_uint4(lt.w[4], lt.w[5], lt.w[6], lt.w[7]); m2 = lt.vm[1]; }
-            if (j == 2) { v = make_uint4(lt.w[8], lt.w[9], lt.w[10], lt.w[11]); m2 = lt.vm[2]; }
-            if (j == 3) { v = make_uint4(lt.w[12], lt.w[13], lt.w[14], lt.w[15]); m2 = lt.vm[3]; }
-            push_vector(st.smem, st.sh_addr, st.caps, v, lane_vec0 + j * 32,
-                        fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
+            if (j == 1) m2 = lt.vm[1];
+            if (j == 2) m2 = lt.vm[2];
+            if (j == 3) m2 = lt.vm[3];
+            stage_vector(st, lane_vec0 + j * 32, fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
         }
     }
 }
@@ -295,41 +288,62 @@ __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Thr
         while (mask) {
             const int j = __ffs(mask) - 1;
             mask &= mask - 1;
-            float a = lt.z[0], b = lt.z[1], c = lt.z[2], d = lt.z[3], m = lt.vm[0];
-            if (j == 1) { a = lt.z[4]; b = lt.z[5]; c = lt.z[6]; d = lt.z[7]; m = lt.vm[1]; }
-            if (j == 2) { a = lt.z[8]; b = lt.z[9]; c = lt.z[10]; d = lt.z[11]; m = lt.vm[2]; }
-            if (j == 3) { a = lt.z[12]; b = lt.z[13]; c = lt.z[14]; d = lt.z[15]; m = lt.vm[3]; }
-            push_vector(st.smem, st.sh_addr, st.caps,
-                        make_uint4(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d)),
-                        lane_vec0 + j * 32, m);
+            float m = lt.vm[0];
+            if (j == 1) m = lt.vm[1];
+            if (j == 2) m = lt.vm[2];
+            if (j == 3) m = lt.vm[3];
+            stage_vector(st, lane_vec0 + j * 32, m);
         }
     }
 }
 
-// All threads: turn the staged vectors into (key, index) candidates, keeping the logits whose bin
-// is >= bin, and empty the staging buffer.  A full candidate list raises the overflow flag.
+// All threads: turn the staged vectors whose largest logit is in a bin >= bin into (key, index)
+// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  The vectors
+// come back from global memory (L2 or HBM), four loads in flight per thread.  A full candidate
+// list raises the overflow flag.
 template <typename T>
-__device__ __noinline__ void expand_staged(const uint4* vdata, const int* vidx, int vcap, Candidates cb, int cap,
-                                           int bin, int V, SparsifyShared* sh, int tid) {
+__device__ __noinline__ void expand_staged(const uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
+                                           Candidates cb, int cap, int bin, int V, SparsifyShared* sh, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
+    constexpr int kInFlight = 4;
     const int nv = min(sh->vec_count, vcap);
     const uint32_t min_key = (uint32_t)bin << kHistShift;
-    for (int i = tid; i < nv; i += kBlockThreads) {
-        const uint4 d = vdata[i];
-        const int e0 = vidx[i] * kPer;
-        float z[kPer];
-        unpack_vec<T>(d, z);
+    for (int base = 0; base < nv; base += kInFlight * kBlockThreads) {
+        uint4 d[kInFlight];
+        int vi[kInFlight];
 #pragma unroll
-        for (int e = 0; e < kPer; ++e) {
-            if (z[e] >= -3.4028234e38f && e0 + e < V) {
-                const uint32_t kk = float_to_key(z[e]);
-                if (kk >= min_key) {
-                    const int pos = atomicAdd(cb.count, 1);
-                    if (pos < cap) {
-                        cb.key[pos] = kk;
-                        cb.idx[pos] = e0 + e;
-                    } else {
-                        sh->overflow = 1;
+        for (int u = 0; u < kInFlight; ++u) {
+            const int i = base + u * kBlockThreads + tid;
+            vi[u] = -1;
+            if (i < nv) {
+                const uint2 s = staged[i];
+                if (s.y >= min_key) vi[u] = (int)s.x;
+            }
+            if (vi[u] >= 0 && vi[u] < ext.nvec_full) d[u] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            if (vi[u] < 0) continue;
+            const int e0 = vi[u] * kPer;
+            float z[kPer];
+            if (vi[u] < ext.nvec_full) {
+                unpack_vec<T>(d[u], z);
+            } else {  // the row's ragged last vector: element by element
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) z[e] = e0 + e < V ? Elt<T>::load(rowp, e0 + e) : -INFINITY;
+            }
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                if (z[e] >= -3.4028234e38f) {
+                    const uint32_t kk = float_to_key(z[e]);
+                    if (kk >= min_key) {
+                        const int pos = atomicAdd(cb.count, 1);
+                        if (pos < cap) {
+                            cb.key[pos] = kk;
+                            cb.idx[pos] = e0 + e;
+                        } else {
+                            sh->overflow = 1;
+                        }
                     }
                 }
             }
@@ -553,9 +567,8 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     unsigned char* arena = smem_raw;
     uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
     uint32_t* coarse = hist + kHistBins;
-    uint4* vec_data = reinterpret_cast<uint4*>(arena + kArenaBytes);
-    int* vec_idx = reinterpret_cast<int*>(vec_data + p.vcap);
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(vec_idx + p.vcap);
+    uint2* staged = reinterpret_cast<uint2*>(arena + kArenaBytes);
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(staged + p.vcap);
     int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
     uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
@@ -649,7 +662,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
                 if (warp == 0) raise_threshold(sh, k);
                 consumer_sync();
                 const int bin = sh->thr_bin;
-                expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, bin, p.V, sh, tid);
+                expand_staged<T>(staged, p.vcap, rowp, ext, cb, p.cap, bin, p.V, sh, tid);
                 if (sh->cand_count > p.high) compact_buffer(cb, bin, sh, tid);
             }
             if (tid == 0) sh->trim_request = 0;
@@ -658,7 +671,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     }
 
     // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
-    if (!sh->overflow) expand_staged<T>(vec_data, vec_idx, p.vcap, cb, p.cap, sh->thr_bin, p.V, sh, tid);
+    if (!sh->overflow) expand_staged<T>(staged, p.vcap, rowp, ext, cb, p.cap, sh->thr_bin, p.V, sh, tid);
     if (sh->overflow) {
         if (warp == 0) raise_threshold(sh, k);
         consumer_sync();
