@@ -49,24 +49,23 @@ constexpr float kRaiseSlack = 32.0f;
 struct LaneSum {
     float2 acc[4];
     float M;     // reference exponent (base 2), -3e38 while the lane has seen nothing finite
-    float zmax;  // logit the reference was last set from
     __device__ __forceinline__ void reset() {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] = make_float2(0.f, 0.f);
         M = -3.0e38f;
-        zmax = -INFINITY;
     }
-    // does a lane tile whose largest logit is lm need a new reference first?
-    __device__ __forceinline__ bool needs_raise(float lm, float c) const { return fmaf(lm, c, -M) > kRaiseSlack; }
-    // raise the reference to the exponent of a new maximum
-    __device__ __forceinline__ void raise(float new_max, float c) {
-        zmax = new_max;
-        const float Mn = new_max * c;
-        const float sc = ex2_approx(M - Mn);
+    // Before a lane tile whose largest logit is lm is added: move the reference to lm's exponent if
+    // that exceeds it by more than the slack.  Branch-free on purpose: the scale is exactly 1 when
+    // nothing moves, and the compiler turns a rarely taken branch here into a longer chain of
+    // selects executed on every step.
+    __device__ __forceinline__ void raise_to(float lm, float c) {
+        const float Mn = lm * c;
+        const bool up = Mn - M > kRaiseSlack;
+        const float sc = up ? ex2_approx(M - Mn) : 1.0f;
         const float2 sc2 = make_float2(sc, sc);
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] = __fmul2_rn(acc[i], sc2);
-        M = Mn;
+        M = up ? Mn : M;
     }
     __device__ __forceinline__ float total() const {
         return ((acc[0].x + acc[0].y) + (acc[1].x + acc[1].y)) + ((acc[2].x + acc[2].y) + (acc[3].x + acc[3].y));

@@ -77,10 +77,10 @@ struct SparsifyShared {
     int vec_count;   // staged vectors
     int overflow;    // a buffer was found full: its contents are no longer complete
     int trim_request;
-    uint32_t hist_addr, coarse_addr;  // shared-space addresses of the two histogram levels
     // --------------------------------------------------------------------------------------------
     int cand_count;  // expanded (key, index) candidates
     int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
+    uint32_t thr_word;  // thr_bin << 16 | the bf16 pattern the packed lane-tile test compares with; only ever rises
     int sel_bin, sel_above;  // bin of the k-th largest logit and the number of logits in higher bins
     int n_win, n_bnd;
     int warp_tot[kWarps];
@@ -91,12 +91,15 @@ struct SparsifyShared {
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // shared-memory carve-up (dynamic):
-//   arena | staged[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k] | SparsifyShared
-__host__ __device__ inline size_t sparsify_shared_off(int cap, int vcap, int k) {
-    return align_up((size_t)kArenaBytes + (size_t)vcap * 8 + (size_t)cap * 8 + (size_t)k * 8, 16);
-}
+//   SparsifyShared | arena | staged[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k]
+// The control block, the histograms and the staging buffer sit at compile-time offsets of the
+// CTA's shared memory, so the streaming loop holds no address of them in a register.
+constexpr uint32_t kSharedBlockBytes = (sizeof(SparsifyShared) + 127) / 128 * 128;
+constexpr uint32_t kHistOff = kSharedBlockBytes;
+constexpr uint32_t kCoarseOff = kHistOff + 4u * kHistBins;
+constexpr uint32_t kStagedOff = kHistOff + kArenaBytes;
 __host__ __device__ inline size_t sparsify_smem_bytes(int cap, int vcap, int k) {
-    return sparsify_shared_off(cap, vcap, k) + align_up(sizeof(SparsifyShared), 16);
+    return align_up((size_t)kStagedOff + (size_t)vcap * 8 + (size_t)cap * 8 + (size_t)k * 8, 16);
 }
 
 // Sources for select_topk: the candidate buffer, or a run of logits in global memory.
@@ -146,26 +149,18 @@ __device__ __forceinline__ void sts_v2(uint32_t addr, uint32_t x, uint32_t y) {
     asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
 }
 
-// Where the staging buffer and the histograms of this CTA are: everything sits at fixed offsets of
-// the CTA's dynamic shared memory, addressed in the shared space.
-struct StageRef {
-    uint32_t smem;     // shared-space address of the dynamic shared memory (the fine histogram)
-    uint32_t sh_addr;  // shared-space address of the SparsifyShared block
-    uint32_t caps;     // vcap | vhigh << 16
-};
-
 // Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax: only its
 // number and the key of that logit are kept (8 bytes), and the logit is counted.  The vector's
 // data is read again from global memory when the staged vectors are expanded, and only if its
 // largest logit still passes the threshold of that moment: a fraction of the staged vectors.
-__device__ __forceinline__ void stage_vector(const StageRef& st, int vec_index, float vmax) {
-    const uint32_t vcap = st.caps & 0xffffu, vhigh = st.caps >> 16;
-    const uint32_t pos = atoms_add(st.sh_addr + offsetof(SparsifyShared, vec_count), 1u);
+// `base` is the shared-space address of the CTA's dynamic shared memory.
+__device__ __forceinline__ void stage_vector(uint32_t base, const SparsifyParams& p, int vec_index, float vmax) {
+    const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
     const uint32_t key = float_to_key(vmax);
-    hist_count(st.smem, st.smem + 4u * kHistBins, (int)(key >> kHistShift), 1u);
-    if (pos < vcap) sts_v2(st.smem + kArenaBytes + 8u * pos, (uint32_t)vec_index, key);
-    else sts_u32(st.sh_addr + offsetof(SparsifyShared, overflow), 1u);
-    if (pos + 1u == vhigh) sts_u32(st.sh_addr + offsetof(SparsifyShared, trim_request), 1u);
+    hist_count(base + kHistOff, base + kCoarseOff, (int)(key >> kHistShift), 1u);
+    if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, (uint32_t)vec_index, key);
+    else sts_u32(base + (uint32_t)offsetof(SparsifyShared, overflow), 1u);
+    if (pos + 1u == (uint32_t)p.vhigh) sts_u32(base + (uint32_t)offsetof(SparsifyShared, trim_request), 1u);
 }
 
 // One warp: the highest fine bin b with (number of counted logits in bins >= b) >= k, or -1 if
@@ -228,12 +223,23 @@ __device__ __noinline__ int scan_boundary(uint32_t hist_addr, uint32_t coarse_ad
     return cbin * 32 + 31 - fl;
 }
 
+// The bf16 side of the threshold word: P = the largest bf16 value below the lower edge of `bin`.
+__device__ __forceinline__ uint32_t threshold_word(int bin) {
+    uint32_t k16 = ((uint32_t)bin << (kHistShift - 16)) - 1u;  // key of the value just below the edge
+    if (k16 == 0x7fffu) k16 = 0x7ffeu;                         // -0 shares +0's key: step past it
+    const uint32_t b16 = (k16 & 0x8000u) ? (k16 & 0x7fffu) : (~k16 & 0xffffu);
+    return ((uint32_t)bin << 16) | b16;
+}
+
 // One warp: raise thr_bin to the bin scan_boundary finds.  Counts that other warps are still adding
 // can only be missed, never invented, so the result is always a valid lower bound.
 __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
     uint32_t above;
-    const int found = scan_boundary(sh->hist_addr, sh->coarse_addr, k, &above);
-    if ((threadIdx.x & 31) == 0 && found > *(volatile int*)&sh->thr_bin) atomicMax(&sh->thr_bin, found);
+    const int found = scan_boundary(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, k, &above);
+    if ((threadIdx.x & 31) == 0 && found > *(volatile int*)&sh->thr_bin) {
+        atomicMax(&sh->thr_bin, found);
+        atomicMax(&sh->thr_word, threshold_word(found));
+    }
 }
 
 // The running threshold in the form the lane-tile test wants.  A logit is a candidate iff its
@@ -244,15 +250,14 @@ __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
 template <typename T> struct Threshold;
 template <> struct Threshold<float> {
     float edge;
-    __device__ __forceinline__ explicit Threshold(int bin) : edge(bin_lower_edge(bin)) {}
+    __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh)
+        : edge(bin_lower_edge(*(const volatile int*)&sh->thr_bin)) {}
 };
 template <> struct Threshold<bf16_t> {
     uint32_t P2;
-    __device__ __forceinline__ explicit Threshold(int bin) {
-        uint32_t k16 = ((uint32_t)bin << (kHistShift - 16)) - 1u;  // key of the value just below the edge
-        if (k16 == 0x7fffu) k16 = 0x7ffeu;                         // -0 shares +0's key: step past it
-        const uint32_t b16 = (k16 & 0x8000u) ? (k16 & 0x7fffu) : (~k16 & 0xffffu);
-        P2 = b16 | (b16 << 16);
+    __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh) {
+        const uint32_t w = *(const volatile uint32_t*)&sh->thr_word;
+        P2 = __byte_perm(w, 0u, 0x1010);
     }
 };
 
@@ -261,7 +266,7 @@ template <> struct Threshold<bf16_t> {
 // and then all of them stage their next marked vector together, whichever of the four it is, so
 // that the staging code runs once per round for the whole warp (almost always a single round).
 __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, int lane_vec0,
-                                            const StageRef& st) {
+                                            uint32_t base, const SparsifyParams& p) {
     const uint32_t P2 = th.P2;
     if (bf16x2_max(lt.lane_max2(), P2) != P2) {
         uint32_t mask = 0;
@@ -274,12 +279,12 @@ __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Th
             if (j == 1) m2 = lt.vm[1];
             if (j == 2) m2 = lt.vm[2];
             if (j == 3) m2 = lt.vm[3];
-            stage_vector(st, lane_vec0 + j * 32, fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
+            stage_vector(base, p, lane_vec0 + j * 32, fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
         }
     }
 }
 __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, int lane_vec0,
-                                            const StageRef& st) {
+                                            uint32_t base, const SparsifyParams& p) {
     const float thr = th.edge;
     if (fmaxf(fmaxf(lt.vm[0], lt.vm[1]), fmaxf(lt.vm[2], lt.vm[3])) >= thr) {
         uint32_t mask = 0;
@@ -292,7 +297,7 @@ __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Thr
             if (j == 1) m = lt.vm[1];
             if (j == 2) m = lt.vm[2];
             if (j == 3) m = lt.vm[3];
-            stage_vector(st, lane_vec0 + j * 32, m);
+            stage_vector(base, p, lane_vec0 + j * 32, m);
         }
     }
 }
@@ -564,16 +569,14 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // every pointer below is derived from smem_raw by plain offsets, so that the compiler keeps
     // them in the shared address space (shared-memory atomics and loads, not generic ones)
-    unsigned char* arena = smem_raw;
-    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
-    uint32_t* coarse = hist + kHistBins;
-    uint2* staged = reinterpret_cast<uint2*>(arena + kArenaBytes);
+    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + kHistOff);
+    uint2* staged = reinterpret_cast<uint2*>(smem_raw + kStagedOff);
     uint32_t* cand_key = reinterpret_cast<uint32_t*>(staged + p.vcap);
     int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
     uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
-    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, p.vcap, p.k));
-    const StageRef stage{smem_u32(smem_raw), smem_u32(sh), (uint32_t)p.vcap | ((uint32_t)p.vhigh << 16)};
+    const uint32_t base = smem_u32(smem_raw);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
@@ -587,12 +590,11 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
     if (tid == 0) {
         sh->thr_bin = kLowestFiniteBin;
+        sh->thr_word = threshold_word(kLowestFiniteBin);
         sh->cand_count = 0;
         sh->vec_count = 0;
         sh->overflow = 0;
         sh->trim_request = 0;
-        sh->hist_addr = smem_u32(hist);
-        sh->coarse_addr = smem_u32(coarse);
     }
     __syncthreads();
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
@@ -613,13 +615,13 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
 #pragma unroll
                 for (int j = 0; j < kVecsPerLane; ++j) {
                     const float z = lt.vec_max(j);
-                    if (z >= -3.4028234e38f) hist_count(sh->hist_addr, sh->coarse_addr, (int)(float_to_key(z) >> kHistShift), 1u);
+                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(float_to_key(z) >> kHistShift), 1u);
                 }
             } else {
 #pragma unroll 4
                 for (int e = 0; e < kVecsPerLane * kPer; ++e) {
                     const float z = lt.elem(e / kPer, e % kPer);
-                    if (z >= -3.4028234e38f) hist_count(sh->hist_addr, sh->coarse_addr, (int)(float_to_key(z) >> kHistShift), 1u);
+                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(float_to_key(z) >> kHistShift), 1u);
                 }
             }
         }
@@ -633,25 +635,28 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     // ---- streaming: no barriers; warp w rescans the histogram on its turn --------------------------
     LaneSum ls;
     ls.reset();
-    int ch = chunk_begin + warp, step = 0;
+    // chunks below pf_end are whole and inside the segment: the only ones asked of L2 ahead of time
+    const int pf_end = min(chunk_end, ext.nvec_full / kVecsPerChunk);
+    int ch = chunk_begin + warp;
     for (;;) {
         while (ch < chunk_end) {
             __syncwarp();
             if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
             LaneTile<T> lt;
             lt.load(rowp, ch * kVecsPerChunk, lane, ext);
-            prefetch_chunk(rowp, ch + kPrefetchSteps * kWarps, chunk_end, lane, ext);
+            if (ch + kPrefetchSteps * kWarps < pf_end && lane == 0)
+                prefetch_l2(rowp + (size_t)(ch + kPrefetchSteps * kWarps) * kChunkBytes, kChunkBytes);
             const float lm = lt.reduce_max();
-            if (ls.needs_raise(lm, c)) ls.raise(lm, c);
+            ls.raise_to(lm, c);
             lt.accumulate(ls, c);
-            const Threshold<T> th(*(volatile int*)&sh->thr_bin);
-            filter_push(lt, th, ch * kVecsPerChunk + lane, stage);
-            if ((step & (kWarps - 1)) == warp) {
+            const Threshold<T> th(sh);
+            filter_push(lt, th, ch * kVecsPerChunk + lane, base, p);
+            // the warps take turns at rescanning the histogram: one of them on every step
+            if ((((ch >> 3) ^ warp) & (kWarps - 1)) == 0) {
                 __syncwarp();
                 raise_threshold(sh, k);
             }
             ch += kWarps;
-            ++step;
         }
         const int all_done = __syncthreads_and(ch >= chunk_end);
         const int want_trim = sh->trim_request;
@@ -714,21 +719,16 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
 template <typename T>
 __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const SparsifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* arena = smem_raw;
-    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(arena + kArenaBytes);
+    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw);
+    unsigned char* arena = smem_raw + kHistOff;
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem_raw + kStagedOff);
     int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
     uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
-    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw + sparsify_shared_off(p.cap, 0, p.k));
     const int tid = threadIdx.x, row = blockIdx.x;
     // the uniforms are needed last: ask for their cache line now
     if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
-    if (tid == 0) {
-        sh->hist_addr = smem_u32(hist);
-        sh->coarse_addr = smem_u32(hist + kHistBins);
-        sh->overflow = 0;
-    }
+    if (tid == 0) sh->overflow = 0;
     wait_for_primary_kernel();  // nothing the streaming kernel wrote is read before this point
     if (row == 0 && tid == 0) *p.status = 0;
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
@@ -772,11 +772,11 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
     consumer_sync();
     for (int i = tid; i < nc; i += kBlockThreads)
-        hist_count(sh->hist_addr, sh->coarse_addr, (int)(cand_key[i] >> kHistShift), 1u);
+        hist_count(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, (int)(cand_key[i] >> kHistShift), 1u);
     consumer_sync();
     if (warp == 0) {
         uint32_t above;
-        const int b = scan_boundary(sh->hist_addr, sh->coarse_addr, k, &above);
+        const int b = scan_boundary(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, k, &above);
         if (lane == 0) {
             sh->sel_bin = b;  // -1: fewer than k candidates exist, all of them are kept
             sh->sel_above = (int)above;

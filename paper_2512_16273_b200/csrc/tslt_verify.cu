@@ -472,10 +472,7 @@ __device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWo
         const float wm = warp_max(lt.reduce_max());
         LaneSum ls;
         ls.reset();
-        if (wm > -INFINITY) {
-            ls.zmax = wm;
-            ls.M = wm * c;
-        }
+        if (wm > -INFINITY) ls.M = wm * c;
         lt.accumulate(ls, c);
         const float Sw = warp_sum(ls.total());
         if (lane == 0) part[ch] = make_float2(ls.M, Sw);
