@@ -264,6 +264,18 @@ template <> __device__ __forceinline__ void unpack_vec<bf16_t>(const uint4& v, f
     z[6] = __uint_as_float(v.w << 16); z[7] = __uint_as_float(v.w & 0xffff0000u);
 }
 
+// The reverse, for values that came from the storage type (exact).
+template <typename T> __device__ __forceinline__ uint4 pack_vec(const float* z);
+template <> __device__ __forceinline__ uint4 pack_vec<float>(const float* z) {
+    return make_uint4(__float_as_uint(z[0]), __float_as_uint(z[1]), __float_as_uint(z[2]), __float_as_uint(z[3]));
+}
+template <> __device__ __forceinline__ uint4 pack_vec<bf16_t>(const float* z) {
+    return make_uint4((__float_as_uint(z[0]) >> 16) | (__float_as_uint(z[1]) & 0xffff0000u),
+                      (__float_as_uint(z[2]) >> 16) | (__float_as_uint(z[3]) & 0xffff0000u),
+                      (__float_as_uint(z[4]) >> 16) | (__float_as_uint(z[5]) & 0xffff0000u),
+                      (__float_as_uint(z[6]) >> 16) | (__float_as_uint(z[7]) & 0xffff0000u));
+}
+
 // The scale c = log2(e) / T that turns a stored logit into a base-2 exponent.  The streaming
 // pass uses its fp32 rounding `f` in one fused multiply-add per logit, y = z * f - M, where M is
 // the fp32 exponent of a running maximum; `d` is the value all fp64 code uses.  |f/d - 1| <=

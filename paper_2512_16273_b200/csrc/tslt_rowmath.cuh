@@ -84,7 +84,22 @@ template <> struct LaneTile<bf16_t> {
     static constexpr int kElems = 32;
     uint32_t w[16];  // vector j holds words 4j..4j+3, each two bf16 (low half = lower index)
     uint32_t vm[4];  // packed maximum of vector j (set by reduce_max)
+    uint32_t m2;     // packed maximum of the lane tile (set by reduce_max)
 
+    // A whole chunk from lane_row = row + 16 * lane, so that the common case needs no lane number.
+    __device__ __forceinline__ void load_lane(const unsigned char* lane_row, int vec0, const RowExtent& ext) {
+        if (vec0 + kVecsPerChunk <= ext.nvec_full) {
+            const uint4* base = reinterpret_cast<const uint4*>(lane_row) + vec0;
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j) {
+                const uint4 v = ldg_stream(base + j * 32);
+                w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+            }
+        } else {
+            const int lane = threadIdx.x & 31;
+            load(lane_row - lane * kVecBytes, vec0, lane, ext);
+        }
+    }
     // Chunk whose first vector is number vec0 of the row at `row`; vectors past the row's end read
     // as -inf, the ragged last vector is fetched element by element.
     __device__ __forceinline__ void load(const unsigned char* row, int vec0, int lane, const RowExtent& ext) {
@@ -115,16 +130,13 @@ template <> struct LaneTile<bf16_t> {
     }
     static __device__ __forceinline__ float lo(uint32_t x) { return __uint_as_float(x << 16); }
     static __device__ __forceinline__ float hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
-    // Fills vm[] and returns the largest logit of the lane tile.
+    // Fills vm[] and m2 and returns the largest logit of the lane tile.
     __device__ __forceinline__ float reduce_max() {
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             vm[j] = bf16x2_max(bf16x2_max(w[4 * j], w[4 * j + 1]), bf16x2_max(w[4 * j + 2], w[4 * j + 3]));
-        const uint32_t m = lane_max2();
-        return fmaxf(lo(m), hi(m));
-    }
-    __device__ __forceinline__ uint32_t lane_max2() const {
-        return bf16x2_max(bf16x2_max(vm[0], vm[1]), bf16x2_max(vm[2], vm[3]));
+        m2 = bf16x2_max(bf16x2_max(vm[0], vm[1]), bf16x2_max(vm[2], vm[3]));
+        return fmaxf(lo(m2), hi(m2));
     }
     __device__ __forceinline__ float vec_max(int j) const { return fmaxf(lo(vm[j]), hi(vm[j])); }
     // s += sum 2^(z * c - M) over the 32 logits
@@ -148,6 +160,20 @@ template <> struct LaneTile<float> {
     float z[16];
     float vm[4];  // maximum of vector j (set by reduce_max)
 
+    __device__ __forceinline__ void load_lane(const unsigned char* lane_row, int vec0, const RowExtent& ext) {
+        if (vec0 + kVecsPerChunk <= ext.nvec_full) {
+            const uint4* base = reinterpret_cast<const uint4*>(lane_row) + vec0;
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j) {
+                const uint4 v = ldg_stream(base + j * 32);
+                z[4 * j] = __uint_as_float(v.x); z[4 * j + 1] = __uint_as_float(v.y);
+                z[4 * j + 2] = __uint_as_float(v.z); z[4 * j + 3] = __uint_as_float(v.w);
+            }
+        } else {
+            const int lane = threadIdx.x & 31;
+            load(lane_row - lane * kVecBytes, vec0, lane, ext);
+        }
+    }
     __device__ __forceinline__ void load(const unsigned char* row, int vec0, int lane, const RowExtent& ext) {
         const uint4* base = reinterpret_cast<const uint4*>(row) + vec0 + lane;
         if (vec0 + kVecsPerChunk <= ext.nvec_full) {

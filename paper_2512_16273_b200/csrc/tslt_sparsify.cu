@@ -43,8 +43,9 @@ constexpr int kRankSortMax = 256;   // up to this many entries are ordered by co
 struct SegStat {
     double S[kWarps];  // per warp: sum of 2^(y - M) over the warp's chunks of the segment
     float M[kWarps];   // per warp: reference exponent (base 2)
-    int n;             // candidates written for the segment
-    int pad;
+    int n;             // entries written for the segment
+    int raw_bin;       // -1: the entries are (key, idx) candidates; else they are staged lane tiles (first vector
+                       // and vector mask, key of the largest logit) and this is the segment's final threshold bin
 };
 
 struct SparsifyParams {
@@ -64,19 +65,22 @@ struct SparsifyParams {
     int nchunks;
     RowSplit split;
     int cap, high;      // candidate (key, index) list: capacity and compaction mark
-    int vcap, vhigh;    // staged vectors: capacity and early-expansion mark
+    int vcap, vhigh;    // staged lane tiles: capacity and early-expansion mark
     int idx_hi_byte;
     int* status;
     SegStat* seg_stats;
-    uint2* seg_entries;  // [rows, nseg, seg_cap] (key, idx)
-    int seg_cap;
+    uint2* seg_entries;  // [rows, nseg, seg_stride]: (key, idx) candidates, or staged lane tiles handed over raw
+    int seg_cap;         // most candidates a segment hands over
+    int seg_stride;      // entries reserved per segment
+    int raw_cap;         // > 0: a segment whose staging buffer never filled hands its staged tiles over unexpanded
 };
 
 struct SparsifyShared {
-    // ---- written by stage_vector through their shared-space addresses --------------------------------
-    int vec_count;   // staged vectors
+    // ---- written by stage_tile through their shared-space addresses ----------------------------------
+    int vec_count;   // staged lane tiles
     int overflow;    // a buffer was found full: its contents are no longer complete
     int trim_request;
+    int n_above;     // logits counted in bins above thr_bin since it last rose (may lag, never leads a rise)
     // --------------------------------------------------------------------------------------------
     int cand_count;  // expanded (key, index) candidates
     int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
@@ -148,17 +152,34 @@ __device__ __forceinline__ void hist_count(uint32_t hist_addr, uint32_t coarse_a
 __device__ __forceinline__ void sts_v2(uint32_t addr, uint32_t x, uint32_t y) {
     asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
 }
+// A warp hands out list positions with one atomic: returns where this lane's cnt entries start.
+__device__ __forceinline__ int warp_reserve(int* counter, int cnt, int lane) {
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    int start = 0;
+    if (lane == 31 && incl > 0) start = atomicAdd(counter, incl);
+    return __shfl_sync(0xffffffffu, start, 31) + incl - cnt;
+}
 
-// Stage one 16-byte vector (number vec_index of its row) whose largest logit is vmax: only its
-// number and the key of that logit are kept (8 bytes), and the logit is counted.  The vector's
-// data is read again from global memory when the staged vectors are expanded, and only if its
-// largest logit still passes the threshold of that moment: a fraction of the staged vectors.
-// `base` is the shared-space address of the CTA's dynamic shared memory.
-__device__ __forceinline__ void stage_vector(uint32_t base, const SparsifyParams& p, int vec_index, float vmax) {
+
+// Stage a lane tile (the four 16-byte vectors vec0, vec0 + 32, vec0 + 64, vec0 + 96 of the row)
+// whose largest logit is vmax: only vec0, which of the four vectors hold a candidate, and the key
+// of that logit are kept (8 bytes), and the logit is counted.  The tile's data is read again from
+// global memory when the staged tiles are expanded, and only if its largest logit still passes
+// the threshold of that moment: a fraction of what is staged.  `base` is the shared-space address
+// of the CTA's dynamic shared memory.
+constexpr int kTileMaskShift = 28;  // a staged tile's word: first vector (below 2^18) | mask of its four vectors << 28
+__device__ __forceinline__ void stage_tile(uint32_t base, const SparsifyParams& p, int thr_bin, uint32_t tile_word,
+                                           float vmax) {
     const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
     const uint32_t key = float_to_key(vmax);
     hist_count(base + kHistOff, base + kCoarseOff, (int)(key >> kHistShift), 1u);
-    if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, (uint32_t)vec_index, key);
+    if ((int)(key >> kHistShift) > thr_bin) reds_add(base + (uint32_t)offsetof(SparsifyShared, n_above), 1u);
+    if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, tile_word, key);
     else sts_u32(base + (uint32_t)offsetof(SparsifyShared, overflow), 1u);
     if (pos + 1u == (uint32_t)p.vhigh) sts_u32(base + (uint32_t)offsetof(SparsifyShared, trim_request), 1u);
 }
@@ -236,9 +257,15 @@ __device__ __forceinline__ uint32_t threshold_word(int bin) {
 __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
     uint32_t above;
     const int found = scan_boundary(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, k, &above);
-    if ((threadIdx.x & 31) == 0 && found > *(volatile int*)&sh->thr_bin) {
-        atomicMax(&sh->thr_bin, found);
-        atomicMax(&sh->thr_word, threshold_word(found));
+    if ((threadIdx.x & 31) == 0) {
+        const int cur = *(volatile int*)&sh->thr_bin;
+        if (found > cur) {
+            atomicMax(&sh->thr_bin, found);
+            atomicMax(&sh->thr_word, threshold_word(found));
+        }
+        // what is counted above the boundary bin starts the count towards the next rise (a stale
+        // value only costs or delays a rescan)
+        if (found >= cur) *(volatile int*)&sh->n_above = (int)above;
     }
 }
 
@@ -249,80 +276,82 @@ __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
 //              word w holds a candidate iff max.bf16x2(w, P) != P (NaN halves never differ).
 template <typename T> struct Threshold;
 template <> struct Threshold<float> {
+    int bin;
     float edge;
     __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh)
-        : edge(bin_lower_edge(*(const volatile int*)&sh->thr_bin)) {}
+        : bin(*(const volatile int*)&sh->thr_bin), edge(bin_lower_edge(bin)) {}
+    __device__ __forceinline__ int bin_value() const { return bin; }
 };
 template <> struct Threshold<bf16_t> {
-    uint32_t P2;
+    uint32_t word, P2;
     __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh) {
-        const uint32_t w = *(const volatile uint32_t*)&sh->thr_word;
-        P2 = __byte_perm(w, 0u, 0x1010);
+        word = *(const volatile uint32_t*)&sh->thr_word;
+        P2 = __byte_perm(word, 0u, 0x1010);
     }
+    __device__ __forceinline__ int bin_value() const { return (int)(word >> 16); }
 };
 
-// Stage the vectors of a lane tile that hold a candidate (reduce_max() already called).  One test
-// on the lane's packed maximum; lanes that pass mark which of their four vectors hold a candidate,
-// and then all of them stage their next marked vector together, whichever of the four it is, so
-// that the staging code runs once per round for the whole warp (almost always a single round).
-__device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, int lane_vec0,
+// Stage the lane tile if it holds a candidate (reduce_max() already called, lm its result): one
+// test on the lane's packed maximum, one staging step for all the lanes of the warp that pass.
+__device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, float lm, int vec0,
                                             uint32_t base, const SparsifyParams& p) {
     const uint32_t P2 = th.P2;
-    if (bf16x2_max(lt.lane_max2(), P2) != P2) {
-        uint32_t mask = 0;
+    if (bf16x2_max(lt.m2, P2) != P2) {
+        uint32_t word = (uint32_t)vec0;
 #pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j) mask |= (bf16x2_max(lt.vm[j], P2) != P2) ? (1u << j) : 0u;
-        while (mask) {
-            const int j = __ffs(mask) - 1;
-            mask &= mask - 1;
-            uint32_t m2 = lt.vm[0];
-            if (j == 1) m2 = lt.vm[1];
-            if (j == 2) m2 = lt.vm[2];
-            if (j == 3) m2 = lt.vm[3];
-            stage_vector(base, p, lane_vec0 + j * 32, fmaxf(LaneTile<bf16_t>::lo(m2), LaneTile<bf16_t>::hi(m2)));
-        }
+        for (int j = 0; j < kVecsPerLane; ++j)
+            if (bf16x2_max(lt.vm[j], P2) != P2) word |= 1u << (kTileMaskShift + j);
+        stage_tile(base, p, th.bin_value(), word, lm);
     }
 }
-__device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, int lane_vec0,
+__device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, float lm, int vec0,
                                             uint32_t base, const SparsifyParams& p) {
-    const float thr = th.edge;
-    if (fmaxf(fmaxf(lt.vm[0], lt.vm[1]), fmaxf(lt.vm[2], lt.vm[3])) >= thr) {
-        uint32_t mask = 0;
+    if (lm >= th.edge) {
+        uint32_t word = (uint32_t)vec0;
 #pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j) mask |= (lt.vm[j] >= thr) ? (1u << j) : 0u;
-        while (mask) {
-            const int j = __ffs(mask) - 1;
-            mask &= mask - 1;
-            float m = lt.vm[0];
-            if (j == 1) m = lt.vm[1];
-            if (j == 2) m = lt.vm[2];
-            if (j == 3) m = lt.vm[3];
-            stage_vector(base, p, lane_vec0 + j * 32, m);
-        }
+        for (int j = 0; j < kVecsPerLane; ++j)
+            if (lt.vec_max(j) >= th.edge) word |= 1u << (kTileMaskShift + j);
+        stage_tile(base, p, th.bin_value(), word, lm);
     }
 }
 
-// All threads: turn the staged vectors whose largest logit is in a bin >= bin into (key, index)
-// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  The vectors
-// come back from global memory (L2 or HBM), four loads in flight per thread.  A full candidate
-// list raises the overflow flag.
+// One 16-byte vector of a row as kPer logits; the row's ragged last vector element by element,
+// -inf beyond the row.
+template <typename T>
+__device__ __forceinline__ void load_row_vector(const unsigned char* rowp, int vi, const RowExtent& ext, int V,
+                                                float (&z)[Elt<T>::kPerVec]) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    if (vi < ext.nvec_full) {
+        unpack_vec<T>(__ldcg(reinterpret_cast<const uint4*>(rowp) + vi), z);
+    } else {
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) z[e] = vi * kPer + e < V ? Elt<T>::load(rowp, vi * kPer + e) : -INFINITY;
+    }
+}
+
+// All threads: turn the staged lane tiles whose largest logit is in a bin >= bin into (key, index)
+// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  One thread
+// per marked 16-byte vector of a tile; the vectors come back from global memory (L2 or HBM), four
+// loads in flight per thread.  A full candidate list raises the overflow flag.
 template <typename T>
 __device__ __noinline__ void expand_staged(const uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
                                            Candidates cb, int cap, int bin, int V, SparsifyShared* sh, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr int kInFlight = 4;
-    const int nv = min(sh->vec_count, vcap);
+    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
+    const int nitems = min(sh->vec_count, vcap) * kVecsPerLane;
     const uint32_t min_key = (uint32_t)bin << kHistShift;
-    for (int base = 0; base < nv; base += kInFlight * kBlockThreads) {
+    for (int base = 0; base < nitems; base += kInFlight * kBlockThreads) {
         uint4 d[kInFlight];
         int vi[kInFlight];
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const int i = base + u * kBlockThreads + tid;
             vi[u] = -1;
-            if (i < nv) {
-                const uint2 s = staged[i];
-                if (s.y >= min_key) vi[u] = (int)s.x;
+            if (i < nitems) {
+                const uint2 s = staged[i / kVecsPerLane];
+                const int j = i % kVecsPerLane;
+                if (s.y >= min_key && ((s.x >> (kTileMaskShift + j)) & 1u)) vi[u] = (int)(s.x & kVecMask) + 32 * j;
             }
             if (vi[u] >= 0 && vi[u] < ext.nvec_full) d[u] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[u]);
         }
@@ -331,12 +360,8 @@ __device__ __noinline__ void expand_staged(const uint2* staged, int vcap, const 
             if (vi[u] < 0) continue;
             const int e0 = vi[u] * kPer;
             float z[kPer];
-            if (vi[u] < ext.nvec_full) {
-                unpack_vec<T>(d[u], z);
-            } else {  // the row's ragged last vector: element by element
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) z[e] = e0 + e < V ? Elt<T>::load(rowp, e0 + e) : -INFINITY;
-            }
+            if (vi[u] < ext.nvec_full) unpack_vec<T>(d[u], z);
+            else load_row_vector<T>(rowp, vi[u], ext, V, z);  // the ragged last vector; nothing beyond it
 #pragma unroll
             for (int e = 0; e < kPer; ++e) {
                 if (z[e] >= -3.4028234e38f) {
@@ -484,7 +509,7 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
     if (nseg == 1 && p.seg_cap <= 8 * kBlockThreads) {
         // one segment: every load is issued before anything is used, so the row costs one trip to memory
         const SegStat* st = &p.seg_stats[slot0];
-        const uint2* ent = p.seg_entries + slot0 * (size_t)p.seg_cap;
+        const uint2* ent = p.seg_entries + slot0 * (size_t)p.seg_stride;
         uint2 e[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -543,7 +568,7 @@ __device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row
     for (int g = 0; g < nseg; ++g) {
         const SegStat* st = &p.seg_stats[slot0 + g];
         const int ng = __ldcg(&st->n);
-        const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_cap;
+        const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_stride;
         const int base = sh->cand_count;
         for (int i = tid; i < ng; i += kBlockThreads) {
             const uint2 e2 = __ldcg(&ent[i]);
@@ -595,6 +620,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         sh->vec_count = 0;
         sh->overflow = 0;
         sh->trim_request = 0;
+        sh->n_above = 0;
     }
     __syncthreads();
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
@@ -629,6 +655,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         if (warp == 0) raise_threshold(sh, k);
         __syncthreads();
         for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+        if (tid == 0) sh->n_above = 0;
         __syncthreads();
     }
 
@@ -637,24 +664,26 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     ls.reset();
     // chunks below pf_end are whole and inside the segment: the only ones asked of L2 ahead of time
     const int pf_end = min(chunk_end, ext.nvec_full / kVecsPerChunk);
+    const unsigned char* lane_rowp = rowp + lane * kVecBytes;  // the loop's loads need no lane number
     int ch = chunk_begin + warp;
     for (;;) {
         while (ch < chunk_end) {
             __syncwarp();
             if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
             LaneTile<T> lt;
-            lt.load(rowp, ch * kVecsPerChunk, lane, ext);
+            lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
             if (ch + kPrefetchSteps * kWarps < pf_end && lane == 0)
                 prefetch_l2(rowp + (size_t)(ch + kPrefetchSteps * kWarps) * kChunkBytes, kChunkBytes);
             const float lm = lt.reduce_max();
+            const Threshold<T> th(sh);
+            filter_push(lt, th, lm, ch * kVecsPerChunk + lane, base, p);  // while the vector maxima are at hand
             ls.raise_to(lm, c);
             lt.accumulate(ls, c);
-            const Threshold<T> th(sh);
-            filter_push(lt, th, ch * kVecsPerChunk + lane, base, p);
-            // the warps take turns at rescanning the histogram: one of them on every step
-            if ((((ch >> 3) ^ warp) & (kWarps - 1)) == 0) {
+            // The warps take turns at looking whether enough has been counted above the threshold
+            // bin for it to rise (ch mod 8 is the warp's own, so the turns differ), and rescan then.
+            if ((((ch >> 3) ^ ch) & (kWarps - 1)) == 0) {
                 __syncwarp();
-                raise_threshold(sh, k);
+                if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->n_above, 0) >= k) raise_threshold(sh, k);
             }
             ch += kWarps;
         }
@@ -675,6 +704,31 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         }
     }
 
+    // ---- hand-over: one (M, S) pair per warp and the segment's entries; the kernel boundary publishes
+    // them to the finish kernel
+    const float Mw = warp_max(ls.M);
+    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
+    const size_t slot = (size_t)row * wk.nseg + wk.seg;
+    uint2* my_entries = p.seg_entries + slot * (size_t)p.seg_stride;
+    SegStat* st = &p.seg_stats[slot];
+    if (lane == 0) {
+        st->S[warp] = Sw;
+        st->M[warp] = Mw;
+    }
+    // (the loop's last barrier ordered every write of the flags read here)
+    if (p.raw_cap > 0 && !sh->overflow && sh->cand_count == 0) {
+        // The staging buffer never filled: its tiles go over as they are, with the final threshold
+        // bin, and the finish kernel reads the few that still pass back from global memory, all
+        // rows at once, instead of this CTA waiting on them now.
+        const int n = sh->vec_count;
+        for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = staged[i];
+        if (tid == 0) {
+            st->n = n;
+            st->raw_bin = sh->thr_bin;
+        }
+        return;
+    }
+
     // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
     if (!sh->overflow) expand_staged<T>(staged, p.vcap, rowp, ext, cb, p.cap, sh->thr_bin, p.V, sh, tid);
     if (sh->overflow) {
@@ -689,11 +743,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         if (tid == 0) sh->overflow = 0;
         consumer_sync();
     }
-
-    // ---- hand-over: candidates (all at or above this segment's final threshold) and one (M, S) pair
-    // per warp; the kernel boundary publishes them to the finish kernel
-    const float Mw = warp_max(ls.M);
-    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
+    // candidates: all at or above this segment's final threshold
     int n = sh->cand_count;
     if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
         compact_buffer(cb, sh->thr_bin, sh, tid);
@@ -703,15 +753,11 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
         n = sh->cand_count;
     }
-    const size_t slot = (size_t)row * wk.nseg + wk.seg;
-    uint2* my_entries = p.seg_entries + slot * (size_t)p.seg_cap;
     for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
-    SegStat* st = &p.seg_stats[slot];
-    if (lane == 0) {
-        st->S[warp] = Sw;
-        st->M[warp] = Mw;
+    if (tid == 0) {
+        st->n = n;
+        st->raw_bin = -1;
     }
-    if (tid == 0) st->n = n;
 }
 
 // Second launch: one CTA per row merges the row's segments and finishes it.
@@ -954,30 +1000,34 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 }
 
 // ---- finish kernel for small k --------------------------------------------------------------------
-// Rows whose hand-over is at most 256 candidates in one segment (k <= 128) are finished by a CTA of
-// 128 threads with 6 KB of shared memory, so that every row of a large batch is resident at once:
-// finishing a row is a chain of a dozen dependent steps (one trip to memory, rank counting, two
-// scans), and what it costs machine-wide is the length of that chain times the number of waves.
-constexpr int kSmallThreads = 128;
-constexpr int kSmallCand = 256;
+// Rows of one segment with k <= 128 are finished by a CTA of 64, 96 or 128 threads (k rounded up
+// to a warp) with 8 KB of shared memory, so that every row of a large batch is resident at once:
+// finishing a row is a chain of dependent steps (trips to memory, rank counting, two scans), and
+// what it costs machine-wide is the length of that chain times the number of waves.
+constexpr int kSmallMaxThreads = 128;
+constexpr int kSmallCand = 256;  // candidates a row may bring
+constexpr int kSmallPass = 512;  // marked vectors in the staged tiles of a row that pass its final threshold
 
 struct SmallShared {
-    uint32_t key[kSmallCand];
-    int idx[kSmallCand];
-    uint32_t wkey[kSmallThreads];  // winners in (key descending, index ascending) order, then in ascending index
-    int widx[kSmallThreads];
-    uint32_t okey[kSmallThreads];
-    int oidx[kSmallThreads];
-    double cum[kSmallThreads];
-    double wv[kSmallThreads];
+    unsigned long long comp[kSmallCand];  // candidates as key << 32 | ~index: larger is earlier in the top-k order
+    uint32_t wkey[kSmallMaxThreads];  // winners in (key descending, index ascending) order, then in ascending index
+    int widx[kSmallMaxThreads];
+    uint32_t okey[kSmallMaxThreads];
+    int oidx[kSmallMaxThreads];
+    double cum[kSmallMaxThreads];
+    double wv[kSmallMaxThreads];
     double red[8];
     int n_cut;
+    // rows handed over as staged lane tiles
+    uint32_t pass[kSmallPass];  // marked vectors of the tiles whose largest logit passes the final threshold
+    int n_pass, n_cand;
+    unsigned long long best[kSmallMaxThreads / 32];
 };
 
-__device__ __forceinline__ void small_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kSmallThreads) : "memory"); }
+template <int NT> __device__ __forceinline__ void small_sync() { asm volatile("bar.sync 2, %0;" ::"n"(NT) : "memory"); }
 
-// inclusive scan of one value per thread over the 128 threads; returns this thread's inclusive sum
-__device__ __forceinline__ double small_scan(double v, int tid, double* red, double* total) {
+// inclusive scan of one value per thread over the NT threads; returns this thread's inclusive sum
+template <int NT> __device__ __forceinline__ double small_scan(double v, int tid, double* red, double* total) {
     const int lane = tid & 31, warp = tid >> 5;
     double incl = v;
 #pragma unroll
@@ -986,31 +1036,176 @@ __device__ __forceinline__ double small_scan(double v, int tid, double* red, dou
         if (lane >= o) incl += t;
     }
     if (lane == 31) red[warp] = incl;
-    small_sync();
+    small_sync<NT>();
     double base = 0.0, tot = 0.0;
 #pragma unroll
-    for (int w = 0; w < kSmallThreads / 32; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         const double t = red[w];
         if (w < warp) base += t;
         tot += t;
     }
-    small_sync();
+    small_sync<NT>();
     *total = tot;
     return base + incl;
 }
-__device__ __forceinline__ double small_max(double v, int tid, double* red) {
+template <int NT> __device__ __forceinline__ double small_max(double v, int tid, double* red) {
     v = warp_max(v);
     if ((tid & 31) == 0) red[tid >> 5] = v;
-    small_sync();
+    small_sync<NT>();
     double m = red[0];
 #pragma unroll
-    for (int w = 1; w < kSmallThreads / 32; ++w) m = fmax(m, red[w]);
-    small_sync();
+    for (int w = 1; w < NT / 32; ++w) m = fmax(m, red[w]);
+    small_sync<NT>();
     return m;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kernel(const SparsifyParams p) {
+// The slow way to a row's k winners from its staged tiles: one winner per round, each round a pass
+// over the marked vectors of the passing tiles.  Only there to be correct when a row has more
+// tied candidates around its k-th logit than the lists of the kernel below hold.
+// composite = key << 32 | ~index: larger is earlier in (logit descending, index ascending)
+template <typename T, int NT>
+__device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
+                                               SmallShared* sm, int tid) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
+    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
+    const RowExtent ext = row_extent<T>(p.V);
+    const uint32_t min_key = (uint32_t)bin << kHistShift;
+    unsigned long long last = ~0ull;
+    int found = 0;
+    for (; found < p.k; ++found) {
+        unsigned long long best = 0ull;
+        for (int i = tid; i < n_tiles * kVecsPerLane; i += NT) {
+            const uint2 e = __ldcg(&ent[i / kVecsPerLane]);
+            const int j = i % kVecsPerLane;
+            if (e.y < min_key || !((e.x >> (kTileMaskShift + j)) & 1u)) continue;
+            const int vi = (int)(e.x & kVecMask) + 32 * j;
+            float z[kPer];
+            load_row_vector<T>(rowp, vi, ext, p.V, z);
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) {
+                if (z[q] >= -3.4028234e38f) {
+                    const unsigned long long comp = ((unsigned long long)float_to_key(z[q]) << 32) |
+                                                    (unsigned long long)(0xffffffffu - (uint32_t)(vi * kPer + q));
+                    if (comp < last && comp > best) best = comp;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long t = __shfl_xor_sync(0xffffffffu, best, o);
+            best = t > best ? t : best;
+        }
+        if ((tid & 31) == 0) sm->best[tid >> 5] = best;
+        small_sync<NT>();
+#pragma unroll
+        for (int w = 0; w < NT / 32; ++w) best = sm->best[w] > best ? sm->best[w] : best;
+        small_sync<NT>();
+        if (best == 0ull || (uint32_t)(best >> 32) < min_key) break;
+        if (tid == 0) sm->comp[found] = best;
+        last = best;
+    }
+    small_sync<NT>();
+    return found;
+}
+
+// NT threads: the row was handed over as n_tiles staged lane tiles and its final threshold bin.
+// Puts the row's candidates (every logit whose bin is >= bin, at least its k largest) into
+// sm->comp and returns their number (<= kSmallCand).  The marked vectors of the tiles that pass
+// (largest logit in a bin >= bin) are listed, then one thread per listed vector reads it back and
+// appends its candidates.  (Inlined into the kernel so that the compiler sees sm in the shared
+// address space: atomics through a generic pointer to shared memory are several times slower.)
+template <typename T, int NT>
+__device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
+                                                     SmallShared* sm, int tid) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
+    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
+    const RowExtent ext = row_extent<T>(p.V);
+    const uint32_t min_key = (uint32_t)bin << kHistShift;
+    const int lane = tid & 31;
+    if (tid == 0) {
+        sm->n_pass = 0;
+        sm->n_cand = 0;
+    }
+    small_sync<NT>();
+    // ---- the marked vectors of the passing tiles, as a list ------------------------------------------
+    for (int base = 0; base < n_tiles; base += 8 * NT) {
+        uint32_t m = 0;  // which of this thread's eight entries pass
+        int cnt = 0;     // marked vectors in them
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * NT + tid;
+            const uint2 e = i < n_tiles ? __ldcg(&ent[i]) : make_uint2(0u, 0u);  // key 0 never passes
+            if (e.y >= min_key) {
+                m |= 1u << u;
+                cnt += __popc(e.x >> kTileMaskShift);
+            }
+        }
+        int pos = warp_reserve(&sm->n_pass, cnt, lane);
+        while (m) {  // few: read them again (cached) rather than keep eight entries in registers
+            const int u = __ffs(m) - 1;
+            m &= m - 1;
+            const uint32_t w = __ldg(&ent[base + u * NT + tid].x);
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j) {
+                if ((w >> (kTileMaskShift + j)) & 1u) {
+                    if (pos < kSmallPass) sm->pass[pos] = (w & kVecMask) + 32u * j;
+                    ++pos;
+                }
+            }
+        }
+    }
+    small_sync<NT>();
+    const int nvec = sm->n_pass;
+    if (nvec <= kSmallPass) {
+        // ---- one thread per listed vector: read it back, append its candidates ----------------------
+        constexpr int kInFlight = 2;
+        static_assert(kInFlight * kPer <= 32, "one mask bit per logit a thread holds");
+        for (int base = 0; base < nvec; base += kInFlight * NT) {
+            float z[kInFlight][kPer];
+            int vi[kInFlight];
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u) {
+                const int i = base + u * NT + tid;
+                vi[u] = i < nvec ? (int)sm->pass[i] : -1;
+                if (vi[u] >= 0) {
+                    load_row_vector<T>(rowp, vi[u], ext, p.V, z[u]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e) z[u][e] = -INFINITY;
+                }
+            }
+            uint32_t m = 0;
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u)
+#pragma unroll
+                for (int e = 0; e < kPer; ++e)
+                    if (z[u][e] >= -3.4028234e38f && float_to_key(z[u][e]) >= min_key) m |= 1u << (u * kPer + e);
+            int pos = warp_reserve(&sm->n_cand, __popc(m), lane);
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u)
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    if ((m >> (u * kPer + e)) & 1u) {
+                        if (pos < kSmallCand)
+                            sm->comp[pos] = ((unsigned long long)float_to_key(z[u][e]) << 32) |
+                                            (unsigned long long)(0xffffffffu - (uint32_t)(vi[u] * kPer + e));
+                        ++pos;
+                    }
+                }
+        }
+        small_sync<NT>();
+        if (sm->n_cand <= kSmallCand) return sm->n_cand;
+    }
+    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, sm, tid);
+}
+
+constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : 12; }
+
+template <typename T, int NT>
+__global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_kernel(const SparsifyParams p) {
+    constexpr int kHeld = (kSmallCand + NT - 1) / NT;  // candidates a thread holds in registers
     __shared__ SmallShared sm;
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
     float u_raw = 0.f;
@@ -1019,11 +1214,16 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     if (row == 0 && tid == 0) *p.status = 0;
     // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
     const SegStat* st = &p.seg_stats[row];
-    const uint2* ent = p.seg_entries + (size_t)row * p.seg_cap;
-    uint2 e0 = make_uint2(0u, 0u), e1 = make_uint2(0u, 0u);
-    if (tid < p.seg_cap) e0 = __ldcg(&ent[tid]);
-    if (tid + kSmallThreads < p.seg_cap) e1 = __ldcg(&ent[tid + kSmallThreads]);
+    const uint2* ent = p.seg_entries + (size_t)row * p.seg_stride;
+    unsigned long long held[kHeld];  // key << 32 | ~index
+#pragma unroll
+    for (int c = 0; c < kHeld; ++c) {
+        const int i = tid + c * NT;
+        const uint2 e = i < p.seg_cap ? __ldcg(&ent[i]) : make_uint2(0u, 0u);
+        held[c] = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
+    }
     int nc = __ldcg(&st->n);
+    const int raw_bin = __ldcg(&st->raw_bin);
     // the log-normaliser once, by one warp (fp64 is scarce): one per-warp pair per lane
     if (tid < 32) {
         const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
@@ -1032,27 +1232,37 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
         const double Srow = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mrow) : 0.0);
         if (tid == 0) sm.red[7] = Mrow + log2(Srow);
     }
-    nc = nc < 0 ? 0 : (nc > kSmallCand ? kSmallCand : nc);
-    if (tid < nc) { sm.key[tid] = e0.x; sm.idx[tid] = (int)e0.y; }
-    if (tid + kSmallThreads < nc) { sm.key[tid + kSmallThreads] = e1.x; sm.idx[tid + kSmallThreads] = (int)e1.y; }
-    small_sync();
+    if (raw_bin >= 0) {  // the entries are staged lane tiles: make the candidates from them first
+        nc = candidates_from_tiles<T, NT>(p, row, ent, nc, raw_bin, &sm, tid);
+#pragma unroll
+        for (int c = 0; c < kHeld; ++c) {
+            const int i = tid + c * NT;
+            held[c] = i < nc ? sm.comp[i] : 0ull;
+        }
+    } else {
+        nc = nc < 0 ? 0 : (nc > kSmallCand ? kSmallCand : nc);
+#pragma unroll
+        for (int c = 0; c < kHeld; ++c) {
+            const int i = tid + c * NT;
+            if (i < nc) sm.comp[i] = held[c];
+        }
+    }
+    small_sync<NT>();
     // ---- exact top-k by counting ranks under (key descending, index ascending) -------------------
     // (only the threads that hold a candidate count; the 64-bit composite makes it one compare per entry)
-    if (tid < nc) {
-        const unsigned long long mine = ((unsigned long long)e0.x << 32) | (unsigned long long)(0xffffffffu - e0.y);
-        int r0 = 0;
-        for (int j = 0; j < nc; ++j)
-            r0 += ((((unsigned long long)sm.key[j] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)sm.idx[j])) > mine) ? 1 : 0;
-        if (r0 < k) { sm.wkey[r0] = e0.x; sm.widx[r0] = (int)e0.y; }
+#pragma unroll
+    for (int c = 0; c < kHeld; ++c) {
+        if (tid + c * NT < nc) {
+            const unsigned long long mine = held[c];
+            int r = 0;
+            for (int j = 0; j < nc; ++j) r += sm.comp[j] > mine ? 1 : 0;
+            if (r < k) {
+                sm.wkey[r] = (uint32_t)(mine >> 32);
+                sm.widx[r] = (int)(0xffffffffu - (uint32_t)mine);
+            }
+        }
     }
-    if (tid + kSmallThreads < nc) {
-        const unsigned long long mine = ((unsigned long long)e1.x << 32) | (unsigned long long)(0xffffffffu - e1.y);
-        int r1 = 0;
-        for (int j = 0; j < nc; ++j)
-            r1 += ((((unsigned long long)sm.key[j] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)sm.idx[j])) > mine) ? 1 : 0;
-        if (r1 < k) { sm.wkey[r1] = e1.x; sm.widx[r1] = (int)e1.y; }
-    }
-    small_sync();
+    small_sync<NT>();
     const int n0 = nc < k ? nc : k;
     const double L2 = sm.red[7];  // written before the barriers above; red[0..3] serve the scans
     const double cd = p.c.d;
@@ -1063,18 +1273,18 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
         double q = 0.0;
         if (tid < n0) q = exp2((double)key_to_float(sm.wkey[tid]) * cd - L2);
         double tot;
-        const double c_incl = small_scan(q, tid, sm.red, &tot);
+        const double c_incl = small_scan<NT>(q, tid, sm.red, &tot);
         if (p.top_p < 1.0f) {
             if (tid == 0) sm.n_cut = n0;
             if (tid < n0) sm.cum[tid] = c_incl;
-            small_sync();
+            small_sync<NT>();
             const double tp = (double)p.top_p;
             // first crossing of the cumulative: exactly one thread, if any
             if (tid < n0 && c_incl >= tp && (tid == 0 || sm.cum[tid - 1] < tp)) sm.n_cut = tid + 1;
-            small_sync();
+            small_sync<NT>();
             n = sm.n_cut;
             mass = n > 0 ? sm.cum[n - 1] : 0.0;
-            small_sync();
+            small_sync<NT>();
         } else {
             mass = tot;
         }
@@ -1087,16 +1297,16 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
         sm.oidx[r] = mine;
         sm.okey[r] = sm.wkey[tid];
     }
-    small_sync();
+    small_sync<NT>();
     // ---- renormalised truncated distribution and its CDF in fp64 -------------------------------------
     double y = -INFINITY;
     if (tid < n) y = (double)key_to_float(sm.okey[tid]) * cd;
-    const double mS = small_max(y, tid, sm.red);
+    const double mS = small_max<NT>(y, tid, sm.red);
     const double w = tid < n ? exp2(y - mS) : 0.0;
     double W;
-    const double cw = small_scan(w, tid, sm.red, &W);
+    const double cw = small_scan<NT>(w, tid, sm.red, &W);
     if (tid < n) { sm.cum[tid] = cw; sm.wv[tid] = w; }
-    small_sync();
+    small_sync<NT>();
     // ---- outputs ----------------------------------------------------------------------------------------
     int* o_idx = p.idx + (size_t)row * k;
     float* o_logit = p.logit + (size_t)row * k;
@@ -1109,7 +1319,7 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
         if (p.lse) p.lse[row] = n0 > 0 ? (float)(L2 * 0.6931471805599453) : -INFINITY;
         if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
     }
-    for (int sidx = tid; sidx < p.num_samples; sidx += kSmallThreads) {
+    for (int sidx = tid; sidx < p.num_samples; sidx += NT) {
         int tok = -1;
         if (n > 0) {
             const float u = clamp_uniform(sidx == tid ? u_raw : p.uniforms[(size_t)row * p.num_samples + sidx]);
@@ -1124,10 +1334,19 @@ __global__ void __launch_bounds__(kSmallThreads, 12) sparsify_finish_small_kerne
     }
 }
 
+// The small finish kernel for this k: a warp's worth of threads per 32 of k, at least two warps.
+template <typename T> static void (*small_finish_kernel(int k, int* threads))(const SparsifyParams) {
+    if (k <= 64) { *threads = 64; return sparsify_finish_small_kernel<T, 64>; }
+    if (k <= 96) { *threads = 96; return sparsify_finish_small_kernel<T, 96>; }
+    *threads = 128;
+    return sparsify_finish_small_kernel<T, 128>;
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
-    int nchunks, cap, high, vcap, vhigh, seg_cap;
+    int nchunks, cap, high, vcap, vhigh, seg_cap, seg_stride, raw_cap;
+    bool small_finish;
     RowSplit split;
     size_t smem;
     size_t ws_stats_off, ws_entries_off, ws_bytes;
@@ -1184,12 +1403,16 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (pl.split.nseg < 1) pl.split.nseg = 1;
     pl.split.cps = cps;
     pl.split.grid = rows * pl.split.nseg;
+    // rows of one segment with k <= 128 go to the small finish kernel, and hand their staged tiles over raw
+    pl.small_finish = pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallMaxThreads;
+    pl.raw_cap = pl.small_finish ? pl.vcap : 0;
+    pl.seg_stride = pl.seg_cap > pl.raw_cap ? pl.seg_cap : pl.raw_cap;
     const size_t split_rows = (size_t)rows;
     size_t off = kWsHeaderBytes;
     pl.ws_stats_off = off;
     off = align_up(off + split_rows * pl.split.nseg * sizeof(SegStat), 256);
     pl.ws_entries_off = off;
-    off = align_up(off + split_rows * pl.split.nseg * pl.seg_cap * sizeof(uint2), 256);
+    off = align_up(off + split_rows * pl.split.nseg * pl.seg_stride * sizeof(uint2), 256);
     pl.ws_bytes = off;
     return pl;
 }
@@ -1248,6 +1471,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
     p.nchunks = pl.nchunks; p.split = pl.split;
     p.cap = pl.cap; p.high = pl.high; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
+    p.seg_stride = pl.seg_stride; p.raw_cap = pl.raw_cap;
     p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
@@ -1261,9 +1485,10 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
         return TSLT_ERR_CUDA;
     kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
-    if (pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallThreads) {
-        auto fin = dtype == TSLT_F32 ? sparsify_finish_small_kernel<float> : sparsify_finish_small_kernel<bf16_t>;
-        if (launch_dependent(fin, rows, kSmallThreads, 0, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
+    if (pl.small_finish) {
+        int threads = 0;
+        auto fin = dtype == TSLT_F32 ? small_finish_kernel<float>(k, &threads) : small_finish_kernel<bf16_t>(k, &threads);
+        if (launch_dependent(fin, rows, threads, 0, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     } else {
         auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
         if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -144,6 +144,12 @@ def adversarial_rows(V, dtype):
     r2 = torch.full((V,), -float("inf")); r2[V // 2] = 1.5; r2[5] = 0.5; rows.append(r2)  # fewer finite than k
     r3 = torch.randn(V, generator=g) * 30; rows.append(r3)  # wide dynamic range
     r4 = torch.randn(V, generator=g); r4[::3] = -0.0; r4[1::3] = 0.0; rows.append(r4)   # signed zeros
+    # a few hundred equal maxima over a low background: more tied candidates than the small finish
+    # kernel lists (400), and more tiles holding one than it lists (700)
+    for n_top in (400, 700):
+        r5 = torch.randn(V, generator=g) * 0.01 - 10.0
+        r5[::max(1, V // n_top)] = 3.0
+        rows.append(r5)
     return torch.stack(rows).to(dtype)
 
 
