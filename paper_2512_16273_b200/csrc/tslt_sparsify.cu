@@ -82,6 +82,7 @@ struct SparsifyShared {
     int trim_request;
     int n_above;     // logits counted in bins above thr_bin since it last rose (may lag, never leads a rise)
     // --------------------------------------------------------------------------------------------
+    int n_list;      // expand_staged: vectors listed for reading back
     int cand_count;  // expanded (key, index) candidates
     int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
     uint32_t thr_word;  // thr_bin << 16 | the bf16 pattern the packed lane-tile test compares with; only ever rises
@@ -173,12 +174,20 @@ __device__ __forceinline__ int warp_reserve(int* counter, int cnt, int lane) {
 // the threshold of that moment: a fraction of what is staged.  `base` is the shared-space address
 // of the CTA's dynamic shared memory.
 constexpr int kTileMaskShift = 28;  // a staged tile's word: first vector (below 2^18) | mask of its four vectors << 28
-__device__ __forceinline__ void stage_tile(uint32_t base, const SparsifyParams& p, int thr_bin, uint32_t tile_word,
-                                           float vmax) {
-    const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
-    const uint32_t key = float_to_key(vmax);
+// Count one logit of the row in the histogram, and towards the next rise of the threshold.
+__device__ __forceinline__ void count_logit(uint32_t base, int thr_bin, uint32_t key) {
     hist_count(base + kHistOff, base + kCoarseOff, (int)(key >> kHistShift), 1u);
     if ((int)(key >> kHistShift) > thr_bin) reds_add(base + (uint32_t)offsetof(SparsifyShared, n_above), 1u);
+}
+// Small k counts the tile's largest logit only (two candidates seldom share a tile); large k, where
+// most tiles hold some, counts the largest logit of every marked vector (count_tile false, the
+// caller does it), or the threshold would sit too low.
+constexpr int kCountPerVectorAboveK = 128;
+__device__ __forceinline__ void stage_tile(uint32_t base, const SparsifyParams& p, int thr_bin, uint32_t tile_word,
+                                           float vmax, bool count_tile) {
+    const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
+    const uint32_t key = float_to_key(vmax);
+    if (count_tile) count_logit(base, thr_bin, key);
     if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, tile_word, key);
     else sts_u32(base + (uint32_t)offsetof(SparsifyShared, overflow), 1u);
     if (pos + 1u == (uint32_t)p.vhigh) sts_u32(base + (uint32_t)offsetof(SparsifyShared, trim_request), 1u);
@@ -301,7 +310,13 @@ __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Th
 #pragma unroll
         for (int j = 0; j < kVecsPerLane; ++j)
             if (bf16x2_max(lt.vm[j], P2) != P2) word |= 1u << (kTileMaskShift + j);
-        stage_tile(base, p, th.bin_value(), word, lm);
+        const bool per_vector = p.k > kCountPerVectorAboveK;
+        stage_tile(base, p, th.bin_value(), word, lm, !per_vector);
+        if (per_vector) {
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j)
+                if ((word >> (kTileMaskShift + j)) & 1u) count_logit(base, th.bin_value(), float_to_key(lt.vec_max(j)));
+        }
     }
 }
 __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, float lm, int vec0,
@@ -311,7 +326,13 @@ __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Thr
 #pragma unroll
         for (int j = 0; j < kVecsPerLane; ++j)
             if (lt.vec_max(j) >= th.edge) word |= 1u << (kTileMaskShift + j);
-        stage_tile(base, p, th.bin_value(), word, lm);
+        const bool per_vector = p.k > kCountPerVectorAboveK;
+        stage_tile(base, p, th.bin_value(), word, lm, !per_vector);
+        if (per_vector) {
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j)
+                if ((word >> (kTileMaskShift + j)) & 1u) count_logit(base, th.bin_value(), float_to_key(lt.vec_max(j)));
+        }
     }
 }
 
@@ -330,29 +351,60 @@ __device__ __forceinline__ void load_row_vector(const unsigned char* rowp, int v
 }
 
 // All threads: turn the staged lane tiles whose largest logit is in a bin >= bin into (key, index)
-// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  One thread
-// per marked 16-byte vector of a tile; the vectors come back from global memory (L2 or HBM), four
-// loads in flight per thread.  A full candidate list raises the overflow flag.
+// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  First the
+// marked vectors of the tiles that pass are listed (over the staging buffer itself, its entries
+// held in registers meanwhile), then one thread per listed vector reads it back from global
+// memory (L2 or HBM), four loads in flight per thread: no load is spent on a tile that fails.
+// A full candidate list raises the overflow flag.
+constexpr int kMaxStagedTiles = 2048;  // largest vcap
 template <typename T>
-__device__ __noinline__ void expand_staged(const uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
+__device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
                                            Candidates cb, int cap, int bin, int V, SparsifyShared* sh, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr int kInFlight = 4;
+    constexpr int kMine = kMaxStagedTiles / kBlockThreads;
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
-    const int nitems = min(sh->vec_count, vcap) * kVecsPerLane;
+    const int nv = min(sh->vec_count, vcap);
     const uint32_t min_key = (uint32_t)bin << kHistShift;
-    for (int base = 0; base < nitems; base += kInFlight * kBlockThreads) {
+    const int lane = tid & 31;
+    uint2 mine[kMine];
+    int cnt = 0;
+#pragma unroll
+    for (int c = 0; c < kMine; ++c) {
+        const int i = tid + c * kBlockThreads;
+        mine[c] = i < nv ? staged[i] : make_uint2(0u, 0u);  // key 0 never passes
+        if (mine[c].y >= min_key) cnt += __popc(mine[c].x >> kTileMaskShift);
+    }
+    if (tid == 0) sh->n_list = 0;
+    consumer_sync();  // every entry is in a register: the buffer can take the list
+    uint32_t* list = reinterpret_cast<uint32_t*>(staged);
+    const int list_cap = 2 * vcap;
+    int pos = warp_reserve(&sh->n_list, cnt, lane);
+#pragma unroll
+    for (int c = 0; c < kMine; ++c) {
+        if (mine[c].y >= min_key) {
+#pragma unroll
+            for (int j = 0; j < kVecsPerLane; ++j) {
+                if ((mine[c].x >> (kTileMaskShift + j)) & 1u) {
+                    if (pos < list_cap) list[pos] = (mine[c].x & kVecMask) + 32u * j;
+                    ++pos;
+                }
+            }
+        }
+    }
+    consumer_sync();
+    int nlist = sh->n_list;
+    if (nlist > list_cap) {  // more than two marked vectors per staged tile: take the second pass over the row
+        if (tid == 0) sh->overflow = 1;
+        nlist = 0;
+    }
+    for (int base = 0; base < nlist; base += kInFlight * kBlockThreads) {
         uint4 d[kInFlight];
         int vi[kInFlight];
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u) {
             const int i = base + u * kBlockThreads + tid;
-            vi[u] = -1;
-            if (i < nitems) {
-                const uint2 s = staged[i / kVecsPerLane];
-                const int j = i % kVecsPerLane;
-                if (s.y >= min_key && ((s.x >> (kTileMaskShift + j)) & 1u)) vi[u] = (int)(s.x & kVecMask) + 32 * j;
-            }
+            vi[u] = i < nlist ? (int)list[i] : -1;
             if (vi[u] >= 0 && vi[u] < ext.nvec_full) d[u] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[u]);
         }
 #pragma unroll
@@ -367,10 +419,10 @@ __device__ __noinline__ void expand_staged(const uint2* staged, int vcap, const 
                 if (z[e] >= -3.4028234e38f) {
                     const uint32_t kk = float_to_key(z[e]);
                     if (kk >= min_key) {
-                        const int pos = atomicAdd(cb.count, 1);
-                        if (pos < cap) {
-                            cb.key[pos] = kk;
-                            cb.idx[pos] = e0 + e;
+                        const int pos2 = atomicAdd(cb.count, 1);
+                        if (pos2 < cap) {
+                            cb.key[pos2] = kk;
+                            cb.idx[pos2] = e0 + e;
                         } else {
                             sh->overflow = 1;
                         }
@@ -1373,8 +1425,12 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.cap = 16 * k;
     if (pl.cap < 1024) pl.cap = 1024;
     if (pl.cap > 4096) pl.cap = 4096;
+    // k <= 128: the staged tiles normally go to the finish kernel unexpanded, so the staging buffer
+    // is sized never to fill on ordinary rows (about 8 k tiles are staged) and the candidate list,
+    // used only when it does, is kept small: four CTAs still fit an SM
+    if (k <= 128) pl.cap = 1024;
     pl.high = pl.cap - pl.cap / 4;
-    pl.vcap = k <= 128 ? 1024 : 2048;
+    pl.vcap = k <= 64 ? 1024 : 2048;
     pl.vhigh = k <= 256 ? pl.vcap - pl.vcap / 4 : pl.vcap / 2;  // large k stages most vectors: leave room to react
     pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above); see below
     pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
