@@ -664,7 +664,13 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     const float c = p.c.f;
 
     allow_dependent_launch();
-    for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+    // the first chunk's loads go out before anything else: their latency covers the set-up below
+    const int ch0 = chunk_begin + warp;
+    LaneTile<T> first;
+    if (ch0 < chunk_end) first.load(rowp, ch0 * kVecsPerChunk, lane, ext);
+    static_assert((kHistBins + kCoarseBins) % 4 == 0, "the histograms are cleared 16 bytes at a time");
+    uint4* hist4 = reinterpret_cast<uint4*>(hist);
+    for (int i = tid; i < (kHistBins + kCoarseBins) / 4; i += kBlockThreads) hist4[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid == 0) {
         sh->thr_bin = kLowestFiniteBin;
         sh->thr_word = threshold_word(kLowestFiniteBin);
@@ -684,10 +690,8 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     // afterwards: the streaming loop below starts again at the first chunk (an L2 hit) and counts
     // what it pushes.
     {
-        const int ch0 = chunk_begin + warp;
         if (ch0 < chunk_end) {
-            LaneTile<T> lt;
-            lt.load(rowp, ch0 * kVecsPerChunk, lane, ext);
+            LaneTile<T>& lt = first;
             lt.reduce_max();
             if (k <= 256) {
 #pragma unroll
@@ -706,7 +710,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         __syncthreads();
         if (warp == 0) raise_threshold(sh, k);
         __syncthreads();
-        for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
+        for (int i = tid; i < (kHistBins + kCoarseBins) / 4; i += kBlockThreads) hist4[i] = make_uint4(0u, 0u, 0u, 0u);
         if (tid == 0) sh->n_above = 0;
         __syncthreads();
     }

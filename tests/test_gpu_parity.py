@@ -256,6 +256,35 @@ def test_determinism_and_canaries():
         assert outs[0][n].tobytes() == outs[1][n].tobytes(), n
 
 
+def test_back_to_back_calls_reuse_workspace_and_outputs():
+    """A serving loop calls the two entry points again and again on the same workspace and the
+    same output buffers, with nothing in between.  Eight such steps on a batch of more rows than
+    the machine holds at once (the small finish kernel and the two-launch verifier) must give the
+    first step's bytes every time and leave both status words at zero."""
+    B, gamma, V, k = 80, 8, 32000, 64
+    zq, zp = synth.sequence_logits(B, gamma, V, torch.bfloat16, 0.5, 21, "cuda")
+    rows = B * gamma
+    ud = synth.uniforms((rows, 1), 21, synth.TID_U_DRAFT, "cuda")
+    ua = synth.uniforms((B, gamma), 21, synth.TID_U_ACCEPT, "cuda")
+    us = synth.uniforms((B,), 21, synth.TID_U_SAMPLE, "cuda")
+    ws_s = torch.empty(tslt.sparsify_workspace_bytes(rows, V, k, 1), dtype=torch.uint8, device="cuda")
+    ws_v = torch.empty(tslt.verify_workspace_bytes(B, gamma, V, k), dtype=torch.uint8, device="cuda")
+    s = tslt.sparsify(zq, k, 1.0, 1.0, ud, ws=ws_s)
+    v = tslt.verify(zp, s["idx"], s["logit"], s["count"], s["token"], 1.0, 1.0, ua, us, ws=ws_v)
+    torch.cuda.synchronize()
+    first = {n: to_np(s[n]).copy() for n in ("idx", "logit", "count", "token", "lse", "mass")}
+    first.update({n: to_np(v[n]).copy() for n in ("accepted_len", "out_token")})
+    for _ in range(8):
+        tslt.sparsify(zq, k, 1.0, 1.0, ud, out=s, ws=ws_s)
+        tslt.verify(zp, s["idx"], s["logit"], s["count"], s["token"], 1.0, 1.0, ua, us, out=v, ws=ws_v)
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(ws_s) == 0 and tslt.workspace_status(ws_v) == 0
+    for n in ("idx", "logit", "count", "token", "lse", "mass"):
+        assert to_np(s[n]).tobytes() == first[n].tobytes(), n
+    for n in ("accepted_len", "out_token"):
+        assert to_np(v[n]).tobytes() == first[n].tobytes(), n
+
+
 def run_tree_case(B, expansion, V, dtype, k, T, seed, sigma_t=0.5, what=""):
     parent, ndr, M, depth = synth.complete_tree(expansion)
     N = len(parent)
