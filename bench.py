@@ -383,6 +383,25 @@ def main():
                                              "sparsify_GBps": (B * gamma * V * eb) / a / 1e6,
                                              "verify_GBps": (B * (gamma + 1) * V * eb) / b / 1e6}
 
+    payload = None
+    if args.extras and rank == 0:
+        # the uplink payload of this step's draft rows (Section 2.2 of the paper: entries * (b_prob + b_idx) bits)
+        s_o = tslt.sparsify(zq, k, top_p, T, ud)
+        fmt = tslt.PROB_BF16 if w["dtype"] == "bf16" else tslt.PROB_F32
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        for it in range(4):  # the last round is the timed one
+            evs[0].record()
+            pk = tslt.pack_payload(s_o["idx"], s_o["logit"], s_o["count"], V, fmt)
+            evs[1].record()
+            tslt.unpack_payload(pk["payload"], k, V, fmt)
+            evs[2].record()
+        torch.cuda.synchronize()
+        words, ebits = tslt.payload_words(k, V, fmt)
+        payload = {"format": "bf16" if fmt == tslt.PROB_BF16 else "f32", "entry_bits": ebits,
+                   "bits_per_row": float(pk["bits"].double().mean().item()),
+                   "dense_row_bits": V * (16 if fmt == tslt.PROB_BF16 else 32), "record_words": words,
+                   "pack_ms": evs[0].elapsed_time(evs[1]), "unpack_ms": evs[1].elapsed_time(evs[2])}
+
     cpu_baseline = None
     if rank == 0 and not args.no_cpu_baseline:
         n_rows, n_seq = B * gamma, B  # the whole step: a few seconds on the host cores
@@ -400,6 +419,8 @@ def main():
                 "e2e": e2e, "cpu_baseline": cpu_baseline, "gpu_launches": 4 * args.steps}
         if extras:
             line["sweep"] = extras
+        if payload:
+            line["payload"] = payload
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist

@@ -179,6 +179,43 @@ int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
                      int max_depth, int* accepted_path, int* accepted_len, int* out_token,
                      void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Uplink payload (Section 2.2: a transmitted distribution costs entries * (b_prob + b_idx) bits,
+ * b_idx = ceil(log2 |V|), b_prob = 32 or 16; Section 3, Solution 1: what is sent are the selected
+ * logits and their token ids).  tslt_pack_payload turns the output of tslt_sparsify into what
+ * goes over the link, tslt_unpack_payload turns it back into the arrays tslt_verify and
+ * tslt_tree_verify take.  The paper fixes the bit widths, not a layout; the layout is:
+ *   one record of `words` 32-bit little-endian words per row, `words` given by
+ *   tslt_payload_words = 1 + ceil(k * (b_idx + b_prob) / 32); word 0 = n, the row's number of
+ *   entries (draft_count); the entries follow as one bit stream, entry e in bits
+ *   [e * w, (e + 1) * w), w = b_idx + b_prob, stream bit i being bit (i mod 32) of word
+ *   1 + i / 32; inside an entry the low b_idx bits are the token index, the next b_prob bits the
+ *   logit's bit pattern in the chosen format.  Bits after the last entry are zero.
+ * prob_format: TSLT_PROB_F32 (32 bits, exact), TSLT_PROB_BF16 or TSLT_PROB_F16 (16 bits, the
+ * fp32 logit rounded to nearest even; exact whenever the logits came from bf16 storage and the
+ * format is bf16).  With a 16-bit format the verifier sees the rounded logits: q~ is the
+ * distribution of the rounded values, which is what the draft side must also have sampled from
+ * for the method's guarantees to hold exactly; tslt_sparsify samples from the unrounded ones,
+ * so with fp32 logits and a 16-bit payload the pair is an approximation (for bf16 logits and a
+ * bf16 payload nothing changes).
+ * Arguments (device pointers): idx [rows, k] int32 padded with -1, logit [rows, k] fp32 padded
+ * with -inf, count [rows] int32 (0 <= count <= k, the first count entries of a row are used),
+ * payload [rows, words] uint32.  payload_bits (may be NULL) [rows] int64 gets the paper's
+ * figure n * (b_idx + b_prob) per row; the count word is not part of it.  V >= 1, 1 <= k <=
+ * TSLT_MAX_K, indices must be in [0, V).  An unpacked count above k (a corrupt record) sets the
+ * status flag returned through *device_flag (may be NULL; int32, set to 1, never cleared) and
+ * the row is treated as empty.  No workspace.  Errors: TSLT_ERR_INVALID_ARG, TSLT_ERR_UNSUPPORTED
+ * (unknown format), TSLT_ERR_CUDA.
+ */
+#define TSLT_PROB_F32 0
+#define TSLT_PROB_BF16 1
+#define TSLT_PROB_F16 2
+int tslt_payload_words(int k, int V, int prob_format, int* words, int* entry_bits);
+int tslt_pack_payload(const int* idx, const float* logit, const int* count, int rows, int k, int V,
+                      int prob_format, unsigned int* payload, long long* payload_bits, void* stream);
+int tslt_unpack_payload(const unsigned int* payload, int rows, int k, int V, int prob_format,
+                        int* idx, float* logit, int* count, int* device_flag, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,10 @@ MAX_K = 1024
 EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status",
            "tslt_sparsify_workspace_bytes", "tslt_sparsify",
            "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
-           "tslt_tree_verify_workspace_bytes", "tslt_tree_verify"]
+           "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
+           "tslt_payload_words", "tslt_pack_payload", "tslt_unpack_payload"]
+
+PROB_F32, PROB_BF16, PROB_F16 = 0, 1, 2
 
 
 class TsltError(RuntimeError):
@@ -71,6 +74,12 @@ def lib() -> ctypes.CDLL:
     L.tslt_tree_verify.restype = i
     L.tslt_tree_verify.argtypes = [p, i, i, i, i, ll, p, p, i, i, p, p, p, p, f, f, p, p, i, p, p, p,
                                    p, sz, p]
+    L.tslt_payload_words.restype = i
+    L.tslt_payload_words.argtypes = [i, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
+    L.tslt_pack_payload.restype = i
+    L.tslt_pack_payload.argtypes = [p, p, p, i, i, i, i, p, p, p]
+    L.tslt_unpack_payload.restype = i
+    L.tslt_unpack_payload.argtypes = [p, i, i, i, i, p, p, p, p, p]
     _lib = L
     return L
 
@@ -350,3 +359,44 @@ def payload_bits(count: int, V: int, b_prob: int = 32) -> int:
     """Uplink payload of one sparse distribution, the per-distribution data volume of Section
     2.2 with the vocabulary size replaced by the retained count: count * (b_prob + ceil(log2 V))."""
     return int(count) * (int(b_prob) + math.ceil(math.log2(V)))
+
+
+def payload_words(k: int, V: int, prob_format: int):
+    """(32-bit words per row record, bits per entry) of the uplink payload."""
+    w, b = ctypes.c_int(0), ctypes.c_int(0)
+    _check(lib().tslt_payload_words(k, V, prob_format, ctypes.byref(w), ctypes.byref(b)), "tslt_payload_words")
+    return int(w.value), int(b.value)
+
+
+def pack_payload(idx: torch.Tensor, logit: torch.Tensor, count: torch.Tensor, V: int, prob_format: int) -> dict:
+    """tslt_pack_payload on the output of sparsify: idx / logit [rows, k], count [rows].
+    Returns dict(payload [rows, words] int32 (bit patterns), bits [rows] int64)."""
+    _cuda(idx, "idx", torch.int32); _cuda(logit, "logit", torch.float32); _cuda(count, "count", torch.int32)
+    k = idx.shape[-1]
+    rows = count.numel()
+    if idx.numel() != rows * k or logit.numel() != rows * k:
+        raise ValueError("idx / logit / count shapes do not match")
+    words, _ = payload_words(k, V, prob_format)
+    payload = torch.empty(rows, words, dtype=torch.int32, device=idx.device)
+    bits = torch.empty(rows, dtype=torch.int64, device=idx.device)
+    _check(lib().tslt_pack_payload(_ptr(idx), _ptr(logit), _ptr(count), rows, k, V, prob_format, _ptr(payload),
+                                   _ptr(bits), _stream()), "tslt_pack_payload")
+    return {"payload": payload, "bits": bits}
+
+
+def unpack_payload(payload: torch.Tensor, k: int, V: int, prob_format: int) -> dict:
+    """tslt_unpack_payload: records [rows, words] -> dict(idx, logit [rows, k], count [rows], flag [1])
+    in the form verify / tree_verify take."""
+    _cuda(payload, "payload", torch.int32)
+    words, _ = payload_words(k, V, prob_format)
+    if payload.dim() != 2 or payload.shape[1] != words:
+        raise ValueError("payload must be [rows, %d] for this k, V and format" % words)
+    rows = payload.shape[0]
+    dev = payload.device
+    o = {"idx": torch.empty(rows, k, dtype=torch.int32, device=dev),
+         "logit": torch.empty(rows, k, dtype=torch.float32, device=dev),
+         "count": torch.empty(rows, dtype=torch.int32, device=dev),
+         "flag": torch.zeros(1, dtype=torch.int32, device=dev)}
+    _check(lib().tslt_unpack_payload(_ptr(payload), rows, k, V, prob_format, _ptr(o["idx"]), _ptr(o["logit"]),
+                                     _ptr(o["count"]), _ptr(o["flag"]), _stream()), "tslt_unpack_payload")
+    return o
