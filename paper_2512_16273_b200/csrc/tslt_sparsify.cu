@@ -1,26 +1,32 @@
 // tslt_sparsify: draft-side sparsify-then-sample (Section 3, Solution 1; the sampling steps
-// of Algorithms 2 and 4) as one kernel.
+// of Algorithms 2 and 4) as two kernels on the caller's stream.
 //
-// One CTA reads one segment of one logits row from HBM exactly once, with 16-byte loads that go
-// straight to registers (each warp instruction covers 512 contiguous bytes).  Warps run freely:
-// there is no barrier in the steady state.  Each lane keeps an online (max, sum) for the softmax
-// normaliser and copies every 16-byte vector that holds a logit at or above a running threshold
-// into a shared staging buffer (the test is on the vector's packed maximum, so a lane tile
-// without a candidate costs a handful of instructions and nothing is searched inside a vector
-// while streaming).  The threshold comes from a 4096-bin histogram of the order-preserving keys
-// (top 12 bits) of the staged vectors' maxima: the highest bin above which at least k distinct
-// logits have been seen is a lower bound on the row's k-th largest logit, so no member of the
-// top-k is ever skipped, whatever the order in which the warps run.  The warps take turns
-// rescanning the histogram, which tightens the threshold as the row streams by.  Staged vectors
-// are later expanded into (key, index) candidates, again filtered against the threshold.  The CTA that holds the whole row (the only
-// one, or the last of the row's segments to finish) then finds the bin that holds the k-th
-// largest logit, keeps everything above it, breaks the tie inside it exactly (logit descending,
-// index ascending), applies the top-rho cut, renormalises in fp64, draws the samples by inverse
-// CDF and writes the (index, logit) pairs in ascending index.
+// Streaming kernel.  One CTA reads one segment of one logits row from HBM exactly once, with
+// 16-byte loads that go straight to registers (each warp instruction covers 512 contiguous
+// bytes).  Warps run freely: there is no barrier in the steady state.  Each lane keeps an online
+// (max, sum) for the softmax normaliser and stages every lane tile (its four 16-byte vectors of a
+// 2 KB chunk) that holds a logit at or above a running threshold: 8 bytes (where the tile is,
+// which of its vectors hold a candidate, the key of its largest logit), no data.  The test is on
+// the tile's packed maximum, so a tile without a candidate costs a handful of instructions and
+// nothing is searched inside a vector while streaming.  The threshold comes from a 4096-bin
+// histogram of the order-preserving keys (top 12 bits) of what is staged: the highest bin above
+// which at least k distinct logits have been counted is a lower bound on the row's k-th largest
+// logit, so no member of the top-k is ever skipped, whatever the order in which the warps run.
+// The warps take turns at checking whether enough has been counted for the threshold to rise,
+// and rescan the histogram then.  At the end the segment hands over its per-warp (max, sum)
+// pairs and either the staged tiles as they are (k <= 128, the usual case) or the (key, index)
+// candidates it expanded from them by reading the marked vectors back.
+//
+// Finish kernel (launched with programmatic stream serialization, so that it is in place when
+// the streaming kernel ends).  One CTA per row: candidates from the hand-over, the bin that holds
+// the k-th largest logit, everything above it, the tie inside it broken exactly (logit
+// descending, index ascending), the top-rho cut, renormalisation in fp64, the samples by inverse
+// CDF, the (index, logit) pairs in ascending index.
 //
 // Rare paths: a staging buffer that fills up is expanded early by all warps together (and the
-// candidate list compacted to the current threshold); a buffer that overflows before they can meet (adversarial
-// rows: sorted ascending, all equal) is abandoned and the segment's exact top-k is selected
+// candidate list compacted to the current threshold); a buffer that overflows before they can
+// meet (adversarial rows: sorted ascending, all equal) is abandoned and the segment is read a
+// second time against the final threshold; a candidate list that overflows even then is selected
 // again from global memory with a radix select.
 #include <math.h>
 
