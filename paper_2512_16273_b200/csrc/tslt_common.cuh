@@ -90,6 +90,32 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 __device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void wait_for_primary_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// A row-ready flag between the two kernels of tslt_sparsify.  The finish kernel is the streaming
+// kernel's programmatic dependent, so by the time one of its CTAs runs, every CTA of the streaming
+// kernel has started (dependents are scheduled once all CTAs of the primary have issued
+// launch_dependents or exited): each streaming CTA still running is resident and finishes on its
+// own, whatever the finish CTAs do.  A finish CTA can therefore begin as soon as its own row has
+// been handed over instead of when the whole streaming kernel has ended.  The wait is bounded all
+// the same: after kReadyPollLimit polls (about a second) the CTA falls back to griddepcontrol.wait,
+// which returns when the streaming kernel has completed.  Without the launch attribute the finish
+// kernel starts after the streaming kernel and finds every flag set.  Each streaming CTA clears
+// its row's flag (and fences) before it issues launch_dependents, so a flag left set by an earlier
+// call on the same workspace is gone before any finish CTA can look at it.
+constexpr int kReadyPollLimit = 1 << 22;
+__device__ __forceinline__ void publish_row_ready(int* flag) {  // one thread, after a barrier that follows the row's writes
+    __threadfence();
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(1) : "memory");
+}
+__device__ __forceinline__ bool poll_row_ready(const int* flag) {  // one thread
+    for (int it = 0; it < kReadyPollLimit; ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v != 0) return true;
+        __nanosleep(200);
+    }
+    return false;
+}
+
 template <typename Params>
 inline cudaError_t launch_dependent(void (*kernel)(const Params), unsigned grid, unsigned block, size_t smem,
                                     cudaStream_t st, const Params& p) {

@@ -79,6 +79,7 @@ struct SparsifyParams {
     int seg_cap;         // most candidates a segment hands over
     int seg_stride;      // entries reserved per segment
     int raw_cap;         // > 0: a segment whose staging buffer never filled hands its staged tiles over unexpanded
+    int* row_ready;      // [rows] (small finish kernel only, else NULL): set to 1 when the row has been handed over
 };
 
 struct SparsifyShared {
@@ -669,7 +670,6 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     const int k = p.k;
     const float c = p.c.f;
 
-    allow_dependent_launch();
     // the first chunk's loads go out before anything else: their latency covers the set-up below
     const int ch0 = chunk_begin + warp;
     LaneTile<T> first;
@@ -685,6 +685,11 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         sh->overflow = 0;
         sh->trim_request = 0;
         sh->n_above = 0;
+        // The row's ready flag is cleared here, by the CTA that will set it; the store is fenced
+        // below, before this CTA lets the finish kernel be scheduled.  A finish CTA runs only after
+        // every streaming CTA has passed that point, so it never sees a flag left by an earlier
+        // call, and the workspace needs no clearing between calls.
+        if (p.row_ready) *(volatile int*)&p.row_ready[row] = 0;
     }
     __syncthreads();
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
@@ -720,6 +725,9 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         if (tid == 0) sh->n_above = 0;
         __syncthreads();
     }
+    // (thread 0's fence comes long after its store of the cleared flag, and holds up only its own warp)
+    if (tid == 0 && p.row_ready) __threadfence();
+    allow_dependent_launch();
 
     // ---- streaming: no barriers; warp w rescans the histogram on its turn --------------------------
     LaneSum ls;
@@ -788,6 +796,8 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             st->n = n;
             st->raw_bin = sh->thr_bin;
         }
+        __syncthreads();  // every thread's part of the hand-over is written
+        if (tid == 0 && p.row_ready) publish_row_ready(&p.row_ready[row]);
         return;
     }
 
@@ -820,6 +830,8 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         st->n = n;
         st->raw_bin = -1;
     }
+    __syncthreads();  // every thread's part of the hand-over is written
+    if (tid == 0 && p.row_ready) publish_row_ready(&p.row_ready[row]);
 }
 
 // Second launch: one CTA per row merges the row's segments and finishes it.
@@ -1208,7 +1220,7 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
         while (m) {  // few: read them again (cached) rather than keep eight entries in registers
             const int u = __ffs(m) - 1;
             m &= m - 1;
-            const uint32_t w = __ldg(&ent[base + u * NT + tid].x);
+            const uint32_t w = __ldcg(&ent[base + u * NT + tid].x);
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j) {
                 if ((w >> (kTileMaskShift + j)) & 1u) {
@@ -1272,7 +1284,12 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
     float u_raw = 0.f;
     if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];  // an input: may be read early
-    wait_for_primary_kernel();  // nothing the streaming kernel wrote is read before this point
+    // Nothing the streaming kernel wrote is read before this point.  The row's own ready flag is
+    // enough to go on (see poll_row_ready); if it does not come, the end of the streaming kernel is.
+    if (tid == 0) sm.n_cut = poll_row_ready(&p.row_ready[row]) ? 1 : 0;
+    small_sync<NT>();
+    if (!sm.n_cut) wait_for_primary_kernel();
+    small_sync<NT>();
     if (row == 0 && tid == 0) *p.status = 0;
     // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
     const SegStat* st = &p.seg_stats[row];
@@ -1394,6 +1411,9 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
         }
         p.token[(size_t)row * p.num_samples + sidx] = tok;
     }
+    // This kernel's completion must imply the streaming kernel's (what follows on the stream relies
+    // on it): one CTA sees to that; the others leave and make room.
+    if (row == 0) wait_for_primary_kernel();
 }
 
 // The small finish kernel for this k: a warp's worth of threads per 32 of k, at least two warps.
@@ -1411,7 +1431,7 @@ struct SparsifyPlan {
     bool small_finish;
     RowSplit split;
     size_t smem;
-    size_t ws_stats_off, ws_entries_off, ws_bytes;
+    size_t ws_stats_off, ws_entries_off, ws_ready_off, ws_bytes;
 };
 
 static int sm_count_cached() {
@@ -1479,6 +1499,8 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     off = align_up(off + split_rows * pl.split.nseg * sizeof(SegStat), 256);
     pl.ws_entries_off = off;
     off = align_up(off + split_rows * pl.split.nseg * pl.seg_stride * sizeof(uint2), 256);
+    pl.ws_ready_off = off;
+    if (pl.small_finish) off = align_up(off + split_rows * sizeof(int), 256);
     pl.ws_bytes = off;
     return pl;
 }
@@ -1543,6 +1565,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.status = (int*)ws;
     p.seg_stats = (SegStat*)(ws + pl.ws_stats_off);
     p.seg_entries = (uint2*)(ws + pl.ws_entries_off);
+    p.row_ready = pl.small_finish ? (int*)(ws + pl.ws_ready_off) : nullptr;
 
     cudaStream_t st = (cudaStream_t)stream;
     auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
