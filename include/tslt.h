@@ -21,8 +21,10 @@
  *   - uniforms are fp32 in [0,1); a value >= 1 is read as the largest float below 1.
  *   - "sample" always means inverse CDF in ascending token index: the first index whose
  *     cumulative mass exceeds u * total.
- *   - no kernel waits on another CTA: CTAs that share a row or a sequence meet through a
- *     ticket counter in the workspace and the last one to arrive carries on.  The first word
+ *   - CTAs that share a row or a sequence meet through a ticket counter in the workspace and
+ *     the last one to arrive carries on; the one wait on another CTA (a row's finish CTA on the
+ *     row's streaming CTA in tslt_sparsify, k <= 128) is one-way, bounded, and falls back to the
+ *     end of the streaming kernel.  The first word
  *     of the workspace is a device status word (0 = fine) that tslt_workspace_status reads
  *     back; a non-zero word is reported as TSLT_ERR_DEVICE_STATUS.
  */
