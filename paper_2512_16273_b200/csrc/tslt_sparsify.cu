@@ -79,7 +79,7 @@ struct SparsifyParams {
     int seg_cap;         // most candidates a segment hands over
     int seg_stride;      // entries reserved per segment
     int raw_cap;         // > 0: a segment whose staging buffer never filled hands its staged tiles over unexpanded
-    int* row_ready;      // [rows] (small finish kernel only, else NULL): set to 1 when the row has been handed over
+    int* row_ready;      // [rows] (rows of one segment only, else NULL): set to 1 when the row has been handed over
 };
 
 struct SparsifyShared {
@@ -849,12 +849,24 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     // the uniforms are needed last: ask for their cache line now
     if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) sh->overflow = 0;
-    wait_for_primary_kernel();  // nothing the streaming kernel wrote is read before this point
+    // Nothing the streaming kernel wrote is read before this point.  A row of one segment goes on
+    // as soon as its own ready flag is set (see poll_row_ready); rows cut into segments, and a
+    // flag that does not come, wait for the end of the streaming kernel.
+    if (p.row_ready) {
+        if (tid == 0) sh->n_list = poll_row_ready(&p.row_ready[row]) ? 1 : 0;
+        __syncthreads();
+        if (!sh->n_list) wait_for_primary_kernel();
+        __syncthreads();
+    } else {
+        wait_for_primary_kernel();
+    }
     if (row == 0 && tid == 0) *p.status = 0;
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
     double Mrow, Srow;
     gather_segments(p, row, p.split.nseg, cb, sh, tid, &Mrow, &Srow);
     finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, tid);
+    // this kernel's completion must imply the streaming kernel's: one CTA sees to that
+    if (row == 0 && p.row_ready) wait_for_primary_kernel();
 }
 
 // Position of entry (key, idx) of the buffer in the order (key descending, idx ascending) /
@@ -1500,7 +1512,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.ws_entries_off = off;
     off = align_up(off + split_rows * pl.split.nseg * pl.seg_stride * sizeof(uint2), 256);
     pl.ws_ready_off = off;
-    if (pl.small_finish) off = align_up(off + split_rows * sizeof(int), 256);
+    if (pl.split.nseg == 1) off = align_up(off + split_rows * sizeof(int), 256);
     pl.ws_bytes = off;
     return pl;
 }
@@ -1565,7 +1577,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.status = (int*)ws;
     p.seg_stats = (SegStat*)(ws + pl.ws_stats_off);
     p.seg_entries = (uint2*)(ws + pl.ws_entries_off);
-    p.row_ready = pl.small_finish ? (int*)(ws + pl.ws_ready_off) : nullptr;
+    p.row_ready = pl.split.nseg == 1 ? (int*)(ws + pl.ws_ready_off) : nullptr;  // rows of one segment only
 
     cudaStream_t st = (cudaStream_t)stream;
     auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
