@@ -685,13 +685,17 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         sh->overflow = 0;
         sh->trim_request = 0;
         sh->n_above = 0;
-        // The row's ready flag is cleared here, by the CTA that will set it; the store is fenced
-        // below, before this CTA lets the finish kernel be scheduled.  A finish CTA runs only after
-        // every streaming CTA has passed that point, so it never sees a flag left by an earlier
-        // call, and the workspace needs no clearing between calls.
-        if (p.row_ready) *(volatile int*)&p.row_ready[row] = 0;
+        // The row's ready flag is cleared here, by the CTA that will set it, and the store is fenced
+        // before the barrier after which the first thread of this CTA lets the finish kernel be
+        // scheduled.  A finish CTA runs only after every streaming CTA has passed that point, so it
+        // never sees a flag left by an earlier call, and the workspace needs no clearing between calls.
+        if (p.row_ready) {
+            *(volatile int*)&p.row_ready[row] = 0;
+            __threadfence();
+        }
     }
     __syncthreads();
+    allow_dependent_launch();
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
 
     // ---- first threshold, from the segment's first chunks (one per warp) ---------------------------
@@ -725,9 +729,6 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         if (tid == 0) sh->n_above = 0;
         __syncthreads();
     }
-    // (thread 0's fence comes long after its store of the cleared flag, and holds up only its own warp)
-    if (tid == 0 && p.row_ready) __threadfence();
-    allow_dependent_launch();
 
     // ---- streaming: no barriers; warp w rescans the histogram on its turn --------------------------
     LaneSum ls;
