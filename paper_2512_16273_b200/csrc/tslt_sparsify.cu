@@ -51,7 +51,10 @@ struct SegStat {
     float M[kWarps];   // per warp: reference exponent (base 2)
     int n;             // entries written for the segment
     int raw_bin;       // -1: the entries are (key, idx) candidates; else they are staged lane tiles (first vector
-                       // and vector mask, key of the largest logit) and this is the segment's final threshold bin
+                       // and vector mask, relative key of the largest logit) and this is the segment's final
+                       // threshold bin
+    float z0;          // the segment's offset: bins are over z - z0 (see rel_key)
+    int pad;
 };
 
 struct SparsifyParams {
@@ -91,7 +94,9 @@ struct SparsifyShared {
     // --------------------------------------------------------------------------------------------
     int n_list;      // expand_staged: vectors listed for reading back
     int cand_count;  // expanded (key, index) candidates
-    int thr_bin;     // candidates are the logits whose key bin is >= thr_bin; only ever rises
+    int thr_bin;     // candidates are the logits whose relative key's bin is >= thr_bin; only ever rises
+    float z0;        // the segment's offset (see rel_key); fixed once the first chunks have been looked at
+    uint32_t thr_edge_key;  // fp32 rows: order-preserving key of the raw-domain threshold the lane-tile test uses
     uint32_t thr_word;  // thr_bin << 16 | the bf16 pattern the packed lane-tile test compares with; only ever rises
     int sel_bin, sel_above;  // bin of the k-th largest logit and the number of logits in higher bins
     int n_win, n_bnd;
@@ -132,12 +137,35 @@ template <typename T> struct GlobalSrc {
 
 __device__ __forceinline__ float bin_lower_edge(int bin) { return key_to_float((uint32_t)bin << kHistShift); }
 
+// The histogram's bins are over the logits RELATIVE to an offset z0 taken from the segment's first
+// chunks (their largest logit): a bin is the top 12 bits of the order-preserving key of z - z0.
+// Float keys are relative (three mantissa bits: 12.5 % of the value), so bins over the raw logits
+// would be as wide as the logits are large: a row of N(20, 1) logits put thousands of them in the
+// threshold's bin and fell off every fast path (5.7 ms for the bench batch instead of 0.23).
+// Relative to a value near the row's maximum the bins are finest exactly where the top-k lives,
+// whatever the offset and scale of the logits.  z - z0 is monotone in z (rounding is), which is all
+// the threshold argument needs.  Candidates always carry their RAW keys: exact selection and
+// ordering never see z0.
+__device__ __forceinline__ uint32_t rel_key(float z, float z0) { return float_to_key(z - z0); }
+
+// A raw-domain value that every logit whose relative bin is >= bin is at or above: the bin's lower
+// edge moved back by z0, less a margin that covers the roundings of z - z0, of edge + z0 and of the
+// subtraction itself (2^-21 of the magnitudes involved; each rounding is at most 2^-24 of one).
+// Being low only lets a few more tiles through the streaming test; what they hold is then judged
+// by its relative key.
+__device__ __forceinline__ float raw_edge_below(int bin, float z0) {
+    const float es = bin_lower_edge(bin);
+    const float er = es + z0;
+    return er - 4.76837158e-7f * (fabsf(es) + fabsf(z0) + fabsf(er));
+}
+
 // ---- shared memory by address: one out-of-line copy of the rare paths, still shared-space code ----
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ float lds_f32(uint32_t addr) { return __uint_as_float(lds_u32(addr)); }
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -193,7 +221,7 @@ constexpr int kCountPerVectorAboveK = 128;
 __device__ __forceinline__ void stage_tile(uint32_t base, const SparsifyParams& p, int thr_bin, uint32_t tile_word,
                                            float vmax, bool count_tile) {
     const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
-    const uint32_t key = float_to_key(vmax);
+    const uint32_t key = rel_key(vmax, lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0)));
     if (count_tile) count_logit(base, thr_bin, key);
     if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, tile_word, key);
     else sts_u32(base + (uint32_t)offsetof(SparsifyShared, overflow), 1u);
@@ -260,10 +288,12 @@ __device__ __noinline__ int scan_boundary(uint32_t hist_addr, uint32_t coarse_ad
     return cbin * 32 + 31 - fl;
 }
 
-// The bf16 side of the threshold word: P = the largest bf16 value below the lower edge of `bin`.
-__device__ __forceinline__ uint32_t threshold_word(int bin) {
-    uint32_t k16 = ((uint32_t)bin << (kHistShift - 16)) - 1u;  // key of the value just below the edge
-    if (k16 == 0x7fffu) k16 = 0x7ffeu;                         // -0 shares +0's key: step past it
+// The bf16 side of the threshold word: P = the largest bf16 value below raw_edge_below(bin, z0),
+// never below -inf (the pattern that lets every finite logit through).
+__device__ __forceinline__ uint32_t threshold_word(int bin, float z0) {
+    uint32_t k16 = float_to_key(raw_edge_below(bin, z0)) >> 16;  // bf16 key at or below the edge ...
+    k16 = k16 > 0x80u ? k16 - 1u : 0x7fu;                       // ... then strictly below; 0x7f is -inf
+    if (k16 == 0x7fffu) k16 = 0x7ffeu;                           // -0 shares +0's key: step past it
     const uint32_t b16 = (k16 & 0x8000u) ? (k16 & 0x7fffu) : (~k16 & 0xffffu);
     return ((uint32_t)bin << 16) | b16;
 }
@@ -276,8 +306,10 @@ __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
     if ((threadIdx.x & 31) == 0) {
         const int cur = *(volatile int*)&sh->thr_bin;
         if (found > cur) {
+            const float z0 = sh->z0;
             atomicMax(&sh->thr_bin, found);
-            atomicMax(&sh->thr_word, threshold_word(found));
+            atomicMax(&sh->thr_word, threshold_word(found, z0));
+            atomicMax(&sh->thr_edge_key, float_to_key(raw_edge_below(found, z0)));
         }
         // what is counted above the boundary bin starts the count towards the next rise (a stale
         // value only costs or delays a rescan)
@@ -285,17 +317,17 @@ __device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
     }
 }
 
-// The running threshold in the form the lane-tile test wants.  A logit is a candidate iff its
-// key bin is >= thr_bin, i.e. iff it is >= the bin's lower edge.
-//   fp32 rows: the edge itself, compared as floats.
-//   bf16 rows: P = the largest bf16 value below the edge, in both halves of a word; a packed
+// The running threshold in the form the lane-tile test wants: a raw-domain bound that lets through
+// every logit whose relative bin is >= thr_bin (and a few more, see raw_edge_below).
+//   fp32 rows: the bound itself, compared as floats.
+//   bf16 rows: P = the largest bf16 value below the bound, in both halves of a word; a packed
 //              word w holds a candidate iff max.bf16x2(w, P) != P (NaN halves never differ).
 template <typename T> struct Threshold;
 template <> struct Threshold<float> {
     int bin;
     float edge;
     __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh)
-        : bin(*(const volatile int*)&sh->thr_bin), edge(bin_lower_edge(bin)) {}
+        : bin(*(const volatile int*)&sh->thr_bin), edge(key_to_float(*(const volatile uint32_t*)&sh->thr_edge_key)) {}
     __device__ __forceinline__ int bin_value() const { return bin; }
 };
 template <> struct Threshold<bf16_t> {
@@ -322,7 +354,9 @@ __device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Th
         if (per_vector) {
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j)
-                if ((word >> (kTileMaskShift + j)) & 1u) count_logit(base, th.bin_value(), float_to_key(lt.vec_max(j)));
+                if ((word >> (kTileMaskShift + j)) & 1u)
+                    count_logit(base, th.bin_value(),
+                                rel_key(lt.vec_max(j), lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0))));
         }
     }
 }
@@ -338,7 +372,9 @@ __device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Thr
         if (per_vector) {
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j)
-                if ((word >> (kTileMaskShift + j)) & 1u) count_logit(base, th.bin_value(), float_to_key(lt.vec_max(j)));
+                if ((word >> (kTileMaskShift + j)) & 1u)
+                    count_logit(base, th.bin_value(),
+                                rel_key(lt.vec_max(j), lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0))));
         }
     }
 }
@@ -373,6 +409,7 @@ __device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsign
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
     const int nv = min(sh->vec_count, vcap);
     const uint32_t min_key = (uint32_t)bin << kHistShift;
+    const float z0 = sh->z0;
     const int lane = tid & 31;
     uint2 mine[kMine];
     int cnt = 0;
@@ -424,11 +461,10 @@ __device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsign
 #pragma unroll
             for (int e = 0; e < kPer; ++e) {
                 if (z[e] >= -3.4028234e38f) {
-                    const uint32_t kk = float_to_key(z[e]);
-                    if (kk >= min_key) {
+                    if (rel_key(z[e], z0) >= min_key) {
                         const int pos2 = atomicAdd(cb.count, 1);
                         if (pos2 < cap) {
-                            cb.key[pos2] = kk;
+                            cb.key[pos2] = float_to_key(z[e]);
                             cb.idx[pos2] = e0 + e;
                         } else {
                             sh->overflow = 1;
@@ -451,6 +487,7 @@ __device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsign
 __device__ __noinline__ void compact_buffer(Candidates cb, int bin, SparsifyShared* sh, int tid) {
     constexpr int E = 16;  // cap <= 4096 = 16 * 256
     const int n = min(*cb.count, E * kBlockThreads);
+    const float z0 = sh->z0;
     uint32_t ek[E];
     int ei[E];
     unsigned keep = 0;
@@ -463,7 +500,7 @@ __device__ __noinline__ void compact_buffer(Candidates cb, int bin, SparsifyShar
         if (i < n) {
             ek[e] = cb.key[i];
             ei[e] = cb.idx[i];
-            if ((int)(ek[e] >> kHistShift) >= bin) {
+            if ((int)(rel_key(key_to_float(ek[e]), z0) >> kHistShift) >= bin) {
                 keep |= 1u << e;
                 ++cnt;
             }
@@ -516,7 +553,9 @@ __device__ __noinline__ void recollect_from_global(const unsigned char* rowp, in
         sh->overflow = 0;
     }
     consumer_sync();
-    const float edge = bin_lower_edge(bin);
+    const float z0 = sh->z0;
+    const float edge = raw_edge_below(bin, z0);  // for the tile and vector tests; a logit is judged by its relative key
+    const uint32_t min_key = (uint32_t)bin << kHistShift;
     for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
         LaneTile<T> lt;
         lt.load(rowp, ch * kVecsPerChunk, lane, ext);
@@ -527,7 +566,7 @@ __device__ __noinline__ void recollect_from_global(const unsigned char* rowp, in
 #pragma unroll
                 for (int e = 0; e < kPer; ++e) {
                     const float z = lt.elem(j, e);
-                    if (z >= edge) {
+                    if (z >= -3.4028234e38f && rel_key(z, z0) >= min_key) {
                         const int pos = atomicAdd(cb.count, 1);
                         if (pos < cap) {
                             cb.key[pos] = float_to_key(z);
@@ -679,7 +718,8 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     for (int i = tid; i < (kHistBins + kCoarseBins) / 4; i += kBlockThreads) hist4[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid == 0) {
         sh->thr_bin = kLowestFiniteBin;
-        sh->thr_word = threshold_word(kLowestFiniteBin);
+        sh->thr_word = threshold_word(kLowestFiniteBin, 0.f);  // P = -inf: every finite logit passes
+        sh->thr_edge_key = float_to_key(-3.4028234e38f);
         sh->cand_count = 0;
         sh->vec_count = 0;
         sh->overflow = 0;
@@ -694,8 +734,18 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
             __threadfence();
         }
     }
+    // the segment's offset for the histogram's bins: the largest logit of its first chunks (see rel_key)
+    float first_max = -INFINITY;
+    if (ch0 < chunk_end) first_max = first.reduce_max();
+    first_max = warp_max(first_max);
+    if (lane == 0) sh->scratch[warp] = (double)first_max;
     __syncthreads();
     allow_dependent_launch();
+    float z0 = (float)sh->scratch[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) z0 = fmaxf(z0, (float)sh->scratch[w]);
+    if (!(z0 >= -3.4028234e38f && z0 <= 3.4028234e38f)) z0 = 0.f;  // nothing finite there: no offset
+    if (tid == 0) sh->z0 = z0;  // read by others only after the barriers below
     Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
 
     // ---- first threshold, from the segment's first chunks (one per warp) ---------------------------
@@ -706,19 +756,18 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
     // what it pushes.
     {
         if (ch0 < chunk_end) {
-            LaneTile<T>& lt = first;
-            lt.reduce_max();
+            LaneTile<T>& lt = first;  // (reduce_max() already called)
             if (k <= 256) {
 #pragma unroll
                 for (int j = 0; j < kVecsPerLane; ++j) {
                     const float z = lt.vec_max(j);
-                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(float_to_key(z) >> kHistShift), 1u);
+                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(rel_key(z, z0) >> kHistShift), 1u);
                 }
             } else {
 #pragma unroll 4
                 for (int e = 0; e < kVecsPerLane * kPer; ++e) {
                     const float z = lt.elem(e / kPer, e % kPer);
-                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(float_to_key(z) >> kHistShift), 1u);
+                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(rel_key(z, z0) >> kHistShift), 1u);
                 }
             }
         }
@@ -796,6 +845,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_ke
         if (tid == 0) {
             st->n = n;
             st->raw_bin = sh->thr_bin;
+            st->z0 = sh->z0;
         }
         __syncthreads();  // every thread's part of the hand-over is written
         if (tid == 0 && p.row_ready) publish_row_ready(&p.row_ready[row]);
@@ -1092,11 +1142,16 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 // finishing a row is a chain of dependent steps (trips to memory, rank counting, two scans), and
 // what it costs machine-wide is the length of that chain times the number of waves.
 constexpr int kSmallMaxThreads = 128;
-constexpr int kSmallCand = 256;  // candidates a row may bring
+constexpr int kSmallCand = 256;      // candidates a row may bring as (key, index) entries
+// Candidates the kernel may make from a row's staged tiles: 256, and 512 for k above 96, where
+// 256 is only 2 k and the threshold bin's share can exceed it on ordinary rows.  (512 everywhere
+// cost the 64-thread kernel 9 us on the bench batch: fewer finish CTAs fit beside the streaming
+// CTAs of the last wave.)
+__host__ __device__ constexpr int small_list_cap(int nt) { return nt > 96 ? 512 : 256; }
 constexpr int kSmallPass = 512;  // marked vectors in the staged tiles of a row that pass its final threshold
 
-struct SmallShared {
-    unsigned long long comp[kSmallCand];  // candidates as key << 32 | ~index: larger is earlier in the top-k order
+template <int kList> struct SmallShared {
+    unsigned long long comp[kList];  // candidates as key << 32 | ~index: larger is earlier in the top-k order
     uint32_t wkey[kSmallMaxThreads];  // winners in (key descending, index ascending) order, then in ascending index
     int widx[kSmallMaxThreads];
     uint32_t okey[kSmallMaxThreads];
@@ -1147,12 +1202,13 @@ template <int NT> __device__ __forceinline__ double small_max(double v, int tid,
 }
 
 // The slow way to a row's k winners from its staged tiles: one winner per round, each round a pass
-// over the marked vectors of the passing tiles.  Only there to be correct when a row has more
-// tied candidates around its k-th logit than the lists of the kernel below hold.
+// over the marked vectors of the passing tiles (the kernel's list of them if it held them all).
+// Only there to be correct when a row has more tied candidates around its k-th logit than the
+// lists of the kernel below hold.
 // composite = key << 32 | ~index: larger is earlier in (logit descending, index ascending)
 template <typename T, int NT>
 __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                               SmallShared* sm, int tid) {
+                                               float z0, int n_listed, SmallShared<small_list_cap(NT)>* sm, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
@@ -1162,16 +1218,24 @@ __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row,
     int found = 0;
     for (; found < p.k; ++found) {
         unsigned long long best = 0ull;
-        for (int i = tid; i < n_tiles * kVecsPerLane; i += NT) {
-            const uint2 e = __ldcg(&ent[i / kVecsPerLane]);
-            const int j = i % kVecsPerLane;
-            if (e.y < min_key || !((e.x >> (kTileMaskShift + j)) & 1u)) continue;
-            const int vi = (int)(e.x & kVecMask) + 32 * j;
+        // the vectors to look at: those listed in sm->pass (n_listed >= 0), else every marked vector
+        // of every passing tile of the hand-over
+        const int n_items = n_listed >= 0 ? n_listed : n_tiles * kVecsPerLane;
+        for (int i = tid; i < n_items; i += NT) {
+            int vi;
+            if (n_listed >= 0) {
+                vi = (int)sm->pass[i];
+            } else {
+                const uint2 e = __ldcg(&ent[i / kVecsPerLane]);
+                const int j = i % kVecsPerLane;
+                if (e.y < min_key || !((e.x >> (kTileMaskShift + j)) & 1u)) continue;
+                vi = (int)(e.x & kVecMask) + 32 * j;
+            }
             float z[kPer];
             load_row_vector<T>(rowp, vi, ext, p.V, z);
 #pragma unroll
             for (int q = 0; q < kPer; ++q) {
-                if (z[q] >= -3.4028234e38f) {
+                if (z[q] >= -3.4028234e38f && rel_key(z[q], z0) >= min_key) {
                     const unsigned long long comp = ((unsigned long long)float_to_key(z[q]) << 32) |
                                                     (unsigned long long)(0xffffffffu - (uint32_t)(vi * kPer + q));
                     if (comp < last && comp > best) best = comp;
@@ -1188,7 +1252,7 @@ __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row,
 #pragma unroll
         for (int w = 0; w < NT / 32; ++w) best = sm->best[w] > best ? sm->best[w] : best;
         small_sync<NT>();
-        if (best == 0ull || (uint32_t)(best >> 32) < min_key) break;
+        if (best == 0ull) break;
         if (tid == 0) sm->comp[found] = best;
         last = best;
     }
@@ -1198,13 +1262,13 @@ __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row,
 
 // NT threads: the row was handed over as n_tiles staged lane tiles and its final threshold bin.
 // Puts the row's candidates (every logit whose bin is >= bin, at least its k largest) into
-// sm->comp and returns their number (<= kSmallCand).  The marked vectors of the tiles that pass
+// sm->comp and returns their number (<= small_list_cap(NT)).  The marked vectors of the tiles that pass
 // (largest logit in a bin >= bin) are listed, then one thread per listed vector reads it back and
 // appends its candidates.  (Inlined into the kernel so that the compiler sees sm in the shared
 // address space: atomics through a generic pointer to shared memory are several times slower.)
 template <typename T, int NT>
 __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                                     SmallShared* sm, int tid) {
+                                                     float z0, SmallShared<small_list_cap(NT)>* sm, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
@@ -1268,14 +1332,14 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
             for (int u = 0; u < kInFlight; ++u)
 #pragma unroll
                 for (int e = 0; e < kPer; ++e)
-                    if (z[u][e] >= -3.4028234e38f && float_to_key(z[u][e]) >= min_key) m |= 1u << (u * kPer + e);
+                    if (z[u][e] >= -3.4028234e38f && rel_key(z[u][e], z0) >= min_key) m |= 1u << (u * kPer + e);
             int pos = warp_reserve(&sm->n_cand, __popc(m), lane);
 #pragma unroll
             for (int u = 0; u < kInFlight; ++u)
 #pragma unroll
                 for (int e = 0; e < kPer; ++e) {
                     if ((m >> (u * kPer + e)) & 1u) {
-                        if (pos < kSmallCand)
+                        if (pos < small_list_cap(NT))
                             sm->comp[pos] = ((unsigned long long)float_to_key(z[u][e]) << 32) |
                                             (unsigned long long)(0xffffffffu - (uint32_t)(vi[u] * kPer + e));
                         ++pos;
@@ -1283,9 +1347,9 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
                 }
         }
         small_sync<NT>();
-        if (sm->n_cand <= kSmallCand) return sm->n_cand;
+        if (sm->n_cand <= small_list_cap(NT)) return sm->n_cand;
     }
-    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, sm, tid);
+    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, z0, nvec <= kSmallPass ? nvec : -1, sm, tid);
 }
 
 constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : 12; }
@@ -1293,7 +1357,7 @@ constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : 12
 template <typename T, int NT>
 __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_kernel(const SparsifyParams p) {
     constexpr int kHeld = (kSmallCand + NT - 1) / NT;  // candidates a thread holds in registers
-    __shared__ SmallShared sm;
+    __shared__ SmallShared<small_list_cap(NT)> sm;
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
     float u_raw = 0.f;
     if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];  // an input: may be read early
@@ -1325,7 +1389,7 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
         if (tid == 0) sm.red[7] = Mrow + log2(Srow);
     }
     if (raw_bin >= 0) {  // the entries are staged lane tiles: make the candidates from them first
-        nc = candidates_from_tiles<T, NT>(p, row, ent, nc, raw_bin, &sm, tid);
+        nc = candidates_from_tiles<T, NT>(p, row, ent, nc, raw_bin, __ldcg(&st->z0), &sm, tid);
 #pragma unroll
         for (int c = 0; c < kHeld; ++c) {
             const int i = tid + c * NT;
@@ -1352,6 +1416,15 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
                 sm.wkey[r] = (uint32_t)(mine >> 32);
                 sm.widx[r] = (int)(0xffffffffu - (uint32_t)mine);
             }
+        }
+    }
+    for (int i = kHeld * NT + tid; i < nc; i += NT) {  // a long list made from tiles: the rest of it
+        const unsigned long long mine = sm.comp[i];
+        int r = 0;
+        for (int j = 0; j < nc; ++j) r += sm.comp[j] > mine ? 1 : 0;
+        if (r < k) {
+            sm.wkey[r] = (uint32_t)(mine >> 32);
+            sm.widx[r] = (int)(0xffffffffu - (uint32_t)mine);
         }
     }
     small_sync<NT>();

@@ -150,6 +150,10 @@ def adversarial_rows(V, dtype):
         r5 = torch.randn(V, generator=g) * 0.01 - 10.0
         r5[::max(1, V // n_top)] = 3.0
         rows.append(r5)
+    # a run of 800 adjacent equal maxima: few vectors, more tied candidates than the finish kernel lists
+    r6 = torch.randn(V, generator=g) * 0.01 - 10.0
+    r6[V // 8: V // 8 + min(800, V // 2)] = 3.0
+    rows.append(r6)
     # large offsets: thousands of logits crowd the threshold's histogram bin (bins are relative to
     # the logit's magnitude), so these rows leave the fast paths
     rows.append(torch.randn(V, generator=g) + 20.0)
