@@ -158,6 +158,11 @@ def adversarial_rows(V, dtype):
     # the logit's magnitude), so these rows leave the fast paths
     rows.append(torch.randn(V, generator=g) + 20.0)
     rows.append(torch.randn(V, generator=g) * 0.5 - 30.0)
+    # the row's first 16 KB say nothing about the rest (masked to a large negative finite value):
+    # the offset taken from them is useless and the bins are coarse again
+    r7 = torch.randn(V, generator=g)
+    r7[:min(V // 2, 8192)] = -1000.0
+    rows.append(r7)
     return torch.stack(rows).to(dtype)
 
 
