@@ -23,7 +23,7 @@
  *     cumulative mass exceeds u * total.
  *   - CTAs that share a row or a sequence meet through a ticket counter in the workspace and
  *     the last one to arrive carries on; the one wait on another CTA (a row's finish CTA on the
- *     row's streaming CTA in tslt_sparsify, k <= 128) is one-way, bounded, and falls back to the
+ *     row's streaming CTA in tslt_sparsify) is one-way, bounded, and falls back to the
  *     end of the streaming kernel.  The first word
  *     of the workspace is a device status word (0 = fine) that tslt_workspace_status reads
  *     back; a non-zero word is reported as TSLT_ERR_DEVICE_STATUS.

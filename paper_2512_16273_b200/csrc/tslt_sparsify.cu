@@ -14,7 +14,7 @@
 // logit, so no member of the top-k is ever skipped, whatever the order in which the warps run.
 // The warps take turns at checking whether enough has been counted for the threshold to rise,
 // and rescan the histogram then.  At the end the segment hands over its per-warp (max, sum)
-// pairs and either the staged tiles as they are (k <= 128, the usual case) or the (key, index)
+// pairs and either the staged tiles as they are (k <= 256, the usual case) or the (key, index)
 // candidates it expanded from them by reading the marked vectors back.
 //
 // Finish kernel (launched with programmatic stream serialization, so that it is in place when
@@ -1137,34 +1137,38 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
 }
 
 // ---- finish kernel for small k --------------------------------------------------------------------
-// Rows of one segment with k <= 128 are finished by a CTA of 64, 96 or 128 threads (k rounded up
-// to a warp) with 8 KB of shared memory, so that every row of a large batch is resident at once:
+// Rows of one segment with k <= 256 are finished by a CTA of 64, 96, 128 or 256 threads (at least
+// k) with 6 to 21 KB of shared memory, so that every row of a large batch is resident at once:
 // finishing a row is a chain of dependent steps (trips to memory, rank counting, two scans), and
 // what it costs machine-wide is the length of that chain times the number of waves.
-constexpr int kSmallMaxThreads = 128;
-constexpr int kSmallCand = 256;      // candidates a row may bring as (key, index) entries
+constexpr int kSmallMaxThreads = 256;  // and so the largest k of this kernel
+// candidates a row may bring as (key, index) entries: 2 k at most (seg_cap)
+__host__ __device__ constexpr int small_cand_cap(int nt) { return nt > 128 ? 512 : 256; }
 // Candidates the kernel may make from a row's staged tiles: 256, and 512 for k above 96, where
 // 256 is only 2 k and the threshold bin's share can exceed it on ordinary rows.  (512 everywhere
 // cost the 64-thread kernel 9 us on the bench batch: fewer finish CTAs fit beside the streaming
 // CTAs of the last wave.)
-__host__ __device__ constexpr int small_list_cap(int nt) { return nt > 96 ? 512 : 256; }
-constexpr int kSmallPass = 512;  // marked vectors in the staged tiles of a row that pass its final threshold
+__host__ __device__ constexpr int small_list_cap(int nt) { return nt > 128 ? 1024 : nt > 96 ? 512 : 256; }
+// marked vectors in the staged tiles of a row that pass its final threshold
+__host__ __device__ constexpr int small_pass_cap(int nt) { return nt > 128 ? 1024 : 512; }
 
-template <int kList> struct SmallShared {
+template <int kList, int kK, int kPass> struct SmallShared {
     unsigned long long comp[kList];  // candidates as key << 32 | ~index: larger is earlier in the top-k order
-    uint32_t wkey[kSmallMaxThreads];  // winners in (key descending, index ascending) order, then in ascending index
-    int widx[kSmallMaxThreads];
-    uint32_t okey[kSmallMaxThreads];
-    int oidx[kSmallMaxThreads];
-    double cum[kSmallMaxThreads];
-    double wv[kSmallMaxThreads];
-    double red[8];
+    uint32_t wkey[kK];  // winners in (key descending, index ascending) order, then in ascending index
+    int widx[kK];
+    uint32_t okey[kK];
+    int oidx[kK];
+    double cum[kK];
+    double wv[kK];
+    double red[8];   // one slot per warp for the block scans
+    double lrow;     // the row's log2-normaliser
     int n_cut;
     // rows handed over as staged lane tiles
-    uint32_t pass[kSmallPass];  // marked vectors of the tiles whose largest logit passes the final threshold
+    uint32_t pass[kPass];  // marked vectors of the tiles whose largest logit passes the final threshold
     int n_pass, n_cand;
     unsigned long long best[kSmallMaxThreads / 32];
 };
+template <int NT> using SmallSharedFor = SmallShared<small_list_cap(NT), NT, small_pass_cap(NT)>;
 
 template <int NT> __device__ __forceinline__ void small_sync() { asm volatile("bar.sync 2, %0;" ::"n"(NT) : "memory"); }
 
@@ -1208,7 +1212,7 @@ template <int NT> __device__ __forceinline__ double small_max(double v, int tid,
 // composite = key << 32 | ~index: larger is earlier in (logit descending, index ascending)
 template <typename T, int NT>
 __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                               float z0, int n_listed, SmallShared<small_list_cap(NT)>* sm, int tid) {
+                                               float z0, int n_listed, SmallSharedFor<NT>* sm, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
@@ -1268,7 +1272,7 @@ __device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row,
 // address space: atomics through a generic pointer to shared memory are several times slower.)
 template <typename T, int NT>
 __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                                     float z0, SmallShared<small_list_cap(NT)>* sm, int tid) {
+                                                     float z0, SmallSharedFor<NT>* sm, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
@@ -1301,7 +1305,7 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
 #pragma unroll
             for (int j = 0; j < kVecsPerLane; ++j) {
                 if ((w >> (kTileMaskShift + j)) & 1u) {
-                    if (pos < kSmallPass) sm->pass[pos] = (w & kVecMask) + 32u * j;
+                    if (pos < small_pass_cap(NT)) sm->pass[pos] = (w & kVecMask) + 32u * j;
                     ++pos;
                 }
             }
@@ -1309,7 +1313,7 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
     }
     small_sync<NT>();
     const int nvec = sm->n_pass;
-    if (nvec <= kSmallPass) {
+    if (nvec <= small_pass_cap(NT)) {
         // ---- one thread per listed vector: read it back, append its candidates ----------------------
         constexpr int kInFlight = 2;
         static_assert(kInFlight * kPer <= 32, "one mask bit per logit a thread holds");
@@ -1349,15 +1353,15 @@ __device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, in
         small_sync<NT>();
         if (sm->n_cand <= small_list_cap(NT)) return sm->n_cand;
     }
-    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, z0, nvec <= kSmallPass ? nvec : -1, sm, tid);
+    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, z0, nvec <= small_pass_cap(NT) ? nvec : -1, sm, tid);
 }
 
-constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : 12; }
+constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : nt == 128 ? 12 : 6; }
 
 template <typename T, int NT>
 __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_kernel(const SparsifyParams p) {
-    constexpr int kHeld = (kSmallCand + NT - 1) / NT;  // candidates a thread holds in registers
-    __shared__ SmallShared<small_list_cap(NT)> sm;
+    constexpr int kHeld = (small_cand_cap(NT) + NT - 1) / NT;  // candidates a thread holds in registers
+    __shared__ SmallSharedFor<NT> sm;
     const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
     float u_raw = 0.f;
     if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];  // an input: may be read early
@@ -1386,7 +1390,7 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
         const double Mw = tid < kWarps ? (double)__ldcg(&st->M[tid]) : -INFINITY;
         const double Mrow = warp_max(Sw > 0.0 ? Mw : -INFINITY);
         const double Srow = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mrow) : 0.0);
-        if (tid == 0) sm.red[7] = Mrow + log2(Srow);
+        if (tid == 0) sm.lrow = Mrow + log2(Srow);
     }
     if (raw_bin >= 0) {  // the entries are staged lane tiles: make the candidates from them first
         nc = candidates_from_tiles<T, NT>(p, row, ent, nc, raw_bin, __ldcg(&st->z0), &sm, tid);
@@ -1396,7 +1400,7 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
             held[c] = i < nc ? sm.comp[i] : 0ull;
         }
     } else {
-        nc = nc < 0 ? 0 : (nc > kSmallCand ? kSmallCand : nc);
+        nc = nc < 0 ? 0 : (nc > small_cand_cap(NT) ? small_cand_cap(NT) : nc);
 #pragma unroll
         for (int c = 0; c < kHeld; ++c) {
             const int i = tid + c * NT;
@@ -1429,7 +1433,7 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
     }
     small_sync<NT>();
     const int n0 = nc < k ? nc : k;
-    const double L2 = sm.red[7];  // written before the barriers above; red[0..3] serve the scans
+    const double L2 = sm.lrow;  // written before the barriers above
     const double cd = p.c.d;
     // ---- nucleus cut on the cumulative q in that order ---------------------------------------------
     int n = n0;
@@ -1506,8 +1510,9 @@ __global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_
 template <typename T> static void (*small_finish_kernel(int k, int* threads))(const SparsifyParams) {
     if (k <= 64) { *threads = 64; return sparsify_finish_small_kernel<T, 64>; }
     if (k <= 96) { *threads = 96; return sparsify_finish_small_kernel<T, 96>; }
-    *threads = 128;
-    return sparsify_finish_small_kernel<T, 128>;
+    if (k <= 128) { *threads = 128; return sparsify_finish_small_kernel<T, 128>; }
+    *threads = 256;
+    return sparsify_finish_small_kernel<T, 256>;
 }
 
 // ---- host side -------------------------------------------------------------------------------
@@ -1541,10 +1546,10 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.cap = 16 * k;
     if (pl.cap < 1024) pl.cap = 1024;
     if (pl.cap > 4096) pl.cap = 4096;
-    // k <= 128: the staged tiles normally go to the finish kernel unexpanded, so the staging buffer
+    // k <= 256: the staged tiles normally go to the finish kernel unexpanded, so the staging buffer
     // is sized never to fill on ordinary rows (about 8 k tiles are staged) and the candidate list,
     // used only when it does, is kept small: four CTAs still fit an SM
-    if (k <= 128) pl.cap = 1024;
+    if (k <= kSmallMaxThreads) pl.cap = 1024;
     pl.high = pl.cap - pl.cap / 4;
     pl.vcap = k <= 64 ? 1024 : 2048;
     pl.vhigh = k <= 256 ? pl.vcap - pl.vcap / 4 : pl.vcap / 2;  // large k stages most vectors: leave room to react
@@ -1575,8 +1580,8 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (pl.split.nseg < 1) pl.split.nseg = 1;
     pl.split.cps = cps;
     pl.split.grid = rows * pl.split.nseg;
-    // rows of one segment with k <= 128 go to the small finish kernel, and hand their staged tiles over raw
-    pl.small_finish = pl.split.nseg == 1 && pl.seg_cap <= kSmallCand && k <= kSmallMaxThreads;
+    // rows of one segment with k <= 256 go to the small finish kernel, and hand their staged tiles over raw
+    pl.small_finish = pl.split.nseg == 1 && k <= kSmallMaxThreads;  // (seg_cap = 2 k fits small_cand_cap)
     pl.raw_cap = pl.small_finish ? pl.vcap : 0;
     pl.seg_stride = pl.seg_cap > pl.raw_cap ? pl.seg_cap : pl.raw_cap;
     const size_t split_rows = (size_t)rows;

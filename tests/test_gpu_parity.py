@@ -171,8 +171,10 @@ def adversarial_rows(V, dtype):
 def test_sparsify_adversarial_rows(V, dtype):
     z = adversarial_rows(V, dtype)
     rows = z.shape[0]
-    # k = 80 / 96 run the 96-thread finish kernel, 128 the 128-thread one, 64 and below the 64-thread one
-    for k, top_p in [(1, 1.0), (7, 1.0), (64, 1.0), (80, 1.0), (96, 0.95), (128, 1.0), (257, 1.0), (1000, 1.0), (128, 0.9)]:
+    # k = 80 / 96 run the 96-thread finish kernel, 128 the 128-thread one, 200 / 256 the 256-thread one,
+    # 64 and below the 64-thread one, 257 and above the generic one
+    for k, top_p in [(1, 1.0), (7, 1.0), (64, 1.0), (80, 1.0), (96, 0.95), (128, 1.0), (200, 1.0), (256, 0.95),
+                     (257, 1.0), (1000, 1.0), (128, 0.9)]:
         u = synth.uniforms((rows, 2), k, synth.TID_U_DRAFT)
         ref = oracle.sparsify(z, k, top_p, 1.0, u.numpy())
         gpu = tslt.sparsify(z.cuda(), k, top_p, 1.0, u.cuda())
