@@ -399,7 +399,7 @@ __device__ __forceinline__ void load_row_vector(const unsigned char* rowp, int v
 // held in registers meanwhile), then one thread per listed vector reads it back from global
 // memory (L2 or HBM), four loads in flight per thread: no load is spent on a tile that fails.
 // A full candidate list raises the overflow flag.
-constexpr int kMaxStagedTiles = 2048;  // largest vcap
+constexpr int kMaxStagedTiles = 4096;  // largest vcap
 template <typename T>
 __device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
                                            Candidates cb, int cap, int bin, int V, SparsifyShared* sh, int tid) {
@@ -1551,8 +1551,10 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     // used only when it does, is kept small: four CTAs still fit an SM
     if (k <= kSmallMaxThreads) pl.cap = 1024;
     pl.high = pl.cap - pl.cap / 4;
-    pl.vcap = k <= 64 ? 1024 : 2048;
-    pl.vhigh = k <= 256 ? pl.vcap - pl.vcap / 4 : pl.vcap / 2;  // large k stages most vectors: leave room to react
+    // (large k stages thousands of tiles per row: a buffer that holds most of them saves the early
+    // expansions, each a rendezvous of the warps and a round of reads back)
+    pl.vcap = k <= 64 ? 1024 : k <= 256 ? 2048 : 4096;
+    pl.vhigh = pl.vcap - pl.vcap / 4;
     pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above); see below
     pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
     // CTAs the machine holds at once: launch bounds and the shared-memory footprint decide
@@ -1661,7 +1663,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     cudaStream_t st = (cudaStream_t)stream;
     auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sparsify_smem_bytes(4096, 2048, TSLT_MAX_K)) != cudaSuccess)
+                             (int)sparsify_smem_bytes(4096, kMaxStagedTiles, TSLT_MAX_K)) != cudaSuccess)
         return TSLT_ERR_CUDA;
     kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
