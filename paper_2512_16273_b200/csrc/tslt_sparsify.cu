@@ -146,7 +146,9 @@ __device__ __forceinline__ float bin_lower_edge(int bin) { return key_to_float((
 // whatever the offset and scale of the logits.  z - z0 is monotone in z (rounding is), which is all
 // the threshold argument needs.  Candidates always carry their RAW keys: exact selection and
 // ordering never see z0.
-__device__ __forceinline__ uint32_t rel_key(float z, float z0) { return float_to_key(z - z0); }
+// (A finite z keeps a finite relative value, so that the lowest finite bin still admits every finite
+// logit: -3e38 relative to +3e38 would otherwise round to -inf.)
+__device__ __forceinline__ uint32_t rel_key(float z, float z0) { return float_to_key(fmaxf(z - z0, -3.4028234e38f)); }
 
 // A raw-domain value that every logit whose relative bin is >= bin is at or above: the bin's lower
 // edge moved back by z0, less a margin that covers the roundings of z - z0, of edge + z0 and of the
