@@ -17,11 +17,11 @@
  *   - logits are row-major [rows, V] in fp32 (TSLT_F32) or bf16 (TSLT_BF16); the base
  *     pointer must be 16-byte aligned and row_stride_elems * sizeof(element) must be a
  *     multiple of 16.  -inf logits are legal (probability 0, never selected).  NaN / +inf
- *     logits give unspecified values but never an out-of-bounds access or a hang.  The
- *     exponent z / T is carried in fp32 while a row streams, so the stated accuracy holds for
- *     |z / T| up to about 2^17; beyond that the selection is still exact but the normaliser
- *     (lse, mass, and through them the sampled token) loses accuracy, and near 2^100 it
- *     overflows.
+ *     logits give unspecified values but never an out-of-bounds access or a hang.  While a
+ *     row streams, the exponent z / T is carried in fp32 relative to a reference exponent,
+ *     itself fp32: offsets cancel, but once |z / T| passes about 2^30 the reference is so
+ *     coarse that the running sum can overflow; the selection is still exact there, the
+ *     normaliser (lse, mass, and through them the sampled token) is not.
  *   - uniforms are fp32 in [0,1); a value >= 1 is read as the largest float below 1.
  *   - "sample" always means inverse CDF in ascending token index: the first index whose
  *     cumulative mass exceeds u * total.
