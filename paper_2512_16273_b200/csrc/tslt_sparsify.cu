@@ -141,7 +141,7 @@ __device__ __forceinline__ float bin_lower_edge(int bin) { return key_to_float((
 // chunks (their largest logit): a bin is the top 12 bits of the order-preserving key of z - z0.
 // Float keys are relative (three mantissa bits: 12.5 % of the value), so bins over the raw logits
 // would be as wide as the logits are large: a row of N(20, 1) logits put thousands of them in the
-// threshold's bin and fell off every fast path (5.7 ms for the bench batch instead of 0.23).
+// threshold's bin and fell off every fast path (5.7 ms for 2048 rows of 256 000 bf16 logits instead of 0.23).
 // Relative to a value near the row's maximum the bins are finest exactly where the top-k lives,
 // whatever the offset and scale of the logits.  z - z0 is monotone in z (rounding is), which is all
 // the threshold argument needs.  Candidates always carry their RAW keys: exact selection and
@@ -1148,7 +1148,7 @@ constexpr int kSmallMaxThreads = 256;  // and so the largest k of this kernel
 __host__ __device__ constexpr int small_cand_cap(int nt) { return nt > 128 ? 512 : 256; }
 // Candidates the kernel may make from a row's staged tiles: 256, and 512 for k above 96, where
 // 256 is only 2 k and the threshold bin's share can exceed it on ordinary rows.  (512 everywhere
-// cost the 64-thread kernel 9 us on the bench batch: fewer finish CTAs fit beside the streaming
+// cost the 64-thread kernel 9 us on 2048 rows of 256 000 logits: fewer finish CTAs fit beside the streaming
 // CTAs of the last wave.)
 __host__ __device__ constexpr int small_list_cap(int nt) { return nt > 128 ? 1024 : nt > 96 ? 512 : 256; }
 // marked vectors in the staged tiles of a row that pass its final threshold
@@ -1567,7 +1567,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     const int max_seg = pl.cap / pl.seg_cap < 16 ? pl.cap / pl.seg_cap : 16;
     // One CTA per row.  Only when there are fewer rows than half the SMs and the rows are long is a
     // row cut into segments (of at least 32 chunks): every segment pays the first threshold and the
-    // hand-over, which on the benchmark's small configurations costs more than it gains.
+    // hand-over, which on small batches (tens of rows) costs more than it gains.
     (void)per_sm;
     pl.split.rows = rows;
     int nseg = 1;
