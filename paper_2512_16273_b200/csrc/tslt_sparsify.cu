@@ -73,7 +73,8 @@ struct SparsifyParams {
     float* mass;
     int nchunks;
     RowSplit split;
-    int cap, high;      // candidate (key, index) list: capacity and compaction mark
+    int cap, high;      // candidate (key, index) list of the streaming kernel: capacity and compaction mark
+    int fin_cap;        // candidate list of the finish kernel: what the row's segments can hand over
     int vcap, vhigh;    // staged lane tiles: capacity and early-expansion mark
     int idx_hi_byte;
     int* status;
@@ -895,8 +896,8 @@ __global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const
     SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw);
     unsigned char* arena = smem_raw + kHistOff;
     uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem_raw + kStagedOff);
-    int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
-    uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
+    int* cand_idx = reinterpret_cast<int*>(cand_key + p.fin_cap);
+    uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.fin_cap);
     int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
     const int tid = threadIdx.x, row = blockIdx.x;
     // the uniforms are needed last: ask for their cache line now
@@ -1520,7 +1521,7 @@ template <typename T> static void (*small_finish_kernel(int k, int* threads))(co
 // ---- host side -------------------------------------------------------------------------------
 
 struct SparsifyPlan {
-    int nchunks, cap, high, vcap, vhigh, seg_cap, seg_stride, raw_cap;
+    int nchunks, cap, high, fin_cap, vcap, vhigh, seg_cap, seg_stride, raw_cap;
     bool small_finish;
     RowSplit split;
     size_t smem;
@@ -1584,6 +1585,9 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     if (pl.split.nseg < 1) pl.split.nseg = 1;
     pl.split.cps = cps;
     pl.split.grid = rows * pl.split.nseg;
+    // the generic finish kernel holds what the row's segments hand over, no more: it fits more CTAs per SM
+    pl.fin_cap = pl.split.nseg * pl.seg_cap;
+    if (pl.fin_cap < 1024) pl.fin_cap = 1024;
     // rows of one segment with k <= 256 go to the small finish kernel, and hand their staged tiles over raw
     pl.small_finish = pl.split.nseg == 1 && k <= kSmallMaxThreads;  // (seg_cap = 2 k fits small_cand_cap)
     pl.raw_cap = pl.small_finish ? pl.vcap : 0;
@@ -1653,7 +1657,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.uniforms = uniforms;
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
     p.nchunks = pl.nchunks; p.split = pl.split;
-    p.cap = pl.cap; p.high = pl.high; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
+    p.cap = pl.cap; p.high = pl.high; p.fin_cap = pl.fin_cap; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
     p.seg_stride = pl.seg_stride; p.raw_cap = pl.raw_cap;
     p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
     unsigned char* ws = (unsigned char*)workspace;
@@ -1678,7 +1682,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
         if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
             return TSLT_ERR_CUDA;
-        if (launch_dependent(fin, rows, kBlockThreads, sparsify_smem_bytes(pl.cap, 0, k), st, p) != cudaSuccess)
+        if (launch_dependent(fin, rows, kBlockThreads, sparsify_smem_bytes(pl.fin_cap, 0, k), st, p) != cudaSuccess)
             return TSLT_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
