@@ -8,7 +8,7 @@ import torch
 import oracle
 from oracle import payload as P
 from paper_2512_16273_b200 import synth, tslt
-from parity_utils import compare_verify, to_gpu_rows, to_np
+from parity_utils import compare_verify, to_gpu_rows, to_np, verify_inputs
 
 pytestmark = pytest.mark.gpu
 
@@ -101,7 +101,8 @@ def test_round_trip_through_the_wire_then_verify(dtype, fmt):
     torch.cuda.synchronize()
     ref_v = oracle.verify(zp, ref_s["idx"].reshape(B, gamma, k), wire_logit.reshape(B, gamma, k),
                           ref_s["count"].reshape(B, gamma), tok, T, T, ua.numpy(), us.numpy())
-    compare_verify(gpu_v, ref_v, "wire %s / %d" % (dtype, gf))
+    inp = verify_inputs(zp, dict(idx=ref_s["idx"], logit=wire_logit, count=ref_s["count"]), B, gamma, k, tok, T, T, ua, us)
+    compare_verify(gpu_v, ref_v, "wire %s / %d" % (dtype, gf), inputs=inp)
 
 
 def test_argument_errors():
