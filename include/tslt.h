@@ -49,6 +49,9 @@ extern "C" {
 #define TSLT_ERR_DEVICE_STATUS (-5)
 #define TSLT_ERR_STATIC_SCRATCH (-6)
 
+/* bits of the device status word (tslt_workspace_status) */
+#define TSLT_STATUS_WAIT_FELL_BACK 1 /* a bounded device-side wait ran out and took its fall-back; results are valid */
+
 #define TSLT_F32 0
 #define TSLT_BF16 1
 
@@ -68,6 +71,13 @@ const char* tslt_status_string(int status);
  * `stream`: waits for the stream, copies the word back and stores it in *device_status
  * (HOST, nullable).  Returns TSLT_OK if it is zero, TSLT_ERR_DEVICE_STATUS otherwise. */
 int tslt_workspace_status(const void* workspace, void* stream, int* device_status);
+
+/* Test and tuning knob, process-wide: how many times (200 ns apart) a finish CTA of tslt_sparsify
+ * polls for its row before it records TSLT_STATUS_WAIT_FELL_BACK and waits for the end of the
+ * streaming kernel instead.  Default 1 << 22 (about a second); 0 sends every CTA through the
+ * fall-back at once.  polls >= 0.  (No counterpart in the paper: it bounds a wait of this
+ * implementation.) */
+int tslt_set_ready_poll_limit(int polls);
 
 /*
  * Draft side: sparsify-then-sample (Section 3, Solution 1; sampling steps of Algorithms 2

@@ -72,6 +72,7 @@ inline RowSplit make_row_split(long long rows, int nchunks, int slots, int max_s
 
 // Workspace header: word 0 is the device status (0 = fine).
 constexpr int kWsHeaderBytes = 256;
+inline size_t align_up256(size_t x) { return (x + 255) / 256 * 256; }
 
 __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync %0, %1;" ::"n"(kConsumerBarrier), "n"(kConsumerThreads) : "memory");
@@ -90,24 +91,25 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 __device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void wait_for_primary_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// A row-ready flag between the two kernels of tslt_sparsify.  The finish kernel is the streaming
-// kernel's programmatic dependent, so by the time one of its CTAs runs, every CTA of the streaming
-// kernel has started (dependents are scheduled once all CTAs of the primary have issued
-// launch_dependents or exited): each streaming CTA still running is resident and finishes on its
-// own, whatever the finish CTAs do.  A finish CTA can therefore begin as soon as its own row has
-// been handed over instead of when the whole streaming kernel has ended.  The wait is bounded all
-// the same: after kReadyPollLimit polls (about a second) the CTA falls back to griddepcontrol.wait,
-// which returns when the streaming kernel has completed.  Without the launch attribute the finish
-// kernel starts after the streaming kernel and finds every flag set.  Each streaming CTA clears
-// its row's flag (and fences) before it issues launch_dependents, so a flag left set by an earlier
-// call on the same workspace is gone before any finish CTA can look at it.
+// Ready flags between the two kernels of tslt_sparsify (one per row segment).  The finish kernel is
+// the streaming kernel's programmatic dependent, so by the time one of its CTAs runs, every CTA of
+// the streaming kernel has started (dependents are scheduled once all CTAs of the primary have
+// issued launch_dependents or exited): each streaming CTA still running is resident and finishes
+// on its own, whatever the finish CTAs do.  A finish CTA can therefore begin as soon as its own
+// row has been handed over instead of when the whole streaming kernel has ended.  The wait is
+// bounded all the same: after `limit` polls (kReadyPollLimit by default, about a second) the CTA
+// records that in the workspace's status word and falls back to griddepcontrol.wait, which returns
+// when the streaming kernel has completed; the results are the same.  Without the launch
+// attribute the finish kernel starts after the streaming kernel and finds every flag set.  Each
+// streaming CTA clears its own flag (and fences) before it issues launch_dependents, so a flag
+// left set by an earlier call on the same workspace is gone before any finish CTA can look at it.
 constexpr int kReadyPollLimit = 1 << 22;
-__device__ __forceinline__ void publish_row_ready(int* flag) {  // one thread, after a barrier that follows the row's writes
+__device__ __forceinline__ void publish_row_ready(int* flag) {  // one thread, after a barrier that follows the segment's writes
     __threadfence();
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(1) : "memory");
 }
-__device__ __forceinline__ bool poll_row_ready(const int* flag) {  // one thread
-    for (int it = 0; it < kReadyPollLimit; ++it) {
+__device__ __forceinline__ bool poll_row_ready(const int* flag, int limit) {  // one thread
+    for (int it = 0; it < limit; ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
         if (v != 0) return true;

@@ -3,31 +3,29 @@
 //
 // Streaming kernel.  One CTA reads one segment of one logits row from HBM exactly once, with
 // 16-byte loads that go straight to registers (each warp instruction covers 512 contiguous
-// bytes).  Warps run freely: there is no barrier in the steady state.  Each lane keeps an online
-// (max, sum) for the softmax normaliser and stages every lane tile (its four 16-byte vectors of a
-// 2 KB chunk) that holds a logit at or above a running threshold: 8 bytes (where the tile is,
-// which of its vectors hold a candidate, the key of its largest logit), no data.  The test is on
-// the tile's packed maximum, so a tile without a candidate costs a handful of instructions and
-// nothing is searched inside a vector while streaming.  The threshold comes from a 4096-bin
-// histogram of the order-preserving keys (top 12 bits) of what is staged: the highest bin above
-// which at least k distinct logits have been counted is a lower bound on the row's k-th largest
-// logit, so no member of the top-k is ever skipped, whatever the order in which the warps run.
-// The warps take turns at checking whether enough has been counted for the threshold to rise,
-// and rescan the histogram then.  At the end the segment hands over its per-warp (max, sum)
-// pairs and either the staged tiles as they are (k <= 256, the usual case) or the (key, index)
-// candidates it expanded from them by reading the marked vectors back.
+// bytes).  It keeps two things: each lane's online (max, sum) for the softmax normaliser, and,
+// for every 64-byte tile of the row (32 bf16 or 16 fp32 logits), the top 16 bits of the tile's
+// largest logit, written to the workspace (2 bytes per 64 read).  Nothing in it depends on k or
+// top_p: there is no threshold, no histogram, no shared memory and no barrier in the loop, so it
+// runs at the occupancy and speed of a plain streaming reduction.
 //
-// Finish kernel (launched with programmatic stream serialization, so that it is in place when
-// the streaming kernel ends).  One CTA per row: candidates from the hand-over, the bin that holds
-// the k-th largest logit, everything above it, the tie inside it broken exactly (logit
-// descending, index ascending), the top-rho cut, renormalisation in fp64, the samples by inverse
-// CDF, the (index, logit) pairs in ascending index.
-//
-// Rare paths: a staging buffer that fills up is expanded early by all warps together (and the
-// candidate list compacted to the current threshold); a buffer that overflows before they can
-// meet (adversarial rows: sorted ascending, all equal) is abandoned and the segment is read a
-// second time against the final threshold; a candidate list that overflows even then is selected
-// again from global memory with a radix select.
+// Finish kernel (launched with programmatic stream serialization; a CTA starts on its row as soon
+// as the row's segments have been handed over).  One CTA per row:
+//   1. a lower bound on the k-th largest TILE maximum: tiles are taken in groups so that there are
+//      a few times k groups, and the k-th largest group maximum is found by bisection on its 16
+//      bits (each of the k groups at or above it holds a tile, and so a logit, at or above it);
+//   2. the tiles at or above that bound are listed in address order ("survivors": a little more
+//      than k of them) and read back from global memory: 64 bytes each, k * 64 bytes of the row's
+//      V * e;
+//   3. the exact k-th largest logit among them by a histogram over the 16-bit keys between the
+//      bound and the row maximum (fp32 rows: a second histogram over the low 16 bits inside the
+//      boundary value), ties at the boundary going to the lower index;
+//   4. the winners are collected by prefix sums over the survivors in address order, so they come
+//      out in ascending token index without any sort;
+//   5. the top-rho cut (a sort of the at most k winners by logit, an fp64 cumulative), the
+//      renormalised distribution and its CDF in fp64, the samples by inverse CDF, the outputs.
+// A row whose survivors do not fit the list (thousands of tied tile maxima: constant rows, rows
+// sorted by value) runs steps 3 and 4 over all of its vectors instead: slower, same code.
 #include <math.h>
 
 #include "tslt_common.cuh"
@@ -36,25 +34,20 @@
 
 namespace tslt {
 
-constexpr int kHistBins = 4096;   // fine bins: key >> 20 (sign, exponent and three mantissa bits)
-constexpr int kHistShift = 20;
-constexpr int kCoarseBins = 128;  // coarse bin = fine bin >> 5: lets a scan find the right 32 fine bins in one step
-constexpr int kLowestFiniteBin = 0x00800000u >> kHistShift;  // bin of -FLT_MAX: every finite logit passes
-constexpr int kBoundaryCap = 960;   // entries of the k-th logit's bin that the direct tie-break handles
-constexpr int kArenaBytes = 24576;  // histograms (16.5 KB) + boundary list (7.5 KB); fp64 work arrays afterwards
-constexpr int kSparsifyCtasPerSm = 4;  // 64 registers per thread
-constexpr int kPrefetchSteps = 1;      // how many of its own steps ahead a warp asks L2 for its chunk
-constexpr int kRankSortMax = 256;   // up to this many entries are ordered by counting, more by a bitonic sort
+constexpr int kTilesPerChunk = 32;        // 64-byte tiles in a 2 KB chunk
+constexpr int kVecsPerTile = 4;           // 16-byte vectors in a tile
+constexpr int kSparsifyStreamCtasPerSm = 6;
+constexpr int kFinishThreads = kBlockThreads;
+constexpr int kMaxGroups = 4096;          // group maxima the finish kernel bisects over
+constexpr int kMaxTileList = 4096;        // survivor tiles it can list
+constexpr int kSelBins = 1024;            // bins of the selection histogram
+constexpr uint32_t kLowestFinite16 = 0x0080u;   // key of -FLT_MAX >> 16
+constexpr uint32_t kHighestFinite16 = 0xff7fu;  // key of +FLT_MAX >> 16
 
+// What a segment hands over besides its tile maxima: one (max, sum) pair per warp.
 struct SegStat {
-    double S[kWarps];  // per warp: sum of 2^(y - M) over the warp's chunks of the segment
-    float M[kWarps];   // per warp: reference exponent (base 2)
-    int n;             // entries written for the segment
-    int raw_bin;       // -1: the entries are (key, idx) candidates; else they are staged lane tiles (first vector
-                       // and vector mask, relative key of the largest logit) and this is the segment's final
-                       // threshold bin
-    float z0;          // the segment's offset: bins are over z - z0 (see rel_key)
-    int pad;
+    double S[kWarps];  // sum of 2^(y - M) over the warp's chunks of the segment
+    float M[kWarps];   // the warp's reference exponent (base 2)
 };
 
 struct SparsifyParams {
@@ -73,314 +66,135 @@ struct SparsifyParams {
     float* mass;
     int nchunks;
     RowSplit split;
-    int cap, high;      // candidate (key, index) list of the streaming kernel: capacity and compaction mark
-    int fin_cap;        // candidate list of the finish kernel: what the row's segments can hand over
-    int vcap, vhigh;    // staged lane tiles: capacity and early-expansion mark
-    int idx_hi_byte;
+    int group_log2;   // tiles per group = 1 << group_log2
+    int ngroups;      // <= kMaxGroups
+    int tile_cap;     // survivor list capacity (<= kMaxTileList)
+    int poll_limit;   // polls of a segment's ready flag before falling back to the end of the streaming kernel
     int* status;
-    SegStat* seg_stats;
-    uint2* seg_entries;  // [rows, nseg, seg_stride]: (key, idx) candidates, or staged lane tiles handed over raw
-    int seg_cap;         // most candidates a segment hands over
-    int seg_stride;      // entries reserved per segment
-    int raw_cap;         // > 0: a segment whose staging buffer never filled hands its staged tiles over unexpanded
-    int* row_ready;      // [rows] (rows of one segment only, else NULL): set to 1 when the row has been handed over
+    int* seg_ready;           // [rows * nseg]
+    SegStat* seg_stats;       // [rows * nseg]
+    unsigned short* tile_max; // [rows, nchunks * 32]: top 16 bits of each tile's largest logit, slot order (see tile_slot)
 };
 
-struct SparsifyShared {
-    // ---- written by stage_tile through their shared-space addresses ----------------------------------
-    int vec_count;   // staged lane tiles
-    int overflow;    // a buffer was found full: its contents are no longer complete
-    int trim_request;
-    int n_above;     // logits counted in bins above thr_bin since it last rose (may lag, never leads a rise)
-    // --------------------------------------------------------------------------------------------
-    int n_list;      // expand_staged: vectors listed for reading back
-    int cand_count;  // expanded (key, index) candidates
-    int thr_bin;     // candidates are the logits whose relative key's bin is >= thr_bin; only ever rises
-    float z0;        // the segment's offset (see rel_key); fixed once the first chunks have been looked at
-    uint32_t thr_edge_key;  // fp32 rows: order-preserving key of the raw-domain threshold the lane-tile test uses
-    uint32_t thr_word;  // thr_bin << 16 | the bf16 pattern the packed lane-tile test compares with; only ever rises
-    int sel_bin, sel_above;  // bin of the k-th largest logit and the number of logits in higher bins
-    int n_win, n_bnd;
-    int warp_tot[kWarps];
+// Tile a of a row is its bytes [64 a, 64 a + 64).  In the streaming kernel vector j * 32 + l of a
+// chunk belongs to lane l, so the tile made of vectors j * 32 + 4 q .. + 3 belongs to the lane
+// quad q, whose leader stores the maxima of its four tiles (j = 0..3) side by side: slot
+// ch * 32 + q * 4 + j holds tile ch * 32 + j * 8 + q.
+__host__ __device__ inline int tile_slot(int a) { return (a & ~31) | ((a & 7) << 2) | ((a >> 3) & 3); }
+
+// Order-preserving 16-bit key of the top half of an fp32 / a bf16 pattern, -0 folded onto +0
+// (equal to float_to_key(value) >> 16 for the value the pattern truncates).
+__device__ __forceinline__ uint32_t raw16_to_key16(uint32_t r) {
+    r = (r == 0x8000u) ? 0u : r;
+    return (r & 0x8000u) ? (~r & 0xffffu) : (r | 0x8000u);
+}
+
+// ---- streaming kernel ------------------------------------------------------------------------------
+template <typename T> struct QuadMax;
+template <> struct QuadMax<bf16_t> {
+    // top 16 bits of the largest logit of each of the quad's four tiles, packed (j = 0, 1 | 2, 3)
+    static __device__ __forceinline__ uint2 keys(const LaneTile<bf16_t>& lt) {
+        uint32_t r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t v = lt.vm[j];
+            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 2));
+            r[j] = bf16x2_max(v, v >> 16) & 0xffffu;
+        }
+        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
+    }
+};
+template <> struct QuadMax<float> {
+    static __device__ __forceinline__ uint2 keys(const LaneTile<float>& lt) {
+        uint32_t r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v = lt.vm[j];
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+            r[j] = __float_as_uint(v) >> 16;
+        }
+        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) sparsify_stream_kernel(const SparsifyParams p) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
+    const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
+    const RowExtent ext = row_extent<T>(p.V);
+    const float c = p.c.f;
+    const unsigned char* lane_rowp = rowp + lane * kVecBytes;
+    int ch = wk.chunk_begin + warp;
+    LaneTile<T> lt;
+    if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);  // in flight during the set-up below
+    // The segment's ready flag is cleared here, by the CTA that will set it, and the store is fenced
+    // before the barrier after which this CTA lets the finish kernel be scheduled.  A finish CTA
+    // runs only after every streaming CTA has passed that point, so it never sees a flag (or a
+    // status word) left by an earlier call, and the workspace needs no clearing between calls.
+    if (tid == 0) {
+        *(volatile int*)&p.seg_ready[blockIdx.x] = 0;
+        if (blockIdx.x == 0) *(volatile int*)p.status = 0;
+        __threadfence();
+    }
+    __syncthreads();
+    allow_dependent_launch();
+
+    LaneSum ls;
+    ls.reset();
+    unsigned short* tmax = p.tile_max + (size_t)wk.row * p.nchunks * kTilesPerChunk;
+    while (ch < wk.chunk_end) {
+        const float lm = lt.reduce_max();
+        const uint2 q = QuadMax<T>::keys(lt);
+        if ((lane & 3) == 0) *reinterpret_cast<uint2*>(tmax + ch * kTilesPerChunk + lane) = q;  // slots (lane >> 2) * 4 ..+3
+        ls.raise_to(lm, c);
+        lt.accumulate(ls, c);
+        ch += kWarps;
+        if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
+    }
+    // hand-over: one (M, S) pair per warp
+    const float Mw = warp_max(ls.M);
+    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
+    if (lane == 0) {
+        SegStat* st = &p.seg_stats[blockIdx.x];
+        st->S[warp] = Sw;
+        st->M[warp] = Mw;
+    }
+    __syncthreads();  // every warp's part of the hand-over is written
+    if (tid == 0) publish_row_ready(&p.seg_ready[blockIdx.x]);
+}
+
+// ---- finish kernel ---------------------------------------------------------------------------------
+__host__ __device__ inline size_t align16(size_t x) { return (x + 15) / 16 * 16; }
+__host__ __device__ inline int pow2_at_least(int n) {
+    int p = 1;
+    while (p < n) p <<= 1;
+    return p;
+}
+constexpr int kFinishHeaderBytes = 512;
+// dynamic shared memory of the finish kernel: header | histogram | region A | region B | winners
+__host__ __device__ inline size_t finish_region_a(int ngroups, int k) {
+    const size_t g = (size_t)ngroups * 4, c = (size_t)pow2_at_least(k) * 8;
+    return align16(g > c ? g : c);
+}
+__host__ __device__ inline size_t finish_region_b(int tile_cap, int k) {
+    const size_t t = (size_t)tile_cap * 4, w = (size_t)k * 16;
+    return align16(t > w ? t : w);
+}
+__host__ __device__ inline size_t sparsify_finish_smem(int ngroups, int tile_cap, int k) {
+    return kFinishHeaderBytes + (size_t)kSelBins * 4 + finish_region_a(ngroups, k) + finish_region_b(tile_cap, k) + (size_t)k * 8;
+}
+
+struct FinishShared {
     double scratch[16];
-    SelectScratch sel;
+    double lrow;            // base-2 log of the row's softmax normaliser
+    int round_count[32];    // one counter per bisection round
+    int iscr[16];
+    int sel_bin, sel_above, sel_eq, sel_total;
+    int ready, n_surv, max16;
 };
-
-__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-// shared-memory carve-up (dynamic):
-//   SparsifyShared | arena | staged[vcap] | cand_key[cap] | cand_idx[cap] | tmp_key[k] | tmp_idx[k]
-// The control block, the histograms and the staging buffer sit at compile-time offsets of the
-// CTA's shared memory, so the streaming loop holds no address of them in a register.
-constexpr uint32_t kSharedBlockBytes = (sizeof(SparsifyShared) + 127) / 128 * 128;
-constexpr uint32_t kHistOff = kSharedBlockBytes;
-constexpr uint32_t kCoarseOff = kHistOff + 4u * kHistBins;
-constexpr uint32_t kStagedOff = kHistOff + kArenaBytes;
-__host__ __device__ inline size_t sparsify_smem_bytes(int cap, int vcap, int k) {
-    return align_up((size_t)kStagedOff + (size_t)vcap * 8 + (size_t)cap * 8 + (size_t)k * 8, 16);
-}
-
-// Sources for select_topk: the candidate buffer, or a run of logits in global memory.
-struct BufferSrc {
-    const uint32_t* k_;
-    const int* i_;
-    __device__ __forceinline__ bool valid(int) const { return true; }
-    __device__ __forceinline__ uint32_t key(int i) const { return k_[i]; }
-    __device__ __forceinline__ int idx(int i) const { return i_[i]; }
-};
-template <typename T> struct GlobalSrc {
-    const unsigned char* row;
-    int elem0;
-    __device__ __forceinline__ bool valid(int i) const { return Elt<T>::load(row, elem0 + i) > -INFINITY; }
-    __device__ __forceinline__ uint32_t key(int i) const { return float_to_key(Elt<T>::load(row, elem0 + i)); }
-    __device__ __forceinline__ int idx(int i) const { return elem0 + i; }
-};
-
-__device__ __forceinline__ float bin_lower_edge(int bin) { return key_to_float((uint32_t)bin << kHistShift); }
-
-// The histogram's bins are over the logits RELATIVE to an offset z0 taken from the segment's first
-// chunks (their largest logit): a bin is the top 12 bits of the order-preserving key of z - z0.
-// Float keys are relative (three mantissa bits: 12.5 % of the value), so bins over the raw logits
-// would be as wide as the logits are large: a row of N(20, 1) logits put thousands of them in the
-// threshold's bin and fell off every fast path (5.7 ms for 2048 rows of 256 000 bf16 logits instead of 0.23).
-// Relative to a value near the row's maximum the bins are finest exactly where the top-k lives,
-// whatever the offset and scale of the logits.  z - z0 is monotone in z (rounding is), which is all
-// the threshold argument needs.  Candidates always carry their RAW keys: exact selection and
-// ordering never see z0.
-// (A finite z keeps a finite relative value, so that the lowest finite bin still admits every finite
-// logit: -3e38 relative to +3e38 would otherwise round to -inf.)
-__device__ __forceinline__ uint32_t rel_key(float z, float z0) { return float_to_key(fmaxf(z - z0, -3.4028234e38f)); }
-
-// A raw-domain value that every logit whose relative bin is >= bin is at or above: the bin's lower
-// edge moved back by z0, less a margin that covers the roundings of z - z0, of edge + z0 and of the
-// subtraction itself (2^-21 of the magnitudes involved; each rounding is at most 2^-24 of one).
-// Being low only lets a few more tiles through the streaming test; what they hold is then judged
-// by its relative key.
-__device__ __forceinline__ float raw_edge_below(int bin, float z0) {
-    const float es = bin_lower_edge(bin);
-    const float er = es + z0;
-    return er - 4.76837158e-7f * (fabsf(es) + fabsf(z0) + fabsf(er));
-}
-
-// ---- shared memory by address: one out-of-line copy of the rare paths, still shared-space code ----
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ float lds_f32(uint32_t addr) { return __uint_as_float(lds_u32(addr)); }
-__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
-    asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t atoms_add(uint32_t addr, uint32_t v) {
-    uint32_t old;
-    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
-    return old;
-}
-__device__ __forceinline__ void reds_add(uint32_t addr, uint32_t v) {
-    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-
-// Count one logit in both histogram levels (fine first: a scan that sees the coarse count also
-// finds the fine one).
-__device__ __forceinline__ void hist_count(uint32_t hist_addr, uint32_t coarse_addr, int bin, uint32_t delta) {
-    reds_add(hist_addr + 4u * (uint32_t)bin, delta);
-    reds_add(coarse_addr + 4u * (uint32_t)(bin >> 5), delta);
-}
-
-__device__ __forceinline__ void sts_v2(uint32_t addr, uint32_t x, uint32_t y) {
-    asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
-}
-// A warp hands out list positions with one atomic: returns where this lane's cnt entries start.
-__device__ __forceinline__ int warp_reserve(int* counter, int cnt, int lane) {
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    int start = 0;
-    if (lane == 31 && incl > 0) start = atomicAdd(counter, incl);
-    return __shfl_sync(0xffffffffu, start, 31) + incl - cnt;
-}
-
-
-// Stage a lane tile (the four 16-byte vectors vec0, vec0 + 32, vec0 + 64, vec0 + 96 of the row)
-// whose largest logit is vmax: only vec0, which of the four vectors hold a candidate, and the key
-// of that logit are kept (8 bytes), and the logit is counted.  The tile's data is read again from
-// global memory when the staged tiles are expanded, and only if its largest logit still passes
-// the threshold of that moment: a fraction of what is staged.  `base` is the shared-space address
-// of the CTA's dynamic shared memory.
-constexpr int kTileMaskShift = 28;  // a staged tile's word: first vector (below 2^18) | mask of its four vectors << 28
-// Count one logit of the row in the histogram, and towards the next rise of the threshold.
-__device__ __forceinline__ void count_logit(uint32_t base, int thr_bin, uint32_t key) {
-    hist_count(base + kHistOff, base + kCoarseOff, (int)(key >> kHistShift), 1u);
-    if ((int)(key >> kHistShift) > thr_bin) reds_add(base + (uint32_t)offsetof(SparsifyShared, n_above), 1u);
-}
-// Small k counts the tile's largest logit only (two candidates seldom share a tile); large k, where
-// most tiles hold some, counts the largest logit of every marked vector (count_tile false, the
-// caller does it), or the threshold would sit too low.
-constexpr int kCountPerVectorAboveK = 128;
-__device__ __forceinline__ void stage_tile(uint32_t base, const SparsifyParams& p, int thr_bin, uint32_t tile_word,
-                                           float vmax, bool count_tile) {
-    const uint32_t pos = atoms_add(base + (uint32_t)offsetof(SparsifyShared, vec_count), 1u);
-    const uint32_t key = rel_key(vmax, lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0)));
-    if (count_tile) count_logit(base, thr_bin, key);
-    if (pos < (uint32_t)p.vcap) sts_v2(base + kStagedOff + 8u * pos, tile_word, key);
-    else sts_u32(base + (uint32_t)offsetof(SparsifyShared, overflow), 1u);
-    if (pos + 1u == (uint32_t)p.vhigh) sts_u32(base + (uint32_t)offsetof(SparsifyShared, trim_request), 1u);
-}
-
-// One warp: the highest fine bin b with (number of counted logits in bins >= b) >= k, or -1 if
-// fewer than k are counted; *above gets the count in the bins above b (the total if none).
-// Two steps whatever the values: the 128 coarse counts, then the 32 fine bins of the coarse bin
-// in which the running count crosses k.
-__device__ __noinline__ int scan_boundary(uint32_t hist_addr, uint32_t coarse_addr, int k, uint32_t* above_out) {
-    const int lane = threadIdx.x & 31;
-    // lane l owns coarse bins 127-4l .. 124-4l (descending)
-    uint32_t c[4], tot = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        c[i] = lds_u32(coarse_addr + 4u * (uint32_t)(127 - 4 * lane - i));
-        tot += c[i];
-    }
-    uint32_t incl = tot;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    const unsigned hit = __ballot_sync(0xffffffffu, incl >= (uint32_t)k);
-    if (!hit) {
-        *above_out = __shfl_sync(0xffffffffu, incl, 31);
-        return -1;
-    }
-    const int l = __ffs(hit) - 1;
-    uint32_t run = incl - tot;  // counted above this lane's bins
-    int cbin = 0;
-    bool done = false;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        if (!done) {
-            if (run + c[i] >= (uint32_t)k) {
-                cbin = 127 - 4 * lane - i;
-                done = true;
-            } else {
-                run += c[i];
-            }
-        }
-    }
-    cbin = __shfl_sync(0xffffffffu, cbin, l);
-    const uint32_t above_c = __shfl_sync(0xffffffffu, run, l);
-    // fine bins of that coarse bin, lane 0 the highest
-    const int fb = cbin * 32 + 31 - lane;
-    const uint32_t f = lds_u32(hist_addr + 4u * (uint32_t)fb);
-    uint32_t fincl = f;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, fincl, o);
-        if (lane >= o) fincl += t;
-    }
-    const unsigned fhit = __ballot_sync(0xffffffffu, above_c + fincl >= (uint32_t)k);
-    if (!fhit) {  // the fine counts lag the coarse one (another warp is mid-push): nothing to report yet
-        *above_out = 0;
-        return -2;
-    }
-    const int fl = __ffs(fhit) - 1;
-    *above_out = above_c + __shfl_sync(0xffffffffu, fincl - f, fl);
-    return cbin * 32 + 31 - fl;
-}
-
-// The bf16 side of the threshold word: P = the largest bf16 value below raw_edge_below(bin, z0),
-// never below -inf (the pattern that lets every finite logit through).
-__device__ __forceinline__ uint32_t threshold_word(int bin, float z0) {
-    uint32_t k16 = float_to_key(raw_edge_below(bin, z0)) >> 16;  // bf16 key at or below the edge ...
-    k16 = k16 > 0x80u ? k16 - 1u : 0x7fu;                       // ... then strictly below; 0x7f is -inf
-    if (k16 == 0x7fffu) k16 = 0x7ffeu;                           // -0 shares +0's key: step past it
-    const uint32_t b16 = (k16 & 0x8000u) ? (k16 & 0x7fffu) : (~k16 & 0xffffu);
-    return ((uint32_t)bin << 16) | b16;
-}
-
-// One warp: raise thr_bin to the bin scan_boundary finds.  Counts that other warps are still adding
-// can only be missed, never invented, so the result is always a valid lower bound.
-__device__ __forceinline__ void raise_threshold(SparsifyShared* sh, int k) {
-    uint32_t above;
-    const int found = scan_boundary(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, k, &above);
-    if ((threadIdx.x & 31) == 0) {
-        const int cur = *(volatile int*)&sh->thr_bin;
-        if (found > cur) {
-            const float z0 = sh->z0;
-            atomicMax(&sh->thr_bin, found);
-            atomicMax(&sh->thr_word, threshold_word(found, z0));
-            atomicMax(&sh->thr_edge_key, float_to_key(raw_edge_below(found, z0)));
-        }
-        // what is counted above the boundary bin starts the count towards the next rise (a stale
-        // value only costs or delays a rescan)
-        if (found >= cur) *(volatile int*)&sh->n_above = (int)above;
-    }
-}
-
-// The running threshold in the form the lane-tile test wants: a raw-domain bound that lets through
-// every logit whose relative bin is >= thr_bin (and a few more, see raw_edge_below).
-//   fp32 rows: the bound itself, compared as floats.
-//   bf16 rows: P = the largest bf16 value below the bound, in both halves of a word; a packed
-//              word w holds a candidate iff max.bf16x2(w, P) != P (NaN halves never differ).
-template <typename T> struct Threshold;
-template <> struct Threshold<float> {
-    int bin;
-    float edge;
-    __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh)
-        : bin(*(const volatile int*)&sh->thr_bin), edge(key_to_float(*(const volatile uint32_t*)&sh->thr_edge_key)) {}
-    __device__ __forceinline__ int bin_value() const { return bin; }
-};
-template <> struct Threshold<bf16_t> {
-    uint32_t word, P2;
-    __device__ __forceinline__ explicit Threshold(const SparsifyShared* sh) {
-        word = *(const volatile uint32_t*)&sh->thr_word;
-        P2 = __byte_perm(word, 0u, 0x1010);
-    }
-    __device__ __forceinline__ int bin_value() const { return (int)(word >> 16); }
-};
-
-// Stage the lane tile if it holds a candidate (reduce_max() already called, lm its result): one
-// test on the lane's packed maximum, one staging step for all the lanes of the warp that pass.
-__device__ __forceinline__ void filter_push(const LaneTile<bf16_t>& lt, const Threshold<bf16_t>& th, float lm, int vec0,
-                                            uint32_t base, const SparsifyParams& p) {
-    const uint32_t P2 = th.P2;
-    if (bf16x2_max(lt.m2, P2) != P2) {
-        uint32_t word = (uint32_t)vec0;
-#pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j)
-            if (bf16x2_max(lt.vm[j], P2) != P2) word |= 1u << (kTileMaskShift + j);
-        const bool per_vector = p.k > kCountPerVectorAboveK;
-        stage_tile(base, p, th.bin_value(), word, lm, !per_vector);
-        if (per_vector) {
-#pragma unroll
-            for (int j = 0; j < kVecsPerLane; ++j)
-                if ((word >> (kTileMaskShift + j)) & 1u)
-                    count_logit(base, th.bin_value(),
-                                rel_key(lt.vec_max(j), lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0))));
-        }
-    }
-}
-__device__ __forceinline__ void filter_push(const LaneTile<float>& lt, const Threshold<float>& th, float lm, int vec0,
-                                            uint32_t base, const SparsifyParams& p) {
-    if (lm >= th.edge) {
-        uint32_t word = (uint32_t)vec0;
-#pragma unroll
-        for (int j = 0; j < kVecsPerLane; ++j)
-            if (lt.vec_max(j) >= th.edge) word |= 1u << (kTileMaskShift + j);
-        const bool per_vector = p.k > kCountPerVectorAboveK;
-        stage_tile(base, p, th.bin_value(), word, lm, !per_vector);
-        if (per_vector) {
-#pragma unroll
-            for (int j = 0; j < kVecsPerLane; ++j)
-                if ((word >> (kTileMaskShift + j)) & 1u)
-                    count_logit(base, th.bin_value(),
-                                rel_key(lt.vec_max(j), lds_f32(base + (uint32_t)offsetof(SparsifyShared, z0))));
-        }
-    }
-}
 
 // One 16-byte vector of a row as kPer logits; the row's ragged last vector element by element,
 // -inf beyond the row.
@@ -396,709 +210,451 @@ __device__ __forceinline__ void load_row_vector(const unsigned char* rowp, int v
     }
 }
 
-// All threads: turn the staged lane tiles whose largest logit is in a bin >= bin into (key, index)
-// candidates, keeping the logits whose bin is >= bin, and empty the staging buffer.  First the
-// marked vectors of the tiles that pass are listed (over the staging buffer itself, its entries
-// held in registers meanwhile), then one thread per listed vector reads it back from global
-// memory (L2 or HBM), four loads in flight per thread: no load is spent on a tile that fails.
-// A full candidate list raises the overflow flag.
-constexpr int kMaxStagedTiles = 4096;  // largest vcap
-template <typename T>
-__device__ __noinline__ void expand_staged(uint2* staged, int vcap, const unsigned char* rowp, const RowExtent ext,
-                                           Candidates cb, int cap, int bin, int V, SparsifyShared* sh, int tid) {
-    constexpr int kPer = Elt<T>::kPerVec;
-    constexpr int kInFlight = 4;
-    constexpr int kMine = kMaxStagedTiles / kBlockThreads;
-    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
-    const int nv = min(sh->vec_count, vcap);
-    const uint32_t min_key = (uint32_t)bin << kHistShift;
-    const float z0 = sh->z0;
-    const int lane = tid & 31;
-    uint2 mine[kMine];
-    int cnt = 0;
-#pragma unroll
-    for (int c = 0; c < kMine; ++c) {
-        const int i = tid + c * kBlockThreads;
-        mine[c] = i < nv ? staged[i] : make_uint2(0u, 0u);  // key 0 never passes
-        if (mine[c].y >= min_key) cnt += __popc(mine[c].x >> kTileMaskShift);
-    }
-    if (tid == 0) sh->n_list = 0;
-    consumer_sync();  // every entry is in a register: the buffer can take the list
-    uint32_t* list = reinterpret_cast<uint32_t*>(staged);
-    const int list_cap = 2 * vcap;
-    int pos = warp_reserve(&sh->n_list, cnt, lane);
-#pragma unroll
-    for (int c = 0; c < kMine; ++c) {
-        if (mine[c].y >= min_key) {
-#pragma unroll
-            for (int j = 0; j < kVecsPerLane; ++j) {
-                if ((mine[c].x >> (kTileMaskShift + j)) & 1u) {
-                    if (pos < list_cap) list[pos] = (mine[c].x & kVecMask) + 32u * j;
-                    ++pos;
-                }
-            }
-        }
-    }
-    consumer_sync();
-    int nlist = sh->n_list;
-    if (nlist > list_cap) {  // more than two marked vectors per staged tile: take the second pass over the row
-        if (tid == 0) sh->overflow = 1;
-        nlist = 0;
-    }
-    for (int base = 0; base < nlist; base += kInFlight * kBlockThreads) {
-        uint4 d[kInFlight];
-        int vi[kInFlight];
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u) {
-            const int i = base + u * kBlockThreads + tid;
-            vi[u] = i < nlist ? (int)list[i] : -1;
-            if (vi[u] >= 0 && vi[u] < ext.nvec_full) d[u] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u) {
-            if (vi[u] < 0) continue;
-            const int e0 = vi[u] * kPer;
-            float z[kPer];
-            if (vi[u] < ext.nvec_full) unpack_vec<T>(d[u], z);
-            else load_row_vector<T>(rowp, vi[u], ext, V, z);  // the ragged last vector; nothing beyond it
-#pragma unroll
-            for (int e = 0; e < kPer; ++e) {
-                if (z[e] >= -3.4028234e38f) {
-                    if (rel_key(z[e], z0) >= min_key) {
-                        const int pos2 = atomicAdd(cb.count, 1);
-                        if (pos2 < cap) {
-                            cb.key[pos2] = float_to_key(z[e]);
-                            cb.idx[pos2] = e0 + e;
-                        } else {
-                            sh->overflow = 1;
-                        }
-                    }
-                }
-            }
-        }
-    }
-    consumer_sync();
-    if (tid == 0) {
-        sh->vec_count = 0;
-        if (*cb.count > cap) *cb.count = cap;
-    }
-    consumer_sync();
-}
-
-// All threads: drop the buffer entries whose bin is below `bin` (entries are held in registers
-// between the read and the write phase, so the compaction is in place).
-__device__ __noinline__ void compact_buffer(Candidates cb, int bin, SparsifyShared* sh, int tid) {
-    constexpr int E = 16;  // cap <= 4096 = 16 * 256
-    const int n = min(*cb.count, E * kBlockThreads);
-    const float z0 = sh->z0;
-    uint32_t ek[E];
-    int ei[E];
-    unsigned keep = 0;
-    int cnt = 0;
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int i = tid * E + e;
-        ek[e] = 0u;
-        ei[e] = 0;
-        if (i < n) {
-            ek[e] = cb.key[i];
-            ei[e] = cb.idx[i];
-            if ((int)(rel_key(key_to_float(ek[e]), z0) >> kHistShift) >= bin) {
-                keep |= 1u << e;
-                ++cnt;
-            }
-        }
-    }
+// Exclusive prefix sum of one int per thread over the block; *total gets the sum.
+__device__ __forceinline__ int block_exscan(int v, int tid, int* scr /* >= 8 */, int* total) {
     const int lane = tid & 31, warp = tid >> 5;
-    int incl = cnt;
+    int incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int t = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += t;
     }
-    if (lane == 31) sh->warp_tot[warp] = incl;
-    consumer_sync();  // every entry has been read, warp totals are in place
-    int off = incl - cnt, total = 0;
+    if (lane == 31) scr[warp] = incl;
+    consumer_sync();
+    int base = 0, tot = 0;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) {
-        const int t = sh->warp_tot[w];
-        if (w < warp) off += t;
-        total += t;
+        const int t = scr[w];
+        if (w < warp) base += t;
+        tot += t;
     }
-#pragma unroll
-    for (int e = 0; e < E; ++e)
-        if (keep & (1u << e)) {
-            cb.key[off] = ek[e];
-            cb.idx[off] = ei[e];
-            ++off;
-        }
     consumer_sync();
-    if (tid == 0) *cb.count = total;
-    consumer_sync();
+    *total = tot;
+    return base + incl - v;
 }
 
-template <typename T>
-__device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* arena, double Mrow, double Srow, int tid);
-
-// All threads: second pass over a segment whose buffers overflowed.  The histogram went on counting,
-// so the final threshold is as tight as ever: read the segment again and append every logit whose
-// bin is >= bin straight to the (emptied) candidate list.  A list that fills up again (a huge tie)
-// leaves the overflow flag set for the radix select.
-template <typename T>
-__device__ __noinline__ void recollect_from_global(const unsigned char* rowp, int chunk_begin, int chunk_end, int bin,
-                                                   const RowExtent ext, Candidates cb, int cap, SparsifyShared* sh,
-                                                   int tid) {
-    constexpr int kPer = Elt<T>::kPerVec;
-    const int lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) {
-        *cb.count = 0;
-        sh->overflow = 0;
-    }
-    consumer_sync();
-    const float z0 = sh->z0;
-    const float edge = raw_edge_below(bin, z0);  // for the tile and vector tests; a logit is judged by its relative key
-    const uint32_t min_key = (uint32_t)bin << kHistShift;
-    for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
-        LaneTile<T> lt;
-        lt.load(rowp, ch * kVecsPerChunk, lane, ext);
-        if (lt.reduce_max() >= edge) {
-#pragma unroll 1
-            for (int j = 0; j < kVecsPerLane; ++j) {
-                if (!(lt.vec_max(j) >= edge)) continue;
+// Which of a chunk's 32 tiles have a key >= bound: bit a of the result is tile a of the chunk in
+// ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the chunk's 64-byte line of maxima).
+__device__ __forceinline__ uint32_t chunk_survivors(const unsigned short* line, uint32_t bound) {
+    uint32_t w[16];
 #pragma unroll
-                for (int e = 0; e < kPer; ++e) {
-                    const float z = lt.elem(j, e);
-                    if (z >= -3.4028234e38f && rel_key(z, z0) >= min_key) {
-                        const int pos = atomicAdd(cb.count, 1);
-                        if (pos < cap) {
-                            cb.key[pos] = float_to_key(z);
-                            cb.idx[pos] = (ch * kVecsPerChunk + j * 32 + lane) * kPer + e;
-                        } else {
-                            sh->overflow = 1;
-                        }
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(line) + i);
+        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+    uint32_t m = 0;
+#pragma unroll
+    for (int a = 0; a < kTilesPerChunk; ++a) {
+        const int slot = ((a & 7) << 2) | (a >> 3);
+        const uint32_t raw = (slot & 1) ? (w[slot >> 1] >> 16) : (w[slot >> 1] & 0xffffu);
+        m |= (raw16_to_key16(raw) >= bound ? 1u : 0u) << a;
+    }
+    return m;
+}
+
+// The vectors a thread works on: units [u0, u1) of the row's survivor tiles (tl: their tile numbers in
+// address order, four vectors each), or of the whole row (tl == nullptr: unit = vector).  f(z, vi)
+// is called for each of them in ascending order with the vector's logits (-inf beyond the row).
+template <typename T, typename F>
+__device__ __forceinline__ void for_my_vectors(const unsigned char* rowp, const RowExtent& ext, int V, const uint32_t* tl,
+                                               int u0, int u1, F f) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    constexpr int kInFlight = 4;
+    for (int u = u0; u < u1; u += kInFlight) {
+        uint4 d[kInFlight];
+        int vi[kInFlight];
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) {
+            const int uu = u + i;
+            vi[i] = -1;
+            if (uu < u1) vi[i] = tl ? (int)(tl[uu >> 2] * (uint32_t)kVecsPerTile) + (uu & 3) : uu;
+            if (vi[i] >= 0 && vi[i] < ext.nvec_full) d[i] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) {
+            if (vi[i] < 0) continue;
+            float z[kPer];
+            if (vi[i] < ext.nvec_full) unpack_vec<T>(d[i], z);
+            else load_row_vector<T>(rowp, vi[i], ext, V, z);
+            f(z, vi[i]);
+        }
+    }
+}
+
+// The kk-th largest of the values value_of(z) in [lo, hi] over the thread block's vectors (values
+// outside the range, or negative, do not take part), by a histogram of kSelBins bins over the
+// range, narrowed once more if the range is wider than the histogram.  Results in sh: sel_bin = the
+// value, sel_above = how many are larger (inside [lo, hi]), sel_eq = how many equal it,
+// sel_total = how many lie in [lo, hi].  If fewer than kk lie in the range, sel_bin = -1 and only
+// sel_total is meaningful.  All threads call it; hist is kSelBins words of shared memory.
+template <typename T, typename VF>
+__device__ __forceinline__ void hist_select(const unsigned char* rowp, const RowExtent& ext, int V, const uint32_t* tl, int u0,
+                                            int u1, VF value_of, int lo, int hi, int kk, FinishShared* sh, uint32_t* hist,
+                                            int tid) {
+    constexpr int kPer = Elt<T>::kPerVec;
+    int above_acc = 0, total_first = -1;
+    for (;;) {
+        int s = 0;
+        while (((hi - lo) >> s) >= kSelBins) ++s;
+        for (int i = tid; i < kSelBins; i += kFinishThreads) hist[i] = 0u;
+        consumer_sync();
+        for_my_vectors<T>(rowp, ext, V, tl, u0, u1, [&](const float(&z)[kPer], int) {
+            int cur = -1;
+            uint32_t run = 0;
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                const int v = value_of(z[e]);
+                if (v >= lo && v <= hi) {
+                    const int b = (v - lo) >> s;
+                    if (b != cur) {  // equal neighbours (ties) cost one atomic, not one each
+                        if (run) atomicAdd(&hist[cur], run);
+                        cur = b;
+                        run = 0;
                     }
+                    ++run;
                 }
             }
-        }
-    }
-    consumer_sync();
-    if (tid == 0 && *cb.count > cap) *cb.count = cap;
-    consumer_sync();
-}
-
-// Radix-select fallbacks, out of line (one copy each).
-template <typename T>
-__device__ __noinline__ void reselect_from_global(const unsigned char* rowp, int e0, int n, int k, int idx_hi_byte,
-                                                  Candidates cb, SparsifyShared* sh, int tid) {
-    uint32_t kth;
-    GlobalSrc<T> src{rowp, e0};
-    select_topk<(Elt<T>::kBytes == 2)>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
-}
-template <bool kKeyHiOnly>
-__device__ __noinline__ void reselect_from_buffer(int n, int k, int idx_hi_byte, Candidates cb, SparsifyShared* sh,
-                                                  int tid) {
-    uint32_t kth;
-    BufferSrc src{cb.key, cb.idx};
-    select_topk<kKeyHiOnly>(src, n, k, idx_hi_byte, cb, &sh->sel, tid, &kth);
-}
-
-// All threads: bring every segment's candidates and statistics of a row into the candidate list.
-__device__ __forceinline__ void gather_segments(const SparsifyParams& p, int row, int nseg, Candidates cb,
-                                                SparsifyShared* sh, int tid, double* Mrow, double* Srow) {
-    const size_t slot0 = (size_t)row * nseg;
-    if (nseg == 1 && p.seg_cap <= 8 * kBlockThreads) {
-        // one segment: every load is issued before anything is used, so the row costs one trip to memory
-        const SegStat* st = &p.seg_stats[slot0];
-        const uint2* ent = p.seg_entries + slot0 * (size_t)p.seg_stride;
-        uint2 e[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int i = tid + j * kBlockThreads;
-            e[j] = i < p.seg_cap ? __ldcg(&ent[i]) : make_uint2(0u, 0u);
-        }
-        const int n = __ldcg(&st->n);
-        // fp64 is scarce (two warp instructions per clock per SM): one warp combines the eight
-        // per-warp pairs, one pair per lane, and leaves (M, S) in shared memory for the others
+            if (run) atomicAdd(&hist[cur], run);
+        });
+        consumer_sync();
         if (tid < 32) {
-            const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
-            const double Mw = tid < kWarps ? (double)__ldcg(&st->M[tid]) : -INFINITY;
-            const double Mall = warp_max(Sw > 0.0 ? Mw : -INFINITY);
-            const double Sall = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mall) : 0.0);
-            if (tid == 0) {
-                sh->scratch[0] = Mall;
-                sh->scratch[1] = Sall;
-            }
-        }
+            // rows of 32 bins from the top; lane l takes bin top - l of the row
+            uint32_t carried = 0;
+            int found_bin = -1;
+            uint32_t found_above = 0, found_eq = 0;
+            const int nb = ((hi - lo) >> s) + 1;
+            for (int top = nb - 1; top >= 0; top -= 32) {
+                const int b = top - tid;
+                const uint32_t cnt = b >= 0 ? hist[b] : 0u;
+                uint32_t incl = cnt;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int i = tid + j * kBlockThreads;
-            if (i < n) {
-                cb.key[i] = e[j].x;
-                cb.idx[i] = (int)e[j].y;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (tid >= o) incl += t;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, carried + incl >= (uint32_t)kk);
+                if (hit && found_bin < 0) {
+                    const int l = __ffs(hit) - 1;
+                    found_bin = top - l;
+                    found_above = carried + __shfl_sync(0xffffffffu, incl - cnt, l);
+                    found_eq = __shfl_sync(0xffffffffu, cnt, l);
+                }
+                carried += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (tid == 0) {
+                sh->sel_bin = found_bin;
+                sh->sel_above = (int)found_above;
+                sh->sel_eq = (int)found_eq;
+                sh->sel_total = (int)carried;
             }
         }
-        if (tid == 0) sh->cand_count = n;
         consumer_sync();
-        *Mrow = sh->scratch[0];
-        *Srow = sh->scratch[1];
+        const int bin = sh->sel_bin, above = sh->sel_above, eq = sh->sel_eq, total = sh->sel_total;
         consumer_sync();
-        return;
+        if (total_first < 0) total_first = total;
+        if (bin < 0 || s == 0) {
+            if (tid == 0) {
+                sh->sel_bin = bin < 0 ? -1 : lo + bin;
+                sh->sel_above = above_acc + above;
+                sh->sel_eq = eq;
+                sh->sel_total = total_first;
+            }
+            consumer_sync();
+            return;
+        }
+        above_acc += above;
+        kk -= above;
+        lo = lo + (bin << s);
+        hi = min(hi, lo + (1 << s) - 1);
     }
-    if (tid == 0) sh->cand_count = 0;
-    consumer_sync();
-    if (tid < 32) {  // one warp combines the nseg * 8 per-warp pairs (fp64 is scarce)
-        double Mall = -INFINITY;
-        for (int i = tid; i < nseg * kWarps; i += 32) {
-            const SegStat* st = &p.seg_stats[slot0 + i / kWarps];
-            if (__ldcg(&st->S[i % kWarps]) > 0.0) Mall = fmax(Mall, (double)__ldcg(&st->M[i % kWarps]));
-        }
-        Mall = warp_max(Mall);
-        double Sall = 0.0;
-        for (int i = tid; i < nseg * kWarps; i += 32) {
-            const SegStat* st = &p.seg_stats[slot0 + i / kWarps];
-            const double Sw = __ldcg(&st->S[i % kWarps]);
-            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st->M[i % kWarps]) - Mall);
-        }
-        Sall = warp_sum(Sall);
-        if (tid == 0) {
-            sh->scratch[0] = Mall;
-            sh->scratch[1] = Sall;
-        }
-    }
-    for (int g = 0; g < nseg; ++g) {
-        const SegStat* st = &p.seg_stats[slot0 + g];
-        const int ng = __ldcg(&st->n);
-        const uint2* ent = p.seg_entries + (slot0 + g) * (size_t)p.seg_stride;
-        const int base = sh->cand_count;
-        for (int i = tid; i < ng; i += kBlockThreads) {
-            const uint2 e2 = __ldcg(&ent[i]);
-            cb.key[base + i] = e2.x;
-            cb.idx[base + i] = (int)e2.y;
-        }
-        consumer_sync();
-        if (tid == 0) sh->cand_count = base + ng;
-        consumer_sync();
-    }
-    *Mrow = sh->scratch[0];
-    *Srow = sh->scratch[1];
-    consumer_sync();
 }
 
-// First launch: every segment streams, hands its candidates and statistics over and ends; the
-// rows are finished by sparsify_finish_kernel, launched next on the stream.
 template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, kSparsifyCtasPerSm) sparsify_kernel(const SparsifyParams p) {
-    constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
+__global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(const SparsifyParams p) {
     constexpr int kPer = Elt<T>::kPerVec;
-    constexpr int kChunkElems = kChunkBytes / Elt<T>::kBytes;
+    constexpr bool kBf16 = (Elt<T>::kBytes == 2);
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // every pointer below is derived from smem_raw by plain offsets, so that the compiler keeps
-    // them in the shared address space (shared-memory atomics and loads, not generic ones)
-    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw);
-    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + kHistOff);
-    uint2* staged = reinterpret_cast<uint2*>(smem_raw + kStagedOff);
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(staged + p.vcap);
-    int* cand_idx = reinterpret_cast<int*>(cand_key + p.cap);
-    uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.cap);
-    int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
-    const uint32_t base = smem_u32(smem_raw);
+    // carve-up (sizes in sparsify_finish_smem): header | hist | region A | region B | win_raw | win_idx
+    //   region A: group maxima, later the sort keys of the top-rho cut
+    //   region B: survivor tile list, later the fp64 work arrays
+    FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
+    static_assert(sizeof(FinishShared) <= kFinishHeaderBytes, "header");
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes);
+    const int k = p.k;
+    const size_t a_bytes = finish_region_a(p.ngroups, k), b_bytes = finish_region_b(p.tile_cap, k);
+    uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4);
+    unsigned long long* comp = reinterpret_cast<unsigned long long*>(gm);
+    uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4 + a_bytes);
+    double* cum = reinterpret_cast<double*>(tl);
+    double* wv = cum + k;
+    uint32_t* win_raw = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4 + a_bytes + b_bytes);
+    int* win_idx = reinterpret_cast<int*>(win_raw + k);
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
-    const int row = wk.row, chunk_begin = wk.chunk_begin, chunk_end = wk.chunk_end;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, row = blockIdx.x;
+    const int nseg = p.split.nseg;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
     const RowExtent ext = row_extent<T>(p.V);
-    const int k = p.k;
-    const float c = p.c.f;
-
-    // the first chunk's loads go out before anything else: their latency covers the set-up below
-    const int ch0 = chunk_begin + warp;
-    LaneTile<T> first;
-    if (ch0 < chunk_end) first.load(rowp, ch0 * kVecsPerChunk, lane, ext);
-    static_assert((kHistBins + kCoarseBins) % 4 == 0, "the histograms are cleared 16 bytes at a time");
-    uint4* hist4 = reinterpret_cast<uint4*>(hist);
-    for (int i = tid; i < (kHistBins + kCoarseBins) / 4; i += kBlockThreads) hist4[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (tid == 0) {
-        sh->thr_bin = kLowestFiniteBin;
-        sh->thr_word = threshold_word(kLowestFiniteBin, 0.f);  // P = -inf: every finite logit passes
-        sh->thr_edge_key = float_to_key(-3.4028234e38f);
-        sh->cand_count = 0;
-        sh->vec_count = 0;
-        sh->overflow = 0;
-        sh->trim_request = 0;
-        sh->n_above = 0;
-        // The row's ready flag is cleared here, by the CTA that will set it, and the store is fenced
-        // before the barrier after which the first thread of this CTA lets the finish kernel be
-        // scheduled.  A finish CTA runs only after every streaming CTA has passed that point, so it
-        // never sees a flag left by an earlier call, and the workspace needs no clearing between calls.
-        if (p.row_ready) {
-            *(volatile int*)&p.row_ready[row] = 0;
-            __threadfence();
-        }
+    if (tid == 0 && p.num_samples > 0)  // the uniforms are needed last: ask for their cache line now
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
+    if (tid < 32) sh->round_count[tid] = 0;
+    // ---- wait for the row's segments --------------------------------------------------------------
+    // Nothing the streaming kernel wrote is read before this point.  The row's own segments being
+    // handed over is enough to go on; a flag that does not come within the poll limit is recorded in
+    // the status word and the CTA waits for the end of the streaming kernel instead.
+    if (tid < 32) {
+        bool ok = true;
+        for (int s = lane; s < nseg; s += 32) ok = poll_row_ready(&p.seg_ready[(size_t)row * nseg + s], p.poll_limit) && ok;
+        ok = __all_sync(0xffffffffu, ok);
+        if (lane == 0) sh->ready = ok ? 1 : 0;
     }
-    // the segment's offset for the histogram's bins: the largest logit of its first chunks (see rel_key)
-    float first_max = -INFINITY;
-    if (ch0 < chunk_end) first_max = first.reduce_max();
-    first_max = warp_max(first_max);
-    if (lane == 0) sh->scratch[warp] = (double)first_max;
     __syncthreads();
-    allow_dependent_launch();
-    float z0 = (float)sh->scratch[0];
-#pragma unroll
-    for (int w = 1; w < kWarps; ++w) z0 = fmaxf(z0, (float)sh->scratch[w]);
-    if (!(z0 >= -3.4028234e38f && z0 <= 3.4028234e38f)) z0 = 0.f;  // nothing finite there: no offset
-    if (tid == 0) sh->z0 = z0;  // read by others only after the barriers below
-    Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
-
-    // ---- first threshold, from the segment's first chunks (one per warp) ---------------------------
-    // For k <= 256 the histogram takes only the maxima of the 1024 16-byte vectors of these chunks:
-    // the k-th largest of them is a lower bound on the k-th largest logit, and close to it while k
-    // is small against 1024.  Larger k counts every logit of the chunks.  The counts are wiped
-    // afterwards: the streaming loop below starts again at the first chunk (an L2 hit) and counts
-    // what it pushes.
-    {
-        if (ch0 < chunk_end) {
-            LaneTile<T>& lt = first;  // (reduce_max() already called)
-            if (k <= 256) {
-#pragma unroll
-                for (int j = 0; j < kVecsPerLane; ++j) {
-                    const float z = lt.vec_max(j);
-                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(rel_key(z, z0) >> kHistShift), 1u);
-                }
-            } else {
-#pragma unroll 4
-                for (int e = 0; e < kVecsPerLane * kPer; ++e) {
-                    const float z = lt.elem(e / kPer, e % kPer);
-                    if (z >= -3.4028234e38f) hist_count(base + kHistOff, base + kCoarseOff, (int)(rel_key(z, z0) >> kHistShift), 1u);
-                }
-            }
-        }
-        __syncthreads();
-        if (warp == 0) raise_threshold(sh, k);
-        __syncthreads();
-        for (int i = tid; i < (kHistBins + kCoarseBins) / 4; i += kBlockThreads) hist4[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (tid == 0) sh->n_above = 0;
-        __syncthreads();
-    }
-
-    // ---- streaming: no barriers; warp w rescans the histogram on its turn --------------------------
-    LaneSum ls;
-    ls.reset();
-    // chunks below pf_end are whole and inside the segment: the only ones asked of L2 ahead of time
-    const int pf_end = min(chunk_end, ext.nvec_full / kVecsPerChunk);
-    const unsigned char* lane_rowp = rowp + lane * kVecBytes;  // the loop's loads need no lane number
-    int ch = chunk_begin + warp;
-    for (;;) {
-        while (ch < chunk_end) {
-            __syncwarp();
-            if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->trim_request, 0)) break;
-            LaneTile<T> lt;
-            lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
-            if (ch + kPrefetchSteps * kWarps < pf_end && lane == 0)
-                prefetch_l2(rowp + (size_t)(ch + kPrefetchSteps * kWarps) * kChunkBytes, kChunkBytes);
-            const float lm = lt.reduce_max();
-            const Threshold<T> th(sh);
-            filter_push(lt, th, lm, ch * kVecsPerChunk + lane, base, p);  // while the vector maxima are at hand
-            ls.raise_to(lm, c);
-            lt.accumulate(ls, c);
-            // The warps take turns at looking whether enough has been counted above the threshold
-            // bin for it to rise (ch mod 8 is the warp's own, so the turns differ), and rescan then.
-            if ((((ch >> 3) ^ ch) & (kWarps - 1)) == 0) {
-                __syncwarp();
-                if (__shfl_sync(0xffffffffu, *(volatile int*)&sh->n_above, 0) >= k) raise_threshold(sh, k);
-            }
-            ch += kWarps;
-        }
-        const int all_done = __syncthreads_and(ch >= chunk_end);
-        const int want_trim = sh->trim_request;
-        __syncthreads();
-        if (all_done) break;
-        if (want_trim) {
-            if (!sh->overflow) {
-                if (warp == 0) raise_threshold(sh, k);
-                consumer_sync();
-                const int bin = sh->thr_bin;
-                expand_staged<T>(staged, p.vcap, rowp, ext, cb, p.cap, bin, p.V, sh, tid);
-                if (sh->cand_count > p.high) compact_buffer(cb, bin, sh, tid);
-            }
-            if (tid == 0) sh->trim_request = 0;
-            __syncthreads();
-        }
-    }
-
-    // ---- hand-over: one (M, S) pair per warp and the segment's entries; the kernel boundary publishes
-    // them to the finish kernel
-    const float Mw = warp_max(ls.M);
-    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
-    const size_t slot = (size_t)row * wk.nseg + wk.seg;
-    uint2* my_entries = p.seg_entries + slot * (size_t)p.seg_stride;
-    SegStat* st = &p.seg_stats[slot];
-    if (lane == 0) {
-        st->S[warp] = Sw;
-        st->M[warp] = Mw;
-    }
-    // (the loop's last barrier ordered every write of the flags read here)
-    if (p.raw_cap > 0 && !sh->overflow && sh->cand_count == 0) {
-        // The staging buffer never filled: its tiles go over as they are, with the final threshold
-        // bin, and the finish kernel reads the few that still pass back from global memory, all
-        // rows at once, instead of this CTA waiting on them now.
-        const int n = sh->vec_count;
-        for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = staged[i];
-        if (tid == 0) {
-            st->n = n;
-            st->raw_bin = sh->thr_bin;
-            st->z0 = sh->z0;
-        }
-        __syncthreads();  // every thread's part of the hand-over is written
-        if (tid == 0 && p.row_ready) publish_row_ready(&p.row_ready[row]);
-        return;
-    }
-
-    // ---- what is still staged becomes candidates; a buffer that overflowed is rebuilt from global memory
-    if (!sh->overflow) expand_staged<T>(staged, p.vcap, rowp, ext, cb, p.cap, sh->thr_bin, p.V, sh, tid);
-    if (sh->overflow) {
-        if (warp == 0) raise_threshold(sh, k);
-        consumer_sync();
-        recollect_from_global<T>(rowp, chunk_begin, chunk_end, sh->thr_bin, ext, cb, p.cap, sh, tid);
-    }
-    if (sh->overflow) {
-        const int e0 = chunk_begin * kChunkElems;
-        const int n = min(p.V, chunk_end * kChunkElems) - e0;
-        reselect_from_global<T>(rowp, e0, n, k, p.idx_hi_byte, cb, sh, tid);
-        if (tid == 0) sh->overflow = 0;
-        consumer_sync();
-    }
-    // candidates: all at or above this segment's final threshold
-    int n = sh->cand_count;
-    if (n > p.seg_cap) {  // earlier expansions used looser thresholds: keep what the final one admits
-        compact_buffer(cb, sh->thr_bin, sh, tid);
-        n = sh->cand_count;
-    }
-    if (n > p.seg_cap) {  // heavy ties at the boundary: hand over the exact k
-        reselect_from_buffer<kHiOnly>(n, k, p.idx_hi_byte, cb, sh, tid);
-        n = sh->cand_count;
-    }
-    for (int i = tid; i < n; i += kBlockThreads) my_entries[i] = make_uint2(cand_key[i], (uint32_t)cand_idx[i]);
-    if (tid == 0) {
-        st->n = n;
-        st->raw_bin = -1;
-    }
-    __syncthreads();  // every thread's part of the hand-over is written
-    if (tid == 0 && p.row_ready) publish_row_ready(&p.row_ready[row]);
-}
-
-// Second launch: one CTA per row merges the row's segments and finishes it.
-// Same shared-memory carve-up as the streaming kernel, with no staging buffer (vcap = 0).
-template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, 6) sparsify_finish_kernel(const SparsifyParams p) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    SparsifyShared* sh = reinterpret_cast<SparsifyShared*>(smem_raw);
-    unsigned char* arena = smem_raw + kHistOff;
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem_raw + kStagedOff);
-    int* cand_idx = reinterpret_cast<int*>(cand_key + p.fin_cap);
-    uint32_t* tmp_key = reinterpret_cast<uint32_t*>(cand_idx + p.fin_cap);
-    int* tmp_idx = reinterpret_cast<int*>(tmp_key + p.k);
-    const int tid = threadIdx.x, row = blockIdx.x;
-    // the uniforms are needed last: ask for their cache line now
-    if (tid == 0 && p.num_samples > 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
-    if (tid == 0) sh->overflow = 0;
-    // Nothing the streaming kernel wrote is read before this point.  A row of one segment goes on
-    // as soon as its own ready flag is set (see poll_row_ready); rows cut into segments, and a
-    // flag that does not come, wait for the end of the streaming kernel.
-    if (p.row_ready) {
-        if (tid == 0) sh->n_list = poll_row_ready(&p.row_ready[row]) ? 1 : 0;
-        __syncthreads();
-        if (!sh->n_list) wait_for_primary_kernel();
-        __syncthreads();
-    } else {
+    if (!sh->ready) {
+        if (tid == 0) atomicOr(p.status, TSLT_STATUS_WAIT_FELL_BACK);
         wait_for_primary_kernel();
     }
-    if (row == 0 && tid == 0) *p.status = 0;
-    Candidates cb{cand_key, cand_idx, tmp_key, tmp_idx, &sh->cand_count};
-    double Mrow, Srow;
-    gather_segments(p, row, p.split.nseg, cb, sh, tid, &Mrow, &Srow);
-    finalize_row<T>(p, row, cb, sh, arena, Mrow, Srow, tid);
-    // this kernel's completion must imply the streaming kernel's: one CTA sees to that
-    if (row == 0 && p.row_ready) wait_for_primary_kernel();
-}
-
-// Position of entry (key, idx) of the buffer in the order (key descending, idx ascending) /
-// (idx ascending), by counting the entries that precede it.
-__device__ __forceinline__ int rank_by_key(const uint32_t* key, const int* idx, int n, uint32_t my_key, int my_idx) {
-    int r = 0;
-    for (int j = 0; j < n; ++j) {
-        const uint32_t kj = key[j];
-        const int ij = idx[j];
-        r += (kj > my_key || (kj == my_key && ij < my_idx)) ? 1 : 0;
-    }
-    return r;
-}
-__device__ __forceinline__ int rank_by_idx(const int* idx, int n, int my_idx) {
-    int r = 0;
-    for (int j = 0; j < n; ++j) r += idx[j] < my_idx ? 1 : 0;
-    return r;
-}
-
-// Exact top-k of the row, nucleus cut, renormalisation, sampling and the ascending-index payload.
-template <typename T>
-__device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Candidates cb, SparsifyShared* sh,
-                                          unsigned char* arena, double Mrow, double Srow, int tid) {
-    constexpr bool kHiOnly = (Elt<T>::kBytes == 2);
-    const int k = p.k;
-    const int lane = tid & 31, warp = tid >> 5;
-    uint32_t* cand_key = cb.key;
-    int* cand_idx = cb.idx;
-    uint32_t* hist = reinterpret_cast<uint32_t*>(arena);
-    uint2* bnd = reinterpret_cast<uint2*>(arena + (kHistBins + kCoarseBins) * 4);
-    const int nc = sh->cand_count;
-
-    // ---- the bin of the k-th largest logit ------------------------------------------------------
-    // exact counts of the candidates (the streaming histogram only counted vector maxima)
-    for (int i = tid; i < kHistBins + kCoarseBins; i += kBlockThreads) hist[i] = 0u;
-    consumer_sync();
-    for (int i = tid; i < nc; i += kBlockThreads)
-        hist_count(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, (int)(cand_key[i] >> kHistShift), 1u);
-    consumer_sync();
-    if (warp == 0) {
-        uint32_t above;
-        const int b = scan_boundary(smem_u32(sh) + kHistOff, smem_u32(sh) + kCoarseOff, k, &above);
-        if (lane == 0) {
-            sh->sel_bin = b;  // -1: fewer than k candidates exist, all of them are kept
-            sh->sel_above = (int)above;
-            sh->n_win = 0;
-            sh->n_bnd = 0;
+    __syncthreads();
+    // ---- the row's log-normaliser, by one warp (fp64 is scarce) -------------------------------------
+    if (warp == 1) {
+        const SegStat* st = p.seg_stats + (size_t)row * nseg;
+        double Mall = -INFINITY;
+        for (int i = lane; i < nseg * kWarps; i += 32)
+            if (__ldcg(&st[i / kWarps].S[i % kWarps]) > 0.0) Mall = fmax(Mall, (double)__ldcg(&st[i / kWarps].M[i % kWarps]));
+        Mall = warp_max(Mall);
+        double Sall = 0.0;
+        for (int i = lane; i < nseg * kWarps; i += 32) {
+            const double Sw = __ldcg(&st[i / kWarps].S[i % kWarps]);
+            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st[i / kWarps].M[i % kWarps]) - Mall);
         }
+        Sall = warp_sum(Sall);
+        if (lane == 0) sh->lrow = Sall > 0.0 ? Mall + log2(Sall) : -INFINITY;
     }
-    consumer_sync();
-    const int sel_bin = sh->sel_bin;
-    // ---- everything above that bin is in; the bin itself goes to the boundary list ---------------
-    for (int i = tid; i < nc; i += kBlockThreads) {
-        const uint32_t kk = cand_key[i];
-        const int bin = (int)(kk >> kHistShift);
-        if (bin > sel_bin) {
-            const int pos = atomicAdd(&sh->n_win, 1);
-            if (pos < k) {
-                cb.tmp_key[pos] = kk;
-                cb.tmp_idx[pos] = cand_idx[i];
+    // ---- 1. group maxima of the tile keys ---------------------------------------------------------------
+    const int ntiles = p.nchunks * kTilesPerChunk;
+    const unsigned short* tmax = p.tile_max + (size_t)row * ntiles;
+    const int glog = p.group_log2, ngroups = p.ngroups;
+    if (glog > 3)
+        for (int i = tid; i < ngroups; i += kFinishThreads) gm[i] = 0u;
+    if (tid == 0) sh->max16 = 0;
+    __syncthreads();
+    {
+        uint32_t my_max = 0;
+        const int nv8 = ntiles / 8;
+        for (int v = tid; v < nv8; v += kFinishThreads) {
+            const uint4 w = __ldcg(reinterpret_cast<const uint4*>(tmax) + v);
+            uint32_t kk[8];
+            kk[0] = raw16_to_key16(w.x & 0xffffu); kk[1] = raw16_to_key16(w.x >> 16);
+            kk[2] = raw16_to_key16(w.y & 0xffffu); kk[3] = raw16_to_key16(w.y >> 16);
+            kk[4] = raw16_to_key16(w.z & 0xffffu); kk[5] = raw16_to_key16(w.z >> 16);
+            kk[6] = raw16_to_key16(w.w & 0xffffu); kk[7] = raw16_to_key16(w.w >> 16);
+            // groups are runs of consecutive SLOTS (any fixed partition of the tiles will do)
+            if (glog == 0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) gm[v * 8 + i] = kk[i];
+            } else if (glog == 1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) gm[v * 4 + i] = max(kk[2 * i], kk[2 * i + 1]);
+            } else if (glog == 2) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) gm[v * 2 + i] = max(max(kk[4 * i], kk[4 * i + 1]), max(kk[4 * i + 2], kk[4 * i + 3]));
             }
-        } else if (bin == sel_bin) {
-            const int pos = atomicAdd(&sh->n_bnd, 1);
-            if (pos < kBoundaryCap) bnd[pos] = make_uint2(kk, (uint32_t)cand_idx[i]);
+            const uint32_t m8 = max(max(max(kk[0], kk[1]), max(kk[2], kk[3])), max(max(kk[4], kk[5]), max(kk[6], kk[7])));
+            if (glog == 3) gm[v] = m8;
+            else if (glog > 3) atomicMax(&gm[v >> (glog - 3)], m8);
+            my_max = max(my_max, m8);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) my_max = max(my_max, __shfl_xor_sync(0xffffffffu, my_max, o));
+        if (lane == 0) atomicMax(&sh->max16, (int)my_max);
+    }
+    __syncthreads();
+    const int max16 = min(sh->max16, (int)kHighestFinite16);
+    const double L2 = sh->lrow;
+    // ---- 2. the k-th largest group maximum, by bisection on its 16 bits -----------------------------------
+    uint32_t bound = 0;
+    if (ngroups >= k) {
+        for (int bit = 15; bit >= 0; --bit) {
+            const uint32_t cand = bound | (1u << bit);
+            int cnt = 0;
+            for (int i = tid; i < ngroups; i += kFinishThreads) cnt += gm[i] >= cand ? 1 : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            if (lane == 0 && cnt) atomicAdd(&sh->round_count[bit], cnt);
+            __syncthreads();
+            if (sh->round_count[bit] >= k) bound = cand;
         }
     }
-    consumer_sync();
-    const int n_above = min(sh->n_win, k), nb = sh->n_bnd;
-    int n0;
-    if (nb > kBoundaryCap) {
-        // heavy ties: radix select over the whole buffer (leaves its winners at the front of the buffer)
-        reselect_from_buffer<kHiOnly>(nc, k, p.idx_hi_byte, cb, sh, tid);
-        n0 = min(sh->cand_count, k);
-    } else {
-        const int need = min(k - n_above, nb);
-        for (int t = tid; t < nb; t += kBlockThreads) {
-            const uint2 me = bnd[t];
-            int r = t;
-            if (nb > need) {
-                r = 0;
-                for (int j = 0; j < nb; ++j) {
-                    const uint2 o = bnd[j];
-                    r += (o.x > me.x || (o.x == me.x && (int)o.y < (int)me.y)) ? 1 : 0;
+    int lo16 = max((int)bound, (int)kLowestFinite16);
+    // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
+    // Thread t takes a run of consecutive chunks; a chunk's 32 tile keys are one 64-byte line.
+    const int cpt = (p.nchunks + kFinishThreads - 1) / kFinishThreads;
+    const int ch0 = min(p.nchunks, tid * cpt), ch1 = min(p.nchunks, ch0 + cpt);
+    int my_surv = 0;
+    for (int ch = ch0; ch < ch1; ++ch) my_surv += __popc(chunk_survivors(tmax + ch * kTilesPerChunk, (uint32_t)lo16));
+    int n_surv;
+    int pos = block_exscan(my_surv, tid, sh->iscr, &n_surv);
+    const bool listed = n_surv <= p.tile_cap;
+    if (listed) {
+        for (int ch = ch0; ch < ch1; ++ch) {
+            uint32_t m = chunk_survivors(tmax + ch * kTilesPerChunk, (uint32_t)lo16);  // bit a: tile a of the chunk
+            while (m) {
+                const int a = __ffs(m) - 1;
+                m &= m - 1;
+                tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
+            }
+        }
+    }
+    __syncthreads();
+    // the vectors this thread works on from here: a contiguous run of the survivors' vectors, or of the row's
+    const uint32_t* units = listed ? tl : nullptr;
+    const int n_units = listed ? n_surv * kVecsPerTile : (p.V + kPer - 1) / kPer;
+    const int upt = (n_units + kFinishThreads - 1) / kFinishThreads;
+    const int u0 = min(n_units, tid * upt), u1 = min(n_units, u0 + upt);
+    if (!listed) lo16 = (int)kLowestFinite16;
+
+    // ---- 4. the exact k-th largest logit --------------------------------------------------------------------
+    // level 1: its 16-bit key among the finite logits of the survivors
+    auto key16_of = [](float z) -> int {
+        const uint32_t k16 = float_to_key(z) >> 16;
+        return (k16 >= kLowestFinite16 && k16 <= kHighestFinite16) ? (int)k16 : -1;
+    };
+    int n0 = 0;                 // winners: min(k, finite logits)
+    uint32_t e32 = 0;           // key of the k-th largest logit
+    int need_ties = 0;          // how many logits equal to it are winners (the lowest indices)
+    if (max16 >= lo16) {
+        hist_select<T>(rowp, ext, p.V, units, u0, u1, key16_of, lo16, max16, k, sh, hist, tid);
+        const int e16 = sh->sel_bin, above = sh->sel_above, eq = sh->sel_eq, total = sh->sel_total;
+        consumer_sync();
+        if (e16 < 0) {  // fewer than k finite logits in the row: all of them win
+            n0 = total;
+            e32 = 0u;
+            need_ties = 0;
+            // every finite logit is "above" the key 0; nothing ties
+        } else if (kBf16) {
+            n0 = k;
+            e32 = ((uint32_t)e16 << 16) | ((e16 & 0x8000) ? 0u : 0xffffu);  // keys of bf16 values: low half follows the sign
+            need_ties = k - above;
+        } else {
+            // level 2 (fp32 rows): the low 16 bits among the logits whose high bits equal e16
+            const uint32_t hi_bits = (uint32_t)e16;
+            auto low16_of = [hi_bits](float z) -> int {
+                const uint32_t kz = float_to_key(z);
+                return (kz >> 16) == hi_bits ? (int)(kz & 0xffffu) : -1;
+            };
+            hist_select<T>(rowp, ext, p.V, units, u0, u1, low16_of, 0, 0xffff, k - above, sh, hist, tid);
+            const int low = sh->sel_bin, above2 = sh->sel_above;
+            consumer_sync();
+            n0 = k;
+            e32 = (hi_bits << 16) | (uint32_t)low;
+            need_ties = k - above - above2;
+            (void)eq;
+        }
+    }
+    // ---- 5. the winners, in ascending index ---------------------------------------------------------------
+    int n = 0;
+    if (n0 > 0) {
+        int c_gt = 0, c_eq = 0;
+        const uint32_t e32c = e32;
+        for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                if (key16_of(z[e]) < lo16) continue;
+                const uint32_t kz = float_to_key(z[e]);
+                c_gt += kz > e32c ? 1 : 0;
+                c_eq += kz == e32c ? 1 : 0;
+            }
+        });
+        int tot_eq, tot_w;
+        const int eq_before = block_exscan(c_eq, tid, sh->iscr, &tot_eq);
+        const int my_ties = max(0, min(c_eq, need_ties - eq_before));
+        int wpos = block_exscan(c_gt + my_ties, tid, sh->iscr, &tot_w);
+        int ties_left = my_ties;
+        for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                if (key16_of(z[e]) < lo16) continue;
+                const uint32_t kz = float_to_key(z[e]);
+                bool win = kz > e32c;
+                if (kz == e32c && ties_left > 0) {
+                    win = true;
+                    --ties_left;
+                }
+                if (win && wpos < k) {
+                    win_raw[wpos] = __float_as_uint(z[e]);
+                    win_idx[wpos] = vi * kPer + e;
+                    ++wpos;
                 }
             }
-            if (r < need) {
-                cb.tmp_key[n_above + r] = me.x;
-                cb.tmp_idx[n_above + r] = (int)me.y;
-            }
-        }
-        consumer_sync();
-        n0 = n_above + need;
-        for (int i = tid; i < n0; i += kBlockThreads) {
-            cand_key[i] = cb.tmp_key[i];
-            cand_idx[i] = cb.tmp_idx[i];
-        }
-        consumer_sync();
+        });
+        n = min(tot_w, k);
+        __syncthreads();
     }
-
-    if (tid == 0) sh->scratch[2] = Mrow + log2(Srow);  // base-2 log of the softmax normaliser (once: fp64 is scarce)
-    consumer_sync();
-    const double L2 = sh->scratch[2];
+    n0 = n;
+    const double cf = (double)p.c.f;  // the scale the streaming sum used: keeps q consistent with the normaliser
     const double cd = p.c.d;
-    // the histogram and the boundary list are no longer needed: their arena holds the fp64 work arrays
-    unsigned long long* comp = reinterpret_cast<unsigned long long*>(arena);          // 1024 * 8
-    double* wv = reinterpret_cast<double*>(arena + 8192);                             // 1024 * 8
-    double* cum = reinterpret_cast<double*>(arena + 16384);                           // 1024 * 8
-    int n = n0;
     double mass = 0.0;
+    // ---- 6. top-rho cut ---------------------------------------------------------------------------------------
     if (n0 > 0 && p.top_p < 1.0f) {
-        // order the candidates by (logit descending, index ascending) and cut at the nucleus
-        if (n0 <= kRankSortMax) {
-            if (tid < n0) {
-                const uint32_t kk = cand_key[tid];
-                const int ii = cand_idx[tid];
-                const int r = rank_by_key(cand_key, cand_idx, n0, kk, ii);
-                comp[r] = ((unsigned long long)kk << 32) | (unsigned long long)(0xffffffffu - (uint32_t)ii);
-            }
-            consumer_sync();
-        } else {
-            const int P = next_pow2(n0);
-            for (int i = tid; i < P; i += kBlockThreads)
-                comp[i] = i < n0 ? (((unsigned long long)cand_key[i] << 32) | (unsigned long long)(0xffffffffu - (uint32_t)cand_idx[i])) : 0ull;
-            consumer_sync();
-            bitonic_sort<true>(comp, P, tid);
-        }
-        for (int i = tid; i < n0; i += kBlockThreads) {
-            const float z = key_to_float((uint32_t)(comp[i] >> 32));
-            cum[i] = exp2((double)z * cd - L2);
-        }
+        const int P = pow2_at_least(n0);
+        for (int i = tid; i < P; i += kFinishThreads)
+            comp[i] = i < n0 ? (((unsigned long long)float_to_key(__uint_as_float(win_raw[i])) << 32) |
+                                (unsigned long long)(0xffffffffu - (uint32_t)win_idx[i])) : 0ull;
+        consumer_sync();
+        bitonic_sort<true>(comp, P, tid);
+        for (int i = tid; i < n0; i += kFinishThreads)
+            cum[i] = exp2((double)key_to_float((uint32_t)(comp[i] >> 32)) * cf - L2);
         consumer_sync();
         block_inclusive_scan(cum, n0, tid, sh->scratch);
-        // n* = first n with c_n >= top_p
         const double tp = (double)p.top_p;
         int lo = 0, hi = n0;
-        while (lo < hi) {
+        while (lo < hi) {  // first n with c_n >= top_p
             const int mid = (lo + hi) >> 1;
             if (cum[mid] >= tp) hi = mid; else lo = mid + 1;
         }
         n = lo < n0 ? lo + 1 : n0;
         mass = cum[n - 1];
         consumer_sync();
-        for (int i = tid; i < n; i += kBlockThreads) {
-            cand_key[i] = (uint32_t)(comp[i] >> 32);
-            cand_idx[i] = (int)(0xffffffffu - (uint32_t)(comp[i] & 0xffffffffull));
-        }
-        consumer_sync();
-    }
-    // ascending index order
-    if (n > 0) {
-        if (n <= kRankSortMax) {
-            if (tid < n) {
-                const int ii = cand_idx[tid];
-                comp[rank_by_idx(cand_idx, n, ii)] = ((unsigned long long)(uint32_t)ii << 32) | (unsigned long long)cand_key[tid];
+        if (n < n0) {
+            // keep what precedes the cut in (logit descending, index ascending): a larger key, or the
+            // cut's key and an index up to the cut's
+            const unsigned long long cutc = comp[n - 1];
+            const uint32_t ckey = (uint32_t)(cutc >> 32);
+            const int cidx = (int)(0xffffffffu - (uint32_t)cutc);
+            const int ipt = (n0 + kFinishThreads - 1) / kFinishThreads;
+            const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
+            uint32_t keep_raw[4];
+            int keep_idx[4];
+            int kept = 0;
+            for (int i = i0; i < i1; ++i) {  // ipt <= 4 (k <= 1024)
+                const uint32_t kz = float_to_key(__uint_as_float(win_raw[i]));
+                if (kz > ckey || (kz == ckey && win_idx[i] <= cidx)) {
+                    keep_raw[kept] = win_raw[i];
+                    keep_idx[kept] = win_idx[i];
+                    ++kept;
+                }
             }
+            int tot;
+            int kp = block_exscan(kept, tid, sh->iscr, &tot);  // (its barriers order the reads above before the writes below)
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < kept) {
+                    win_raw[kp + i] = keep_raw[i];
+                    win_idx[kp + i] = keep_idx[i];
+                }
             consumer_sync();
-        } else {
-            const int P = next_pow2(n);
-            for (int i = tid; i < P; i += kBlockThreads)
-                comp[i] = i < n ? (((unsigned long long)(uint32_t)cand_idx[i] << 32) | (unsigned long long)cand_key[i]) : ~0ull;
-            consumer_sync();
-            bitonic_sort<false>(comp, P, tid);
         }
     }
-    // renormalised truncated distribution in fp64: w_i = 2^(y_i - m_S), CDF by inclusive scan
+    // ---- 7. renormalised truncated distribution in fp64, CDF, samples, outputs ----------------------------
     double my_max = -INFINITY;
-    for (int i = tid; i < n; i += kBlockThreads) {
-        const float z = key_to_float((uint32_t)(comp[i] & 0xffffffffull));
-        const double y = (double)z * cd;
+    for (int i = tid; i < n; i += kFinishThreads) {
+        const double y = (double)__uint_as_float(win_raw[i]) * cd;
         wv[i] = y;
         my_max = fmax(my_max, y);
     }
     const double mS = block_max(my_max, tid, sh->scratch);
     double my_mass = 0.0;
-    for (int i = tid; i < n; i += kBlockThreads) {
-        const double y = wv[i];
-        if (!(p.top_p < 1.0f)) my_mass += exp2(y - L2);
-        const double w = exp2(y - mS);
+    for (int i = tid; i < n; i += kFinishThreads) {
+        if (!(p.top_p < 1.0f)) my_mass += exp2((double)__uint_as_float(win_raw[i]) * cf - L2);
+        const double w = exp2(wv[i] - mS);
         wv[i] = w;
         cum[i] = w;
     }
@@ -1106,17 +662,11 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
     else consumer_sync();
     block_inclusive_scan(cum, n, tid, sh->scratch);
 
-    // ---- outputs ------------------------------------------------------------------------------
     int* o_idx = p.idx + (size_t)row * k;
     float* o_logit = p.logit + (size_t)row * k;
-    for (int i = tid; i < k; i += kBlockThreads) {
-        if (i < n) {
-            o_idx[i] = (int)(comp[i] >> 32);
-            o_logit[i] = key_to_float((uint32_t)(comp[i] & 0xffffffffull));
-        } else {
-            o_idx[i] = -1;
-            o_logit[i] = -INFINITY;
-        }
+    for (int i = tid; i < k; i += kFinishThreads) {
+        o_idx[i] = i < n ? win_idx[i] : -1;
+        o_logit[i] = i < n ? __uint_as_float(win_raw[i]) : -INFINITY;
     }
     if (tid == 0) {
         p.count[row] = n;
@@ -1124,408 +674,34 @@ __device__ __noinline__ void finalize_row(const SparsifyParams& p, int row, Cand
         if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
     }
     const double W = n > 0 ? cum[n - 1] : 0.0;
-    for (int sidx = tid; sidx < p.num_samples; sidx += kBlockThreads) {
+    for (int sidx = tid; sidx < p.num_samples; sidx += kFinishThreads) {
         int tok = -1;
         if (n > 0) {
             const float u = clamp_uniform(p.uniforms[(size_t)row * p.num_samples + sidx]);
-            int pos = first_greater(cum, n, (double)u * W);
-            if (pos >= n) {
-                pos = n - 1;
-                while (pos > 0 && !(wv[pos] > 0.0)) --pos;
+            int pos2 = first_greater(cum, n, (double)u * W);
+            if (pos2 >= n) {
+                pos2 = n - 1;
+                while (pos2 > 0 && !(wv[pos2] > 0.0)) --pos2;
             }
-            tok = (int)(comp[pos] >> 32);
+            tok = win_idx[pos2];
         }
         p.token[(size_t)row * p.num_samples + sidx] = tok;
     }
-}
-
-// ---- finish kernel for small k --------------------------------------------------------------------
-// Rows of one segment with k <= 256 are finished by a CTA of 64, 96, 128 or 256 threads (at least
-// k) with 6 to 21 KB of shared memory, so that every row of a large batch is resident at once:
-// finishing a row is a chain of dependent steps (trips to memory, rank counting, two scans), and
-// what it costs machine-wide is the length of that chain times the number of waves.
-constexpr int kSmallMaxThreads = 256;  // and so the largest k of this kernel
-// candidates a row may bring as (key, index) entries: 2 k at most (seg_cap)
-__host__ __device__ constexpr int small_cand_cap(int nt) { return nt > 128 ? 512 : 256; }
-// Candidates the kernel may make from a row's staged tiles: 256, and 512 for k above 96, where
-// 256 is only 2 k and the threshold bin's share can exceed it on ordinary rows.  (512 everywhere
-// cost the 64-thread kernel 9 us on 2048 rows of 256 000 logits: fewer finish CTAs fit beside the streaming
-// CTAs of the last wave.)
-__host__ __device__ constexpr int small_list_cap(int nt) { return nt > 128 ? 1024 : nt > 96 ? 512 : 256; }
-// marked vectors in the staged tiles of a row that pass its final threshold
-__host__ __device__ constexpr int small_pass_cap(int nt) { return nt > 128 ? 1024 : 512; }
-
-template <int kList, int kK, int kPass> struct SmallShared {
-    unsigned long long comp[kList];  // candidates as key << 32 | ~index: larger is earlier in the top-k order
-    uint32_t wkey[kK];  // winners in (key descending, index ascending) order, then in ascending index
-    int widx[kK];
-    uint32_t okey[kK];
-    int oidx[kK];
-    double cum[kK];
-    double wv[kK];
-    double red[8];   // one slot per warp for the block scans
-    double lrow;     // the row's log2-normaliser
-    int n_cut;
-    // rows handed over as staged lane tiles
-    uint32_t pass[kPass];  // marked vectors of the tiles whose largest logit passes the final threshold
-    int n_pass, n_cand;
-    unsigned long long best[kSmallMaxThreads / 32];
-};
-template <int NT> using SmallSharedFor = SmallShared<small_list_cap(NT), NT, small_pass_cap(NT)>;
-
-template <int NT> __device__ __forceinline__ void small_sync() { asm volatile("bar.sync 2, %0;" ::"n"(NT) : "memory"); }
-
-// inclusive scan of one value per thread over the NT threads; returns this thread's inclusive sum
-template <int NT> __device__ __forceinline__ double small_scan(double v, int tid, double* red, double* total) {
-    const int lane = tid & 31, warp = tid >> 5;
-    double incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) red[warp] = incl;
-    small_sync<NT>();
-    double base = 0.0, tot = 0.0;
-#pragma unroll
-    for (int w = 0; w < NT / 32; ++w) {
-        const double t = red[w];
-        if (w < warp) base += t;
-        tot += t;
-    }
-    small_sync<NT>();
-    *total = tot;
-    return base + incl;
-}
-template <int NT> __device__ __forceinline__ double small_max(double v, int tid, double* red) {
-    v = warp_max(v);
-    if ((tid & 31) == 0) red[tid >> 5] = v;
-    small_sync<NT>();
-    double m = red[0];
-#pragma unroll
-    for (int w = 1; w < NT / 32; ++w) m = fmax(m, red[w]);
-    small_sync<NT>();
-    return m;
-}
-
-// The slow way to a row's k winners from its staged tiles: one winner per round, each round a pass
-// over the marked vectors of the passing tiles (the kernel's list of them if it held them all).
-// Only there to be correct when a row has more tied candidates around its k-th logit than the
-// lists of the kernel below hold.
-// composite = key << 32 | ~index: larger is earlier in (logit descending, index ascending)
-template <typename T, int NT>
-__device__ __noinline__ int winners_one_by_one(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                               float z0, int n_listed, SmallSharedFor<NT>* sm, int tid) {
-    constexpr int kPer = Elt<T>::kPerVec;
-    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
-    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const RowExtent ext = row_extent<T>(p.V);
-    const uint32_t min_key = (uint32_t)bin << kHistShift;
-    unsigned long long last = ~0ull;
-    int found = 0;
-    for (; found < p.k; ++found) {
-        unsigned long long best = 0ull;
-        // the vectors to look at: those listed in sm->pass (n_listed >= 0), else every marked vector
-        // of every passing tile of the hand-over
-        const int n_items = n_listed >= 0 ? n_listed : n_tiles * kVecsPerLane;
-        for (int i = tid; i < n_items; i += NT) {
-            int vi;
-            if (n_listed >= 0) {
-                vi = (int)sm->pass[i];
-            } else {
-                const uint2 e = __ldcg(&ent[i / kVecsPerLane]);
-                const int j = i % kVecsPerLane;
-                if (e.y < min_key || !((e.x >> (kTileMaskShift + j)) & 1u)) continue;
-                vi = (int)(e.x & kVecMask) + 32 * j;
-            }
-            float z[kPer];
-            load_row_vector<T>(rowp, vi, ext, p.V, z);
-#pragma unroll
-            for (int q = 0; q < kPer; ++q) {
-                if (z[q] >= -3.4028234e38f && rel_key(z[q], z0) >= min_key) {
-                    const unsigned long long comp = ((unsigned long long)float_to_key(z[q]) << 32) |
-                                                    (unsigned long long)(0xffffffffu - (uint32_t)(vi * kPer + q));
-                    if (comp < last && comp > best) best = comp;
-                }
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long t = __shfl_xor_sync(0xffffffffu, best, o);
-            best = t > best ? t : best;
-        }
-        if ((tid & 31) == 0) sm->best[tid >> 5] = best;
-        small_sync<NT>();
-#pragma unroll
-        for (int w = 0; w < NT / 32; ++w) best = sm->best[w] > best ? sm->best[w] : best;
-        small_sync<NT>();
-        if (best == 0ull) break;
-        if (tid == 0) sm->comp[found] = best;
-        last = best;
-    }
-    small_sync<NT>();
-    return found;
-}
-
-// NT threads: the row was handed over as n_tiles staged lane tiles and its final threshold bin.
-// Puts the row's candidates (every logit whose bin is >= bin, at least its k largest) into
-// sm->comp and returns their number (<= small_list_cap(NT)).  The marked vectors of the tiles that pass
-// (largest logit in a bin >= bin) are listed, then one thread per listed vector reads it back and
-// appends its candidates.  (Inlined into the kernel so that the compiler sees sm in the shared
-// address space: atomics through a generic pointer to shared memory are several times slower.)
-template <typename T, int NT>
-__device__ __forceinline__ int candidates_from_tiles(const SparsifyParams& p, int row, const uint2* ent, int n_tiles, int bin,
-                                                     float z0, SmallSharedFor<NT>* sm, int tid) {
-    constexpr int kPer = Elt<T>::kPerVec;
-    constexpr uint32_t kVecMask = (1u << kTileMaskShift) - 1u;
-    const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
-    const RowExtent ext = row_extent<T>(p.V);
-    const uint32_t min_key = (uint32_t)bin << kHistShift;
-    const int lane = tid & 31;
-    if (tid == 0) {
-        sm->n_pass = 0;
-        sm->n_cand = 0;
-    }
-    small_sync<NT>();
-    // ---- the marked vectors of the passing tiles, as a list ------------------------------------------
-    for (int base = 0; base < n_tiles; base += 8 * NT) {
-        uint32_t m = 0;  // which of this thread's eight entries pass
-        int cnt = 0;     // marked vectors in them
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = base + u * NT + tid;
-            const uint2 e = i < n_tiles ? __ldcg(&ent[i]) : make_uint2(0u, 0u);  // key 0 never passes
-            if (e.y >= min_key) {
-                m |= 1u << u;
-                cnt += __popc(e.x >> kTileMaskShift);
-            }
-        }
-        int pos = warp_reserve(&sm->n_pass, cnt, lane);
-        while (m) {  // few: read them again (cached) rather than keep eight entries in registers
-            const int u = __ffs(m) - 1;
-            m &= m - 1;
-            const uint32_t w = __ldcg(&ent[base + u * NT + tid].x);
-#pragma unroll
-            for (int j = 0; j < kVecsPerLane; ++j) {
-                if ((w >> (kTileMaskShift + j)) & 1u) {
-                    if (pos < small_pass_cap(NT)) sm->pass[pos] = (w & kVecMask) + 32u * j;
-                    ++pos;
-                }
-            }
-        }
-    }
-    small_sync<NT>();
-    const int nvec = sm->n_pass;
-    if (nvec <= small_pass_cap(NT)) {
-        // ---- one thread per listed vector: read it back, append its candidates ----------------------
-        constexpr int kInFlight = 2;
-        static_assert(kInFlight * kPer <= 32, "one mask bit per logit a thread holds");
-        for (int base = 0; base < nvec; base += kInFlight * NT) {
-            float z[kInFlight][kPer];
-            int vi[kInFlight];
-#pragma unroll
-            for (int u = 0; u < kInFlight; ++u) {
-                const int i = base + u * NT + tid;
-                vi[u] = i < nvec ? (int)sm->pass[i] : -1;
-                if (vi[u] >= 0) {
-                    load_row_vector<T>(rowp, vi[u], ext, p.V, z[u]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e) z[u][e] = -INFINITY;
-                }
-            }
-            uint32_t m = 0;
-#pragma unroll
-            for (int u = 0; u < kInFlight; ++u)
-#pragma unroll
-                for (int e = 0; e < kPer; ++e)
-                    if (z[u][e] >= -3.4028234e38f && rel_key(z[u][e], z0) >= min_key) m |= 1u << (u * kPer + e);
-            int pos = warp_reserve(&sm->n_cand, __popc(m), lane);
-#pragma unroll
-            for (int u = 0; u < kInFlight; ++u)
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) {
-                    if ((m >> (u * kPer + e)) & 1u) {
-                        if (pos < small_list_cap(NT))
-                            sm->comp[pos] = ((unsigned long long)float_to_key(z[u][e]) << 32) |
-                                            (unsigned long long)(0xffffffffu - (uint32_t)(vi[u] * kPer + e));
-                        ++pos;
-                    }
-                }
-        }
-        small_sync<NT>();
-        if (sm->n_cand <= small_list_cap(NT)) return sm->n_cand;
-    }
-    return winners_one_by_one<T, NT>(p, row, ent, n_tiles, bin, z0, nvec <= small_pass_cap(NT) ? nvec : -1, sm, tid);
-}
-
-constexpr int small_resident(int nt) { return nt == 64 ? 24 : nt == 96 ? 16 : nt == 128 ? 12 : 6; }
-
-template <typename T, int NT>
-__global__ void __launch_bounds__(NT, small_resident(NT)) sparsify_finish_small_kernel(const SparsifyParams p) {
-    constexpr int kHeld = (small_cand_cap(NT) + NT - 1) / NT;  // candidates a thread holds in registers
-    __shared__ SmallSharedFor<NT> sm;
-    const int tid = threadIdx.x, row = blockIdx.x, k = p.k;
-    float u_raw = 0.f;
-    if (tid < p.num_samples) u_raw = p.uniforms[(size_t)row * p.num_samples + tid];  // an input: may be read early
-    // Nothing the streaming kernel wrote is read before this point.  The row's own ready flag is
-    // enough to go on (see poll_row_ready); if it does not come, the end of the streaming kernel is.
-    if (tid == 0) sm.n_cut = poll_row_ready(&p.row_ready[row]) ? 1 : 0;
-    small_sync<NT>();
-    if (!sm.n_cut) wait_for_primary_kernel();
-    small_sync<NT>();
-    if (row == 0 && tid == 0) *p.status = 0;
-    // ---- one trip to memory: the candidates, their count, the per-warp statistics, the uniforms' line
-    const SegStat* st = &p.seg_stats[row];
-    const uint2* ent = p.seg_entries + (size_t)row * p.seg_stride;
-    unsigned long long held[kHeld];  // key << 32 | ~index
-#pragma unroll
-    for (int c = 0; c < kHeld; ++c) {
-        const int i = tid + c * NT;
-        const uint2 e = i < p.seg_cap ? __ldcg(&ent[i]) : make_uint2(0u, 0u);
-        held[c] = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
-    }
-    int nc = __ldcg(&st->n);
-    const int raw_bin = __ldcg(&st->raw_bin);
-    // the log-normaliser once, by one warp (fp64 is scarce): one per-warp pair per lane
-    if (tid < 32) {
-        const double Sw = tid < kWarps ? __ldcg(&st->S[tid]) : 0.0;
-        const double Mw = tid < kWarps ? (double)__ldcg(&st->M[tid]) : -INFINITY;
-        const double Mrow = warp_max(Sw > 0.0 ? Mw : -INFINITY);
-        const double Srow = warp_sum(Sw > 0.0 ? Sw * exp2(Mw - Mrow) : 0.0);
-        if (tid == 0) sm.lrow = Mrow + log2(Srow);
-    }
-    if (raw_bin >= 0) {  // the entries are staged lane tiles: make the candidates from them first
-        nc = candidates_from_tiles<T, NT>(p, row, ent, nc, raw_bin, __ldcg(&st->z0), &sm, tid);
-#pragma unroll
-        for (int c = 0; c < kHeld; ++c) {
-            const int i = tid + c * NT;
-            held[c] = i < nc ? sm.comp[i] : 0ull;
-        }
-    } else {
-        nc = nc < 0 ? 0 : (nc > small_cand_cap(NT) ? small_cand_cap(NT) : nc);
-#pragma unroll
-        for (int c = 0; c < kHeld; ++c) {
-            const int i = tid + c * NT;
-            if (i < nc) sm.comp[i] = held[c];
-        }
-    }
-    small_sync<NT>();
-    // ---- exact top-k by counting ranks under (key descending, index ascending) -------------------
-    // (only the threads that hold a candidate count; the 64-bit composite makes it one compare per entry)
-#pragma unroll
-    for (int c = 0; c < kHeld; ++c) {
-        if (tid + c * NT < nc) {
-            const unsigned long long mine = held[c];
-            int r = 0;
-            for (int j = 0; j < nc; ++j) r += sm.comp[j] > mine ? 1 : 0;
-            if (r < k) {
-                sm.wkey[r] = (uint32_t)(mine >> 32);
-                sm.widx[r] = (int)(0xffffffffu - (uint32_t)mine);
-            }
-        }
-    }
-    for (int i = kHeld * NT + tid; i < nc; i += NT) {  // a long list made from tiles: the rest of it
-        const unsigned long long mine = sm.comp[i];
-        int r = 0;
-        for (int j = 0; j < nc; ++j) r += sm.comp[j] > mine ? 1 : 0;
-        if (r < k) {
-            sm.wkey[r] = (uint32_t)(mine >> 32);
-            sm.widx[r] = (int)(0xffffffffu - (uint32_t)mine);
-        }
-    }
-    small_sync<NT>();
-    const int n0 = nc < k ? nc : k;
-    const double L2 = sm.lrow;  // written before the barriers above
-    const double cd = p.c.d;
-    // ---- nucleus cut on the cumulative q in that order ---------------------------------------------
-    int n = n0;
-    double mass = 0.0;
-    {
-        double q = 0.0;
-        if (tid < n0) q = exp2((double)key_to_float(sm.wkey[tid]) * cd - L2);
-        double tot;
-        const double c_incl = small_scan<NT>(q, tid, sm.red, &tot);
-        if (p.top_p < 1.0f) {
-            if (tid == 0) sm.n_cut = n0;
-            if (tid < n0) sm.cum[tid] = c_incl;
-            small_sync<NT>();
-            const double tp = (double)p.top_p;
-            // first crossing of the cumulative: exactly one thread, if any
-            if (tid < n0 && c_incl >= tp && (tid == 0 || sm.cum[tid - 1] < tp)) sm.n_cut = tid + 1;
-            small_sync<NT>();
-            n = sm.n_cut;
-            mass = n > 0 ? sm.cum[n - 1] : 0.0;
-            small_sync<NT>();
-        } else {
-            mass = tot;
-        }
-    }
-    // ---- ascending index order -----------------------------------------------------------------------
-    if (tid < n) {
-        const int mine = sm.widx[tid];
-        int r = 0;
-        for (int j = 0; j < n; ++j) r += sm.widx[j] < mine ? 1 : 0;
-        sm.oidx[r] = mine;
-        sm.okey[r] = sm.wkey[tid];
-    }
-    small_sync<NT>();
-    // ---- renormalised truncated distribution and its CDF in fp64 -------------------------------------
-    double y = -INFINITY;
-    if (tid < n) y = (double)key_to_float(sm.okey[tid]) * cd;
-    const double mS = small_max<NT>(y, tid, sm.red);
-    const double w = tid < n ? exp2(y - mS) : 0.0;
-    double W;
-    const double cw = small_scan<NT>(w, tid, sm.red, &W);
-    if (tid < n) { sm.cum[tid] = cw; sm.wv[tid] = w; }
-    small_sync<NT>();
-    // ---- outputs ----------------------------------------------------------------------------------------
-    int* o_idx = p.idx + (size_t)row * k;
-    float* o_logit = p.logit + (size_t)row * k;
-    if (tid < k) {
-        o_idx[tid] = tid < n ? sm.oidx[tid] : -1;
-        o_logit[tid] = tid < n ? key_to_float(sm.okey[tid]) : -INFINITY;
-    }
-    if (tid == 0) {
-        p.count[row] = n;
-        if (p.lse) p.lse[row] = n0 > 0 ? (float)(L2 * 0.6931471805599453) : -INFINITY;
-        if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
-    }
-    for (int sidx = tid; sidx < p.num_samples; sidx += NT) {
-        int tok = -1;
-        if (n > 0) {
-            const float u = clamp_uniform(sidx == tid ? u_raw : p.uniforms[(size_t)row * p.num_samples + sidx]);
-            int pos = first_greater(sm.cum, n, (double)u * W);
-            if (pos >= n) {
-                pos = n - 1;
-                while (pos > 0 && !(sm.wv[pos] > 0.0)) --pos;
-            }
-            tok = sm.oidx[pos];
-        }
-        p.token[(size_t)row * p.num_samples + sidx] = tok;
-    }
-    // This kernel's completion must imply the streaming kernel's (what follows on the stream relies
-    // on it): one CTA sees to that; the others leave and make room.
+    // this kernel's completion must imply the streaming kernel's (what follows on the stream relies
+    // on it): one CTA sees to that; the others leave and make room
     if (row == 0) wait_for_primary_kernel();
 }
 
-// The small finish kernel for this k: a warp's worth of threads per 32 of k, at least two warps.
-template <typename T> static void (*small_finish_kernel(int k, int* threads))(const SparsifyParams) {
-    if (k <= 64) { *threads = 64; return sparsify_finish_small_kernel<T, 64>; }
-    if (k <= 96) { *threads = 96; return sparsify_finish_small_kernel<T, 96>; }
-    if (k <= 128) { *threads = 128; return sparsify_finish_small_kernel<T, 128>; }
-    *threads = 256;
-    return sparsify_finish_small_kernel<T, 256>;
-}
+}  // namespace tslt
 
 // ---- host side -------------------------------------------------------------------------------
+namespace tslt {
 
 struct SparsifyPlan {
-    int nchunks, cap, high, fin_cap, vcap, vhigh, seg_cap, seg_stride, raw_cap;
-    bool small_finish;
+    int nchunks, group_log2, ngroups, tile_cap;
     RowSplit split;
-    size_t smem;
-    size_t ws_stats_off, ws_entries_off, ws_ready_off, ws_bytes;
+    size_t fin_smem;
+    size_t ws_ready_off, ws_stats_off, ws_tiles_off, ws_bytes;
 };
 
 static int sm_count_cached() {
@@ -1540,66 +716,45 @@ static int sm_count_cached() {
     return sms;
 }
 
-constexpr int kSmemPerSm = 227 * 1024;
-
 static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     SparsifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
     pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
-    pl.cap = 16 * k;
-    if (pl.cap < 1024) pl.cap = 1024;
-    if (pl.cap > 4096) pl.cap = 4096;
-    // k <= 256: the staged tiles normally go to the finish kernel unexpanded, so the staging buffer
-    // is sized never to fill on ordinary rows (about 8 k tiles are staged) and the candidate list,
-    // used only when it does, is kept small: four CTAs still fit an SM
-    if (k <= kSmallMaxThreads) pl.cap = 1024;
-    pl.high = pl.cap - pl.cap / 4;
-    // (large k stages thousands of tiles per row: a buffer that holds most of them saves the early
-    // expansions, each a rendezvous of the warps and a round of reads back)
-    pl.vcap = k <= 64 ? 1024 : k <= 256 ? 2048 : 4096;
-    pl.vhigh = pl.vcap - pl.vcap / 4;
-    pl.seg_cap = 2 * k;  // what one segment of a split row hands over (its k-th bin and above); see below
-    pl.smem = sparsify_smem_bytes(pl.cap, pl.vcap, k);
-    // CTAs the machine holds at once: launch bounds and the shared-memory footprint decide
-    int per_sm = (int)(kSmemPerSm / (pl.smem + 1024));
-    if (per_sm > kSparsifyCtasPerSm) per_sm = kSparsifyCtasPerSm;
-    if (per_sm < 1) per_sm = 1;
-    // a split row's segments must fit the candidate list of the CTA that merges them
-    const int max_seg = pl.cap / pl.seg_cap < 16 ? pl.cap / pl.seg_cap : 16;
-    // One CTA per row.  Only when there are fewer rows than half the SMs and the rows are long is a
-    // row cut into segments (of at least 32 chunks): every segment pays the first threshold and the
-    // hand-over, which on small batches (tens of rows) costs more than it gains.
-    (void)per_sm;
-    pl.split.rows = rows;
+    const long long ntiles = (long long)pl.nchunks * kTilesPerChunk;
+    // tiles per group: the largest power of two that still leaves 2 k groups (the k-th largest group
+    // maximum is then a selective bound), and no more groups than the finish kernel holds
+    int glog = 0;
+    while ((ntiles >> (glog + 1)) >= 2LL * k) ++glog;
+    while (((ntiles + (1LL << glog) - 1) >> glog) > kMaxGroups) ++glog;
+    pl.group_log2 = glog;
+    pl.ngroups = (int)((ntiles + (1LL << glog) - 1) >> glog);
+    pl.tile_cap = 8 * k < 512 ? 512 : (8 * k > kMaxTileList ? kMaxTileList : 8 * k);
+    pl.fin_smem = sparsify_finish_smem(pl.ngroups, pl.tile_cap, k);
+    // One CTA per row when the rows fill the machine; fewer rows are cut into segments (at least one
+    // chunk per warp each) so that every CTA slot has work.  A segment costs nothing but its own
+    // hand-over (8 (max, sum) pairs and a flag).
+    const int slots = kSparsifyStreamCtasPerSm * sm_count_cached();
     int nseg = 1;
-    if (rows > 0 && 2 * rows < sm_count_cached()) {
-        nseg = sm_count_cached() / rows;
-        if (nseg > pl.nchunks / 32) nseg = pl.nchunks / 32;
-        if (nseg > max_seg) nseg = max_seg;
+    if (rows > 0 && rows < slots) {
+        nseg = (slots + rows - 1) / rows;
+        const int by_len = pl.nchunks / kWarps;
+        if (nseg > by_len) nseg = by_len;
+        if (nseg > 64) nseg = 64;
         if (nseg < 1) nseg = 1;
     }
     int cps = (pl.nchunks + nseg - 1) / nseg;
-    cps = (cps + kWarps - 1) / kWarps * kWarps;
-    if (cps < kWarps) cps = kWarps;
-    pl.split.nseg = (pl.nchunks + cps - 1) / cps;
-    if (pl.split.nseg < 1) pl.split.nseg = 1;
+    if (cps < 1) cps = 1;
+    pl.split.rows = rows;
     pl.split.cps = cps;
+    pl.split.nseg = (pl.nchunks + cps - 1) / cps;
     pl.split.grid = rows * pl.split.nseg;
-    // the generic finish kernel holds what the row's segments hand over, no more: it fits more CTAs per SM
-    pl.fin_cap = pl.split.nseg * pl.seg_cap;
-    if (pl.fin_cap < 1024) pl.fin_cap = 1024;
-    // rows of one segment with k <= 256 go to the small finish kernel, and hand their staged tiles over raw
-    pl.small_finish = pl.split.nseg == 1 && k <= kSmallMaxThreads;  // (seg_cap = 2 k fits small_cand_cap)
-    pl.raw_cap = pl.small_finish ? pl.vcap : 0;
-    pl.seg_stride = pl.seg_cap > pl.raw_cap ? pl.seg_cap : pl.raw_cap;
-    const size_t split_rows = (size_t)rows;
     size_t off = kWsHeaderBytes;
-    pl.ws_stats_off = off;
-    off = align_up(off + split_rows * pl.split.nseg * sizeof(SegStat), 256);
-    pl.ws_entries_off = off;
-    off = align_up(off + split_rows * pl.split.nseg * pl.seg_stride * sizeof(uint2), 256);
     pl.ws_ready_off = off;
-    if (pl.split.nseg == 1) off = align_up(off + split_rows * sizeof(int), 256);
+    off = align_up256(off + (size_t)rows * pl.split.nseg * sizeof(int));
+    pl.ws_stats_off = off;
+    off = align_up256(off + (size_t)rows * pl.split.nseg * sizeof(SegStat));
+    pl.ws_tiles_off = off;
+    off = align_up256(off + (size_t)rows * (size_t)ntiles * sizeof(unsigned short));
     pl.ws_bytes = off;
     return pl;
 }
@@ -1612,6 +767,9 @@ ScaleC make_scale(float temperature) {
     return s;
 }
 
+// Polls of a ready flag before a finish CTA gives up on it (about a second at 200 ns per poll).
+static int g_sparsify_poll_limit = kReadyPollLimit;
+
 }  // namespace tslt
 
 using namespace tslt;
@@ -1621,6 +779,12 @@ extern "C" int tslt_sparsify_workspace_bytes(int rows, int V, int k, int num_sam
         return TSLT_ERR_INVALID_ARG;
     SparsifyPlan a = make_sparsify_plan(rows, V, k, 2), b = make_sparsify_plan(rows, V, k, 4);
     *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
+    return TSLT_OK;
+}
+
+extern "C" int tslt_set_ready_poll_limit(int polls) {
+    if (polls < 0) return TSLT_ERR_INVALID_ARG;
+    g_sparsify_poll_limit = polls;
     return TSLT_OK;
 }
 
@@ -1636,7 +800,8 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
         return TSLT_ERR_INVALID_ARG;
     if (k > TSLT_MAX_K) return TSLT_ERR_UNSUPPORTED;
     const long long rows_ll = (long long)B * gamma;
-    if (rows_ll > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    if (rows_ll > 0x7fffffffLL / 64) return TSLT_ERR_UNSUPPORTED;
+    if ((long long)V * eb > (1LL << 30)) return TSLT_ERR_UNSUPPORTED;  // tile and vector numbers stay well inside 32 bits
     const int rows = (int)rows_ll;
     if (rows == 0) return TSLT_OK;
     if (!logits || !idx || !logit || !count || !workspace || (num_samples > 0 && (!uniforms || !token)))
@@ -1657,34 +822,21 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.uniforms = uniforms;
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
     p.nchunks = pl.nchunks; p.split = pl.split;
-    p.cap = pl.cap; p.high = pl.high; p.fin_cap = pl.fin_cap; p.vcap = pl.vcap; p.vhigh = pl.vhigh; p.seg_cap = pl.seg_cap;
-    p.seg_stride = pl.seg_stride; p.raw_cap = pl.raw_cap;
-    p.idx_hi_byte = (V - 1) >= (1 << 24) ? 3 : (V - 1) >= (1 << 16) ? 2 : (V - 1) >= (1 << 8) ? 1 : 0;
+    p.group_log2 = pl.group_log2; p.ngroups = pl.ngroups; p.tile_cap = pl.tile_cap;
+    p.poll_limit = g_sparsify_poll_limit;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
+    p.seg_ready = (int*)(ws + pl.ws_ready_off);
     p.seg_stats = (SegStat*)(ws + pl.ws_stats_off);
-    p.seg_entries = (uint2*)(ws + pl.ws_entries_off);
-    p.row_ready = pl.split.nseg == 1 ? (int*)(ws + pl.ws_ready_off) : nullptr;  // rows of one segment only
+    p.tile_max = (unsigned short*)(ws + pl.ws_tiles_off);
 
     cudaStream_t st = (cudaStream_t)stream;
-    auto kern = dtype == TSLT_F32 ? sparsify_kernel<float> : sparsify_kernel<bf16_t>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sparsify_smem_bytes(4096, kMaxStagedTiles, TSLT_MAX_K)) != cudaSuccess)
-        return TSLT_ERR_CUDA;
-    kern<<<pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
+    if (dtype == TSLT_F32) sparsify_stream_kernel<float><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
+    else sparsify_stream_kernel<bf16_t><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
-    if (pl.small_finish) {
-        int threads = 0;
-        auto fin = dtype == TSLT_F32 ? small_finish_kernel<float>(k, &threads) : small_finish_kernel<bf16_t>(k, &threads);
-        if (launch_dependent(fin, rows, threads, 0, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
-    } else {
-        auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
-        if (cudaFuncSetAttribute(fin, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)sparsify_smem_bytes(4096, 0, TSLT_MAX_K)) != cudaSuccess)
-            return TSLT_ERR_CUDA;
-        if (launch_dependent(fin, rows, kBlockThreads, sparsify_smem_bytes(pl.fin_cap, 0, k), st, p) != cudaSuccess)
-            return TSLT_ERR_CUDA;
-    }
-    if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+    auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
+    static_assert(kFinishHeaderBytes + kSelBins * 4 + kMaxGroups * 4 + TSLT_MAX_K * 16 + TSLT_MAX_K * 8 <= 48 * 1024,
+                  "the finish kernel's shared memory stays under the default limit");
+    if (launch_dependent(fin, rows, kFinishThreads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }

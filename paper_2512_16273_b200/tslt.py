@@ -8,7 +8,6 @@ built library, or calling it with CPU tensors, raises.
 from __future__ import annotations
 
 import ctypes
-import math
 import os
 from typing import Dict, Optional, Sequence
 
@@ -24,7 +23,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 F32, BF16 = 0, 1
 MAX_K = 1024
 
-EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status",
+EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status", "tslt_set_ready_poll_limit",
            "tslt_sparsify_workspace_bytes", "tslt_sparsify",
            "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
@@ -59,6 +58,8 @@ def lib() -> ctypes.CDLL:
     L.tslt_status_string.argtypes = [i]
     L.tslt_workspace_status.restype = i
     L.tslt_workspace_status.argtypes = [p, p, ctypes.POINTER(i)]
+    L.tslt_set_ready_poll_limit.restype = i
+    L.tslt_set_ready_poll_limit.argtypes = [i]
     L.tslt_sparsify_workspace_bytes.restype = i
     L.tslt_sparsify_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_sparsify.restype = i
@@ -188,6 +189,15 @@ def workspace_status(ws: torch.Tensor) -> int:
     if rc not in (OK, ERR_DEVICE_STATUS):
         raise TsltError(rc, "tslt_workspace_status")
     return int(word.value)
+
+
+STATUS_WAIT_FELL_BACK = 1
+
+
+def set_ready_poll_limit(polls: int) -> None:
+    """Process-wide: polls a finish CTA of tslt_sparsify spends on its row's ready flags before it
+    takes the fall-back (and sets STATUS_WAIT_FELL_BACK in the status word).  0: at once."""
+    _check(lib().tslt_set_ready_poll_limit(int(polls)), "tslt_set_ready_poll_limit")
 
 
 def sparsify(logits: torch.Tensor, k: int, top_p: float = 1.0, temperature: float = 1.0,
@@ -353,12 +363,6 @@ def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_r
     _check(rc, "tslt_tree_verify")
     o["workspace"] = ws
     return o
-
-
-def payload_bits(count: int, V: int, b_prob: int = 32) -> int:
-    """Uplink payload of one sparse distribution, the per-distribution data volume of Section
-    2.2 with the vocabulary size replaced by the retained count: count * (b_prob + ceil(log2 V))."""
-    return int(count) * (int(b_prob) + math.ceil(math.log2(V)))
 
 
 def payload_words(k: int, V: int, prob_format: int):

@@ -112,5 +112,6 @@ def test_payload_accounting_matches_paper_formula():
     """Section 2.2: one distribution costs |V| (b_prob + b_idx) bits with b_idx = ceil(log2 |V|);
     the sparse payload replaces |V| by the retained count."""
     from paper_2512_16273_b200 import tslt
-    assert tslt.payload_bits(32000, 32000, 16) == 32000 * (16 + 15)
-    assert tslt.payload_bits(320, 32000, 16) == 9920
+    words, entry_bits = tslt.payload_words(320, 32000, tslt.PROB_F16)   # host-only query of the C ABI
+    assert entry_bits == 16 + 15 and 320 * entry_bits == 9920
+    assert words == 1 + (320 * entry_bits + 31) // 32
