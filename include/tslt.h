@@ -18,19 +18,24 @@
  *     pointer must be 16-byte aligned and row_stride_elems * sizeof(element) must be a
  *     multiple of 16.  -inf logits are legal (probability 0, never selected).  NaN / +inf
  *     logits give unspecified values but never an out-of-bounds access or a hang.  While a
- *     row streams, the exponent z / T is carried in fp32 relative to a reference exponent,
- *     itself fp32: offsets cancel, but once |z / T| passes about 2^30 the reference is so
- *     coarse that the running sum can overflow; the selection is still exact there, the
- *     normaliser (lse, mass, and through them the sampled token) is not.
+ *     row streams, the exponent z * c (c = log2(e) / T rounded to fp32) is carried in fp32
+ *     relative to a reference exponent; every probability that is later formed against the
+ *     row's normaliser uses the same rounded c, so a common offset of the logits cancels and
+ *     what is left of the rounding (2^-25 relative on c) acts on z minus the row's mean only.
+ *     The fp32 product z * c itself is good to 2^-24 relative: lse, mass and the acceptance
+ *     probabilities keep their 1e-5 accuracy while |z / T| stays below a few hundred; the
+ *     selection (which compares stored logits) is exact whatever their size.
  *   - uniforms are fp32 in [0,1); a value >= 1 is read as the largest float below 1.
  *   - "sample" always means inverse CDF in ascending token index: the first index whose
  *     cumulative mass exceeds u * total.
- *   - CTAs that share a row or a sequence meet through a ticket counter in the workspace and
- *     the last one to arrive carries on; the one wait on another CTA (a row's finish CTA on the
- *     row's streaming CTA in tslt_sparsify) is one-way, bounded, and falls back to the
- *     end of the streaming kernel.  The first word
- *     of the workspace is a device status word (0 = fine) that tslt_workspace_status reads
- *     back; a non-zero word is reported as TSLT_ERR_DEVICE_STATUS.
+ *   - kernels of one call hand work over at kernel boundaries; where CTAs of one kernel share a
+ *     row (tslt_tree_verify_walk) they meet through a ticket counter in the workspace and the
+ *     last one to arrive carries on.  The one wait on another CTA (a row's finish CTA on the
+ *     row's streaming CTAs in tslt_sparsify) is one-way and bounded: when it runs out, the CTA
+ *     sets TSLT_STATUS_WAIT_FELL_BACK in the status word and waits for the end of the streaming
+ *     kernel instead; the results are the same.  The first word of the workspace is that device
+ *     status word (0 = nothing to report; every call's first kernel clears it), which
+ *     tslt_workspace_status reads back; a non-zero word is reported as TSLT_ERR_DEVICE_STATUS.
  */
 #ifndef TSLT_H_
 #define TSLT_H_
@@ -194,6 +199,28 @@ int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
                      float target_temperature, const float* u_accept, const float* u_sample,
                      int max_depth, int* accepted_path, int* accepted_len, int* out_token,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same verification by a root-to-leaf PATH WALK (the "new sequence searching" loop that ends
+ * Algorithm 8; Section 4.2): the search only ever uses the nodes on one path, and the uniforms
+ * are indexed by node, so verifying just the node each sequence's walk has reached gives the
+ * outputs of tslt_tree_verify exactly, while reading at most depth + 1 of the N target rows of a
+ * sequence.  One launch per tree level on the caller's stream: the rows of the current nodes are
+ * streamed, Algorithm 5 runs at each of them, the walks move to the accepted children; a
+ * sequence whose walk has stopped costs nothing in later levels.  Arguments, results and rules
+ * are those of tslt_tree_verify; the workspace is smaller (chunk partials of B rows, not B * N)
+ * and has its own size query.  Use it when latency or bytes read matter (the rows it skips are
+ * never touched); tslt_tree_verify, one streaming pass over all B * N rows, is the form the
+ * paper's "in parallel" node loop describes.
+ */
+int tslt_tree_verify_walk_workspace_bytes(int B, int N, int V, int k, size_t* bytes);
+int tslt_tree_verify_walk(const void* target_logits, int dtype, int B, int N, int V,
+                          long long row_stride_elems, const int* parent, const int* node_draft_row,
+                          int M, int k, const int* node_token, const int* draft_idx,
+                          const float* draft_logit, const int* draft_count, float draft_temperature,
+                          float target_temperature, const float* u_accept, const float* u_sample,
+                          int max_depth, int* accepted_path, int* accepted_len, int* out_token,
+                          void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Uplink payload (Section 2.2: a transmitted distribution costs entries * (b_prob + b_idx) bits,

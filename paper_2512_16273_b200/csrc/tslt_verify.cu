@@ -1,16 +1,20 @@
-// tslt_verify / tslt_tree_verify: verifier-side speculative sampling against a sparse draft
-// (Algorithm 3; Algorithm 5 along the walk of Algorithm 8) as one kernel each.
+// tslt_verify / tslt_tree_verify / tslt_tree_verify_walk: verifier-side speculative sampling
+// against a sparse draft (Algorithm 3; Algorithm 5 along the walk of Algorithm 8).
 //
-// Every target row is read from HBM exactly once, with 16-byte loads that go straight to
-// registers (each warp instruction covers 512 contiguous bytes); warps run freely, one 2 KB
-// chunk per step.  The streaming pass keeps nothing but one (max, sum) pair per chunk of the
-// row, written to the workspace.  The CTA that finishes a sequence's last segment (found with a ticket
-// counter, no waiting) resolves the sequence: it turns the chunk partials into each row's
+// Every target row that is looked at is read from HBM exactly once, with 16-byte loads that go
+// straight to registers (each warp instruction covers 512 contiguous bytes); warps run freely, one
+// 2 KB chunk per step.  The streaming pass keeps nothing but one (max, sum) pair per chunk of the
+// row, written to the workspace.  A resolve step then turns the chunk partials into each row's
 // log-normaliser, rebuilds the sparse q~ in fp64, runs the acceptance tests, and samples the
 // correction token from the full-vocabulary residual.  Because q~ is sparse, the residual is
 // a multiple of p outside the draft set S and explicit values on S, so its CDF is the chunk
 // partials corrected by at most k entries; only the one chunk that holds the sampled token is
 // read a second time.
+//   tslt_verify, tslt_tree_verify: a streaming kernel over all rows, then (programmatic dependent
+//     launch) a resolve kernel with one CTA per sequence.
+//   tslt_tree_verify_walk: one launch per tree level; only the row of the node each sequence's
+//     walk has reached is streamed, and the CTA that completes it (a ticket counter, no waiting)
+//     runs Algorithm 5 at that node and moves the walk on.
 #include <math.h>
 
 #include <mutex>
@@ -51,8 +55,14 @@ struct VerifyParams {
     int* accepted_path;
     // workspace
     int* status;
-    int* tickets;
-    float2* partials;  // [B * rows_per_seq, nchunks]
+    int* tickets;      // path walk only: [levels, B]
+    float2* partials;  // [B * rows_per_seq, nchunks]; path walk: [B, nchunks], the row each walk is at
+    struct WalkState* walk;  // path walk only: [B]
+};
+
+// Where a sequence's walk stands between two levels of tslt_tree_verify_walk.
+struct WalkState {
+    int node, len, done, pad;
 };
 
 struct VerifyShared {
@@ -109,12 +119,15 @@ __device__ __forceinline__ double row_log2_norm(const float2* part, int nchunks,
     return s > 0.0 ? mx + log2(s) : -INFINITY;
 }
 
+// p(v) of a streamed row.  cs is the scale AS THE STREAMING PASS USED IT (the fp32 rounding of
+// log2(e) / T, widened): the row's log-normaliser L2 was accumulated with it, and only the same
+// scale in the numerator makes a common offset of the logits cancel exactly.
 template <typename T>
-__device__ __forceinline__ double token_prob(const unsigned char* rowp, int v, int V, double cd, double L2) {
+__device__ __forceinline__ double token_prob(const unsigned char* rowp, int v, int V, double cs, double L2) {
     if (v < 0 || v >= V || !(L2 > -INFINITY)) return 0.0;
     const float z = Elt<T>::load(rowp, v);
     if (!(fabsf(z) <= 3.4028234e38f)) return 0.0;  // non-finite logit: probability 0
-    return exp2((double)z * cd - L2);
+    return exp2((double)z * cs - L2);
 }
 
 // Rebuild q~ from the transmitted pairs of one draft row into s_idx / s_q; returns n.
@@ -204,7 +217,7 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
     // second touch of one chunk: exact weights of its elements
     const int v0 = c * kChunkElems;
     const int ne = min(kChunkElems, p.V - v0);
-    for (int e = tid; e < ne; e += kBlockThreads) A.r[e] = c_out * token_prob<T>(rowp, v0 + e, p.V, p.cp.d, L2);
+    for (int e = tid; e < ne; e += kBlockThreads) A.r[e] = c_out * token_prob<T>(rowp, v0 + e, p.V, (double)p.cp.f, L2);
     consumer_sync();
     for (int i = tid; i < n; i += kBlockThreads) {
         const int v = A.s_idx[i];
@@ -280,11 +293,11 @@ __device__ __forceinline__ double position_accept_prob(const VerifyParams& p, si
         for (int i = lane; i < n; i += 32) {
             const float l = dl[i];
             const double e = fabsf(l) <= 3.4028234e38f ? exp2((double)l * p.cq.d - mx) : 0.0;
-            bh += fmin(token_prob<T>(rowp, di[i], p.V, p.cp.d, L2), W > 0.0 ? e / W : 0.0);
+            bh += fmin(token_prob<T>(rowp, di[i], p.V, (double)p.cp.f, L2), W > 0.0 ? e / W : 0.0);
         }
         *beta_hat_out = warp_sum(bh);
     }
-    return accept_probability(token_prob<T>(rowp, x, p.V, p.cp.d, L2), qx);
+    return accept_probability(token_prob<T>(rowp, x, p.V, (double)p.cp.f, L2), qx);
 }
 
 template <typename T>
@@ -350,7 +363,7 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
     if (a < gamma) {
         n = load_draft(p, (size_t)b * gamma + a, A, tid, sh->scratch);
         for (int i = tid; i < n; i += kBlockThreads) {
-            const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2_stop);
+            const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, (double)p.cp.f, L2_stop);
             A.s_p[i] = pv;
             const double d = pv - A.s_q[i];
             A.s_a[i] = d > 0.0 ? d : 0.0;
@@ -366,91 +379,99 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
     }
 }
 
+// Algorithm 5 at one node of sequence b's walk (Algorithm 8): `part` holds the chunk partials of the
+// node's target row.  Returns the accepted child, where the walk goes on, or -1 if the walk stops
+// at this node, *tok_out then being the final token (a leaf's bonus token, or a sample of p^(k+1)).
 template <typename T>
-__device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* arena, VerifyShared* sh, int tid) {
-    const ResolverArrays A = carve(arena);
+__device__ int resolve_tree_node(const VerifyParams& p, int b, int node, const float2* part, const ResolverArrays& A,
+                                 VerifyShared* sh, int tid, int* tok_out) {
     const int N = p.N;
     const int* child_begin = p.tree_meta;
     const int* child_list = p.tree_meta + (N + 1);
     const int* node_draft_row = p.tree_meta + (N + 1) + (N - 1);
+    const size_t r = (size_t)b * N + node;
+    const unsigned char* rowp = p.logits + (long long)r * p.row_stride_bytes;
+    const double L2 = row_log2_norm(part, p.nchunks, tid, sh->scratch);
+    const int dr = node_draft_row[node];
+    const float u = p.u_sample[r];
+    if (dr < 0) {
+        *tok_out = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);  // leaf: bonus from its own row
+        return -1;
+    }
+    const int n = load_draft(p, (size_t)b * p.M + dr, A, tid, sh->scratch);
+    double ps = 0.0;
+    for (int i = tid; i < n; i += kBlockThreads) {
+        const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, (double)p.cp.f, L2);
+        A.s_p[i] = pv;
+        A.s_a[i] = pv;
+        ps += pv;
+    }
+    const double PS = block_sum(ps, tid, sh->scratch);
+    const double out_mass = 1.0 - PS > 0.0 ? 1.0 - PS : 0.0;  // mass of p outside S
+    double c_out = 1.0;
+    for (int ci = child_begin[node]; ci < child_begin[node + 1]; ++ci) {
+        const int c = child_list[ci];
+        const int x = p.node_token[(size_t)b * N + c];
+        if (tid == 0) sh->slot_found = 0;
+        consumer_sync();
+        for (int i = tid; i < n; i += kBlockThreads)
+            if (A.s_idx[i] == x) {
+                sh->slot_a = A.s_a[i];
+                sh->slot_q = A.s_q[i];
+                sh->slot_found = 1;
+            }
+        consumer_sync();
+        double pa, qx;
+        if (sh->slot_found) {
+            pa = sh->slot_a;
+            qx = sh->slot_q;
+        } else {
+            pa = c_out * token_prob<T>(rowp, x, p.V, (double)p.cp.f, L2);
+            qx = 0.0;
+        }
+        const double ap = accept_probability(pa, qx);
+        const double rr = (double)clamp_uniform(p.u_accept[(size_t)b * N + c]);
+        if (rr < ap) {
+            consumer_sync();
+            return c;
+        }
+        // rejected: p^(i+1) = norm(max(0, p^(i) - q~)), on S explicitly, elsewhere by the scalar
+        double zs = 0.0;
+        for (int i = tid; i < n; i += kBlockThreads) {
+            const double d = A.s_a[i] - A.s_q[i];
+            zs += d > 0.0 ? d : 0.0;
+        }
+        const double Z = block_sum(zs, tid, sh->scratch) + c_out * out_mass;
+        if (Z > 0.0) {
+            for (int i = tid; i < n; i += kBlockThreads) {
+                const double d = A.s_a[i] - A.s_q[i];
+                A.s_a[i] = d > 0.0 ? d / Z : 0.0;
+            }
+            c_out /= Z;
+        }
+        consumer_sync();
+    }
+    int tok = sample_full_vocab<T>(p, rowp, part, L2, c_out, n, A, u, tid, sh);
+    if (tok < 0) tok = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);
+    *tok_out = tok;
+    return -1;
+}
+
+// The whole walk of one sequence when every node's row has been streamed (tslt_tree_verify).
+template <typename T>
+__device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* arena, VerifyShared* sh, int tid) {
+    const ResolverArrays A = carve(arena);
     int* path = p.accepted_path + (size_t)b * p.max_depth;
     for (int d = tid; d < p.max_depth; d += kBlockThreads) path[d] = -1;
     consumer_sync();
     int node = 0, len = 0, tok = -1;
     for (int depth = 0; depth <= p.max_depth; ++depth) {
-        const size_t r = (size_t)b * N + node;
-        const unsigned char* rowp = p.logits + (long long)r * p.row_stride_bytes;
-        const float2* part = p.partials + r * (size_t)p.nchunks;
-        const double L2 = row_log2_norm(part, p.nchunks, tid, sh->scratch);
-        const int dr = node_draft_row[node];
-        const float u = p.u_sample[r];
-        if (dr < 0) {
-            tok = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);  // leaf: bonus from its own row
-            break;
-        }
-        const int n = load_draft(p, (size_t)b * p.M + dr, A, tid, sh->scratch);
-        double ps = 0.0;
-        for (int i = tid; i < n; i += kBlockThreads) {
-            const double pv = token_prob<T>(rowp, A.s_idx[i], p.V, p.cp.d, L2);
-            A.s_p[i] = pv;
-            A.s_a[i] = pv;
-            ps += pv;
-        }
-        const double PS = block_sum(ps, tid, sh->scratch);
-        const double out_mass = 1.0 - PS > 0.0 ? 1.0 - PS : 0.0;  // mass of p outside S
-        double c_out = 1.0;
-        bool accepted = false;
-        for (int ci = child_begin[node]; ci < child_begin[node + 1]; ++ci) {
-            const int c = child_list[ci];
-            const int x = p.node_token[(size_t)b * N + c];
-            if (tid == 0) sh->slot_found = 0;
-            consumer_sync();
-            for (int i = tid; i < n; i += kBlockThreads)
-                if (A.s_idx[i] == x) {
-                    sh->slot_a = A.s_a[i];
-                    sh->slot_q = A.s_q[i];
-                    sh->slot_found = 1;
-                }
-            consumer_sync();
-            double pa, qx;
-            if (sh->slot_found) {
-                pa = sh->slot_a;
-                qx = sh->slot_q;
-            } else {
-                pa = c_out * token_prob<T>(rowp, x, p.V, p.cp.d, L2);
-                qx = 0.0;
-            }
-            const double ap = accept_probability(pa, qx);
-            const double rr = (double)clamp_uniform(p.u_accept[(size_t)b * N + c]);
-            if (rr < ap) {
-                if (len < p.max_depth && tid == 0) path[len] = c;
-                ++len;
-                node = c;
-                accepted = true;
-                consumer_sync();
-                break;
-            }
-            // rejected: p^(i+1) = norm(max(0, p^(i) - q~)), on S explicitly, elsewhere by the scalar
-            double zs = 0.0;
-            for (int i = tid; i < n; i += kBlockThreads) {
-                const double d = A.s_a[i] - A.s_q[i];
-                zs += d > 0.0 ? d : 0.0;
-            }
-            const double Z = block_sum(zs, tid, sh->scratch) + c_out * out_mass;
-            if (Z > 0.0) {
-                for (int i = tid; i < n; i += kBlockThreads) {
-                    const double d = A.s_a[i] - A.s_q[i];
-                    A.s_a[i] = d > 0.0 ? d / Z : 0.0;
-                }
-                c_out /= Z;
-            }
-            consumer_sync();
-        }
-        if (!accepted) {
-            tok = sample_full_vocab<T>(p, rowp, part, L2, c_out, n, A, u, tid, sh);
-            if (tok < 0) tok = sample_full_vocab<T>(p, rowp, part, L2, 1.0, 0, A, u, tid, sh);
-            break;
-        }
+        const float2* part = p.partials + ((size_t)b * p.N + node) * (size_t)p.nchunks;
+        const int next = resolve_tree_node<T>(p, b, node, part, A, sh, tid, &tok);
+        if (next < 0) break;
+        if (len < p.max_depth && tid == 0) path[len] = next;
+        ++len;
+        node = next;
     }
     if (tid == 0) {
         p.accepted_len[b] = len;
@@ -458,15 +479,14 @@ __device__ void resolve_tree(const VerifyParams& p, int b, unsigned char* arena,
     }
 }
 
-// Streaming pass over chunks [chunk_begin, chunk_end) of one row: (max, sum) of every chunk, the
-// chunk's own maximum as the reference exponent.
+// Streaming pass over chunks [chunk_begin, chunk_end) of the row at rowp: (max, sum) of every chunk,
+// the chunk's own maximum as the reference exponent, into part[chunk].
 template <typename T>
-__device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWork& wk, int lane, int warp) {
-    const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
+__device__ __forceinline__ void stream_chunks(const VerifyParams& p, const unsigned char* rowp, float2* part,
+                                              int chunk_begin, int chunk_end, int lane, int warp) {
     const RowExtent ext = row_extent<T>(p.V);
     const float c = p.cp.f;
-    float2* part = p.partials + (size_t)wk.row * p.nchunks;
-    for (int ch = wk.chunk_begin + warp; ch < wk.chunk_end; ch += kWarps) {
+    for (int ch = chunk_begin + warp; ch < chunk_end; ch += kWarps) {
         LaneTile<T> lt;
         lt.load(rowp, ch * kVecsPerChunk, lane, ext);
         const float wm = warp_max(lt.reduce_max());
@@ -479,62 +499,92 @@ __device__ __forceinline__ void stream_chunks(const VerifyParams& p, const RowWo
     }
 }
 
-// Small problems, one launch: stream, then the CTA that completes a sequence resolves it.
-template <typename T, bool kTree>
-__global__ void __launch_bounds__(kBlockThreads, 4) verify_kernel(const VerifyParams p) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
-    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
-    const int tid = threadIdx.x;
-    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
-    stream_chunks<T>(p, wk, tid & 31, tid >> 5);
-    // ---- ticket: the CTA that completes the sequence resolves it ---------------------------------
-    // (the barrier orders every warp's partials before thread 0's fence, which publishes them)
-    __syncthreads();
-    const int b = wk.row / p.rows_per_seq;
-    if (tid == 0) {
-        __threadfence();
-        sh->ticket = atomicAdd(&p.tickets[b], 1);
-    }
-    __syncthreads();
-    if (sh->ticket != p.rows_per_seq * p.split.nseg - 1) return;
-    __threadfence();
-    if (kTree) resolve_tree<T>(p, b, arena, sh, tid);
-    else resolve_sequence<T>(p, b, arena, sh, tid);
-}
+constexpr int kStreamCtasPerSm = 6;  // streaming-only kernel: 40 registers per thread, no shared memory
 
-constexpr int kStreamCtasPerSm = 6;  // streaming-only kernel: 42 registers per thread, no shared memory
-
-// Large problems, two launches on the stream: the streaming pass alone (no shared memory, no
-// ticket, no fence: the kernel boundary publishes the partials) ...
+// First launch: the streaming pass alone (no shared memory, no ticket, no fence: the kernel boundary
+// publishes the partials).  Block 0 clears the workspace's status word before it lets the resolve
+// kernel be scheduled, so the word never carries over from an earlier call.
 template <typename T>
 __global__ void __launch_bounds__(kBlockThreads, kStreamCtasPerSm) verify_stream_kernel(const VerifyParams p) {
+    if (blockIdx.x == 0) {
+        if (threadIdx.x == 0) {
+            *(volatile int*)p.status = 0;
+            __threadfence();
+        }
+        __syncthreads();
+    }
     allow_dependent_launch();
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
-    stream_chunks<T>(p, wk, threadIdx.x & 31, threadIdx.x >> 5);
+    stream_chunks<T>(p, p.logits + (long long)wk.row * p.row_stride_bytes, p.partials + (size_t)wk.row * p.nchunks,
+                     wk.chunk_begin, wk.chunk_end, threadIdx.x & 31, threadIdx.x >> 5);
 }
-// ... then one CTA per sequence resolves it.
+// Second launch: one CTA per sequence resolves it.
 template <typename T, bool kTree>
 __global__ void __launch_bounds__(kBlockThreads, 4) verify_resolve_kernel(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* arena = smem_raw;
+    unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
     VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
     wait_for_primary_kernel();  // the partials come from the streaming kernel
     if (kTree) resolve_tree<T>(p, blockIdx.x, arena, sh, threadIdx.x);
     else resolve_sequence<T>(p, blockIdx.x, arena, sh, threadIdx.x);
 }
 
+// One level of the path walk: every sequence whose walk is still going has the row of its current
+// node streamed by the CTAs of its segments; the CTA that completes the row (a ticket counter: the
+// last to arrive carries on, nobody waits) runs Algorithm 5 at the node and either moves the walk
+// to the accepted child or ends it with the final token.  Launched once per tree level, in stream
+// order; the walk state, zeroed on the stream before the first level, carries over in the workspace.
+template <typename T>
+__global__ void __launch_bounds__(kBlockThreads, 4) tree_walk_level_kernel(const VerifyParams p, int level) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* arena = smem_raw;
+    VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
+    const int tid = threadIdx.x;
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);  // "row" = sequence
+    const int b = wk.row;
+    WalkState* ws = p.walk + b;
+    if (__ldcg(&ws->done)) return;  // (the same for every thread of the CTA)
+    const int node = __ldcg(&ws->node), len = __ldcg(&ws->len);
+    float2* part = p.partials + (size_t)b * p.nchunks;
+    stream_chunks<T>(p, p.logits + (long long)((size_t)b * p.N + node) * p.row_stride_bytes, part, wk.chunk_begin,
+                     wk.chunk_end, tid & 31, tid >> 5);
+    // (the barrier orders every warp's partials before thread 0's fence, which publishes them)
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        sh->ticket = atomicAdd(&p.tickets[(size_t)level * p.B + b], 1);
+    }
+    __syncthreads();
+    if (sh->ticket != wk.nseg - 1) return;
+    __threadfence();
+    const ResolverArrays A = carve(arena);
+    int* path = p.accepted_path + (size_t)b * p.max_depth;
+    if (level == 0)
+        for (int d = tid; d < p.max_depth; d += kBlockThreads) path[d] = -1;
+    int tok = -1;
+    const int next = resolve_tree_node<T>(p, b, node, part, A, sh, tid, &tok);
+    if (tid == 0) {
+        if (next >= 0) {
+            if (len < p.max_depth) path[len] = next;
+            ws->node = next;
+            ws->len = len + 1;
+        } else {
+            ws->done = 1;
+            p.accepted_len[b] = len;
+            p.out_token[b] = tok;
+        }
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 struct VerifyPlan {
     int nchunks;
-    bool two_launches;  // enough rows to fill the machine: stream kernel + resolve kernel
     RowSplit split;
     size_t smem;
-    size_t ws_tickets_off, ws_meta_off, ws_partials_off, ws_bytes;
+    size_t ws_state_off, ws_tickets_off, ws_meta_off, ws_partials_off, ws_bytes;
+    size_t ws_clear_bytes;  // path walk: what is zeroed on the stream before the first level (state, tickets)
 };
-
-static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 static int sm_count_v() {
     static int sms = 0;
@@ -547,24 +597,42 @@ static int sm_count_v() {
     return sms;
 }
 
-constexpr int kVerifyCtasPerSm = 4;  // fused kernel: what the launch bounds and the shared-memory footprint allow
-
-static VerifyPlan make_verify_plan(int B, int rows_per_seq, int V, int elt_bytes, int meta_ints) {
+// rows_streamed: rows the streaming pass covers per launch (all target rows; B for the path walk).
+// levels > 0: the path walk, with its state and one ticket counter per sequence and level.
+static VerifyPlan make_verify_plan(int B, long long rows_streamed, int V, int elt_bytes, int meta_ints, int levels) {
     VerifyPlan pl;
     const long long row_bytes = (long long)V * elt_bytes;
     pl.nchunks = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
-    const long long rows = (long long)B * rows_per_seq;
-    const int slots = kVerifyCtasPerSm * sm_count_v();
-    pl.two_launches = rows >= slots;
-    pl.split = make_row_split(rows, pl.nchunks, slots, pl.two_launches ? 64 : 16, 32);
+    // Rows that fill the machine are cut into 64 KB segments; fewer rows into as many segments as give
+    // every CTA slot about two CTAs, a segment keeping at least one chunk per warp.
+    const int slots = (levels > 0 ? 4 : kStreamCtasPerSm) * sm_count_v();
+    int nseg;
+    if (rows_streamed >= slots) {
+        nseg = (pl.nchunks + 31) / 32;
+    } else {
+        nseg = (int)((2LL * slots + rows_streamed - 1) / (rows_streamed > 0 ? rows_streamed : 1));
+        const int by_len = pl.nchunks / kWarps;
+        if (nseg > by_len) nseg = by_len;
+        if (nseg > 64) nseg = 64;
+    }
+    if (nseg < 1) nseg = 1;
+    int cps = (pl.nchunks + nseg - 1) / nseg;
+    if (cps < 1) cps = 1;
+    pl.split.rows = (int)rows_streamed;
+    pl.split.cps = cps;
+    pl.split.nseg = (pl.nchunks + cps - 1) / cps;
+    pl.split.grid = pl.split.rows * pl.split.nseg;
     pl.smem = kVerifyArena + sizeof(VerifyShared) + 256;
     size_t off = kWsHeaderBytes;
+    pl.ws_state_off = off;
+    if (levels > 0) off = align_up256(off + (size_t)B * sizeof(WalkState));
     pl.ws_tickets_off = off;
-    off = up256(off + (size_t)B * sizeof(int));
+    if (levels > 0) off = align_up256(off + (size_t)levels * B * sizeof(int));
+    pl.ws_clear_bytes = off;
     pl.ws_meta_off = off;
-    off = up256(off + (size_t)meta_ints * sizeof(int));
+    off = align_up256(off + (size_t)meta_ints * sizeof(int));
     pl.ws_partials_off = off;
-    off = up256(off + (size_t)rows * pl.nchunks * sizeof(float2));
+    off = align_up256(off + (size_t)rows_streamed * pl.nchunks * sizeof(float2));
     pl.ws_bytes = off;
     return pl;
 }
@@ -586,22 +654,57 @@ static int check_common(const void* logits, int dtype, int V, long long row_stri
     return TSLT_OK;
 }
 
+// The resolver's shared memory exceeds the default limit: raise the kernel's limit once per device
+// (slot: one per kernel instantiation), not on every call.
+template <typename K> static bool raise_smem_limit_once(K kern, int slot, size_t bytes) {
+    constexpr int kMaxDevices = 64;
+    static bool done[8][kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached && done[slot][dev]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+    if (cached) done[slot][dev] = true;
+    return true;
+}
+
 template <bool kTree>
 static int launch_verify(VerifyParams& p, const VerifyPlan& pl, int dtype, cudaStream_t st) {
-    auto kern = dtype == TSLT_F32 ? verify_kernel<float, kTree> : verify_kernel<bf16_t, kTree>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
-        return TSLT_ERR_CUDA;
-    if (!pl.two_launches) {
-        kern<<<(unsigned)pl.split.grid, kBlockThreads, pl.smem, st>>>(p);
-        return cudaGetLastError() == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
-    }
     auto resolve = dtype == TSLT_F32 ? verify_resolve_kernel<float, kTree> : verify_resolve_kernel<bf16_t, kTree>;
-    if (cudaFuncSetAttribute(resolve, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess)
-        return TSLT_ERR_CUDA;
+    if (!raise_smem_limit_once(resolve, (kTree ? 2 : 0) + (dtype == TSLT_F32 ? 0 : 1), pl.smem)) return TSLT_ERR_CUDA;
     if (dtype == TSLT_F32) verify_stream_kernel<float><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     else verify_stream_kernel<bf16_t><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     return launch_dependent(resolve, (unsigned)p.B, kBlockThreads, pl.smem, st, p) == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+}
+
+// Host check of the tree arrays and the child lists in the form the kernels read:
+// child_begin[N+1] | child_list[N-1] | node_draft_row[N].  Returns the tree's depth, or -1.
+static int build_tree_meta(int N, int M, const int* parent, const int* node_draft_row, std::vector<int>& meta) {
+    if (parent[0] != -1) return -1;
+    std::vector<int> nchild(N, 0), depth(N, 0);
+    int maxd = 0;
+    for (int n = 1; n < N; ++n) {
+        if (parent[n] < 0 || parent[n] >= n) return -1;
+        nchild[parent[n]]++;
+        depth[n] = depth[parent[n]] + 1;
+        if (depth[n] > maxd) maxd = depth[n];
+    }
+    for (int n = 0; n < N; ++n) {
+        const bool internal = nchild[n] > 0;
+        if (internal != (node_draft_row[n] >= 0)) return -1;
+        if (node_draft_row[n] >= M) return -1;
+    }
+    meta.assign(3 * (size_t)N, 0);
+    int* child_begin = meta.data();
+    int* child_list = meta.data() + (N + 1);
+    int* ndr = meta.data() + (N + 1) + (N - 1);
+    child_begin[0] = 0;
+    for (int n = 0; n < N; ++n) child_begin[n + 1] = child_begin[n] + nchild[n];
+    std::vector<int> fill(child_begin, child_begin + N);
+    for (int n = 1; n < N; ++n) child_list[fill[parent[n]]++] = n;
+    for (int n = 0; n < N; ++n) ndr[n] = node_draft_row[n];
+    return maxd;
 }
 
 }  // namespace tslt
@@ -610,7 +713,8 @@ using namespace tslt;
 
 extern "C" int tslt_verify_workspace_bytes(int B, int gamma, int V, int k, size_t* bytes) {
     if (!bytes || B < 0 || gamma < 0 || V <= 0 || k <= 0 || k > V || k > TSLT_MAX_K) return TSLT_ERR_INVALID_ARG;
-    VerifyPlan a = make_verify_plan(B, gamma + 1, V, 2, 0), b = make_verify_plan(B, gamma + 1, V, 4, 0);
+    VerifyPlan a = make_verify_plan(B, (long long)B * (gamma + 1), V, 2, 0, 0),
+               b = make_verify_plan(B, (long long)B * (gamma + 1), V, 4, 0, 0);
     *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
     return TSLT_OK;
 }
@@ -631,7 +735,7 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
         return TSLT_ERR_INVALID_ARG;
     if ((long long)B * (gamma + 1) > 0x7fffffffLL / 16 || gamma >= 1024) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
-    VerifyPlan pl = make_verify_plan(B, gamma + 1, V, eb, 0);
+    VerifyPlan pl = make_verify_plan(B, (long long)B * (gamma + 1), V, eb, 0, 0);
     if (workspace_bytes < pl.ws_bytes) return TSLT_ERR_WORKSPACE;
     VerifyParams p = {};
     p.logits = (const unsigned char*)target_logits;
@@ -646,11 +750,8 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     p.accept_prob = accept_prob; p.beta_hat = beta_hat; p.lse_p = lse_p;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
-    p.tickets = (int*)(ws + pl.ws_tickets_off);
     p.partials = (float2*)(ws + pl.ws_partials_off);
-    cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(ws, 0, pl.ws_meta_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
-    return launch_verify<false>(p, pl, dtype, st);
+    return launch_verify<false>(p, pl, dtype, (cudaStream_t)stream);
 }
 
 // ---- tslt_verify_static: the same verification with the scratch memory built into the library ----
@@ -688,52 +789,51 @@ extern "C" int tslt_verify_static(const void* target_logits, int dtype, int B, i
     if (dtype != TSLT_F32 && dtype != TSLT_BF16) return TSLT_ERR_UNSUPPORTED;
     if (B < 0 || gamma < 0 || V <= 0 || k <= 0 || k > V) return TSLT_ERR_INVALID_ARG;
     if (k > TSLT_MAX_K || (long long)B * (gamma + 1) > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
-    const size_t need = make_verify_plan(B, gamma + 1, V, dtype == TSLT_F32 ? 4 : 2, 0).ws_bytes;
+    const size_t need = make_verify_plan(B, (long long)B * (gamma + 1), V, dtype == TSLT_F32 ? 4 : 2, 0, 0).ws_bytes;
     if (need > (size_t)TSLT_STATIC_SCRATCH_BYTES) return TSLT_ERR_STATIC_SCRATCH;
     if (B == 0) return TSLT_OK;
     void* scratch = nullptr;
     const int rs = static_scratch_address(&scratch);
     if (rs != TSLT_OK) return rs;
-    // tslt_verify zeroes the status word and the ticket counters on the stream before its kernel,
-    // so whatever the previous call left in the array does no harm
+    // tslt_verify's first kernel clears the status word, and nothing else in the array is read before
+    // it has been written, so whatever the previous call left there does no harm
     return tslt_verify(target_logits, dtype, B, gamma, V, row_stride_elems, k, draft_idx, draft_logit, draft_count,
                        draft_token, draft_temperature, target_temperature, u_accept, u_sample, accepted_len,
                        out_token, accept_prob, beta_hat, lse_p, scratch, (size_t)TSLT_STATIC_SCRATCH_BYTES, stream);
 }
 
+// levels the path walk can need for a tree of N nodes: one per node on a root-to-leaf path
+static int walk_levels_bound(int N) { return N; }
+
 extern "C" int tslt_tree_verify_workspace_bytes(int B, int N, int V, int k, size_t* bytes) {
     if (!bytes || B < 0 || N <= 0 || N > kMaxTreeNodes || V <= 0 || k <= 0 || k > V || k > TSLT_MAX_K)
         return TSLT_ERR_INVALID_ARG;
-    VerifyPlan a = make_verify_plan(B, N, V, 2, 3 * N), b = make_verify_plan(B, N, V, 4, 3 * N);
+    VerifyPlan a = make_verify_plan(B, (long long)B * N, V, 2, 3 * N, 0), b = make_verify_plan(B, (long long)B * N, V, 4, 3 * N, 0);
     *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
     return TSLT_OK;
 }
 
-extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
-                                long long row_stride_elems, const int* parent, const int* node_draft_row,
-                                int M, int k, const int* node_token, const int* draft_idx,
-                                const float* draft_logit, const int* draft_count, float draft_temperature,
-                                float target_temperature, const float* u_accept, const float* u_sample,
-                                int max_depth, int* accepted_path, int* accepted_len, int* out_token,
-                                void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int tslt_tree_verify_walk_workspace_bytes(int B, int N, int V, int k, size_t* bytes) {
+    if (!bytes || B < 0 || N <= 0 || N > kMaxTreeNodes || V <= 0 || k <= 0 || k > V || k > TSLT_MAX_K)
+        return TSLT_ERR_INVALID_ARG;
+    VerifyPlan a = make_verify_plan(B, B, V, 2, 3 * N, walk_levels_bound(N)), b = make_verify_plan(B, B, V, 4, 3 * N, walk_levels_bound(N));
+    *bytes = a.ws_bytes > b.ws_bytes ? a.ws_bytes : b.ws_bytes;
+    return TSLT_OK;
+}
+
+// Both tree entry points: walk = false streams every node's row and walks afterwards; walk = true
+// streams, level by level, only the rows the walks reach.
+static int tree_verify_impl(bool walk, const void* target_logits, int dtype, int B, int N, int V,
+                            long long row_stride_elems, const int* parent, const int* node_draft_row, int M, int k,
+                            const int* node_token, const int* draft_idx, const float* draft_logit,
+                            const int* draft_count, float draft_temperature, float target_temperature,
+                            const float* u_accept, const float* u_sample, int max_depth, int* accepted_path,
+                            int* accepted_len, int* out_token, void* workspace, size_t workspace_bytes, void* stream) {
     if (B < 0 || N <= 0 || M < 0 || max_depth < 0 || !parent || !node_draft_row) return TSLT_ERR_INVALID_ARG;
     if (N > kMaxTreeNodes) return TSLT_ERR_UNSUPPORTED;
-    // ---- tree structure, checked on the host ----------------------------------------------------
-    if (parent[0] != -1) return TSLT_ERR_INVALID_ARG;
-    std::vector<int> nchild(N, 0), depth(N, 0);
-    int maxd = 0;
-    for (int n = 1; n < N; ++n) {
-        if (parent[n] < 0 || parent[n] >= n) return TSLT_ERR_INVALID_ARG;
-        nchild[parent[n]]++;
-        depth[n] = depth[parent[n]] + 1;
-        if (depth[n] > maxd) maxd = depth[n];
-    }
-    if (maxd > max_depth) return TSLT_ERR_INVALID_ARG;
-    for (int n = 0; n < N; ++n) {
-        const bool internal = nchild[n] > 0;
-        if (internal != (node_draft_row[n] >= 0)) return TSLT_ERR_INVALID_ARG;
-        if (node_draft_row[n] >= M) return TSLT_ERR_INVALID_ARG;
-    }
+    std::vector<int> meta;
+    const int depth = build_tree_meta(N, M, parent, node_draft_row, meta);  // tree structure, checked on the host
+    if (depth < 0 || depth > max_depth) return TSLT_ERR_INVALID_ARG;
     if (B == 0) return TSLT_OK;
     int rc = check_common(target_logits, dtype, V, row_stride_elems, k, draft_temperature, target_temperature,
                           workspace);
@@ -741,20 +841,12 @@ extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int
     if (!u_sample || !accepted_len || !out_token || (max_depth > 0 && !accepted_path) ||
         (N > 1 && (!node_token || !u_accept)) || (M > 0 && (!draft_idx || !draft_logit || !draft_count)))
         return TSLT_ERR_INVALID_ARG;
-    if ((long long)B * N > 0x7fffffffLL / 16) return TSLT_ERR_UNSUPPORTED;
+    if ((long long)B * N > 0x7fffffffLL / 64) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
-    VerifyPlan pl = make_verify_plan(B, N, V, eb, 3 * N);
+    const int levels = depth + 1;  // nodes on the longest root-to-leaf path
+    VerifyPlan pl = walk ? make_verify_plan(B, B, V, eb, 3 * N, walk_levels_bound(N))
+                         : make_verify_plan(B, (long long)B * N, V, eb, 3 * N, 0);
     if (workspace_bytes < pl.ws_bytes) return TSLT_ERR_WORKSPACE;
-    // children of every node in ascending id: child_begin[N+1] | child_list[N-1] | node_draft_row[N]
-    std::vector<int> meta(3 * N, 0);
-    int* child_begin = meta.data();
-    int* child_list = meta.data() + (N + 1);
-    int* ndr = meta.data() + (N + 1) + (N - 1);
-    child_begin[0] = 0;
-    for (int n = 0; n < N; ++n) child_begin[n + 1] = child_begin[n] + nchild[n];
-    std::vector<int> fill(child_begin, child_begin + N);
-    for (int n = 1; n < N; ++n) child_list[fill[parent[n]]++] = n;
-    for (int n = 0; n < N; ++n) ndr[n] = node_draft_row[n];
 
     VerifyParams p = {};
     p.logits = (const unsigned char*)target_logits;
@@ -770,14 +862,49 @@ extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int
     p.node_token = node_token; p.accepted_path = accepted_path;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
+    p.walk = (WalkState*)(ws + pl.ws_state_off);
     p.tickets = (int*)(ws + pl.ws_tickets_off);
     p.tree_meta = (const int*)(ws + pl.ws_meta_off);
     p.partials = (float2*)(ws + pl.ws_partials_off);
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(ws, 0, pl.ws_meta_off, st) != cudaSuccess) return TSLT_ERR_CUDA;
     // pageable source: the runtime stages it before returning, so `meta` may go out of scope
     if (cudaMemcpyAsync(ws + pl.ws_meta_off, meta.data(), meta.size() * sizeof(int), cudaMemcpyHostToDevice, st) !=
         cudaSuccess)
         return TSLT_ERR_CUDA;
-    return launch_verify<true>(p, pl, dtype, st);
+    if (!walk) return launch_verify<true>(p, pl, dtype, st);
+    // status word, walk state (node 0, length 0, not done) and ticket counters start at zero
+    if (cudaMemsetAsync(ws, 0, pl.ws_clear_bytes, st) != cudaSuccess) return TSLT_ERR_CUDA;
+    auto kern = dtype == TSLT_F32 ? tree_walk_level_kernel<float> : tree_walk_level_kernel<bf16_t>;
+    if (!raise_smem_limit_once(kern, 4 + (dtype == TSLT_F32 ? 0 : 1), pl.smem)) return TSLT_ERR_CUDA;
+    for (int level = 0; level < levels; ++level) {
+        kern<<<(unsigned)pl.split.grid, kBlockThreads, pl.smem, st>>>(p, level);
+        if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
+    }
+    return TSLT_OK;
+}
+
+extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int N, int V,
+                                long long row_stride_elems, const int* parent, const int* node_draft_row,
+                                int M, int k, const int* node_token, const int* draft_idx,
+                                const float* draft_logit, const int* draft_count, float draft_temperature,
+                                float target_temperature, const float* u_accept, const float* u_sample,
+                                int max_depth, int* accepted_path, int* accepted_len, int* out_token,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    return tree_verify_impl(false, target_logits, dtype, B, N, V, row_stride_elems, parent, node_draft_row, M, k,
+                            node_token, draft_idx, draft_logit, draft_count, draft_temperature, target_temperature,
+                            u_accept, u_sample, max_depth, accepted_path, accepted_len, out_token, workspace,
+                            workspace_bytes, stream);
+}
+
+extern "C" int tslt_tree_verify_walk(const void* target_logits, int dtype, int B, int N, int V,
+                                     long long row_stride_elems, const int* parent, const int* node_draft_row,
+                                     int M, int k, const int* node_token, const int* draft_idx,
+                                     const float* draft_logit, const int* draft_count, float draft_temperature,
+                                     float target_temperature, const float* u_accept, const float* u_sample,
+                                     int max_depth, int* accepted_path, int* accepted_len, int* out_token,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+    return tree_verify_impl(true, target_logits, dtype, B, N, V, row_stride_elems, parent, node_draft_row, M, k,
+                            node_token, draft_idx, draft_logit, draft_count, draft_temperature, target_temperature,
+                            u_accept, u_sample, max_depth, accepted_path, accepted_len, out_token, workspace,
+                            workspace_bytes, stream);
 }

@@ -27,6 +27,7 @@ EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status", "tslt_
            "tslt_sparsify_workspace_bytes", "tslt_sparsify",
            "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
+           "tslt_tree_verify_walk_workspace_bytes", "tslt_tree_verify_walk",
            "tslt_payload_words", "tslt_pack_payload", "tslt_unpack_payload"]
 
 PROB_F32, PROB_BF16, PROB_F16 = 0, 1, 2
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
     L.tslt_tree_verify.restype = i
     L.tslt_tree_verify.argtypes = [p, i, i, i, i, ll, p, p, i, i, p, p, p, p, f, f, p, p, i, p, p, p,
                                    p, sz, p]
+    L.tslt_tree_verify_walk_workspace_bytes.restype = i
+    L.tslt_tree_verify_walk_workspace_bytes.argtypes = [i, i, i, i, psz]
+    L.tslt_tree_verify_walk.restype = i
+    L.tslt_tree_verify_walk.argtypes = L.tslt_tree_verify.argtypes
     L.tslt_payload_words.restype = i
     L.tslt_payload_words.argtypes = [i, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.tslt_pack_payload.restype = i
@@ -116,6 +121,18 @@ def _cuda(t: Optional[torch.Tensor], name: str, dtype=None) -> Optional[torch.Te
     if not t.is_contiguous():
         raise ValueError("%s must be contiguous" % name)
     return t
+
+
+def _out(o: dict, name: str, dtype, numel: int, required: bool = True) -> None:
+    """An output buffer the kernels will write: CUDA, contiguous, the right dtype and size."""
+    t = o.get(name)
+    if t is None:
+        if required:
+            raise ValueError("output %s is missing" % name)
+        return
+    _cuda(t, name, dtype)
+    if t.numel() != numel:
+        raise ValueError("output %s must have %d elements, has %d" % (name, numel, t.numel()))
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -227,6 +244,10 @@ def sparsify(logits: torch.Tensor, k: int, top_p: float = 1.0, temperature: floa
         if want_stats:
             o["lse"] = torch.empty(rows, dtype=torch.float32, device=dev)
             o["mass"] = torch.empty(rows, dtype=torch.float32, device=dev)
+    for name, dt, ne, req in (("idx", torch.int32, rows * k, True), ("logit", torch.float32, rows * k, True),
+                              ("count", torch.int32, rows, True), ("token", torch.int32, rows * ns, True),
+                              ("lse", torch.float32, rows, False), ("mass", torch.float32, rows, False)):
+        _out(o, name, dt, ne, req)
     if ws is None:
         ws = workspace(sparsify_workspace_bytes(rows, V, k, ns), dev)
     rc = lib().tslt_sparsify(_ptr(flat), _dtype_code(logits), rows, 1, V, stride, k, top_p, temperature,
@@ -236,6 +257,14 @@ def sparsify(logits: torch.Tensor, k: int, top_p: float = 1.0, temperature: floa
     _check(rc, "tslt_sparsify")
     o["workspace"] = ws
     return o
+
+
+def _check_verify_outputs(o: dict, B: int, gamma: int) -> None:
+    for name, dt, ne, req in (("accepted_len", torch.int32, B, True), ("out_token", torch.int32, B, True),
+                              ("accept_prob", torch.float32, B * gamma, False),
+                              ("beta_hat", torch.float32, B * gamma, False),
+                              ("lse_p", torch.float32, B * (gamma + 1), False)):
+        _out(o, name, dt, ne, req)
 
 
 def verify(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_logit: torch.Tensor,
@@ -274,6 +303,7 @@ def verify(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_logit: to
             o["accept_prob"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
             o["beta_hat"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
             o["lse_p"] = torch.empty(B, gamma + 1, dtype=torch.float32, device=dev)
+    _check_verify_outputs(o, B, gamma)
     if ws is None:
         ws = workspace(verify_workspace_bytes(B, gamma, V, k), dev)
     rc = lib().tslt_verify(_ptr(target_logits), _dtype_code(target_logits), B, gamma, V, stride, k,
@@ -311,6 +341,7 @@ def verify_static(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_lo
             u_accept.numel() != B * gamma or u_sample.numel() != B or \
             out["accepted_len"].numel() != B or out["out_token"].numel() != B:
         raise ValueError("draft / uniform / output shapes do not match target_logits")
+    _check_verify_outputs(out, B, gamma)
     rc = lib().tslt_verify_static(_ptr(target_logits), _dtype_code(target_logits), B, gamma, V, stride, k,
                                   _ptr(draft_idx), _ptr(draft_logit), _ptr(draft_count), _ptr(draft_token),
                                   draft_temperature, target_temperature, _ptr(u_accept), _ptr(u_sample),
@@ -320,13 +351,22 @@ def verify_static(target_logits: torch.Tensor, draft_idx: torch.Tensor, draft_lo
     return out
 
 
+def tree_verify_walk_workspace_bytes(B: int, N: int, V: int, k: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().tslt_tree_verify_walk_workspace_bytes(B, N, V, k, ctypes.byref(n)),
+           "tslt_tree_verify_walk_workspace_bytes")
+    return int(n.value)
+
+
 def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_row: Sequence[int],
                 node_token: torch.Tensor, draft_idx: torch.Tensor, draft_logit: torch.Tensor,
                 draft_count: torch.Tensor, draft_temperature: float, target_temperature: float,
                 u_accept: torch.Tensor, u_sample: torch.Tensor, max_depth: int, *,
-                out: Optional[dict] = None, ws: Optional[torch.Tensor] = None) -> dict:
-    """tslt_tree_verify.  target_logits [B, N, V]; parent / node_draft_row are host sequences [N];
-    drafts [B, M, k].  Returns dict(accepted_path [B, max_depth], accepted_len [B], out_token [B])."""
+                out: Optional[dict] = None, ws: Optional[torch.Tensor] = None, walk: bool = False) -> dict:
+    """tslt_tree_verify (walk=False: every node's row is streamed) or tslt_tree_verify_walk (walk=True:
+    only the rows on each sequence's path).  target_logits [B, N, V]; parent / node_draft_row are host
+    sequences [N]; drafts [B, M, k].  Returns dict(accepted_path [B, max_depth], accepted_len [B],
+    out_token [B])."""
     if not target_logits.is_cuda:
         raise ValueError("target_logits must be a CUDA tensor (libtslt has no CPU path)")
     if target_logits.dim() != 3:
@@ -352,15 +392,19 @@ def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_r
         o["accepted_path"] = torch.empty(B, max_depth, dtype=torch.int32, device=dev)
         o["accepted_len"] = torch.empty(B, dtype=torch.int32, device=dev)
         o["out_token"] = torch.empty(B, dtype=torch.int32, device=dev)
+    for name, dt, ne in (("accepted_path", torch.int32, B * max_depth), ("accepted_len", torch.int32, B),
+                         ("out_token", torch.int32, B)):
+        _out(o, name, dt, ne)
     if ws is None:
-        ws = workspace(tree_verify_workspace_bytes(B, N, V, k), dev)
-    rc = lib().tslt_tree_verify(_ptr(target_logits), _dtype_code(target_logits), B, N, V, stride,
+        ws = workspace((tree_verify_walk_workspace_bytes if walk else tree_verify_workspace_bytes)(B, N, V, k), dev)
+    entry = lib().tslt_tree_verify_walk if walk else lib().tslt_tree_verify
+    rc = entry(_ptr(target_logits), _dtype_code(target_logits), B, N, V, stride,
                                 par.ctypes.data_as(ctypes.c_void_p), ndr.ctypes.data_as(ctypes.c_void_p),
                                 M, k, _ptr(node_token), _ptr(draft_idx), _ptr(draft_logit), _ptr(draft_count),
                                 draft_temperature, target_temperature, _ptr(u_accept), _ptr(u_sample),
                                 max_depth, _ptr(o["accepted_path"]), _ptr(o["accepted_len"]),
                                 _ptr(o["out_token"]), _ptr(ws), ws.numel(), _stream())
-    _check(rc, "tslt_tree_verify")
+    _check(rc, "tslt_tree_verify_walk" if walk else "tslt_tree_verify")
     o["workspace"] = ws
     return o
 

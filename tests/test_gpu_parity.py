@@ -126,6 +126,12 @@ def test_tree_config3_full_batch_every_sequence():
     ref_t = oracle_tree_parallel(zp_c, parent, ndr, inp["toks"], inp["idx"], inp["logit"], inp["count"], 1.0, 1.0,
                                  inp["ua"], inp["us"], depth)
     compare_tree(gt, ref_t, "config 3 trees", inputs=inp)
+    gw = tslt.tree_verify(zp, parent, ndr, toks, gs["idx"].view(B, M, k), gs["logit"].view(B, M, k),
+                          gs["count"].view(B, M), 1.0, 1.0, ua, us, depth, walk=True)
+    torch.cuda.synchronize()
+    compare_tree(gw, ref_t, "config 3 trees (path walk)", inputs=inp)
+    for n in ("accepted_path", "accepted_len", "out_token"):
+        assert torch.equal(gw[n], gt[n]), n  # the two entry points agree bit for bit
 
 
 def adversarial_rows(V, dtype):
@@ -219,6 +225,45 @@ def test_identical_models_accept_everything():
     zp2 = torch.cat([zq2, zq2[:, :1]], dim=1).contiguous()
     _, _, ref_s, ref_v = run_sequence_case(zq2, zp2, 512, 1.0, 1.0, seed=4, what="identical k=V")
     assert (ref_v["accepted_len"] == 2).all()
+
+
+@pytest.mark.parametrize("offset,T", [(300.0, 1.0), (1000.0, 1.0), (-700.0, 1.0), (0.0, 0.3), (300.0, 0.3)])
+def test_large_common_offsets_and_low_temperature(offset, T):
+    """fp32 rows shifted by a large common offset, and a low temperature: the offset must cancel in
+    every probability (the streaming pass and the per-token exponent use one and the same scale)."""
+    B, gamma, V, k = 4, 3, 20011, 48
+    zq, zp = synth.sequence_logits(B, gamma, V, torch.float32, 0.5, 31, "cpu")
+    run_sequence_case(zq + offset, zp + offset, k, 1.0, T, seed=int(abs(offset)) + 3, what="offset %g T=%g" % (offset, T))
+    run_sequence_case(zq + offset, zp + offset, 256, 0.9, T, seed=int(abs(offset)) + 4, what="offset %g T=%g top-p" % (offset, T))
+
+
+def test_ready_wait_fall_back_sets_the_status_word_and_changes_nothing():
+    """With a poll limit of 0 every finish CTA of tslt_sparsify gives up on its row's ready flags at
+    once, records that in the status word and waits for the end of the streaming kernel instead:
+    same outputs, status word non-zero (reported as TSLT_ERR_DEVICE_STATUS).  Nothing is left
+    waiting: the fall-back is an ordinary kernel-boundary wait."""
+    B, gamma, V, k = 40, 4, 32000, 64
+    zq, _ = synth.sequence_logits(B, gamma, V, torch.bfloat16, 0.5, 17, "cuda")
+    u = synth.uniforms((B * gamma, 1), 17, synth.TID_U_DRAFT, "cuda")
+    ref = tslt.sparsify(zq, k, 0.95, 1.0, u)
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(ref["workspace"]) == 0
+    ws = torch.empty(tslt.sparsify_workspace_bytes(B * gamma, V, k, 1), dtype=torch.uint8, device="cuda")
+    try:
+        tslt.set_ready_poll_limit(0)
+        got = tslt.sparsify(zq, k, 0.95, 1.0, u, ws=ws)
+        torch.cuda.synchronize()
+    finally:
+        tslt.set_ready_poll_limit(1 << 22)
+    assert tslt.workspace_status(ws) & tslt.STATUS_WAIT_FELL_BACK
+    rc = tslt.lib().tslt_workspace_status(ws.data_ptr(), None, None)
+    assert rc == tslt.ERR_DEVICE_STATUS
+    for n in ("idx", "logit", "count", "token", "lse", "mass"):
+        assert to_np(got[n]).tobytes() == to_np(ref[n]).tobytes(), n
+    # the next ordinary call on the same workspace clears the word again
+    tslt.sparsify(zq, k, 0.95, 1.0, u, ws=ws)
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(ws) == 0
 
 
 def test_strided_rows_and_zero_rows():
@@ -328,6 +373,16 @@ def run_tree_case(B, expansion, V, dtype, k, T, seed, sigma_t=0.5, what=""):
     inp = dict(zp=zp, parent=parent, ndr=ndr, toks=toks, idx=ref_s["idx"].reshape(B, M, k),
                logit=ref_s["logit"].reshape(B, M, k), count=ref_s["count"].reshape(B, M), Tq=T, Tp=T,
                ua=ua.numpy(), us=us.numpy(), depth=depth)
+    # the path walk (only the rows on each sequence's path are read) must give the same outputs
+    walk = tslt.tree_verify(to_gpu_rows(zp), parent, ndr, torch.from_numpy(toks).cuda(),
+                            torch.from_numpy(ref_s["idx"]).cuda().view(B, M, k),
+                            torch.from_numpy(ref_s["logit"]).cuda().view(B, M, k),
+                            torch.from_numpy(ref_s["count"]).cuda().view(B, M), T, T, ua.cuda(), us.cuda(), depth,
+                            walk=True, ws=torch.empty(tslt.tree_verify_walk_workspace_bytes(B, N, V, k) + 256,
+                                                      dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(walk["workspace"]) == 0
+    compare_tree(walk, ref, what + " (path walk)", inputs=inp)
     return compare_tree(gpu, ref, what, inputs=inp), ref
 
 
@@ -372,6 +427,12 @@ def test_tree_duplicate_children_and_single_node():
                logit=ref_s["logit"].reshape(B, M, k), count=ref_s["count"].reshape(B, M), Tq=1.0, Tp=1.0,
                ua=ua.numpy(), us=us.numpy(), depth=depth)
     compare_tree(gpu, ref, "duplicates", inputs=inp)
+    gw = tslt.tree_verify(zp.cuda(), parent, ndr, torch.from_numpy(toks).cuda(),
+                          torch.from_numpy(ref_s["idx"]).cuda().view(B, M, k),
+                          torch.from_numpy(ref_s["logit"]).cuda().view(B, M, k),
+                          torch.from_numpy(ref_s["count"]).cuda().view(B, M), 1.0, 1.0, ua.cuda(), us.cuda(), depth, walk=True)
+    torch.cuda.synchronize()
+    compare_tree(gw, ref, "duplicates (path walk)", inputs=inp)
     # root only: the "tree" is a leaf, the token is a plain sample of the root row
     z1 = zp[:, :1].contiguous()
     ref = oracle.tree_verify(z1, [-1], [-1], np.zeros((B, 1), np.int32), np.zeros((B, 0, 1), np.int32),
@@ -382,6 +443,11 @@ def test_tree_duplicate_children_and_single_node():
                            torch.empty(0, device="cuda"), e_i, 1.0, 1.0, torch.zeros(B, 1, device="cuda"),
                            us[:, :1].contiguous().cuda(), 0)
     torch.cuda.synchronize()
+    gw = tslt.tree_verify(z1.cuda(), [-1], [-1], torch.zeros(B, 1, dtype=torch.int32, device="cuda"), e_i,
+                          torch.empty(0, device="cuda"), e_i, 1.0, 1.0, torch.zeros(B, 1, device="cuda"),
+                          us[:, :1].contiguous().cuda(), 0, walk=True)
+    torch.cuda.synchronize()
+    assert torch.equal(gw["out_token"], gpu["out_token"]) and (to_np(gw["accepted_len"]) == 0).all()
     assert (to_np(gpu["accepted_len"]) == 0).all()
     inp = dict(zp=z1, parent=[-1], ndr=[-1], toks=np.zeros((B, 1), np.int32), idx=np.zeros((B, 0, 1), np.int32),
                logit=np.zeros((B, 0, 1), np.float32), count=np.zeros((B, 0), np.int32), Tq=1.0, Tp=1.0,
