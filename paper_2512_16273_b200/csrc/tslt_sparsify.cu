@@ -10,34 +10,33 @@
 // runs at the occupancy and speed of a plain streaming reduction.
 //
 // Finish kernel (launched with programmatic stream serialization; a CTA starts on its row as soon
-// as the row's segments have been handed over).  One CTA per row:
-//   1. a lower bound on the k-th largest TILE maximum: tiles are taken in groups so that there are
-//      a few times k groups, and the k-th largest group maximum is found by bisection on its 16
-//      bits (each of the k groups at or above it holds a tile, and so a logit, at or above it);
-//   2. the tiles at or above that bound are listed in address order ("survivors": a little more
-//      than k of them) and read back from global memory: 64 bytes each, k * 64 bytes of the row's
-//      V * e;
-//   3. the exact k-th largest logit among them by a histogram over the 16-bit keys between the
-//      bound and the row maximum (fp32 rows: a second histogram over the low 16 bits inside the
-//      boundary value), ties at the boundary going to the lower index;
-//   4. the winners are collected by prefix sums over the survivors in address order, so they come
-//      out in ascending token index without any sort;
+// as the row's segments have been handed over).  One CTA of 64 to 256 threads per row:
+//   1. a lower bound on the k-th largest logit from the TILE maxima: tiles are taken in groups so
+//      that there are two to four times k groups, and the k-th largest group maximum is found by
+//      bisection on its bits (each of the k groups at or above it holds a logit at or above it);
+//   2. the tiles at or above that bound are listed in address order ("survivors": about 1.2 k of
+//      them) and read back from global memory: 64 bytes each, some k * 64 bytes of the row's V * e;
+//   3. their logits at or above the bound (the candidates, a little more than k) go to shared memory
+//      in index order, by prefix sums over the survivors;
+//   4. the exact k-th largest among them: by counting ranks while they are few, else by bisection on
+//      the 16-bit key between the bound and the row maximum (fp32 rows: once more on the low 16
+//      bits); ties at the k-th logit go to the lower index; the winners are compacted in place and
+//      so come out in ascending token index without any sort;
 //   5. the top-rho cut (a sort of the at most k winners by logit, an fp64 cumulative), the
 //      renormalised distribution and its CDF in fp64, the samples by inverse CDF, the outputs.
-// A row whose survivors do not fit the list (thousands of tied tile maxima: constant rows, rows
-// sorted by value) runs steps 3 and 4 over all of its vectors instead: slower, same code.
+// A row whose survivors or candidates do not fit their lists (thousands of tied maxima: constant
+// rows, rows sorted by value; k close to V) runs the selection over the survivors' vectors, or all
+// of the row's, in global memory instead: a histogram select and two more passes, slower, exact.
 #include <math.h>
 
 #include "tslt_common.cuh"
 #include "tslt_rowmath.cuh"
-#include "tslt_select.cuh"
 
 namespace tslt {
 
 constexpr int kTilesPerChunk = 32;        // 64-byte tiles in a 2 KB chunk
 constexpr int kVecsPerTile = 4;           // 16-byte vectors in a tile
 constexpr int kSparsifyStreamCtasPerSm = 6;
-constexpr int kFinishThreads = kBlockThreads;
 constexpr int kMaxGroups = 4096;          // group maxima the finish kernel bisects over
 constexpr int kMaxTileList = 4096;        // survivor tiles it can list
 constexpr int kSelBins = 1024;            // bins of the selection histogram
@@ -69,6 +68,7 @@ struct SparsifyParams {
     int group_log2;   // tiles per group = 1 << group_log2
     int ngroups;      // <= kMaxGroups
     int tile_cap;     // survivor list capacity (<= kMaxTileList)
+    int cand_cap;     // candidate list capacity (<= 8 * the finish kernel's threads)
     int poll_limit;   // polls of a segment's ready flag before falling back to the end of the streaming kernel
     int* status;
     int* seg_ready;           // [rows * nseg]
@@ -167,34 +167,53 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
 }
 
 // ---- finish kernel ---------------------------------------------------------------------------------
+// NT threads per row: 64 (k <= 64), 128 (k <= 128) or 256.  Finishing a row is a chain of dependent
+// steps (trips to L2 / HBM, bisection rounds, prefix sums), so what it costs machine-wide is the
+// chain's length times the number of waves: small CTAs keep every row of a large batch resident at
+// once (14 CTAs of 64 threads per SM hold 2048 rows on 148 SMs).
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) / 16 * 16; }
 __host__ __device__ inline int pow2_at_least(int n) {
     int p = 1;
     while (p < n) p <<= 1;
     return p;
 }
+__host__ __device__ constexpr int finish_threads(int k) { return k <= 64 ? 64 : k <= 128 ? 128 : 256; }
+__host__ __device__ constexpr int finish_resident(int nt) { return nt == 64 ? 14 : nt == 128 ? 8 : 4; }
 constexpr int kFinishHeaderBytes = 512;
-// dynamic shared memory of the finish kernel: header | histogram | region A | region B | winners
-__host__ __device__ inline size_t finish_region_a(int ngroups, int k) {
-    const size_t g = (size_t)ngroups * 4, c = (size_t)pow2_at_least(k) * 8;
-    return align16(g > c ? g : c);
-}
-__host__ __device__ inline size_t finish_region_b(int tile_cap, int k) {
-    const size_t t = (size_t)tile_cap * 4, w = (size_t)k * 16;
-    return align16(t > w ? t : w);
-}
-__host__ __device__ inline size_t sparsify_finish_smem(int ngroups, int tile_cap, int k) {
-    return kFinishHeaderBytes + (size_t)kSelBins * 4 + finish_region_a(ngroups, k) + finish_region_b(tile_cap, k) + (size_t)k * 8;
+constexpr int kRankListMax = 512;  // candidates up to which the k-th is found by counting ranks
+
+// Dynamic shared memory of the finish kernel:
+//   header | histogram | region A | region B | region C | line maxima
+//   histogram: the selection histogram of the all-vectors path; else the rank-counting keys
+//   region A:  group maxima, later the sort keys of the top-rho cut
+//   region B:  survivor tile list, later the fp64 work arrays (weights, CDF)
+//   region C:  candidates (raw logit bits, token index), compacted in place to the winners
+struct FinishLayout {
+    size_t hist, a, b, c, lines, total;
+};
+__host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap, int cand_cap, int k, int nchunks) {
+    FinishLayout L;
+    L.hist = kFinishHeaderBytes;
+    L.a = L.hist + (size_t)kSelBins * 4;
+    const size_t ga = (size_t)ngroups * 4, ca = (size_t)pow2_at_least(k) * 8;
+    L.b = L.a + align16(ga > ca ? ga : ca);
+    const size_t tb = (size_t)tile_cap * 4, wb = (size_t)k * 16;
+    L.c = L.b + align16(tb > wb ? tb : wb);
+    L.lines = L.c + (size_t)cand_cap * 8;
+    L.total = L.lines + align16((size_t)nchunks * 2);
+    return L;
 }
 
 struct FinishShared {
     double scratch[16];
-    double lrow;            // base-2 log of the row's softmax normaliser
-    int round_count[32];    // one counter per bisection round
+    double lrow;  // base-2 log of the row's softmax normaliser
+    int round_count[48];  // one counter per bisection round: three bisections of at most 16 rounds
     int iscr[16];
     int sel_bin, sel_above, sel_eq, sel_total;
-    int ready, n_surv, max16;
+    int ready, gmin, gmax;
 };
+
+template <int NT> __device__ __forceinline__ void fsync() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); }
 
 // One 16-byte vector of a row as kPer logits; the row's ragged last vector element by element,
 // -inf beyond the row.
@@ -210,8 +229,8 @@ __device__ __forceinline__ void load_row_vector(const unsigned char* rowp, int v
     }
 }
 
-// Exclusive prefix sum of one int per thread over the block; *total gets the sum.
-__device__ __forceinline__ int block_exscan(int v, int tid, int* scr /* >= 8 */, int* total) {
+// Exclusive prefix sum of one int per thread over the NT threads; *total gets the sum.
+template <int NT> __device__ __forceinline__ int block_exscan(int v, int tid, int* scr /* >= NT / 32 */, int* total) {
     const int lane = tid & 31, warp = tid >> 5;
     int incl = v;
 #pragma unroll
@@ -220,36 +239,106 @@ __device__ __forceinline__ int block_exscan(int v, int tid, int* scr /* >= 8 */,
         if (lane >= o) incl += t;
     }
     if (lane == 31) scr[warp] = incl;
-    consumer_sync();
+    fsync<NT>();
     int base = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         const int t = scr[w];
         if (w < warp) base += t;
         tot += t;
     }
-    consumer_sync();
+    fsync<NT>();
     *total = tot;
     return base + incl - v;
 }
-
-// Which of a chunk's 32 tiles have a key >= bound: bit a of the result is tile a of the chunk in
-// ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the chunk's 64-byte line of maxima).
-__device__ __forceinline__ uint32_t chunk_survivors(const unsigned short* line, uint32_t bound) {
-    uint32_t w[16];
+template <int NT> __device__ __forceinline__ double block_max_f64(double v, int tid, double* scr) {
+    v = warp_max(v);
+    if ((tid & 31) == 0) scr[tid >> 5] = v;
+    fsync<NT>();
+    double m = scr[0];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(line) + i);
-        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
-    }
-    uint32_t m = 0;
-#pragma unroll
-    for (int a = 0; a < kTilesPerChunk; ++a) {
-        const int slot = ((a & 7) << 2) | (a >> 3);
-        const uint32_t raw = (slot & 1) ? (w[slot >> 1] >> 16) : (w[slot >> 1] & 0xffffu);
-        m |= (raw16_to_key16(raw) >= bound ? 1u : 0u) << a;
-    }
+    for (int w = 1; w < NT / 32; ++w) m = fmax(m, scr[w]);
+    fsync<NT>();
     return m;
+}
+template <int NT> __device__ __forceinline__ double block_sum_f64(double v, int tid, double* scr) {
+    v = warp_sum(v);
+    if ((tid & 31) == 0) scr[tid >> 5] = v;
+    fsync<NT>();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) t += scr[w];
+    fsync<NT>();
+    return t;
+}
+// In-place inclusive scan of a[0..n) (shared memory, fp64).  Each thread owns a contiguous run, so
+// the sums have a fixed order: deterministic.
+template <int NT> __device__ __forceinline__ void block_inclusive_scan_f64(double* a, int n, int tid, double* scr) {
+    const int per = (n + NT - 1) / NT;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    double run = 0.0;
+    for (int i = lo; i < hi; ++i) run += a[i];
+    double incl = run;
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) scr[warp] = incl;
+    fsync<NT>();
+    double base = 0.0;
+    for (int w = 0; w < warp; ++w) base += scr[w];
+    double acc = base + (incl - run);
+    for (int i = lo; i < hi; ++i) {
+        acc += a[i];
+        a[i] = acc;
+    }
+    fsync<NT>();
+}
+// Bitonic sort of a[0..P) (P a power of two, shared memory), descending.
+template <int NT> __device__ __forceinline__ void bitonic_sort_desc(unsigned long long* a, int P, int tid) {
+    for (int size = 2; size <= P; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = tid; i < (P >> 1); i += NT) {
+                const int lo = 2 * i - (i & (stride - 1));
+                const int hi = lo + stride;
+                const bool up = ((lo & size) == 0);
+                const unsigned long long x = a[lo], y = a[hi];
+                if (up ? x < y : x > y) {
+                    a[lo] = y;
+                    a[hi] = x;
+                }
+            }
+            fsync<NT>();
+        }
+    }
+}
+
+// The largest d in [0, range] such that at least kk of the thread block's values are >= d, given
+// that at least kk are >= 0: bisection on the bits of d, one barrier per bit that needs a count.
+// count_ge(d) returns how many of THIS thread's values are >= d.  *above gets the number of values
+// > the result.  counters: one zeroed int per round (at most 32), consumed here.
+template <int NT, typename CountGe>
+__device__ __forceinline__ uint32_t bisect_kth(uint32_t range, int kk, CountGe count_ge, int* counters, int tid, int* above) {
+    uint32_t d = 0;
+    int last_rejected = 0, round = 0;
+    for (int bit = 31 - __clz((int)(range | 1u)); bit >= 0; --bit) {
+        const uint32_t cand = d | (1u << bit);
+        if (cand > range) {  // nothing lies above the range: rejected without counting
+            last_rejected = 0;
+            continue;
+        }
+        const int cnt = __reduce_add_sync(0xffffffffu, count_ge(cand));
+        if ((tid & 31) == 0 && cnt) atomicAdd(&counters[round], cnt);
+        fsync<NT>();
+        const int total = counters[round];
+        ++round;
+        if (total >= kk) d = cand;
+        else last_rejected = total;
+    }
+    *above = last_rejected;
+    return d;
 }
 
 // The vectors a thread works on: units [u0, u1) of the row's survivor tiles (tl: their tile numbers in
@@ -281,13 +370,13 @@ __device__ __forceinline__ void for_my_vectors(const unsigned char* rowp, const 
     }
 }
 
-// The kk-th largest of the values value_of(z) in [lo, hi] over the thread block's vectors (values
-// outside the range, or negative, do not take part), by a histogram of kSelBins bins over the
-// range, narrowed once more if the range is wider than the histogram.  Results in sh: sel_bin = the
-// value, sel_above = how many are larger (inside [lo, hi]), sel_eq = how many equal it,
-// sel_total = how many lie in [lo, hi].  If fewer than kk lie in the range, sel_bin = -1 and only
-// sel_total is meaningful.  All threads call it; hist is kSelBins words of shared memory.
-template <typename T, typename VF>
+// All-vectors path only.  The kk-th largest of the values value_of(z) in [lo, hi] over the thread
+// block's vectors (values outside the range, or negative, do not take part), by a histogram of
+// kSelBins bins over the range, narrowed once more if the range is wider than the histogram.
+// Results in sh: sel_bin = the value, sel_above = how many are larger (inside [lo, hi]), sel_eq =
+// how many equal it, sel_total = how many lie in [lo, hi].  If fewer than kk lie in the range,
+// sel_bin = -1 and only sel_total is meaningful.  All threads call it.
+template <typename T, int NT, typename VF>
 __device__ __forceinline__ void hist_select(const unsigned char* rowp, const RowExtent& ext, int V, const uint32_t* tl, int u0,
                                             int u1, VF value_of, int lo, int hi, int kk, FinishShared* sh, uint32_t* hist,
                                             int tid) {
@@ -296,8 +385,8 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
     for (;;) {
         int s = 0;
         while (((hi - lo) >> s) >= kSelBins) ++s;
-        for (int i = tid; i < kSelBins; i += kFinishThreads) hist[i] = 0u;
-        consumer_sync();
+        for (int i = tid; i < kSelBins; i += NT) hist[i] = 0u;
+        fsync<NT>();
         for_my_vectors<T>(rowp, ext, V, tl, u0, u1, [&](const float(&z)[kPer], int) {
             int cur = -1;
             uint32_t run = 0;
@@ -316,7 +405,7 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
             }
             if (run) atomicAdd(&hist[cur], run);
         });
-        consumer_sync();
+        fsync<NT>();
         if (tid < 32) {
             // rows of 32 bins from the top; lane l takes bin top - l of the row
             uint32_t carried = 0;
@@ -348,9 +437,9 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
                 sh->sel_total = (int)carried;
             }
         }
-        consumer_sync();
+        fsync<NT>();
         const int bin = sh->sel_bin, above = sh->sel_above, eq = sh->sel_eq, total = sh->sel_total;
-        consumer_sync();
+        fsync<NT>();
         if (total_first < 0) total_first = total;
         if (bin < 0 || s == 0) {
             if (tid == 0) {
@@ -359,7 +448,7 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
                 sh->sel_eq = eq;
                 sh->sel_total = total_first;
             }
-            consumer_sync();
+            fsync<NT>();
             return;
         }
         above_acc += above;
@@ -369,34 +458,104 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
     }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(const SparsifyParams p) {
+// 16-bit key of a finite logit (its order-preserving key's top half), -1 otherwise.
+__device__ __forceinline__ int finite_key16(float z) {
+    const uint32_t k16 = float_to_key(z) >> 16;
+    return (k16 >= kLowestFinite16 && k16 <= kHighestFinite16) ? (int)k16 : -1;
+}
+
+// Group maxima of one 64-byte line of tile maxima (32 slots, two per word): the packed bf16 maximum
+// works on the raw top-16-bit patterns whatever the logits' type.  Writes the line's 32 >> glog group
+// maxima (as keys) to gm_line, for 0 <= glog <= 5; returns the line's maximum as a raw pattern.
+__device__ __forceinline__ uint32_t half_max(uint32_t w) { return bf16x2_max(w, w >> 16) & 0xffffu; }
+__device__ __forceinline__ uint32_t line_group_maxima(const uint32_t (&w)[16], int glog, uint32_t* gm_line) {
+    uint32_t t8[8], t4[4], t2[2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t8[i] = bf16x2_max(w[2 * i], w[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) t4[i] = bf16x2_max(t8[2 * i], t8[2 * i + 1]);
+    t2[0] = bf16x2_max(t4[0], t4[1]);
+    t2[1] = bf16x2_max(t4[2], t4[3]);
+    const uint32_t t1 = bf16x2_max(t2[0], t2[1]);
+    if (glog == 0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            gm_line[2 * i] = raw16_to_key16(w[i] & 0xffffu);
+            gm_line[2 * i + 1] = raw16_to_key16(w[i] >> 16);
+        }
+    } else if (glog == 1) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) gm_line[i] = raw16_to_key16(half_max(w[i]));
+    } else if (glog == 2) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gm_line[i] = raw16_to_key16(half_max(t8[i]));
+    } else if (glog == 3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gm_line[i] = raw16_to_key16(half_max(t4[i]));
+    } else if (glog == 4) {
+        gm_line[0] = raw16_to_key16(half_max(t2[0]));
+        gm_line[1] = raw16_to_key16(half_max(t2[1]));
+    } else if (glog == 5) {
+        gm_line[0] = raw16_to_key16(half_max(t1));
+    }
+    return half_max(t1);
+}
+
+// Which of a line's 32 tiles have a key >= bound: bit a of the result is tile a of the chunk in
+// ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the line).
+__device__ __forceinline__ uint32_t line_survivors(const uint32_t (&w)[16], uint32_t bound) {
+    uint32_t m = 0;
+#pragma unroll
+    for (int a = 0; a < kTilesPerChunk; ++a) {
+        const int slot = ((a & 7) << 2) | (a >> 3);
+        const uint32_t raw = (slot & 1) ? (w[slot >> 1] >> 16) : (w[slot >> 1] & 0xffffu);
+        m |= (raw16_to_key16(raw) >= bound ? 1u : 0u) << a;
+    }
+    return m;
+}
+__device__ __forceinline__ void load_line(const unsigned short* line, uint32_t (&w)[16]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(line) + i);
+        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+}
+
+template <typename T, int NT>
+__global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kernel(const SparsifyParams p) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
+    constexpr int kHeld = 8;  // most list entries a thread owns (cand_cap <= 8 * NT, see the plan)
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // carve-up (sizes in sparsify_finish_smem): header | hist | region A | region B | win_raw | win_idx
-    //   region A: group maxima, later the sort keys of the top-rho cut
-    //   region B: survivor tile list, later the fp64 work arrays
     FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
     static_assert(sizeof(FinishShared) <= kFinishHeaderBytes, "header");
-    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes);
     const int k = p.k;
-    const size_t a_bytes = finish_region_a(p.ngroups, k), b_bytes = finish_region_b(p.tile_cap, k);
-    uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4);
+    const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + L.hist);
+    unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
+    uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + L.a);
     unsigned long long* comp = reinterpret_cast<unsigned long long*>(gm);
-    uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4 + a_bytes);
+    uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + L.b);
     double* cum = reinterpret_cast<double*>(tl);
     double* wv = cum + k;
-    uint32_t* win_raw = reinterpret_cast<uint32_t*>(smem_raw + kFinishHeaderBytes + kSelBins * 4 + a_bytes + b_bytes);
-    int* win_idx = reinterpret_cast<int*>(win_raw + k);
+    uint32_t* c_raw = reinterpret_cast<uint32_t*>(smem_raw + L.c);
+    int* c_idx = reinterpret_cast<int*>(c_raw + p.cand_cap);
+    unsigned short* lmax = reinterpret_cast<unsigned short*>(smem_raw + L.lines);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, row = blockIdx.x;
-    const int nseg = p.split.nseg;
+    const int nseg = p.split.nseg, nchunks = p.nchunks;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
     const RowExtent ext = row_extent<T>(p.V);
     if (tid == 0 && p.num_samples > 0)  // the uniforms are needed last: ask for their cache line now
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
-    if (tid < 32) sh->round_count[tid] = 0;
+    if (tid < 48) sh->round_count[tid] = 0;
+    if (tid == 0) {
+        sh->gmin = 0xffff;
+        sh->gmax = 0;
+    }
+    const int glog = p.group_log2, ngroups = p.ngroups;
+    if (glog > 5)
+        for (int i = tid; i < ngroups; i += NT) gm[i] = 0u;
     // ---- wait for the row's segments --------------------------------------------------------------
     // Nothing the streaming kernel wrote is read before this point.  The row's own segments being
     // handed over is enough to go on; a flag that does not come within the poll limit is recorded in
@@ -407,12 +566,12 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
         ok = __all_sync(0xffffffffu, ok);
         if (lane == 0) sh->ready = ok ? 1 : 0;
     }
-    __syncthreads();
+    fsync<NT>();
     if (!sh->ready) {
         if (tid == 0) atomicOr(p.status, TSLT_STATUS_WAIT_FELL_BACK);
         wait_for_primary_kernel();
     }
-    __syncthreads();
+    fsync<NT>();
     // ---- the row's log-normaliser, by one warp (fp64 is scarce) -------------------------------------
     if (warp == 1) {
         const SegStat* st = p.seg_stats + (size_t)row * nseg;
@@ -428,74 +587,65 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
         Sall = warp_sum(Sall);
         if (lane == 0) sh->lrow = Sall > 0.0 ? Mall + log2(Sall) : -INFINITY;
     }
-    // ---- 1. group maxima of the tile keys ---------------------------------------------------------------
-    const int ntiles = p.nchunks * kTilesPerChunk;
-    const unsigned short* tmax = p.tile_max + (size_t)row * ntiles;
-    const int glog = p.group_log2, ngroups = p.ngroups;
-    if (glog > 3)
-        for (int i = tid; i < ngroups; i += kFinishThreads) gm[i] = 0u;
-    if (tid == 0) sh->max16 = 0;
-    __syncthreads();
-    {
-        uint32_t my_max = 0;
-        const int nv8 = ntiles / 8;
-        for (int v = tid; v < nv8; v += kFinishThreads) {
-            const uint4 w = __ldcg(reinterpret_cast<const uint4*>(tmax) + v);
-            uint32_t kk[8];
-            kk[0] = raw16_to_key16(w.x & 0xffffu); kk[1] = raw16_to_key16(w.x >> 16);
-            kk[2] = raw16_to_key16(w.y & 0xffffu); kk[3] = raw16_to_key16(w.y >> 16);
-            kk[4] = raw16_to_key16(w.z & 0xffffu); kk[5] = raw16_to_key16(w.z >> 16);
-            kk[6] = raw16_to_key16(w.w & 0xffffu); kk[7] = raw16_to_key16(w.w >> 16);
-            // groups are runs of consecutive SLOTS (any fixed partition of the tiles will do)
-            if (glog == 0) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) gm[v * 8 + i] = kk[i];
-            } else if (glog == 1) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) gm[v * 4 + i] = max(kk[2 * i], kk[2 * i + 1]);
-            } else if (glog == 2) {
-#pragma unroll
-                for (int i = 0; i < 2; ++i) gm[v * 2 + i] = max(max(kk[4 * i], kk[4 * i + 1]), max(kk[4 * i + 2], kk[4 * i + 3]));
-            }
-            const uint32_t m8 = max(max(max(kk[0], kk[1]), max(kk[2], kk[3])), max(max(kk[4], kk[5]), max(kk[6], kk[7])));
-            if (glog == 3) gm[v] = m8;
-            else if (glog > 3) atomicMax(&gm[v >> (glog - 3)], m8);
-            my_max = max(my_max, m8);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) my_max = max(my_max, __shfl_xor_sync(0xffffffffu, my_max, o));
-        if (lane == 0) atomicMax(&sh->max16, (int)my_max);
+    // ---- 1. group maxima of the tile maxima; each line's maximum is kept for step 3 -------------------
+    // Thread t takes a run of consecutive chunks; a chunk's 32 tile maxima are one 64-byte line.
+    const unsigned short* tmax = p.tile_max + (size_t)row * nchunks * kTilesPerChunk;
+    const int cpt = (nchunks + NT - 1) / NT;
+    const int ch0 = min(nchunks, tid * cpt), ch1 = min(nchunks, ch0 + cpt);
+    for (int ch = ch0; ch < ch1; ++ch) {
+        uint32_t w[16];
+        load_line(tmax + ch * kTilesPerChunk, w);
+        const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+        if (glog > 5) atomicMax(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
+        lmax[ch] = (unsigned short)lm;
     }
-    __syncthreads();
-    const int max16 = min(sh->max16, (int)kHighestFinite16);
+    fsync<NT>();
+    {
+        uint32_t mn = 0xffffu, mx = 0u;
+        for (int i = tid; i < ngroups; i += NT) {
+            const uint32_t v = gm[i];
+            mn = min(mn, v);
+            mx = max(mx, v);
+        }
+        mn = __reduce_min_sync(0xffffffffu, mn);
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (lane == 0) {
+            atomicMin(&sh->gmin, (int)mn);
+            atomicMax(&sh->gmax, (int)mx);
+        }
+    }
+    fsync<NT>();
+    const uint32_t gmin = (uint32_t)sh->gmin, gmax = (uint32_t)sh->gmax;
+    const int max16 = min((int)gmax, (int)kHighestFinite16);
     const double L2 = sh->lrow;
-    // ---- 2. the k-th largest group maximum, by bisection on its 16 bits -----------------------------------
+    // ---- 2. the k-th largest group maximum: a lower bound on the k-th largest logit's key ---------------
     uint32_t bound = 0;
     if (ngroups >= k) {
-        for (int bit = 15; bit >= 0; --bit) {
-            const uint32_t cand = bound | (1u << bit);
-            int cnt = 0;
-            for (int i = tid; i < ngroups; i += kFinishThreads) cnt += gm[i] >= cand ? 1 : 0;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-            if (lane == 0 && cnt) atomicAdd(&sh->round_count[bit], cnt);
-            __syncthreads();
-            if (sh->round_count[bit] >= k) bound = cand;
-        }
+        int unused;
+        bound = gmin + bisect_kth<NT>(gmax - gmin, k, [&](uint32_t d) {
+            int c = 0;
+            for (int i = tid; i < ngroups; i += NT) c += (gm[i] - gmin) >= d ? 1 : 0;
+            return c;
+        }, sh->round_count, tid, &unused);
     }
     int lo16 = max((int)bound, (int)kLowestFinite16);
     // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
-    // Thread t takes a run of consecutive chunks; a chunk's 32 tile keys are one 64-byte line.
-    const int cpt = (p.nchunks + kFinishThreads - 1) / kFinishThreads;
-    const int ch0 = min(p.nchunks, tid * cpt), ch1 = min(p.nchunks, ch0 + cpt);
     int my_surv = 0;
-    for (int ch = ch0; ch < ch1; ++ch) my_surv += __popc(chunk_survivors(tmax + ch * kTilesPerChunk, (uint32_t)lo16));
+    for (int ch = ch0; ch < ch1; ++ch) {
+        if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+        uint32_t w[16];
+        load_line(tmax + ch * kTilesPerChunk, w);
+        my_surv += __popc(line_survivors(w, (uint32_t)lo16));
+    }
     int n_surv;
-    int pos = block_exscan(my_surv, tid, sh->iscr, &n_surv);
+    int pos = block_exscan<NT>(my_surv, tid, sh->iscr, &n_surv);
     const bool listed = n_surv <= p.tile_cap;
     if (listed) {
         for (int ch = ch0; ch < ch1; ++ch) {
-            uint32_t m = chunk_survivors(tmax + ch * kTilesPerChunk, (uint32_t)lo16);  // bit a: tile a of the chunk
+            if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+            uint32_t w[16];
+            load_line(tmax + ch * kTilesPerChunk, w);
+            uint32_t m = line_survivors(w, (uint32_t)lo16);  // bit a: tile a of the chunk
             while (m) {
                 const int a = __ffs(m) - 1;
                 m &= m - 1;
@@ -503,107 +653,204 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
             }
         }
     }
-    __syncthreads();
+    fsync<NT>();
     // the vectors this thread works on from here: a contiguous run of the survivors' vectors, or of the row's
     const uint32_t* units = listed ? tl : nullptr;
     const int n_units = listed ? n_surv * kVecsPerTile : (p.V + kPer - 1) / kPer;
-    const int upt = (n_units + kFinishThreads - 1) / kFinishThreads;
+    const int upt = (n_units + NT - 1) / NT;
     const int u0 = min(n_units, tid * upt), u1 = min(n_units, u0 + upt);
     if (!listed) lo16 = (int)kLowestFinite16;
+    const float lo_f = key_to_float((uint32_t)lo16 << 16);  // the smallest float whose 16-bit key is lo16
+    auto is_candidate = [lo_f](float z) { return z >= lo_f && z <= 3.4028234e38f; };
 
-    // ---- 4. the exact k-th largest logit --------------------------------------------------------------------
-    // level 1: its 16-bit key among the finite logits of the survivors
-    auto key16_of = [](float z) -> int {
-        const uint32_t k16 = float_to_key(z) >> 16;
-        return (k16 >= kLowestFinite16 && k16 <= kHighestFinite16) ? (int)k16 : -1;
-    };
-    int n0 = 0;                 // winners: min(k, finite logits)
-    uint32_t e32 = 0;           // key of the k-th largest logit
-    int need_ties = 0;          // how many logits equal to it are winners (the lowest indices)
-    if (max16 >= lo16) {
-        hist_select<T>(rowp, ext, p.V, units, u0, u1, key16_of, lo16, max16, k, sh, hist, tid);
-        const int e16 = sh->sel_bin, above = sh->sel_above, eq = sh->sel_eq, total = sh->sel_total;
-        consumer_sync();
-        if (e16 < 0) {  // fewer than k finite logits in the row: all of them win
-            n0 = total;
-            e32 = 0u;
-            need_ties = 0;
-            // every finite logit is "above" the key 0; nothing ties
-        } else if (kBf16) {
-            n0 = k;
-            e32 = ((uint32_t)e16 << 16) | ((e16 & 0x8000) ? 0u : 0xffffu);  // keys of bf16 values: low half follows the sign
-            need_ties = k - above;
-        } else {
-            // level 2 (fp32 rows): the low 16 bits among the logits whose high bits equal e16
-            const uint32_t hi_bits = (uint32_t)e16;
-            auto low16_of = [hi_bits](float z) -> int {
-                const uint32_t kz = float_to_key(z);
-                return (kz >> 16) == hi_bits ? (int)(kz & 0xffffu) : -1;
-            };
-            hist_select<T>(rowp, ext, p.V, units, u0, u1, low16_of, 0, 0xffff, k - above, sh, hist, tid);
-            const int low = sh->sel_bin, above2 = sh->sel_above;
-            consumer_sync();
-            n0 = k;
-            e32 = (hi_bits << 16) | (uint32_t)low;
-            need_ties = k - above - above2;
-            (void)eq;
-        }
-    }
-    // ---- 5. the winners, in ascending index ---------------------------------------------------------------
-    int n = 0;
-    if (n0 > 0) {
-        int c_gt = 0, c_eq = 0;
-        const uint32_t e32c = e32;
+    // ---- 4. candidates: the finite logits of the survivors at or above the bound, in index order --------
+    bool in_smem = false;
+    int n_c = 0;
+    if (listed && max16 >= lo16) {
+        int cnt = 0;
         for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
 #pragma unroll
-            for (int e = 0; e < kPer; ++e) {
-                if (key16_of(z[e]) < lo16) continue;
-                const uint32_t kz = float_to_key(z[e]);
-                c_gt += kz > e32c ? 1 : 0;
-                c_eq += kz == e32c ? 1 : 0;
-            }
+            for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
         });
-        int tot_eq, tot_w;
-        const int eq_before = block_exscan(c_eq, tid, sh->iscr, &tot_eq);
-        const int my_ties = max(0, min(c_eq, need_ties - eq_before));
-        int wpos = block_exscan(c_gt + my_ties, tid, sh->iscr, &tot_w);
-        int ties_left = my_ties;
-        for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+        int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+        if (n_c <= p.cand_cap) {
+            in_smem = true;
+            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
 #pragma unroll
-            for (int e = 0; e < kPer; ++e) {
-                if (key16_of(z[e]) < lo16) continue;
-                const uint32_t kz = float_to_key(z[e]);
-                bool win = kz > e32c;
-                if (kz == e32c && ties_left > 0) {
+                for (int e = 0; e < kPer; ++e)
+                    if (is_candidate(z[e])) {
+                        c_raw[cpos] = __float_as_uint(z[e]);
+                        c_idx[cpos] = vi * kPer + e;
+                        ++cpos;
+                    }
+            });
+            fsync<NT>();
+        }
+    }
+    // ---- 5. the exact top-k (ties at the k-th logit to the lower index), left in ascending index ----------
+    int n = 0;
+    if (in_smem) {
+        // the candidates sit in shared memory in index order; thread t owns entries [i0, i1)
+        const int ipt = (n_c + NT - 1) / NT;  // <= kHeld
+        const int i0 = min(n_c, tid * ipt), i1 = min(n_c, i0 + ipt);
+        uint32_t winmask = 0;  // bit j: entry i0 + j is a winner
+        if (n_c <= k) {
+            winmask = (i1 - i0) >= 32 ? 0xffffffffu : ((1u << (i1 - i0)) - 1u);
+        } else if (n_c <= kRankListMax) {
+            // few candidates: count each one's rank under (logit descending, index ascending)
+            for (int i = tid; i < n_c; i += NT)
+                rkeys[i] = ((unsigned long long)float_to_key(__uint_as_float(c_raw[i])) << 32) |
+                           (unsigned long long)(0xffffffffu - (uint32_t)c_idx[i]);
+            fsync<NT>();
+            for (int i = i0; i < i1; ++i) {
+                const unsigned long long mine = rkeys[i];
+                int r = 0;
+                for (int j = 0; j < n_c; ++j) r += rkeys[j] > mine ? 1 : 0;
+                if (r < k) winmask |= 1u << (i - i0);
+            }
+        } else {
+            // many candidates: bisection on the 16-bit key between the bound and the row maximum,
+            // (fp32 rows) again on the low 16 bits inside the boundary value; ties by position
+            int above = 0;
+            const uint32_t base16 = (uint32_t)lo16;
+            const uint32_t e16 = base16 + bisect_kth<NT>((uint32_t)(max16 - lo16), k, [&](uint32_t d) {
+                int c = 0;
+                for (int i = i0; i < i1; ++i) c += ((float_to_key(__uint_as_float(c_raw[i])) >> 16) - base16) >= d ? 1 : 0;
+                return c;
+            }, sh->round_count + 16, tid, &above);
+            int need = k - above;
+            uint32_t e32;
+            if (kBf16) {
+                e32 = (e16 << 16) | ((e16 & 0x8000u) ? 0u : 0xffffu);  // keys of bf16 values: the low half follows the sign
+            } else {
+                int above2 = 0;
+                const uint32_t low = bisect_kth<NT>(0xffffu, need, [&](uint32_t d) {
+                    int c = 0;
+                    for (int i = i0; i < i1; ++i) {
+                        const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
+                        c += ((kz >> 16) == e16 && (kz & 0xffffu) >= d) ? 1 : 0;
+                    }
+                    return c;
+                }, sh->round_count + 32, tid, &above2);
+                e32 = (e16 << 16) | low;
+                need -= above2;
+            }
+            int c_eq = 0;
+            for (int i = i0; i < i1; ++i) c_eq += float_to_key(__uint_as_float(c_raw[i])) == e32 ? 1 : 0;
+            int tot_eq;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            int ties_left = max(0, min(c_eq, need - eq_before));
+            for (int i = i0; i < i1; ++i) {
+                const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
+                bool win = kz > e32;
+                if (kz == e32 && ties_left > 0) {
                     win = true;
                     --ties_left;
                 }
-                if (win && wpos < k) {
-                    win_raw[wpos] = __float_as_uint(z[e]);
-                    win_idx[wpos] = vi * kPer + e;
-                    ++wpos;
-                }
+                if (win) winmask |= 1u << (i - i0);
             }
-        });
-        n = min(tot_w, k);
-        __syncthreads();
+        }
+        // compact the winners in place: every thread reads its own first, then all write
+        uint32_t my_raw[kHeld];
+        int my_idx[kHeld];
+        int my_wins = 0;
+#pragma unroll
+        for (int j = 0; j < kHeld; ++j)
+            if ((winmask >> j) & 1u) {
+                my_raw[my_wins] = c_raw[i0 + j];
+                my_idx[my_wins] = c_idx[i0 + j];
+                ++my_wins;
+            }
+        int wpos = block_exscan<NT>(my_wins, tid, sh->iscr, &n);
+#pragma unroll
+        for (int j = 0; j < kHeld; ++j)
+            if (j < my_wins) {
+                c_raw[wpos + j] = my_raw[j];
+                c_idx[wpos + j] = my_idx[j];
+            }
+        fsync<NT>();
+    } else if (max16 >= lo16) {
+        // The survivors do not fit (thousands of tied tile maxima, or more candidates than the list
+        // holds): the same selection over the survivors' vectors, or all of the row's, in global
+        // memory: a histogram for the 16-bit key (fp32 rows: another for the low 16 bits), a count
+        // and a collecting pass.
+        auto key16_of = [](float z) -> int { return finite_key16(z); };
+        hist_select<T, NT>(rowp, ext, p.V, units, u0, u1, key16_of, lo16, max16, k, sh, hist, tid);
+        const int e16 = sh->sel_bin, above = sh->sel_above, total = sh->sel_total;
+        fsync<NT>();
+        uint32_t e32 = 0;   // key of the k-th largest logit (0: fewer than k finite logits, all of them win)
+        int need_ties = 0;  // how many logits equal to it are winners (the lowest indices)
+        if (e16 >= 0) {
+            if (kBf16) {
+                e32 = ((uint32_t)e16 << 16) | ((e16 & 0x8000) ? 0u : 0xffffu);
+                need_ties = k - above;
+            } else {
+                const uint32_t hi_bits = (uint32_t)e16;
+                auto low16_of = [hi_bits](float z) -> int {
+                    const uint32_t kz = float_to_key(z);
+                    return (kz >> 16) == hi_bits ? (int)(kz & 0xffffu) : -1;
+                };
+                hist_select<T, NT>(rowp, ext, p.V, units, u0, u1, low16_of, 0, 0xffff, k - above, sh, hist, tid);
+                const int low = sh->sel_bin, above2 = sh->sel_above;
+                fsync<NT>();
+                e32 = (hi_bits << 16) | (uint32_t)low;
+                need_ties = k - above - above2;
+            }
+        }
+        if (total > 0) {
+            int c_gt = 0, c_eq = 0;
+            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    if (!is_candidate(z[e])) continue;
+                    const uint32_t kz = float_to_key(z[e]);
+                    c_gt += kz > e32 ? 1 : 0;
+                    c_eq += kz == e32 ? 1 : 0;
+                }
+            });
+            int tot_eq, tot_w;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            const int my_ties = max(0, min(c_eq, need_ties - eq_before));
+            int wpos = block_exscan<NT>(c_gt + my_ties, tid, sh->iscr, &tot_w);
+            int ties_left = my_ties;
+            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    if (!is_candidate(z[e])) continue;
+                    const uint32_t kz = float_to_key(z[e]);
+                    bool win = kz > e32;
+                    if (kz == e32 && ties_left > 0) {
+                        win = true;
+                        --ties_left;
+                    }
+                    if (win && wpos < k) {
+                        c_raw[wpos] = __float_as_uint(z[e]);
+                        c_idx[wpos] = vi * kPer + e;
+                        ++wpos;
+                    }
+                }
+            });
+            n = min(tot_w, k);
+            fsync<NT>();
+        }
     }
-    n0 = n;
+    const int n0 = n;
+    uint32_t* win_raw = c_raw;
+    int* win_idx = c_idx;
     const double cf = (double)p.c.f;  // the scale the streaming sum used: keeps q consistent with the normaliser
     const double cd = p.c.d;
     double mass = 0.0;
     // ---- 6. top-rho cut ---------------------------------------------------------------------------------------
     if (n0 > 0 && p.top_p < 1.0f) {
         const int P = pow2_at_least(n0);
-        for (int i = tid; i < P; i += kFinishThreads)
+        for (int i = tid; i < P; i += NT)
             comp[i] = i < n0 ? (((unsigned long long)float_to_key(__uint_as_float(win_raw[i])) << 32) |
                                 (unsigned long long)(0xffffffffu - (uint32_t)win_idx[i])) : 0ull;
-        consumer_sync();
-        bitonic_sort<true>(comp, P, tid);
-        for (int i = tid; i < n0; i += kFinishThreads)
-            cum[i] = exp2((double)key_to_float((uint32_t)(comp[i] >> 32)) * cf - L2);
-        consumer_sync();
-        block_inclusive_scan(cum, n0, tid, sh->scratch);
+        fsync<NT>();
+        bitonic_sort_desc<NT>(comp, P, tid);
+        for (int i = tid; i < n0; i += NT) cum[i] = exp2((double)key_to_float((uint32_t)(comp[i] >> 32)) * cf - L2);
+        fsync<NT>();
+        block_inclusive_scan_f64<NT>(cum, n0, tid, sh->scratch);
         const double tp = (double)p.top_p;
         int lo = 0, hi = n0;
         while (lo < hi) {  // first n with c_n >= top_p
@@ -612,59 +859,59 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
         }
         n = lo < n0 ? lo + 1 : n0;
         mass = cum[n - 1];
-        consumer_sync();
+        fsync<NT>();
         if (n < n0) {
             // keep what precedes the cut in (logit descending, index ascending): a larger key, or the
             // cut's key and an index up to the cut's
             const unsigned long long cutc = comp[n - 1];
             const uint32_t ckey = (uint32_t)(cutc >> 32);
             const int cidx = (int)(0xffffffffu - (uint32_t)cutc);
-            const int ipt = (n0 + kFinishThreads - 1) / kFinishThreads;
+            const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
             const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
             uint32_t keep_raw[4];
             int keep_idx[4];
             int kept = 0;
-            for (int i = i0; i < i1; ++i) {  // ipt <= 4 (k <= 1024)
+            for (int i = i0; i < i1; ++i) {
                 const uint32_t kz = float_to_key(__uint_as_float(win_raw[i]));
-                if (kz > ckey || (kz == ckey && win_idx[i] <= cidx)) {
+                if (kept < 4 && (kz > ckey || (kz == ckey && win_idx[i] <= cidx))) {
                     keep_raw[kept] = win_raw[i];
                     keep_idx[kept] = win_idx[i];
                     ++kept;
                 }
             }
             int tot;
-            int kp = block_exscan(kept, tid, sh->iscr, &tot);  // (its barriers order the reads above before the writes below)
+            const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot);  // (its barriers order the reads above before the writes below)
 #pragma unroll
             for (int i = 0; i < 4; ++i)
                 if (i < kept) {
                     win_raw[kp + i] = keep_raw[i];
                     win_idx[kp + i] = keep_idx[i];
                 }
-            consumer_sync();
+            fsync<NT>();
         }
     }
     // ---- 7. renormalised truncated distribution in fp64, CDF, samples, outputs ----------------------------
     double my_max = -INFINITY;
-    for (int i = tid; i < n; i += kFinishThreads) {
+    for (int i = tid; i < n; i += NT) {
         const double y = (double)__uint_as_float(win_raw[i]) * cd;
         wv[i] = y;
         my_max = fmax(my_max, y);
     }
-    const double mS = block_max(my_max, tid, sh->scratch);
+    const double mS = block_max_f64<NT>(my_max, tid, sh->scratch);
     double my_mass = 0.0;
-    for (int i = tid; i < n; i += kFinishThreads) {
+    for (int i = tid; i < n; i += NT) {
         if (!(p.top_p < 1.0f)) my_mass += exp2((double)__uint_as_float(win_raw[i]) * cf - L2);
         const double w = exp2(wv[i] - mS);
         wv[i] = w;
         cum[i] = w;
     }
-    if (!(p.top_p < 1.0f)) mass = block_sum(my_mass, tid, sh->scratch);
-    else consumer_sync();
-    block_inclusive_scan(cum, n, tid, sh->scratch);
+    if (!(p.top_p < 1.0f)) mass = block_sum_f64<NT>(my_mass, tid, sh->scratch);
+    else fsync<NT>();
+    block_inclusive_scan_f64<NT>(cum, n, tid, sh->scratch);
 
     int* o_idx = p.idx + (size_t)row * k;
     float* o_logit = p.logit + (size_t)row * k;
-    for (int i = tid; i < k; i += kFinishThreads) {
+    for (int i = tid; i < k; i += NT) {
         o_idx[i] = i < n ? win_idx[i] : -1;
         o_logit[i] = i < n ? __uint_as_float(win_raw[i]) : -INFINITY;
     }
@@ -674,7 +921,7 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
         if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
     }
     const double W = n > 0 ? cum[n - 1] : 0.0;
-    for (int sidx = tid; sidx < p.num_samples; sidx += kFinishThreads) {
+    for (int sidx = tid; sidx < p.num_samples; sidx += NT) {
         int tok = -1;
         if (n > 0) {
             const float u = clamp_uniform(p.uniforms[(size_t)row * p.num_samples + sidx]);
@@ -698,7 +945,7 @@ __global__ void __launch_bounds__(kFinishThreads, 4) sparsify_finish_kernel(cons
 namespace tslt {
 
 struct SparsifyPlan {
-    int nchunks, group_log2, ngroups, tile_cap;
+    int nchunks, group_log2, ngroups, tile_cap, cand_cap, fin_threads;
     RowSplit split;
     size_t fin_smem;
     size_t ws_ready_off, ws_stats_off, ws_tiles_off, ws_bytes;
@@ -729,7 +976,9 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.group_log2 = glog;
     pl.ngroups = (int)((ntiles + (1LL << glog) - 1) >> glog);
     pl.tile_cap = 8 * k < 512 ? 512 : (8 * k > kMaxTileList ? kMaxTileList : 8 * k);
-    pl.fin_smem = sparsify_finish_smem(pl.ngroups, pl.tile_cap, k);
+    pl.cand_cap = 2 * k < 512 ? 512 : (2 * k > 2048 ? 2048 : 2 * k);
+    pl.fin_threads = finish_threads(k);
+    pl.fin_smem = finish_layout(pl.ngroups, pl.tile_cap, pl.cand_cap, k, pl.nchunks).total;
     // One CTA per row when the rows fill the machine; fewer rows are cut into segments (at least one
     // chunk per warp each) so that every CTA slot has work.  A segment costs nothing but its own
     // hand-over (8 (max, sum) pairs and a flag).
@@ -765,6 +1014,21 @@ ScaleC make_scale(float temperature) {
     s.f = (float)c;
     s.d = c;
     return s;
+}
+
+// Largest k and long rows take the finish kernel's shared memory past the default 48 KB: the kernel's
+// limit is raised once per device (slot: one per kernel instantiation), not on every call.
+constexpr size_t kFinishSmemLimit = 96 * 1024;
+static bool raise_smem_limit_once(void (*kern)(const SparsifyParams), int slot) {
+    constexpr int kMaxDevices = 64;
+    static bool done[6][kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    if (cached && done[slot][dev]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemLimit) != cudaSuccess) return false;
+    if (cached) done[slot][dev] = true;
+    return true;
 }
 
 // Polls of a ready flag before a finish CTA gives up on it (about a second at 200 ns per poll).
@@ -822,7 +1086,7 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.uniforms = uniforms;
     p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
     p.nchunks = pl.nchunks; p.split = pl.split;
-    p.group_log2 = pl.group_log2; p.ngroups = pl.ngroups; p.tile_cap = pl.tile_cap;
+    p.group_log2 = pl.group_log2; p.ngroups = pl.ngroups; p.tile_cap = pl.tile_cap; p.cand_cap = pl.cand_cap;
     p.poll_limit = g_sparsify_poll_limit;
     unsigned char* ws = (unsigned char*)workspace;
     p.status = (int*)ws;
@@ -834,9 +1098,14 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     if (dtype == TSLT_F32) sparsify_stream_kernel<float><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
     else sparsify_stream_kernel<bf16_t><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
-    auto fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float> : sparsify_finish_kernel<bf16_t>;
-    static_assert(kFinishHeaderBytes + kSelBins * 4 + kMaxGroups * 4 + TSLT_MAX_K * 16 + TSLT_MAX_K * 8 <= 48 * 1024,
-                  "the finish kernel's shared memory stays under the default limit");
-    if (launch_dependent(fin, rows, kFinishThreads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
+    void (*fin)(const SparsifyParams);
+    if (pl.fin_threads == 64) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 64> : sparsify_finish_kernel<bf16_t, 64>;
+    else if (pl.fin_threads == 128) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 128> : sparsify_finish_kernel<bf16_t, 128>;
+    else fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 256> : sparsify_finish_kernel<bf16_t, 256>;
+    if (pl.fin_smem > kFinishSmemLimit) return TSLT_ERR_UNSUPPORTED;  // (rows of tens of millions of logits: the line maxima no longer fit)
+    if (pl.fin_smem > 48 * 1024 &&
+        !raise_smem_limit_once(fin, (pl.fin_threads == 64 ? 0 : pl.fin_threads == 128 ? 2 : 4) + (dtype == TSLT_F32 ? 0 : 1)))
+        return TSLT_ERR_CUDA;
+    if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }

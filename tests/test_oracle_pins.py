@@ -649,3 +649,31 @@ def test_argument_errors():
     for k, top_p, T in [(0, 1.0, 1.0), (9, 1.0, 1.0), (2, 0.0, 1.0), (2, 1.0, 0.0)]:
         with pytest.raises(ValueError):
             oracle.sparsify(z, k, top_p, T, u)
+
+
+def test_degenerate_residual_falls_back_to_the_target():
+    """The one branch exact arithmetic never reaches from a well-formed round: the residual mass is
+    zero.  Built by hand: the target equals the truncated draft on S (p = q~ there, -inf elsewhere)
+    and the drafted token lies outside S, so it is rejected whatever the uniform (p(x) = 0) and
+    max(0, p - q~) vanishes everywhere.  The oracle must flag DEGEN and sample the unmodified p by
+    the usual inverse CDF (brute force below)."""
+    V, k = 8, 3
+    S = np.array([1, 3, 5], np.int32)
+    lg = np.array([0.5, 1.25, -0.75], np.float32)          # exactly representable: p == q~ bit for bit
+    zp = np.full((1, 2, V), -np.inf, np.float32)
+    zp[0, 0, S] = lg
+    zp[0, 1] = np.arange(V, dtype=np.float32)               # bonus row, unused
+    idx, logit, count = S[None, None, :], lg[None, None, :], np.array([[k]], np.int32)
+    p = softmax64(lg)
+    cdf = np.cumsum(p)
+    for u in (0.0, 0.3, float(cdf[0]) + 1e-3, 0.999):
+        o = oracle.verify(zp, idx, logit, count, np.array([[0]], np.int32), 1.0, 1.0,
+                          np.array([[0.0]], np.float32), np.array([u], np.float32), want_dense=True)
+        assert o["accepted_len"][0] == 0 and o["accept_prob"][0, 0] == 0.0
+        assert o["flags"][0] & oracle.FLAG_DEGEN
+        assert o["out_token"][0] == S[int(np.searchsorted(cdf, u, side="right"))]
+        assert np.allclose(o["final_pmf"][0, S], p, atol=1e-15) and o["final_pmf"][0].sum() == pytest.approx(1.0)
+    # the same payload with a token inside S is an ordinary round: accepted with probability 1, no flag
+    o = oracle.verify(zp, idx, logit, count, np.array([[3]], np.int32), 1.0, 1.0,
+                      np.array([[0.5]], np.float32), np.array([0.5], np.float32))
+    assert o["accepted_len"][0] == 1 and not (o["flags"][0] & oracle.FLAG_DEGEN)
