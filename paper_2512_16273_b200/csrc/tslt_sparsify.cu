@@ -167,18 +167,19 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
 }
 
 // ---- finish kernel ---------------------------------------------------------------------------------
-// NT threads per row: 64 (k <= 64), 128 (k <= 128) or 256.  Finishing a row is a chain of dependent
-// steps (trips to L2 / HBM, bisection rounds, prefix sums), so what it costs machine-wide is the
-// chain's length times the number of waves: small CTAs keep every row of a large batch resident at
-// once (14 CTAs of 64 threads per SM hold 2048 rows on 148 SMs).
+// NT threads per row: 128 (k <= 128) or 256.  Finishing a row is a chain of dependent steps (trips
+// to L2 / HBM, bisection rounds, prefix sums), and most finish CTAs of a large batch only find room
+// on an SM once the streaming kernel's last wave drains, so what the finish costs is the chain's
+// length times the number of waves left then: the chain is kept to three trips to memory (the
+// hand-over, the survivors' vectors, the outputs).
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) / 16 * 16; }
 __host__ __device__ inline int pow2_at_least(int n) {
     int p = 1;
     while (p < n) p <<= 1;
     return p;
 }
-__host__ __device__ constexpr int finish_threads(int k) { return k <= 64 ? 64 : k <= 128 ? 128 : 256; }
-__host__ __device__ constexpr int finish_resident(int nt) { return nt == 64 ? 14 : nt == 128 ? 8 : 4; }
+__host__ __device__ constexpr int finish_threads(int k) { return k <= 128 ? 128 : 256; }
+__host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
 constexpr int kFinishHeaderBytes = 512;
 constexpr int kRankListMax = 512;  // candidates up to which the k-th is found by counting ranks
 
@@ -207,11 +208,22 @@ __host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap,
 struct FinishShared {
     double scratch[16];
     double lrow;  // base-2 log of the row's softmax normaliser
-    int round_count[48];  // one counter per bisection round: three bisections of at most 16 rounds
     int iscr[16];
     int sel_bin, sel_above, sel_eq, sel_total;
-    int ready, gmin, gmax;
+    int ready, gmax;
 };
+
+// Atomics on shared memory through the shared-space address: a generic-address atomic that happens to
+// hit shared memory is several times slower, and the compiler cannot always tell.
+__device__ __forceinline__ void smem_add(void* p, uint32_t v) {
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ void smem_max(void* p, uint32_t v) {
+    asm volatile("red.shared.max.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ void smem_min(void* p, uint32_t v) {
+    asm volatile("red.shared.min.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
 
 template <int NT> __device__ __forceinline__ void fsync() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); }
 
@@ -315,30 +327,59 @@ template <int NT> __device__ __forceinline__ void bitonic_sort_desc(unsigned lon
     }
 }
 
-// The largest d in [0, range] such that at least kk of the thread block's values are >= d, given
-// that at least kk are >= 0: bisection on the bits of d, one barrier per bit that needs a count.
-// count_ge(d) returns how many of THIS thread's values are >= d.  *above gets the number of values
-// > the result.  counters: one zeroed int per round (at most 32), consumed here.
-template <int NT, typename CountGe>
-__device__ __forceinline__ uint32_t bisect_kth(uint32_t range, int kk, CountGe count_ge, int* counters, int tid, int* above) {
-    uint32_t d = 0;
-    int last_rejected = 0, round = 0;
-    for (int bit = 31 - __clz((int)(range | 1u)); bit >= 0; --bit) {
-        const uint32_t cand = d | (1u << bit);
-        if (cand > range) {  // nothing lies above the range: rejected without counting
-            last_rejected = 0;
-            continue;
-        }
-        const int cnt = __reduce_add_sync(0xffffffffu, count_ge(cand));
-        if ((tid & 31) == 0 && cnt) atomicAdd(&counters[round], cnt);
+// The kk-th largest of the thread block's 16-bit values (at least kk of them exist), by two histogram
+// passes of 256 bins: the high byte, then the low byte among the values that share it.  A bisection
+// on the value's bits would take one barrier per bit, and the keys of logits that straddle zero
+// differ in nearly all sixteen.  for_each(f) calls f(v) for every value v of THIS thread.  *above
+// gets the number of values larger than the result.  hist: 256 words of shared memory.
+template <int NT, typename ForEach>
+__device__ __forceinline__ uint32_t radix_kth16(int kk, ForEach for_each, uint32_t* hist, FinishShared* sh, int tid, int* above) {
+    uint32_t prefix = 0;
+    int above_acc = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int i = tid; i < 256; i += NT) hist[i] = 0u;
         fsync<NT>();
-        const int total = counters[round];
-        ++round;
-        if (total >= kk) d = cand;
-        else last_rejected = total;
+        if (pass == 0) for_each([&](uint32_t v) { smem_add(&hist[v >> 8], 1u); });
+        else for_each([&](uint32_t v) { if ((v >> 8) == prefix) smem_add(&hist[v & 255u], 1u); });
+        fsync<NT>();
+        if (tid < 32) {
+            // rows of 32 bins from the top; lane l takes bin top - l of the row
+            uint32_t carried = 0;
+            int found_bin = 0;
+            uint32_t found_above = 0;
+            bool found = false;
+            for (int top = 255; top >= 0; top -= 32) {
+                const uint32_t cnt = hist[top - tid];
+                uint32_t incl = cnt;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (tid >= o) incl += t;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, carried + incl >= (uint32_t)kk);
+                if (hit) {
+                    const int l = __ffs(hit) - 1;
+                    found_bin = top - l;
+                    found_above = carried + __shfl_sync(0xffffffffu, incl - cnt, l);
+                    found = true;
+                    break;
+                }
+                carried += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (tid == 0) {
+                sh->sel_bin = found ? found_bin : 0;
+                sh->sel_above = found ? (int)found_above : 0;
+            }
+        }
+        fsync<NT>();
+        const int bin = sh->sel_bin, ab = sh->sel_above;
+        above_acc += ab;
+        kk -= ab;
+        prefix = pass == 0 ? (uint32_t)bin : ((prefix << 8) | (uint32_t)bin);
     }
-    *above = last_rejected;
-    return d;
+    *above = above_acc;
+    return prefix;
 }
 
 // The vectors a thread works on: units [u0, u1) of the row's survivor tiles (tl: their tile numbers in
@@ -396,14 +437,14 @@ __device__ __forceinline__ void hist_select(const unsigned char* rowp, const Row
                 if (v >= lo && v <= hi) {
                     const int b = (v - lo) >> s;
                     if (b != cur) {  // equal neighbours (ties) cost one atomic, not one each
-                        if (run) atomicAdd(&hist[cur], run);
+                        if (run) smem_add(&hist[cur], run);
                         cur = b;
                         run = 0;
                     }
                     ++run;
                 }
             }
-            if (run) atomicAdd(&hist[cur], run);
+            if (run) smem_add(&hist[cur], run);
         });
         fsync<NT>();
         if (tid < 32) {
@@ -505,6 +546,13 @@ __device__ __forceinline__ uint32_t line_group_maxima(const uint32_t (&w)[16], i
 // ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the line).
 __device__ __forceinline__ uint32_t line_survivors(const uint32_t (&w)[16], uint32_t bound) {
     uint32_t m = 0;
+    {   // most lines hold no survivor: their maximum settles it
+        uint32_t t = bf16x2_max(bf16x2_max(bf16x2_max(w[0], w[1]), bf16x2_max(w[2], w[3])),
+                                bf16x2_max(bf16x2_max(w[4], w[5]), bf16x2_max(w[6], w[7])));
+        t = bf16x2_max(t, bf16x2_max(bf16x2_max(bf16x2_max(w[8], w[9]), bf16x2_max(w[10], w[11])),
+                                     bf16x2_max(bf16x2_max(w[12], w[13]), bf16x2_max(w[14], w[15]))));
+        if (raw16_to_key16(half_max(t)) < bound) return 0u;
+    }
 #pragma unroll
     for (int a = 0; a < kTilesPerChunk; ++a) {
         const int slot = ((a & 7) << 2) | (a >> 3);
@@ -548,11 +596,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     const RowExtent ext = row_extent<T>(p.V);
     if (tid == 0 && p.num_samples > 0)  // the uniforms are needed last: ask for their cache line now
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
-    if (tid < 48) sh->round_count[tid] = 0;
-    if (tid == 0) {
-        sh->gmin = 0xffff;
-        sh->gmax = 0;
-    }
+    if (tid == 0) sh->gmax = 0;
     const int glog = p.group_log2, ngroups = p.ngroups;
     if (glog > 5)
         for (int i = tid; i < ngroups; i += NT) gm[i] = 0u;
@@ -574,17 +618,31 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     fsync<NT>();
     // ---- the row's log-normaliser, by one warp (fp64 is scarce) -------------------------------------
     if (warp == 1) {
+        // every (max, sum) pair is asked for before any is used: one trip to memory
         const SegStat* st = p.seg_stats + (size_t)row * nseg;
-        double Mall = -INFINITY;
-        for (int i = lane; i < nseg * kWarps; i += 32)
-            if (__ldcg(&st[i / kWarps].S[i % kWarps]) > 0.0) Mall = fmax(Mall, (double)__ldcg(&st[i / kWarps].M[i % kWarps]));
-        Mall = warp_max(Mall);
-        double Sall = 0.0;
-        for (int i = lane; i < nseg * kWarps; i += 32) {
-            const double Sw = __ldcg(&st[i / kWarps].S[i % kWarps]);
-            if (Sw > 0.0) Sall += Sw * exp2((double)__ldcg(&st[i / kWarps].M[i % kWarps]) - Mall);
+        constexpr int kPairs = 4;  // per lane and round: 128 pairs = 16 segments a round
+        double Mall = -INFINITY, Sall = 0.0;
+        for (int base = 0; base < nseg * kWarps; base += 32 * kPairs) {
+            double Sw[kPairs], Mw[kPairs];
+#pragma unroll
+            for (int j = 0; j < kPairs; ++j) {
+                const int i = base + j * 32 + lane;
+                const bool in = i < nseg * kWarps;
+                Sw[j] = in ? __ldcg(&st[i / kWarps].S[i % kWarps]) : 0.0;
+                Mw[j] = in ? (double)__ldcg(&st[i / kWarps].M[i % kWarps]) : -INFINITY;
+            }
+            double Mnew = Mall;
+#pragma unroll
+            for (int j = 0; j < kPairs; ++j)
+                if (Sw[j] > 0.0) Mnew = fmax(Mnew, Mw[j]);
+            Mnew = warp_max(Mnew);
+            double add = 0.0;
+#pragma unroll
+            for (int j = 0; j < kPairs; ++j)
+                if (Sw[j] > 0.0) add += Sw[j] * exp2(Mw[j] - Mnew);
+            Sall = (Sall > 0.0 ? Sall * exp2(Mall - Mnew) : 0.0) + warp_sum(add);
+            Mall = Mnew;
         }
-        Sall = warp_sum(Sall);
         if (lane == 0) sh->lrow = Sall > 0.0 ? Mall + log2(Sall) : -INFINITY;
     }
     // ---- 1. group maxima of the tile maxima; each line's maximum is kept for step 3 -------------------
@@ -592,64 +650,102 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     const unsigned short* tmax = p.tile_max + (size_t)row * nchunks * kTilesPerChunk;
     const int cpt = (nchunks + NT - 1) / NT;
     const int ch0 = min(nchunks, tid * cpt), ch1 = min(nchunks, ch0 + cpt);
-    for (int ch = ch0; ch < ch1; ++ch) {
-        uint32_t w[16];
-        load_line(tmax + ch * kTilesPerChunk, w);
-        const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
-        if (glog > 5) atomicMax(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
-        lmax[ch] = (unsigned short)lm;
+    // up to kKeep lines stay in registers for step 3 (rows up to kKeep * NT chunks: 512 KB with
+    // 128 threads); longer rows read their lines again there
+    constexpr int kKeep = 2;
+    uint32_t kept[kKeep][16];
+    const bool keep_lines = cpt <= kKeep;
+#pragma unroll
+    for (int j = 0; j < kKeep; ++j) {
+        const int ch = ch0 + j;
+        if (keep_lines && ch < ch1) {
+            load_line(tmax + ch * kTilesPerChunk, kept[j]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) kept[j][i] = 0xff80ff80u;  // -inf: never a survivor
+        }
+    }
+    if (keep_lines) {
+#pragma unroll
+        for (int j = 0; j < kKeep; ++j) {
+            const int ch = ch0 + j;
+            if (ch < ch1) {
+                const uint32_t lm = line_group_maxima(kept[j], glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+                if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
+                lmax[ch] = (unsigned short)lm;
+            }
+        }
+    } else {
+        for (int ch = ch0; ch < ch1; ++ch) {
+            uint32_t w[16];
+            load_line(tmax + ch * kTilesPerChunk, w);
+            const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+            if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
+            lmax[ch] = (unsigned short)lm;
+        }
     }
     fsync<NT>();
     {
-        uint32_t mn = 0xffffu, mx = 0u;
-        for (int i = tid; i < ngroups; i += NT) {
-            const uint32_t v = gm[i];
-            mn = min(mn, v);
-            mx = max(mx, v);
-        }
-        mn = __reduce_min_sync(0xffffffffu, mn);
+        uint32_t mx = 0u;
+        for (int i = tid; i < ngroups; i += NT) mx = max(mx, gm[i]);
         mx = __reduce_max_sync(0xffffffffu, mx);
-        if (lane == 0) {
-            atomicMin(&sh->gmin, (int)mn);
-            atomicMax(&sh->gmax, (int)mx);
-        }
+        if (lane == 0) smem_max(&sh->gmax, mx);
     }
     fsync<NT>();
-    const uint32_t gmin = (uint32_t)sh->gmin, gmax = (uint32_t)sh->gmax;
+    const uint32_t gmax = (uint32_t)sh->gmax;
     const int max16 = min((int)gmax, (int)kHighestFinite16);
     const double L2 = sh->lrow;
     // ---- 2. the k-th largest group maximum: a lower bound on the k-th largest logit's key ---------------
     uint32_t bound = 0;
     if (ngroups >= k) {
         int unused;
-        bound = gmin + bisect_kth<NT>(gmax - gmin, k, [&](uint32_t d) {
-            int c = 0;
-            for (int i = tid; i < ngroups; i += NT) c += (gm[i] - gmin) >= d ? 1 : 0;
-            return c;
-        }, sh->round_count, tid, &unused);
+        bound = radix_kth16<NT>(k, [&](auto f) {
+            for (int i = tid; i < ngroups; i += NT) f(gm[i]);
+        }, hist, sh, tid, &unused);
     }
     int lo16 = max((int)bound, (int)kLowestFinite16);
     // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
     int my_surv = 0;
-    for (int ch = ch0; ch < ch1; ++ch) {
-        if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
-        uint32_t w[16];
-        load_line(tmax + ch * kTilesPerChunk, w);
-        my_surv += __popc(line_survivors(w, (uint32_t)lo16));
+    uint32_t kept_mask[kKeep];
+    if (keep_lines) {
+#pragma unroll
+        for (int j = 0; j < kKeep; ++j) {
+            kept_mask[j] = line_survivors(kept[j], (uint32_t)lo16);  // bit a: tile a of the chunk (none beyond the row)
+            my_surv += __popc(kept_mask[j]);
+        }
+    } else {
+        for (int ch = ch0; ch < ch1; ++ch) {
+            if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+            uint32_t w[16];
+            load_line(tmax + ch * kTilesPerChunk, w);
+            my_surv += __popc(line_survivors(w, (uint32_t)lo16));
+        }
     }
     int n_surv;
     int pos = block_exscan<NT>(my_surv, tid, sh->iscr, &n_surv);
     const bool listed = n_surv <= p.tile_cap;
     if (listed) {
-        for (int ch = ch0; ch < ch1; ++ch) {
-            if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
-            uint32_t w[16];
-            load_line(tmax + ch * kTilesPerChunk, w);
-            uint32_t m = line_survivors(w, (uint32_t)lo16);  // bit a: tile a of the chunk
-            while (m) {
-                const int a = __ffs(m) - 1;
-                m &= m - 1;
-                tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
+        if (keep_lines) {
+#pragma unroll
+            for (int j = 0; j < kKeep; ++j) {
+                uint32_t m = kept_mask[j];
+                while (m) {
+                    const int a = __ffs(m) - 1;
+                    m &= m - 1;
+                    tl[pos++] = (uint32_t)((ch0 + j) * kTilesPerChunk + a);
+                }
+            }
+        } else {
+            for (int ch = ch0; ch < ch1; ++ch) {
+                if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+                uint32_t w[16];
+                load_line(tmax + ch * kTilesPerChunk, w);
+                uint32_t m = line_survivors(w, (uint32_t)lo16);
+                while (m) {
+                    const int a = __ffs(m) - 1;
+                    m &= m - 1;
+                    tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
+                }
             }
         }
     }
@@ -667,24 +763,70 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     bool in_smem = false;
     int n_c = 0;
     if (listed && max16 >= lo16) {
-        int cnt = 0;
-        for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
+        constexpr int kRegVecs = 4;
+        if (upt <= kRegVecs) {
+            // few vectors per thread (small k): one trip to memory, the vectors wait in registers
+            // while the prefix sum finds where their candidates go
+            uint4 d[kRegVecs];
+            int vi[kRegVecs];
 #pragma unroll
-            for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
-        });
-        int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
-        if (n_c <= p.cand_cap) {
-            in_smem = true;
-            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+            for (int j = 0; j < kRegVecs; ++j) {
+                const int u = u0 + j;
+                vi[j] = u < u1 ? (int)(tl[u >> 2] * (uint32_t)kVecsPerTile) + (u & 3) : -1;
+                if (vi[j] >= 0 && vi[j] < ext.nvec_full) d[j] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[j]);
+            }
+            int cnt = 0;
 #pragma unroll
-                for (int e = 0; e < kPer; ++e)
-                    if (is_candidate(z[e])) {
-                        c_raw[cpos] = __float_as_uint(z[e]);
-                        c_idx[cpos] = vi * kPer + e;
-                        ++cpos;
-                    }
+            for (int j = 0; j < kRegVecs; ++j) {
+                if (vi[j] < 0) continue;
+                float z[kPer];
+                if (vi[j] < ext.nvec_full) {
+                    unpack_vec<T>(d[j], z);
+                } else {  // the row's ragged last vector: fetched element by element, kept in the same form
+                    load_row_vector<T>(rowp, vi[j], ext, p.V, z);
+                    d[j] = pack_vec<T>(z);
+                }
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
+            }
+            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+            if (n_c <= p.cand_cap) {
+                in_smem = true;
+#pragma unroll
+                for (int j = 0; j < kRegVecs; ++j) {
+                    if (vi[j] < 0) continue;
+                    float z[kPer];
+                    unpack_vec<T>(d[j], z);
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e)
+                        if (is_candidate(z[e])) {
+                            c_raw[cpos] = __float_as_uint(z[e]);
+                            c_idx[cpos] = vi[j] * kPer + e;
+                            ++cpos;
+                        }
+                }
+                fsync<NT>();
+            }
+        } else {
+            int cnt = 0;
+            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
             });
-            fsync<NT>();
+            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+            if (n_c <= p.cand_cap) {
+                in_smem = true;
+                for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e)
+                        if (is_candidate(z[e])) {
+                            c_raw[cpos] = __float_as_uint(z[e]);
+                            c_idx[cpos] = vi * kPer + e;
+                            ++cpos;
+                        }
+                });
+                fsync<NT>();
+            }
         }
     }
     // ---- 5. the exact top-k (ties at the k-th logit to the lower index), left in ascending index ----------
@@ -709,29 +851,24 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
                 if (r < k) winmask |= 1u << (i - i0);
             }
         } else {
-            // many candidates: bisection on the 16-bit key between the bound and the row maximum,
-            // (fp32 rows) again on the low 16 bits inside the boundary value; ties by position
+            // many candidates: the k-th largest 16-bit key by two histogram passes, (fp32 rows) the low
+            // 16 bits inside that key the same way; ties by position
             int above = 0;
-            const uint32_t base16 = (uint32_t)lo16;
-            const uint32_t e16 = base16 + bisect_kth<NT>((uint32_t)(max16 - lo16), k, [&](uint32_t d) {
-                int c = 0;
-                for (int i = i0; i < i1; ++i) c += ((float_to_key(__uint_as_float(c_raw[i])) >> 16) - base16) >= d ? 1 : 0;
-                return c;
-            }, sh->round_count + 16, tid, &above);
+            const uint32_t e16 = radix_kth16<NT>(k, [&](auto f) {
+                for (int i = i0; i < i1; ++i) f(float_to_key(__uint_as_float(c_raw[i])) >> 16);
+            }, hist, sh, tid, &above);
             int need = k - above;
             uint32_t e32;
             if (kBf16) {
                 e32 = (e16 << 16) | ((e16 & 0x8000u) ? 0u : 0xffffu);  // keys of bf16 values: the low half follows the sign
             } else {
                 int above2 = 0;
-                const uint32_t low = bisect_kth<NT>(0xffffu, need, [&](uint32_t d) {
-                    int c = 0;
+                const uint32_t low = radix_kth16<NT>(need, [&](auto f) {
                     for (int i = i0; i < i1; ++i) {
                         const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
-                        c += ((kz >> 16) == e16 && (kz & 0xffffu) >= d) ? 1 : 0;
+                        if ((kz >> 16) == e16) f(kz & 0xffffu);
                     }
-                    return c;
-                }, sh->round_count + 32, tid, &above2);
+                }, hist, sh, tid, &above2);
                 e32 = (e16 << 16) | low;
                 need -= above2;
             }
@@ -1095,16 +1232,19 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.tile_max = (unsigned short*)(ws + pl.ws_tiles_off);
 
     cudaStream_t st = (cudaStream_t)stream;
+    if (!(dtype == TSLT_F32 ? prefer_shared_carveout_once(sparsify_stream_kernel<float>, 0)
+                            : prefer_shared_carveout_once(sparsify_stream_kernel<bf16_t>, 1)))
+        return TSLT_ERR_CUDA;
     if (dtype == TSLT_F32) sparsify_stream_kernel<float><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
     else sparsify_stream_kernel<bf16_t><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     void (*fin)(const SparsifyParams);
-    if (pl.fin_threads == 64) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 64> : sparsify_finish_kernel<bf16_t, 64>;
-    else if (pl.fin_threads == 128) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 128> : sparsify_finish_kernel<bf16_t, 128>;
+    if (pl.fin_threads == 128) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 128> : sparsify_finish_kernel<bf16_t, 128>;
     else fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 256> : sparsify_finish_kernel<bf16_t, 256>;
+    if (!prefer_shared_carveout_once(fin, 2 + (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1))) return TSLT_ERR_CUDA;
     if (pl.fin_smem > kFinishSmemLimit) return TSLT_ERR_UNSUPPORTED;  // (rows of tens of millions of logits: the line maxima no longer fit)
     if (pl.fin_smem > 48 * 1024 &&
-        !raise_smem_limit_once(fin, (pl.fin_threads == 64 ? 0 : pl.fin_threads == 128 ? 2 : 4) + (dtype == TSLT_F32 ? 0 : 1)))
+        !raise_smem_limit_once(fin, (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1)))
         return TSLT_ERR_CUDA;
     if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;

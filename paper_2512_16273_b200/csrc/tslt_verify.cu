@@ -672,6 +672,10 @@ template <bool kTree>
 static int launch_verify(VerifyParams& p, const VerifyPlan& pl, int dtype, cudaStream_t st) {
     auto resolve = dtype == TSLT_F32 ? verify_resolve_kernel<float, kTree> : verify_resolve_kernel<bf16_t, kTree>;
     if (!raise_smem_limit_once(resolve, (kTree ? 2 : 0) + (dtype == TSLT_F32 ? 0 : 1), pl.smem)) return TSLT_ERR_CUDA;
+    if (!prefer_shared_carveout_once(resolve, 8 + (kTree ? 2 : 0) + (dtype == TSLT_F32 ? 0 : 1))) return TSLT_ERR_CUDA;
+    if (!(dtype == TSLT_F32 ? prefer_shared_carveout_once(verify_stream_kernel<float>, 12)
+                            : prefer_shared_carveout_once(verify_stream_kernel<bf16_t>, 13)))
+        return TSLT_ERR_CUDA;
     if (dtype == TSLT_F32) verify_stream_kernel<float><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     else verify_stream_kernel<bf16_t><<<(unsigned)pl.split.grid, kBlockThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
