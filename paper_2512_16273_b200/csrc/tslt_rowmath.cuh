@@ -55,12 +55,13 @@ struct LaneSum {
         M = -3.0e38f;
     }
     // Before a lane tile whose largest logit is lm is added: move the reference to lm's exponent if
-    // that exceeds it by more than the slack.  Branch-free on purpose: the scale is exactly 1 when
-    // nothing moves, and the compiler turns a rarely taken branch here into a longer chain of
-    // selects executed on every step.
+    // that exceeds it by more than the slack.  Called by all lanes of a warp; the rescaling is
+    // skipped by the whole warp unless some lane needs it (a handful of times per row), which a
+    // per-lane branch would not achieve: the compiler turns it into selects executed on every step.
     __device__ __forceinline__ void raise_to(float lm, float c) {
         const float Mn = lm * c;
         const bool up = Mn - M > kRaiseSlack;
+        if (!__any_sync(0xffffffffu, up)) return;
         const float sc = up ? ex2_approx(M - Mn) : 1.0f;
         const float2 sc2 = make_float2(sc, sc);
 #pragma unroll

@@ -36,18 +36,24 @@ namespace tslt {
 
 constexpr int kTilesPerChunk = 32;        // 64-byte tiles in a 2 KB chunk
 constexpr int kVecsPerTile = 4;           // 16-byte vectors in a tile
-constexpr int kSparsifyStreamCtasPerSm = 6;
+constexpr int kSparsifyStreamCtasPerSm = 5;  // 51 registers, no spills (6 CTAs of 40 registers spill and run 8 % slower)
 constexpr int kMaxGroups = 4096;          // group maxima the finish kernel bisects over
 constexpr int kMaxTileList = 4096;        // survivor tiles it can list
 constexpr int kSelBins = 1024;            // bins of the selection histogram
 constexpr uint32_t kLowestFinite16 = 0x0080u;   // key of -FLT_MAX >> 16
 constexpr uint32_t kHighestFinite16 = 0xff7fu;  // key of +FLT_MAX >> 16
 
-// What a segment hands over besides its tile maxima: one (max, sum) pair per warp.
+// What a segment hands over besides its tile maxima or its survivor list: one (max, sum) pair per
+// warp and, from a segment that is a whole row, the outcome of its own selection.
 struct SegStat {
     double S[kWarps];  // sum of 2^(y - M) over the warp's chunks of the segment
     float M[kWarps];   // the warp's reference exponent (base 2)
+    int n_list;        // survivor tiles listed (-1: they did not fit the list)
+    int bound16;       // 16-bit key at or below the row's k-th largest logit's (0: none)
+    int max16;         // 16-bit key of the row's largest tile maximum
+    int pad[5];
 };
+static_assert(sizeof(SegStat) == 128, "one record per 128 bytes");
 
 struct SparsifyParams {
     const unsigned char* logits;
@@ -73,7 +79,9 @@ struct SparsifyParams {
     int* status;
     int* seg_ready;           // [rows * nseg]
     SegStat* seg_stats;       // [rows * nseg]
-    unsigned short* tile_max; // [rows, nchunks * 32]: top 16 bits of each tile's largest logit, slot order (see tile_slot)
+    unsigned short* tile_max; // rows cut into segments: [rows, nchunks * 32], top 16 bits of each tile's largest logit, slot order
+    uint32_t* row_list;       // whole-row CTAs: [rows, tile_cap] survivor tiles in address order
+    int local_bound;          // 1: each row is one streaming CTA, which finds the bound and lists the survivors itself
 };
 
 // Tile a of a row is its bytes [64 a, 64 a + 64).  In the streaming kernel vector j * 32 + l of a
@@ -88,130 +96,6 @@ __device__ __forceinline__ uint32_t raw16_to_key16(uint32_t r) {
     r = (r == 0x8000u) ? 0u : r;
     return (r & 0x8000u) ? (~r & 0xffffu) : (r | 0x8000u);
 }
-
-// ---- streaming kernel ------------------------------------------------------------------------------
-template <typename T> struct QuadMax;
-template <> struct QuadMax<bf16_t> {
-    // top 16 bits of the largest logit of each of the quad's four tiles, packed (j = 0, 1 | 2, 3)
-    static __device__ __forceinline__ uint2 keys(const LaneTile<bf16_t>& lt) {
-        uint32_t r[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t v = lt.vm[j];
-            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 1));
-            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 2));
-            r[j] = bf16x2_max(v, v >> 16) & 0xffffu;
-        }
-        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
-    }
-};
-template <> struct QuadMax<float> {
-    static __device__ __forceinline__ uint2 keys(const LaneTile<float>& lt) {
-        uint32_t r[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float v = lt.vm[j];
-            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
-            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
-            r[j] = __float_as_uint(v) >> 16;
-        }
-        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
-    }
-};
-
-template <typename T>
-__global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) sparsify_stream_kernel(const SparsifyParams p) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
-    const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
-    const RowExtent ext = row_extent<T>(p.V);
-    const float c = p.c.f;
-    const unsigned char* lane_rowp = rowp + lane * kVecBytes;
-    int ch = wk.chunk_begin + warp;
-    LaneTile<T> lt;
-    if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);  // in flight during the set-up below
-    // The segment's ready flag is cleared here, by the CTA that will set it, and the store is fenced
-    // before the barrier after which this CTA lets the finish kernel be scheduled.  A finish CTA
-    // runs only after every streaming CTA has passed that point, so it never sees a flag (or a
-    // status word) left by an earlier call, and the workspace needs no clearing between calls.
-    if (tid == 0) {
-        *(volatile int*)&p.seg_ready[blockIdx.x] = 0;
-        if (blockIdx.x == 0) *(volatile int*)p.status = 0;
-        __threadfence();
-    }
-    __syncthreads();
-    allow_dependent_launch();
-
-    LaneSum ls;
-    ls.reset();
-    unsigned short* tmax = p.tile_max + (size_t)wk.row * p.nchunks * kTilesPerChunk;
-    while (ch < wk.chunk_end) {
-        const float lm = lt.reduce_max();
-        const uint2 q = QuadMax<T>::keys(lt);
-        if ((lane & 3) == 0) *reinterpret_cast<uint2*>(tmax + ch * kTilesPerChunk + lane) = q;  // slots (lane >> 2) * 4 ..+3
-        ls.raise_to(lm, c);
-        lt.accumulate(ls, c);
-        ch += kWarps;
-        if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
-    }
-    // hand-over: one (M, S) pair per warp
-    const float Mw = warp_max(ls.M);
-    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
-    if (lane == 0) {
-        SegStat* st = &p.seg_stats[blockIdx.x];
-        st->S[warp] = Sw;
-        st->M[warp] = Mw;
-    }
-    __syncthreads();  // every warp's part of the hand-over is written
-    if (tid == 0) publish_row_ready(&p.seg_ready[blockIdx.x]);
-}
-
-// ---- finish kernel ---------------------------------------------------------------------------------
-// NT threads per row: 128 (k <= 128) or 256.  Finishing a row is a chain of dependent steps (trips
-// to L2 / HBM, bisection rounds, prefix sums), and most finish CTAs of a large batch only find room
-// on an SM once the streaming kernel's last wave drains, so what the finish costs is the chain's
-// length times the number of waves left then: the chain is kept to three trips to memory (the
-// hand-over, the survivors' vectors, the outputs).
-__host__ __device__ inline size_t align16(size_t x) { return (x + 15) / 16 * 16; }
-__host__ __device__ inline int pow2_at_least(int n) {
-    int p = 1;
-    while (p < n) p <<= 1;
-    return p;
-}
-__host__ __device__ constexpr int finish_threads(int k) { return k <= 128 ? 128 : 256; }
-__host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
-constexpr int kFinishHeaderBytes = 512;
-constexpr int kRankListMax = 512;  // candidates up to which the k-th is found by counting ranks
-
-// Dynamic shared memory of the finish kernel:
-//   header | histogram | region A | region B | region C | line maxima
-//   histogram: the selection histogram of the all-vectors path; else the rank-counting keys
-//   region A:  group maxima, later the sort keys of the top-rho cut
-//   region B:  survivor tile list, later the fp64 work arrays (weights, CDF)
-//   region C:  candidates (raw logit bits, token index), compacted in place to the winners
-struct FinishLayout {
-    size_t hist, a, b, c, lines, total;
-};
-__host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap, int cand_cap, int k, int nchunks) {
-    FinishLayout L;
-    L.hist = kFinishHeaderBytes;
-    L.a = L.hist + (size_t)kSelBins * 4;
-    const size_t ga = (size_t)ngroups * 4, ca = (size_t)pow2_at_least(k) * 8;
-    L.b = L.a + align16(ga > ca ? ga : ca);
-    const size_t tb = (size_t)tile_cap * 4, wb = (size_t)k * 16;
-    L.c = L.b + align16(tb > wb ? tb : wb);
-    L.lines = L.c + (size_t)cand_cap * 8;
-    L.total = L.lines + align16((size_t)nchunks * 2);
-    return L;
-}
-
-struct FinishShared {
-    double scratch[16];
-    double lrow;  // base-2 log of the row's softmax normaliser
-    int iscr[16];
-    int sel_bin, sel_above, sel_eq, sel_total;
-    int ready, gmax;
-};
 
 // Atomics on shared memory through the shared-space address: a generic-address atomic that happens to
 // hit shared memory is several times slower, and the compiler cannot always tell.
@@ -331,9 +215,10 @@ template <int NT> __device__ __forceinline__ void bitonic_sort_desc(unsigned lon
 // passes of 256 bins: the high byte, then the low byte among the values that share it.  A bisection
 // on the value's bits would take one barrier per bit, and the keys of logits that straddle zero
 // differ in nearly all sixteen.  for_each(f) calls f(v) for every value v of THIS thread.  *above
-// gets the number of values larger than the result.  hist: 256 words of shared memory.
+// gets the number of values larger than the result.  hist: 256 words of shared memory.  Ends with
+// a barrier after the last read of sel, so both can be reused right away.
 template <int NT, typename ForEach>
-__device__ __forceinline__ uint32_t radix_kth16(int kk, ForEach for_each, uint32_t* hist, FinishShared* sh, int tid, int* above) {
+__device__ __forceinline__ uint32_t radix_kth16(int kk, ForEach for_each, uint32_t* hist, int* sel /* 2 words of shared memory */, int tid, int* above) {
     uint32_t prefix = 0;
     int above_acc = 0;
 #pragma unroll 1
@@ -368,19 +253,323 @@ __device__ __forceinline__ uint32_t radix_kth16(int kk, ForEach for_each, uint32
                 carried += __shfl_sync(0xffffffffu, incl, 31);
             }
             if (tid == 0) {
-                sh->sel_bin = found ? found_bin : 0;
-                sh->sel_above = found ? (int)found_above : 0;
+                sel[0] = found ? found_bin : 0;
+                sel[1] = found ? (int)found_above : 0;
             }
         }
         fsync<NT>();
-        const int bin = sh->sel_bin, ab = sh->sel_above;
+        const int bin = sel[0], ab = sel[1];
         above_acc += ab;
         kk -= ab;
         prefix = pass == 0 ? (uint32_t)bin : ((prefix << 8) | (uint32_t)bin);
+        fsync<NT>();
     }
     *above = above_acc;
     return prefix;
 }
+
+// ---- streaming kernel ------------------------------------------------------------------------------
+template <typename T> struct QuadMax;
+template <> struct QuadMax<bf16_t> {
+    // top 16 bits of the largest logit of each of the quad's four tiles, packed (j = 0, 1 | 2, 3)
+    static __device__ __forceinline__ uint2 keys(const LaneTile<bf16_t>& lt) {
+        uint32_t r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t v = lt.vm[j];
+            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            v = bf16x2_max(v, __shfl_xor_sync(0xffffffffu, v, 2));
+            r[j] = bf16x2_max(v, v >> 16) & 0xffffu;
+        }
+        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
+    }
+};
+template <> struct QuadMax<float> {
+    static __device__ __forceinline__ uint2 keys(const LaneTile<float>& lt) {
+        uint32_t r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v = lt.vm[j];
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+            r[j] = __float_as_uint(v) >> 16;
+        }
+        return make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
+    }
+};
+
+// Group maxima of one 64-byte line of tile maxima (32 slots, two per word): the packed bf16 maximum
+// works on the raw top-16-bit patterns whatever the logits' type.  Writes the line's 32 >> glog group
+// maxima (as keys) to gm_line, for 0 <= glog <= 5; returns the line's maximum as a raw pattern.
+__device__ __forceinline__ uint32_t half_max(uint32_t w) { return bf16x2_max(w, w >> 16) & 0xffffu; }
+__device__ __forceinline__ uint32_t line_group_maxima(const uint32_t (&w)[16], int glog, uint32_t* gm_line) {
+    uint32_t t8[8], t4[4], t2[2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t8[i] = bf16x2_max(w[2 * i], w[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) t4[i] = bf16x2_max(t8[2 * i], t8[2 * i + 1]);
+    t2[0] = bf16x2_max(t4[0], t4[1]);
+    t2[1] = bf16x2_max(t4[2], t4[3]);
+    const uint32_t t1 = bf16x2_max(t2[0], t2[1]);
+    if (glog == 0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            gm_line[2 * i] = raw16_to_key16(w[i] & 0xffffu);
+            gm_line[2 * i + 1] = raw16_to_key16(w[i] >> 16);
+        }
+    } else if (glog == 1) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) gm_line[i] = raw16_to_key16(half_max(w[i]));
+    } else if (glog == 2) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gm_line[i] = raw16_to_key16(half_max(t8[i]));
+    } else if (glog == 3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) gm_line[i] = raw16_to_key16(half_max(t4[i]));
+    } else if (glog == 4) {
+        gm_line[0] = raw16_to_key16(half_max(t2[0]));
+        gm_line[1] = raw16_to_key16(half_max(t2[1]));
+    } else if (glog == 5) {
+        gm_line[0] = raw16_to_key16(half_max(t1));
+    }
+    return half_max(t1);
+}
+
+// Which of a line's 32 tiles have a key >= bound: bit a of the result is tile a of the chunk in
+// ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the line).
+__device__ __forceinline__ uint32_t line_survivors(const uint32_t (&w)[16], uint32_t bound) {
+    uint32_t m = 0;
+    {   // most lines hold no survivor: their maximum settles it
+        uint32_t t = bf16x2_max(bf16x2_max(bf16x2_max(w[0], w[1]), bf16x2_max(w[2], w[3])),
+                                bf16x2_max(bf16x2_max(w[4], w[5]), bf16x2_max(w[6], w[7])));
+        t = bf16x2_max(t, bf16x2_max(bf16x2_max(bf16x2_max(w[8], w[9]), bf16x2_max(w[10], w[11])),
+                                     bf16x2_max(bf16x2_max(w[12], w[13]), bf16x2_max(w[14], w[15]))));
+        if (raw16_to_key16(half_max(t)) < bound) return 0u;
+    }
+#pragma unroll
+    for (int a = 0; a < kTilesPerChunk; ++a) {
+        const int slot = ((a & 7) << 2) | (a >> 3);
+        const uint32_t raw = (slot & 1) ? (w[slot >> 1] >> 16) : (w[slot >> 1] & 0xffffu);
+        m |= (raw16_to_key16(raw) >= bound ? 1u : 0u) << a;
+    }
+    return m;
+}
+__device__ __forceinline__ void load_line(const unsigned short* line, uint32_t (&w)[16]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(line) + i);
+        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+}
+
+// Shared memory of a whole-row streaming CTA (kLocal): header | histogram (256 words) | the row's tile
+// maxima (2 bytes per tile, slot order) | the group maxima (2 bytes per group).
+struct StreamShared {
+    int sel[2];
+    int iscr[8];
+    int gmax;
+    int pad[5];
+};
+constexpr int kStreamHeaderBytes = 64 + 256 * 4;
+__host__ __device__ inline size_t stream_smem_bytes(int nchunks, int ngroups) {
+    return kStreamHeaderBytes + (size_t)nchunks * kTilesPerChunk * 2 + (((size_t)ngroups * 4 + 15) / 16) * 16;
+}
+
+// kLocal: the CTA streams a whole row, keeps the tile maxima in shared memory and, at the end of the
+// row, finds the bound (the k-th largest group maximum) and lists the survivor tiles itself: the
+// finish kernel then starts from the list, and no tile maximum ever goes to global memory.
+// Otherwise (rows cut into segments, small batches) the tile maxima go to the workspace and the
+// finish kernel, which sees the whole row, does that part.
+template <typename T, bool kLocal>
+__global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) sparsify_stream_kernel(const SparsifyParams p) {
+    extern __shared__ __align__(16) unsigned char stream_smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
+    const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
+    const RowExtent ext = row_extent<T>(p.V);
+    const float c = p.c.f;
+    const unsigned char* lane_rowp = rowp + lane * kVecBytes;
+    int ch = wk.chunk_begin + warp;
+    LaneTile<T> lt;
+    if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);  // in flight during the set-up below
+    // The segment's ready flag is cleared here, by the CTA that will set it, and the store is fenced
+    // before the barrier after which this CTA lets the finish kernel be scheduled.  A finish CTA
+    // runs only after every streaming CTA has passed that point, so it never sees a flag (or a
+    // status word) left by an earlier call, and the workspace needs no clearing between calls.
+    if (tid == 0) {
+        *(volatile int*)&p.seg_ready[blockIdx.x] = 0;
+        if (blockIdx.x == 0) *(volatile int*)p.status = 0;
+        __threadfence();
+    }
+    __syncthreads();
+    allow_dependent_launch();
+
+    LaneSum ls;
+    ls.reset();
+    unsigned short* tmax = kLocal ? reinterpret_cast<unsigned short*>(stream_smem + kStreamHeaderBytes)
+                                  : p.tile_max + (size_t)wk.row * p.nchunks * kTilesPerChunk;
+    while (ch < wk.chunk_end) {
+        const float lm = lt.reduce_max();
+        const uint2 q = QuadMax<T>::keys(lt);
+        if ((lane & 3) == 0) *reinterpret_cast<uint2*>(tmax + ch * kTilesPerChunk + lane) = q;  // slots (lane >> 2) * 4 ..+3
+        ls.raise_to(lm, c);
+        lt.accumulate(ls, c);
+        ch += kWarps;
+        if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
+    }
+    // hand-over: one (M, S) pair per warp
+    const float Mw = warp_max(ls.M);
+    const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
+    SegStat* st = &p.seg_stats[blockIdx.x];
+    if (lane == 0) {
+        st->S[warp] = Sw;
+        st->M[warp] = Mw;
+    }
+    if (kLocal) {
+        // ---- the row's bound and survivor list, from the tile maxima in shared memory -------------------
+        StreamShared* sh = reinterpret_cast<StreamShared*>(stream_smem);
+        uint32_t* hist = reinterpret_cast<uint32_t*>(stream_smem + 64);
+        const int ntiles = p.nchunks * kTilesPerChunk;
+        unsigned short* gm = tmax + ntiles;
+        uint32_t* gmw = reinterpret_cast<uint32_t*>(gm);  // groups of several lines (glog > 5): few, kept as words
+        const int glog = p.group_log2, ngroups = p.ngroups, k = p.k;
+        if (tid == 0) sh->gmax = 0;
+        if (glog > 5)
+            for (int i = tid; i < ngroups; i += kBlockThreads) gmw[i] = 0u;
+        __syncthreads();  // every warp's tile maxima are in place
+        // thread t takes lines t, t + 256, ...; a line (the 32 tile maxima of a chunk, 64 bytes) is read
+        // with four 16-byte loads and worked on in registers.  Rows of up to 256 chunks (512 KB) keep
+        // their one line per thread in registers from here to the listing.
+        uint32_t mx = 0;
+        uint32_t w0[16];
+        const bool one_line = p.nchunks <= kBlockThreads;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) w0[i] = 0xff80ff80u;  // -inf: never a survivor
+        for (int cl = tid; cl < p.nchunks; cl += kBlockThreads) {
+            uint32_t w[16];
+            const uint4* line = reinterpret_cast<const uint4*>(tmax + cl * kTilesPerChunk);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = line[i];
+                w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+            }
+            uint32_t gl[32];  // (only the first 32 >> glog are written, and only for glog <= 5)
+            const uint32_t lm = raw16_to_key16(line_group_maxima(w, glog, gl));
+            if (glog <= 5) {
+                for (int i = 0; i < (kTilesPerChunk >> glog); ++i) gm[((cl * kTilesPerChunk) >> glog) + i] = (unsigned short)gl[i];
+            } else {
+                smem_max(&gmw[cl >> (glog - 5)], lm);  // groups of several lines: 32-bit words, see below
+            }
+            mx = max(mx, lm);
+            if (one_line) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) w0[i] = w[i];
+            }
+        }
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (lane == 0) smem_max(&sh->gmax, mx);
+        __syncthreads();
+        uint32_t bound = 0;
+        if (ngroups >= k) {
+            int unused;
+            if (glog <= 5) {
+                bound = radix_kth16<kBlockThreads>(k, [&](auto f) {
+                    for (int i = tid; i < ngroups; i += kBlockThreads) f((uint32_t)gm[i]);
+                }, hist, sh->sel, tid, &unused);
+            } else {
+                bound = radix_kth16<kBlockThreads>(k, [&](auto f) {
+                    for (int i = tid; i < ngroups; i += kBlockThreads) f(gmw[i]);
+                }, hist, sh->sel, tid, &unused);
+            }
+        }
+        const uint32_t lo16 = max(bound, kLowestFinite16);
+        // survivors in address order, positions by a prefix sum per round of 256 lines
+        uint32_t* list = p.row_list + (size_t)wk.row * p.tile_cap;
+        int base = 0;
+        bool fits = true;
+        for (int c0 = 0; c0 < p.nchunks; c0 += kBlockThreads) {
+            const int cl = c0 + tid;
+            uint32_t m = 0;
+            if (one_line) {
+                m = line_survivors(w0, lo16);
+            } else if (cl < p.nchunks) {
+                uint32_t w[16];
+                const uint4* line = reinterpret_cast<const uint4*>(tmax + cl * kTilesPerChunk);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 v = line[i];
+                    w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+                }
+                m = line_survivors(w, lo16);
+            }
+            int round_total;
+            int pos = base + block_exscan<kBlockThreads>(__popc(m), tid, sh->iscr, &round_total);
+            if (base + round_total > p.tile_cap) fits = false;
+            if (fits) {
+                while (m) {
+                    const int a = __ffs(m) - 1;
+                    m &= m - 1;
+                    list[pos++] = (uint32_t)(cl * kTilesPerChunk + a);
+                }
+            }
+            base += round_total;
+        }
+        if (tid == 0) {
+            st->n_list = fits ? base : -1;
+            st->bound16 = (int)bound;
+            st->max16 = sh->gmax;
+        }
+    }
+    __syncthreads();  // every warp's part of the hand-over is written
+    if (tid == 0) publish_row_ready(&p.seg_ready[blockIdx.x]);
+}
+
+// ---- finish kernel ---------------------------------------------------------------------------------
+// NT threads per row: 128 (k <= 128) or 256.  Finishing a row is a chain of dependent steps (trips
+// to L2 / HBM, bisection rounds, prefix sums), and most finish CTAs of a large batch only find room
+// on an SM once the streaming kernel's last wave drains, so what the finish costs is the chain's
+// length times the number of waves left then: the chain is kept to three trips to memory (the
+// hand-over, the survivors' vectors, the outputs).
+__host__ __device__ inline size_t align16(size_t x) { return (x + 15) / 16 * 16; }
+__host__ __device__ inline int pow2_at_least(int n) {
+    int p = 1;
+    while (p < n) p <<= 1;
+    return p;
+}
+__host__ __device__ constexpr int finish_threads(int k) { return k <= 128 ? 128 : 256; }
+__host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
+constexpr int kFinishHeaderBytes = 512;
+constexpr int kRankListMax = 512;  // candidates up to which the k-th is found by counting ranks
+
+// Dynamic shared memory of the finish kernel:
+//   header | histogram | region A | region B | region C | line maxima
+//   histogram: the selection histogram of the all-vectors path; else the rank-counting keys
+//   region A:  group maxima, later the sort keys of the top-rho cut
+//   region B:  survivor tile list, later the fp64 work arrays (weights, CDF)
+//   region C:  candidates (raw logit bits, token index), compacted in place to the winners
+struct FinishLayout {
+    size_t hist, a, b, c, lines, total;
+};
+__host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap, int cand_cap, int k, int nchunks) {
+    FinishLayout L;
+    L.hist = kFinishHeaderBytes;
+    L.a = L.hist + (size_t)kSelBins * 4;
+    const size_t ga = (size_t)ngroups * 4, ca = (size_t)pow2_at_least(k) * 8;
+    L.b = L.a + align16(ga > ca ? ga : ca);
+    const size_t tb = (size_t)tile_cap * 4, wb = (size_t)k * 16;
+    L.c = L.b + align16(tb > wb ? tb : wb);
+    L.lines = L.c + (size_t)cand_cap * 8;
+    L.total = L.lines + align16((size_t)nchunks * 2);
+    return L;
+}
+
+struct FinishShared {
+    double scratch[16];
+    double lrow;  // base-2 log of the row's softmax normaliser
+    int iscr[16];
+    int sel_bin, sel_above, sel_eq, sel_total;
+    int ready, gmax;
+};
 
 // The vectors a thread works on: units [u0, u1) of the row's survivor tiles (tl: their tile numbers in
 // address order, four vectors each), or of the whole row (tl == nullptr: unit = vector).  f(z, vi)
@@ -505,70 +694,6 @@ __device__ __forceinline__ int finite_key16(float z) {
     return (k16 >= kLowestFinite16 && k16 <= kHighestFinite16) ? (int)k16 : -1;
 }
 
-// Group maxima of one 64-byte line of tile maxima (32 slots, two per word): the packed bf16 maximum
-// works on the raw top-16-bit patterns whatever the logits' type.  Writes the line's 32 >> glog group
-// maxima (as keys) to gm_line, for 0 <= glog <= 5; returns the line's maximum as a raw pattern.
-__device__ __forceinline__ uint32_t half_max(uint32_t w) { return bf16x2_max(w, w >> 16) & 0xffffu; }
-__device__ __forceinline__ uint32_t line_group_maxima(const uint32_t (&w)[16], int glog, uint32_t* gm_line) {
-    uint32_t t8[8], t4[4], t2[2];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) t8[i] = bf16x2_max(w[2 * i], w[2 * i + 1]);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) t4[i] = bf16x2_max(t8[2 * i], t8[2 * i + 1]);
-    t2[0] = bf16x2_max(t4[0], t4[1]);
-    t2[1] = bf16x2_max(t4[2], t4[3]);
-    const uint32_t t1 = bf16x2_max(t2[0], t2[1]);
-    if (glog == 0) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            gm_line[2 * i] = raw16_to_key16(w[i] & 0xffffu);
-            gm_line[2 * i + 1] = raw16_to_key16(w[i] >> 16);
-        }
-    } else if (glog == 1) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) gm_line[i] = raw16_to_key16(half_max(w[i]));
-    } else if (glog == 2) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) gm_line[i] = raw16_to_key16(half_max(t8[i]));
-    } else if (glog == 3) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) gm_line[i] = raw16_to_key16(half_max(t4[i]));
-    } else if (glog == 4) {
-        gm_line[0] = raw16_to_key16(half_max(t2[0]));
-        gm_line[1] = raw16_to_key16(half_max(t2[1]));
-    } else if (glog == 5) {
-        gm_line[0] = raw16_to_key16(half_max(t1));
-    }
-    return half_max(t1);
-}
-
-// Which of a line's 32 tiles have a key >= bound: bit a of the result is tile a of the chunk in
-// ADDRESS order (tile j * 8 + q sits in slot q * 4 + j of the line).
-__device__ __forceinline__ uint32_t line_survivors(const uint32_t (&w)[16], uint32_t bound) {
-    uint32_t m = 0;
-    {   // most lines hold no survivor: their maximum settles it
-        uint32_t t = bf16x2_max(bf16x2_max(bf16x2_max(w[0], w[1]), bf16x2_max(w[2], w[3])),
-                                bf16x2_max(bf16x2_max(w[4], w[5]), bf16x2_max(w[6], w[7])));
-        t = bf16x2_max(t, bf16x2_max(bf16x2_max(bf16x2_max(w[8], w[9]), bf16x2_max(w[10], w[11])),
-                                     bf16x2_max(bf16x2_max(w[12], w[13]), bf16x2_max(w[14], w[15]))));
-        if (raw16_to_key16(half_max(t)) < bound) return 0u;
-    }
-#pragma unroll
-    for (int a = 0; a < kTilesPerChunk; ++a) {
-        const int slot = ((a & 7) << 2) | (a >> 3);
-        const uint32_t raw = (slot & 1) ? (w[slot >> 1] >> 16) : (w[slot >> 1] & 0xffffu);
-        m |= (raw16_to_key16(raw) >= bound ? 1u : 0u) << a;
-    }
-    return m;
-}
-__device__ __forceinline__ void load_line(const unsigned short* line, uint32_t (&w)[16]) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(line) + i);
-        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
-    }
-}
-
 template <typename T, int NT>
 __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kernel(const SparsifyParams p) {
     constexpr int kPer = Elt<T>::kPerVec;
@@ -645,111 +770,125 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         }
         if (lane == 0) sh->lrow = Sall > 0.0 ? Mall + log2(Sall) : -INFINITY;
     }
-    // ---- 1. group maxima of the tile maxima; each line's maximum is kept for step 3 -------------------
-    // Thread t takes a run of consecutive chunks; a chunk's 32 tile maxima are one 64-byte line.
-    const unsigned short* tmax = p.tile_max + (size_t)row * nchunks * kTilesPerChunk;
-    const int cpt = (nchunks + NT - 1) / NT;
-    const int ch0 = min(nchunks, tid * cpt), ch1 = min(nchunks, ch0 + cpt);
-    // up to kKeep lines stay in registers for step 3 (rows up to kKeep * NT chunks: 512 KB with
-    // 128 threads); longer rows read their lines again there
-    constexpr int kKeep = 2;
-    uint32_t kept[kKeep][16];
-    const bool keep_lines = cpt <= kKeep;
-#pragma unroll
-    for (int j = 0; j < kKeep; ++j) {
-        const int ch = ch0 + j;
-        if (keep_lines && ch < ch1) {
-            load_line(tmax + ch * kTilesPerChunk, kept[j]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) kept[j][i] = 0xff80ff80u;  // -inf: never a survivor
-        }
-    }
-    if (keep_lines) {
-#pragma unroll
+    int lo16, max16, n_surv;
+    bool listed;
+    if (p.local_bound) {
+        // ---- 1-3 done by the row's streaming CTA: its bound, its survivor list ------------------------------
+        const SegStat* st = p.seg_stats + row;
+        const int n_list = __ldcg(&st->n_list);
+        lo16 = max(__ldcg(&st->bound16), (int)kLowestFinite16);
+        max16 = min(__ldcg(&st->max16), (int)kHighestFinite16);
+        listed = n_list >= 0 && n_list <= p.tile_cap;
+        n_surv = listed ? n_list : 0;
+        const uint32_t* list = p.row_list + (size_t)row * p.tile_cap;
+        for (int i = tid; i < n_surv; i += NT) tl[i] = __ldcg(list + i);
+        fsync<NT>();
+    } else {
+        // ---- 1. group maxima of the tile maxima; each line's maximum is kept for step 3 -------------------
+        // Thread t takes a run of consecutive chunks; a chunk's 32 tile maxima are one 64-byte line.
+        const unsigned short* tmax = p.tile_max + (size_t)row * nchunks * kTilesPerChunk;
+        const int cpt = (nchunks + NT - 1) / NT;
+        const int ch0 = min(nchunks, tid * cpt), ch1 = min(nchunks, ch0 + cpt);
+        // up to kKeep lines stay in registers for step 3 (rows up to kKeep * NT chunks: 512 KB with
+        // 128 threads); longer rows read their lines again there
+        constexpr int kKeep = 2;
+        uint32_t kept[kKeep][16];
+        const bool keep_lines = cpt <= kKeep;
+    #pragma unroll
         for (int j = 0; j < kKeep; ++j) {
             const int ch = ch0 + j;
-            if (ch < ch1) {
-                const uint32_t lm = line_group_maxima(kept[j], glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+            if (keep_lines && ch < ch1) {
+                load_line(tmax + ch * kTilesPerChunk, kept[j]);
+            } else {
+    #pragma unroll
+                for (int i = 0; i < 16; ++i) kept[j][i] = 0xff80ff80u;  // -inf: never a survivor
+            }
+        }
+        if (keep_lines) {
+    #pragma unroll
+            for (int j = 0; j < kKeep; ++j) {
+                const int ch = ch0 + j;
+                if (ch < ch1) {
+                    const uint32_t lm = line_group_maxima(kept[j], glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+                    if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
+                    lmax[ch] = (unsigned short)lm;
+                }
+            }
+        } else {
+            for (int ch = ch0; ch < ch1; ++ch) {
+                uint32_t w[16];
+                load_line(tmax + ch * kTilesPerChunk, w);
+                const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
                 if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
                 lmax[ch] = (unsigned short)lm;
             }
         }
-    } else {
-        for (int ch = ch0; ch < ch1; ++ch) {
-            uint32_t w[16];
-            load_line(tmax + ch * kTilesPerChunk, w);
-            const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
-            if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
-            lmax[ch] = (unsigned short)lm;
+        fsync<NT>();
+        {
+            uint32_t mx = 0u;
+            for (int i = tid; i < ngroups; i += NT) mx = max(mx, gm[i]);
+            mx = __reduce_max_sync(0xffffffffu, mx);
+            if (lane == 0) smem_max(&sh->gmax, mx);
         }
-    }
-    fsync<NT>();
-    {
-        uint32_t mx = 0u;
-        for (int i = tid; i < ngroups; i += NT) mx = max(mx, gm[i]);
-        mx = __reduce_max_sync(0xffffffffu, mx);
-        if (lane == 0) smem_max(&sh->gmax, mx);
-    }
-    fsync<NT>();
-    const uint32_t gmax = (uint32_t)sh->gmax;
-    const int max16 = min((int)gmax, (int)kHighestFinite16);
-    const double L2 = sh->lrow;
-    // ---- 2. the k-th largest group maximum: a lower bound on the k-th largest logit's key ---------------
-    uint32_t bound = 0;
-    if (ngroups >= k) {
-        int unused;
-        bound = radix_kth16<NT>(k, [&](auto f) {
-            for (int i = tid; i < ngroups; i += NT) f(gm[i]);
-        }, hist, sh, tid, &unused);
-    }
-    int lo16 = max((int)bound, (int)kLowestFinite16);
-    // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
-    int my_surv = 0;
-    uint32_t kept_mask[kKeep];
-    if (keep_lines) {
-#pragma unroll
-        for (int j = 0; j < kKeep; ++j) {
-            kept_mask[j] = line_survivors(kept[j], (uint32_t)lo16);  // bit a: tile a of the chunk (none beyond the row)
-            my_surv += __popc(kept_mask[j]);
+        fsync<NT>();
+        const uint32_t gmax = (uint32_t)sh->gmax;
+        max16 = min((int)gmax, (int)kHighestFinite16);
+        // ---- 2. the k-th largest group maximum: a lower bound on the k-th largest logit's key ---------------
+        uint32_t bound = 0;
+        if (ngroups >= k) {
+            int unused;
+            bound = radix_kth16<NT>(k, [&](auto f) {
+                for (int i = tid; i < ngroups; i += NT) f(gm[i]);
+            }, hist, &sh->sel_bin, tid, &unused);
         }
-    } else {
-        for (int ch = ch0; ch < ch1; ++ch) {
-            if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
-            uint32_t w[16];
-            load_line(tmax + ch * kTilesPerChunk, w);
-            my_surv += __popc(line_survivors(w, (uint32_t)lo16));
-        }
-    }
-    int n_surv;
-    int pos = block_exscan<NT>(my_surv, tid, sh->iscr, &n_surv);
-    const bool listed = n_surv <= p.tile_cap;
-    if (listed) {
+        lo16 = max((int)bound, (int)kLowestFinite16);
+        // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
+        int my_surv = 0;
+        uint32_t kept_mask[kKeep];
         if (keep_lines) {
-#pragma unroll
+    #pragma unroll
             for (int j = 0; j < kKeep; ++j) {
-                uint32_t m = kept_mask[j];
-                while (m) {
-                    const int a = __ffs(m) - 1;
-                    m &= m - 1;
-                    tl[pos++] = (uint32_t)((ch0 + j) * kTilesPerChunk + a);
-                }
+                kept_mask[j] = line_survivors(kept[j], (uint32_t)lo16);  // bit a: tile a of the chunk (none beyond the row)
+                my_surv += __popc(kept_mask[j]);
             }
         } else {
             for (int ch = ch0; ch < ch1; ++ch) {
                 if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
                 uint32_t w[16];
                 load_line(tmax + ch * kTilesPerChunk, w);
-                uint32_t m = line_survivors(w, (uint32_t)lo16);
-                while (m) {
-                    const int a = __ffs(m) - 1;
-                    m &= m - 1;
-                    tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
+                my_surv += __popc(line_survivors(w, (uint32_t)lo16));
+            }
+        }
+        int pos = block_exscan<NT>(my_surv, tid, sh->iscr, &n_surv);
+        listed = n_surv <= p.tile_cap;
+        if (listed) {
+            if (keep_lines) {
+    #pragma unroll
+                for (int j = 0; j < kKeep; ++j) {
+                    uint32_t m = kept_mask[j];
+                    while (m) {
+                        const int a = __ffs(m) - 1;
+                        m &= m - 1;
+                        tl[pos++] = (uint32_t)((ch0 + j) * kTilesPerChunk + a);
+                    }
+                }
+            } else {
+                for (int ch = ch0; ch < ch1; ++ch) {
+                    if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+                    uint32_t w[16];
+                    load_line(tmax + ch * kTilesPerChunk, w);
+                    uint32_t m = line_survivors(w, (uint32_t)lo16);
+                    while (m) {
+                        const int a = __ffs(m) - 1;
+                        m &= m - 1;
+                        tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
+                    }
                 }
             }
         }
+        fsync<NT>();
     }
-    fsync<NT>();
+    const double L2 = sh->lrow;
     // the vectors this thread works on from here: a contiguous run of the survivors' vectors, or of the row's
     const uint32_t* units = listed ? tl : nullptr;
     const int n_units = listed ? n_surv * kVecsPerTile : (p.V + kPer - 1) / kPer;
@@ -856,7 +995,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
             int above = 0;
             const uint32_t e16 = radix_kth16<NT>(k, [&](auto f) {
                 for (int i = i0; i < i1; ++i) f(float_to_key(__uint_as_float(c_raw[i])) >> 16);
-            }, hist, sh, tid, &above);
+            }, hist, &sh->sel_bin, tid, &above);
             int need = k - above;
             uint32_t e32;
             if (kBf16) {
@@ -868,7 +1007,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
                         const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
                         if ((kz >> 16) == e16) f(kz & 0xffffu);
                     }
-                }, hist, sh, tid, &above2);
+                }, hist, &sh->sel_bin, tid, &above2);
                 e32 = (e16 << 16) | low;
                 need -= above2;
             }
@@ -1084,9 +1223,12 @@ namespace tslt {
 struct SparsifyPlan {
     int nchunks, group_log2, ngroups, tile_cap, cand_cap, fin_threads;
     RowSplit split;
+    bool local_bound;    // whole-row streaming CTAs find the bound and list the survivors themselves
+    size_t stream_smem;  // their shared memory
     size_t fin_smem;
     size_t ws_ready_off, ws_stats_off, ws_tiles_off, ws_bytes;
 };
+constexpr size_t kStreamSmemLimit = 100 * 1024;
 
 static int sm_count_cached() {
     static int sms = 0;
@@ -1120,6 +1262,9 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     // chunk per warp each) so that every CTA slot has work.  A segment costs nothing but its own
     // hand-over (8 (max, sum) pairs and a flag).
     const int slots = kSparsifyStreamCtasPerSm * sm_count_cached();
+    // (Cutting the rows of a large batch as well, into segments of 64 to 256 KB, was measured and
+    // dropped: the finish kernel is only scheduled once every streaming CTA has started, which with
+    // eight times the CTAs is the very end of the streaming kernel.)
     int nseg = 1;
     if (rows > 0 && rows < slots) {
         nseg = (slots + rows - 1) / rows;
@@ -1134,13 +1279,18 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.split.cps = cps;
     pl.split.nseg = (pl.nchunks + cps - 1) / cps;
     pl.split.grid = rows * pl.split.nseg;
+    pl.stream_smem = stream_smem_bytes(pl.nchunks, pl.ngroups);
+    pl.local_bound = pl.split.nseg == 1 && pl.stream_smem <= kStreamSmemLimit;
+    if (!pl.local_bound) pl.stream_smem = 0;
     size_t off = kWsHeaderBytes;
     pl.ws_ready_off = off;
     off = align_up256(off + (size_t)rows * pl.split.nseg * sizeof(int));
     pl.ws_stats_off = off;
     off = align_up256(off + (size_t)rows * pl.split.nseg * sizeof(SegStat));
     pl.ws_tiles_off = off;
-    off = align_up256(off + (size_t)rows * (size_t)ntiles * sizeof(unsigned short));
+    // whole-row CTAs hand a survivor list over, segments their tile maxima
+    off = align_up256(off + (pl.local_bound ? (size_t)rows * pl.tile_cap * sizeof(uint32_t)
+                                            : (size_t)rows * (size_t)ntiles * sizeof(unsigned short)));
     pl.ws_bytes = off;
     return pl;
 }
@@ -1156,14 +1306,14 @@ ScaleC make_scale(float temperature) {
 // Largest k and long rows take the finish kernel's shared memory past the default 48 KB: the kernel's
 // limit is raised once per device (slot: one per kernel instantiation), not on every call.
 constexpr size_t kFinishSmemLimit = 96 * 1024;
-static bool raise_smem_limit_once(void (*kern)(const SparsifyParams), int slot) {
+static bool raise_smem_limit_once(void (*kern)(const SparsifyParams), int slot, size_t limit) {
     constexpr int kMaxDevices = 64;
-    static bool done[6][kMaxDevices] = {};
+    static bool done[12][kMaxDevices] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     const bool cached = dev >= 0 && dev < kMaxDevices;
     if (cached && done[slot][dev]) return true;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemLimit) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit) != cudaSuccess) return false;
     if (cached) done[slot][dev] = true;
     return true;
 }
@@ -1230,21 +1380,25 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.seg_ready = (int*)(ws + pl.ws_ready_off);
     p.seg_stats = (SegStat*)(ws + pl.ws_stats_off);
     p.tile_max = (unsigned short*)(ws + pl.ws_tiles_off);
+    p.row_list = (uint32_t*)(ws + pl.ws_tiles_off);
+    p.local_bound = pl.local_bound ? 1 : 0;
 
     cudaStream_t st = (cudaStream_t)stream;
-    if (!(dtype == TSLT_F32 ? prefer_shared_carveout_once(sparsify_stream_kernel<float>, 0)
-                            : prefer_shared_carveout_once(sparsify_stream_kernel<bf16_t>, 1)))
-        return TSLT_ERR_CUDA;
-    if (dtype == TSLT_F32) sparsify_stream_kernel<float><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
-    else sparsify_stream_kernel<bf16_t><<<pl.split.grid, kBlockThreads, 0, st>>>(p);
+    void (*strm)(const SparsifyParams);
+    if (pl.local_bound) strm = dtype == TSLT_F32 ? sparsify_stream_kernel<float, true> : sparsify_stream_kernel<bf16_t, true>;
+    else strm = dtype == TSLT_F32 ? sparsify_stream_kernel<float, false> : sparsify_stream_kernel<bf16_t, false>;
+    const int strm_slot = (pl.local_bound ? 2 : 0) + (dtype == TSLT_F32 ? 0 : 1);
+    if (!prefer_shared_carveout_once(strm, strm_slot)) return TSLT_ERR_CUDA;
+    if (pl.stream_smem > 48 * 1024 && !raise_smem_limit_once(strm, 4 + strm_slot, kStreamSmemLimit)) return TSLT_ERR_CUDA;
+    strm<<<pl.split.grid, kBlockThreads, pl.stream_smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     void (*fin)(const SparsifyParams);
     if (pl.fin_threads == 128) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 128> : sparsify_finish_kernel<bf16_t, 128>;
     else fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 256> : sparsify_finish_kernel<bf16_t, 256>;
-    if (!prefer_shared_carveout_once(fin, 2 + (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1))) return TSLT_ERR_CUDA;
+    if (!prefer_shared_carveout_once(fin, 4 + (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1))) return TSLT_ERR_CUDA;
     if (pl.fin_smem > kFinishSmemLimit) return TSLT_ERR_UNSUPPORTED;  // (rows of tens of millions of logits: the line maxima no longer fit)
     if (pl.fin_smem > 48 * 1024 &&
-        !raise_smem_limit_once(fin, (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1)))
+        !raise_smem_limit_once(fin, (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1), kFinishSmemLimit))
         return TSLT_ERR_CUDA;
     if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
