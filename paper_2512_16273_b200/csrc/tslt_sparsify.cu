@@ -371,6 +371,7 @@ struct StreamShared {
     int pad[5];
 };
 constexpr int kStreamHeaderBytes = 64 + 256 * 4;
+constexpr int kWarpSelectMax = 512;  // group maxima up to which one warp selects the bound
 __host__ __device__ inline size_t stream_smem_bytes(int nchunks, int ngroups) {
     return kStreamHeaderBytes + (size_t)nchunks * kTilesPerChunk * 2 + (((size_t)ngroups * 4 + 15) / 16) * 16;
 }
@@ -470,7 +471,30 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
         if (lane == 0) smem_max(&sh->gmax, mx);
         __syncthreads();
         uint32_t bound = 0;
-        if (ngroups >= k) {
+        if (ngroups >= k && ngroups <= kWarpSelectMax) {
+            // few groups: one warp bisects on the 16 bits of the key, its values in registers, with no
+            // block barrier per step (a barrier costs this CTA a good part of a microsecond while
+            // four other CTAs stream on the SM); the others wait at the barrier below
+            if (warp == 0) {
+                uint32_t v[kWarpSelectMax / 32];
+#pragma unroll
+                for (int j = 0; j < kWarpSelectMax / 32; ++j) {
+                    const int i = lane + 32 * j;
+                    v[j] = i < ngroups ? (glog <= 5 ? (uint32_t)gm[i] : gmw[i]) : 0u;
+                }
+                uint32_t b = 0;
+                for (int bit = 15; bit >= 0; --bit) {
+                    const uint32_t cand = b | (1u << bit);
+                    int cnt = 0;
+#pragma unroll
+                    for (int j = 0; j < kWarpSelectMax / 32; ++j) cnt += v[j] >= cand ? 1 : 0;
+                    if (__reduce_add_sync(0xffffffffu, cnt) >= k) b = cand;
+                }
+                if (lane == 0) sh->sel[0] = (int)b;
+            }
+            __syncthreads();
+            bound = (uint32_t)sh->sel[0];
+        } else if (ngroups >= k) {
             int unused;
             if (glog <= 5) {
                 bound = radix_kth16<kBlockThreads>(k, [&](auto f) {
