@@ -102,6 +102,9 @@ __device__ __forceinline__ uint32_t raw16_to_key16(uint32_t r) {
 __device__ __forceinline__ void smem_add(void* p, uint32_t v) {
     asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
+__device__ __forceinline__ void smem_add64(void* p, unsigned long long v) {
+    asm volatile("red.shared.add.u64 [%0], %1;" ::"r"(smem_u32(p)), "l"(v) : "memory");
+}
 __device__ __forceinline__ void smem_max(void* p, uint32_t v) {
     asm volatile("red.shared.max.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
@@ -192,25 +195,6 @@ template <int NT> __device__ __forceinline__ void block_inclusive_scan_f64(doubl
     }
     fsync<NT>();
 }
-// Bitonic sort of a[0..P) (P a power of two, shared memory), descending.
-template <int NT> __device__ __forceinline__ void bitonic_sort_desc(unsigned long long* a, int P, int tid) {
-    for (int size = 2; size <= P; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int i = tid; i < (P >> 1); i += NT) {
-                const int lo = 2 * i - (i & (stride - 1));
-                const int hi = lo + stride;
-                const bool up = ((lo & size) == 0);
-                const unsigned long long x = a[lo], y = a[hi];
-                if (up ? x < y : x > y) {
-                    a[lo] = y;
-                    a[hi] = x;
-                }
-            }
-            fsync<NT>();
-        }
-    }
-}
-
 // The kk-th largest of the thread block's 16-bit values (at least kk of them exist), by two histogram
 // passes of 256 bins: the high byte, then the low byte among the values that share it.  A bisection
 // on the value's bits would take one barrier per bit, and the keys of logits that straddle zero
@@ -567,23 +551,23 @@ constexpr int kRankListMax = 512;  // candidates up to which the k-th is found b
 
 // Dynamic shared memory of the finish kernel:
 //   header | histogram | region A | region B | region C | line maxima
-//   histogram: the selection histogram of the all-vectors path; else the rank-counting keys
-//   region A:  group maxima, later the sort keys of the top-rho cut
-//   region B:  survivor tile list, later the fp64 work arrays (weights, CDF)
+//   histogram: the selection histogram of the all-vectors path; else the rank-counting keys, the
+//              256 bins of the radix selects and of the top-rho mass descent
+//   region A:  group maxima (rows cut into segments only)
+//   region B:  survivor tile list, later the CDF (fp64)
 //   region C:  candidates (raw logit bits, token index), compacted in place to the winners
 struct FinishLayout {
     size_t hist, a, b, c, lines, total;
 };
-__host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap, int cand_cap, int k, int nchunks) {
+__host__ __device__ inline FinishLayout finish_layout(int ngroups, int tile_cap, int cand_cap, int k, int nchunks, bool local) {
     FinishLayout L;
     L.hist = kFinishHeaderBytes;
     L.a = L.hist + (size_t)kSelBins * 4;
-    const size_t ga = (size_t)ngroups * 4, ca = (size_t)pow2_at_least(k) * 8;
-    L.b = L.a + align16(ga > ca ? ga : ca);
-    const size_t tb = (size_t)tile_cap * 4, wb = (size_t)k * 16;
+    L.b = L.a + align16(local ? 0 : (size_t)ngroups * 4);
+    const size_t tb = (size_t)tile_cap * 4, wb = (size_t)k * 8;
     L.c = L.b + align16(tb > wb ? tb : wb);
     L.lines = L.c + (size_t)cand_cap * 8;
-    L.total = L.lines + align16((size_t)nchunks * 2);
+    L.total = L.lines + (local ? 0 : align16((size_t)nchunks * 2));
     return L;
 }
 
@@ -602,7 +586,7 @@ template <typename T, typename F>
 __device__ __forceinline__ void for_my_vectors(const unsigned char* rowp, const RowExtent& ext, int V, const uint32_t* tl,
                                                int u0, int u1, F f) {
     constexpr int kPer = Elt<T>::kPerVec;
-    constexpr int kInFlight = 4;
+    constexpr int kInFlight = 6;
     for (int u = u0; u < u1; u += kInFlight) {
         uint4 d[kInFlight];
         int vi[kInFlight];
@@ -727,14 +711,12 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
     static_assert(sizeof(FinishShared) <= kFinishHeaderBytes, "header");
     const int k = p.k;
-    const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks);
+    const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks, p.local_bound != 0);
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + L.hist);
     unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
     uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + L.a);
-    unsigned long long* comp = reinterpret_cast<unsigned long long*>(gm);
     uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + L.b);
     double* cum = reinterpret_cast<double*>(tl);
-    double* wv = cum + k;
     uint32_t* c_raw = reinterpret_cast<uint32_t*>(smem_raw + L.c);
     int* c_idx = reinterpret_cast<int*>(c_raw + p.cand_cap);
     unsigned short* lmax = reinterpret_cast<unsigned short*>(smem_raw + L.lines);
@@ -747,7 +729,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) sh->gmax = 0;
     const int glog = p.group_log2, ngroups = p.ngroups;
-    if (glog > 5)
+    if (glog > 5 && !p.local_bound)
         for (int i = tid; i < ngroups; i += NT) gm[i] = 0u;
     // ---- wait for the row's segments --------------------------------------------------------------
     // Nothing the streaming kernel wrote is read before this point.  The row's own segments being
@@ -971,23 +953,44 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
                 fsync<NT>();
             }
         } else {
+            // many vectors per thread: one pass; the first candidates a thread finds wait in a small
+            // stash while the prefix sum finds where they go.  Only if some thread found more than
+            // its stash holds are the vectors read a second time (from L2).
+            constexpr int kStash = 12;
+            uint32_t st_raw[kStash];
+            int st_idx[kStash];
             int cnt = 0;
-            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
+            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
 #pragma unroll
-                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
+                for (int e = 0; e < kPer; ++e)
+                    if (is_candidate(z[e])) {
+                        if (cnt < kStash) {
+                            st_raw[cnt] = __float_as_uint(z[e]);
+                            st_idx[cnt] = vi * kPer + e;
+                        }
+                        ++cnt;
+                    }
             });
             int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+            const int over = __syncthreads_or(cnt > kStash ? 1 : 0);
             if (n_c <= p.cand_cap) {
                 in_smem = true;
-                for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+                if (!over) {
+                    for (int j = 0; j < cnt; ++j) {
+                        c_raw[cpos + j] = st_raw[j];
+                        c_idx[cpos + j] = st_idx[j];
+                    }
+                } else {
+                    for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
 #pragma unroll
-                    for (int e = 0; e < kPer; ++e)
-                        if (is_candidate(z[e])) {
-                            c_raw[cpos] = __float_as_uint(z[e]);
-                            c_idx[cpos] = vi * kPer + e;
-                            ++cpos;
-                        }
-                });
+                        for (int e = 0; e < kPer; ++e)
+                            if (is_candidate(z[e])) {
+                                c_raw[cpos] = __float_as_uint(z[e]);
+                                c_idx[cpos] = vi * kPer + e;
+                                ++cpos;
+                            }
+                    });
+                }
                 fsync<NT>();
             }
         }
@@ -1141,69 +1144,128 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     const double cd = p.c.d;
     double mass = 0.0;
     // ---- 6. top-rho cut ---------------------------------------------------------------------------------------
+    // The smallest n whose cumulative q, in the order (logit descending, index ascending), reaches
+    // top_p.  No sort: the key of the entry at which the cumulative crosses is the largest t with
+    // mass(key >= t) >= top_p, found bit by bit with one block reduction per bit; then the ties of
+    // that key, which all carry the same q, are counted off in index order.  Masses are summed as
+    // 2^-62 fixed point, so the sums do not depend on the order of the adds: deterministic.  (A
+    // histogram of mass per key byte needs 64-bit shared atomics on a handful of hot bins and was
+    // three times slower than the sort it replaced; the bisection is three times faster.)
     if (n0 > 0 && p.top_p < 1.0f) {
-        const int P = pow2_at_least(n0);
-        for (int i = tid; i < P; i += NT)
-            comp[i] = i < n0 ? (((unsigned long long)float_to_key(__uint_as_float(win_raw[i])) << 32) |
-                                (unsigned long long)(0xffffffffu - (uint32_t)win_idx[i])) : 0ull;
-        fsync<NT>();
-        bitonic_sort_desc<NT>(comp, P, tid);
-        for (int i = tid; i < n0; i += NT) cum[i] = exp2((double)key_to_float((uint32_t)(comp[i] >> 32)) * cf - L2);
-        fsync<NT>();
-        block_inclusive_scan_f64<NT>(cum, n0, tid, sh->scratch);
-        const double tp = (double)p.top_p;
-        int lo = 0, hi = n0;
-        while (lo < hi) {  // first n with c_n >= top_p
-            const int mid = (lo + hi) >> 1;
-            if (cum[mid] >= tp) hi = mid; else lo = mid + 1;
+        constexpr double kFix = 4611686018427387904.0;  // 2^62
+        unsigned long long* mhist = reinterpret_cast<unsigned long long*>(hist);  // 256 bins
+        const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
+        const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
+        uint32_t kz[4];
+        unsigned long long qf[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            kz[j] = 0u;
+            qf[j] = 0ull;
+            if (i0 + j < i1) {
+                const float z = __uint_as_float(win_raw[i0 + j]);
+                kz[j] = float_to_key(z);
+                qf[j] = __double2ull_rn(fmin(exp2((double)z * cf - L2), 1.0) * kFix);
+            }
         }
-        n = lo < n0 ? lo + 1 : n0;
-        mass = cum[n - 1];
+        const unsigned long long target = __double2ull_rn((double)p.top_p * kFix);
+        // mass of the entries whose key is >= t, over the block (fixed point: any order gives the same sum)
+        auto mass_from = [&](uint32_t t, int slot) -> unsigned long long {
+            unsigned long long m = 0ull;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1 && kz[j] >= t) m += qf[j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+            if (lane == 0 && m) smem_add64(&mhist[slot], m);  // one add per warp: 4 or 8 in all
+            fsync<NT>();
+            return mhist[slot];
+        };
+        for (int i = tid; i < 40; i += NT) mhist[i] = 0ull;
+        if (tid == 0) sh->scratch[1] = 0.0;
         fsync<NT>();
-        if (n < n0) {
-            // keep what precedes the cut in (logit descending, index ascending): a larger key, or the
-            // cut's key and an index up to the cut's
-            const unsigned long long cutc = comp[n - 1];
-            const uint32_t ckey = (uint32_t)(cutc >> 32);
-            const int cidx = (int)(0xffffffffu - (uint32_t)cutc);
-            const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
-            const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
+        unsigned long long mass_above = 0ull;
+        uint32_t prefix = 0u;
+        bool crossed = mass_from(0u, 0) >= target;
+        if (!crossed) {
+            mass_above = mhist[0];  // the whole mass: the cumulative never reaches top_p, everything is kept
+        } else {
+            // the crossing key: the largest t with mass(key >= t) >= top_p, bit by bit
+            int slot = 1;
+            unsigned long long last_rejected = 0ull;
+#pragma unroll 1
+            for (int bit = 31; bit >= (kBf16 ? 16 : 0); --bit) {
+                const uint32_t cand = prefix | (1u << bit);
+                const unsigned long long m = mass_from(cand, slot++);
+                if (m >= target) prefix = cand;
+                else last_rejected = m;
+            }
+            mass_above = last_rejected;  // mass of the keys above the crossing key (the last candidate refused is that key + 1 ulp)
+        }
+        if (!crossed) {
+            mass = (double)mass_above / kFix;
+        } else {
+            // (keys of bf16 values: the low half follows the sign and was not searched)
+            const uint32_t ckey = kBf16 ? ((prefix & 0xffff0000u) | ((prefix & 0x80000000u) ? 0u : 0xffffu)) : prefix;
+            // the ties of the crossing key share one q: how many of them, in index order, it takes
+            int c_gt = 0, c_eq = 0;
+            unsigned long long qk = 0ull;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1) {
+                    c_gt += kz[j] > ckey ? 1 : 0;
+                    if (kz[j] == ckey) {
+                        ++c_eq;
+                        qk = qf[j];
+                    }
+                }
+            if (qk) sh->scratch[1] = __longlong_as_double((long long)qk);  // (every writer writes the same value)
+            int tot_eq, tot_keep;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            qk = (unsigned long long)__double_as_longlong(sh->scratch[1]);
+            const unsigned long long missing = target - mass_above;  // > 0: the bins above did not reach it
+            int need = qk ? (int)min((unsigned long long)tot_eq, (missing + qk - 1ull) / qk) : tot_eq;
+            if (need < 1) need = 1;
+            const int my_ties = max(0, min(c_eq, need - eq_before));
+            // keep the larger keys and the first `need` ties: read mine, then (after the scan's barriers) write
             uint32_t keep_raw[4];
             int keep_idx[4];
-            int kept = 0;
-            for (int i = i0; i < i1; ++i) {
-                const uint32_t kz = float_to_key(__uint_as_float(win_raw[i]));
-                if (kept < 4 && (kz > ckey || (kz == ckey && win_idx[i] <= cidx))) {
-                    keep_raw[kept] = win_raw[i];
-                    keep_idx[kept] = win_idx[i];
-                    ++kept;
-                }
-            }
-            int tot;
-            const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot);  // (its barriers order the reads above before the writes below)
+            int kept = 0, ties_left = my_ties;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (i < kept) {
-                    win_raw[kp + i] = keep_raw[i];
-                    win_idx[kp + i] = keep_idx[i];
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1) {
+                    bool keep = kz[j] > ckey;
+                    if (kz[j] == ckey && ties_left > 0) {
+                        keep = true;
+                        --ties_left;
+                    }
+                    if (keep) {
+                        keep_raw[kept] = win_raw[i0 + j];
+                        keep_idx[kept] = win_idx[i0 + j];
+                        ++kept;
+                    }
                 }
+            const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot_keep);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < kept) {
+                    win_raw[kp + j] = keep_raw[j];
+                    win_idx[kp + j] = keep_idx[j];
+                }
+            n = tot_keep;
+            mass = (double)(mass_above + (unsigned long long)need * qk) / kFix;
             fsync<NT>();
         }
     }
     // ---- 7. renormalised truncated distribution in fp64, CDF, samples, outputs ----------------------------
     double my_max = -INFINITY;
-    for (int i = tid; i < n; i += NT) {
-        const double y = (double)__uint_as_float(win_raw[i]) * cd;
-        wv[i] = y;
-        my_max = fmax(my_max, y);
-    }
+    for (int i = tid; i < n; i += NT) my_max = fmax(my_max, (double)__uint_as_float(win_raw[i]) * cd);
     const double mS = block_max_f64<NT>(my_max, tid, sh->scratch);
     double my_mass = 0.0;
     for (int i = tid; i < n; i += NT) {
-        if (!(p.top_p < 1.0f)) my_mass += exp2((double)__uint_as_float(win_raw[i]) * cf - L2);
-        const double w = exp2(wv[i] - mS);
-        wv[i] = w;
-        cum[i] = w;
+        const double z = (double)__uint_as_float(win_raw[i]);
+        if (!(p.top_p < 1.0f)) my_mass += exp2(z * cf - L2);
+        cum[i] = exp2(z * cd - mS);
     }
     if (!(p.top_p < 1.0f)) mass = block_sum_f64<NT>(my_mass, tid, sh->scratch);
     else fsync<NT>();
@@ -1228,7 +1290,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
             int pos2 = first_greater(cum, n, (double)u * W);
             if (pos2 >= n) {
                 pos2 = n - 1;
-                while (pos2 > 0 && !(wv[pos2] > 0.0)) --pos2;
+                while (pos2 > 0 && !(cum[pos2] - cum[pos2 - 1] > 0.0)) --pos2;  // the last entry with positive mass
             }
             tok = win_idx[pos2];
         }
@@ -1278,10 +1340,10 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     while (((ntiles + (1LL << glog) - 1) >> glog) > kMaxGroups) ++glog;
     pl.group_log2 = glog;
     pl.ngroups = (int)((ntiles + (1LL << glog) - 1) >> glog);
-    pl.tile_cap = 8 * k < 512 ? 512 : (8 * k > kMaxTileList ? kMaxTileList : 8 * k);
+    pl.tile_cap = 2 * k < 512 ? 512 : (2 * k > kMaxTileList ? kMaxTileList : 2 * k);  // some 1.1 to 1.4 k survive
     pl.cand_cap = 2 * k < 512 ? 512 : (2 * k > 2048 ? 2048 : 2 * k);
     pl.fin_threads = finish_threads(k);
-    pl.fin_smem = finish_layout(pl.ngroups, pl.tile_cap, pl.cand_cap, k, pl.nchunks).total;
+    pl.fin_smem = 0;  // (set below, once the split is known)
     // One CTA per row when the rows fill the machine; fewer rows are cut into segments (at least one
     // chunk per warp each) so that every CTA slot has work.  A segment costs nothing but its own
     // hand-over (8 (max, sum) pairs and a flag).
@@ -1306,6 +1368,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.stream_smem = stream_smem_bytes(pl.nchunks, pl.ngroups);
     pl.local_bound = pl.split.nseg == 1 && pl.stream_smem <= kStreamSmemLimit;
     if (!pl.local_bound) pl.stream_smem = 0;
+    pl.fin_smem = finish_layout(pl.ngroups, pl.tile_cap, pl.cand_cap, k, pl.nchunks, pl.local_bound).total;
     size_t off = kWsHeaderBytes;
     pl.ws_ready_off = off;
     off = align_up256(off + (size_t)rows * pl.split.nseg * sizeof(int));
