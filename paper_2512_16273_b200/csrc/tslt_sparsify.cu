@@ -960,6 +960,11 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
             uint32_t st_raw[kStash];
             int st_idx[kStash];
             int cnt = 0;
+            // every tile of this thread is asked of L2 first, so that the batches of loads below (six
+            // vectors in flight per thread) do not each pay a trip to HBM
+            for (int u = u0; u < u1; ++u)
+                if (u == u0 || (u & 3) == 0)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + (size_t)tl[u >> 2] * (kVecsPerTile * kVecBytes)));
             for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
 #pragma unroll
                 for (int e = 0; e < kPer; ++e)
