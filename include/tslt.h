@@ -119,6 +119,9 @@ int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
  *   draft_token[b, j]; accepted_len[b] = a = number of leading accepted positions;
  *   a < gamma:  out_token[b] ~ norm(max(0, p_a - q~_a)) over the FULL vocabulary;
  *   a = gamma:  out_token[b] ~ p_gamma (the bonus row); both use u_sample[b].
+ *   A residual whose total mass is at most 4e-7 (below the accuracy to which p is known; exact
+ *   arithmetic gives 0 there, e.g. a draft that equals the target on its support) is taken as
+ *   empty and out_token is drawn from the unmodified p_a instead.
  * Optional outputs (nullable): accept_prob[b, j] = min(1, p_j(x_j)/q~_j(x_j)),
  * beta_hat[b, j] = sum_{S_j} min(p_j, q~_j) (the truncated acceptance rate of Section
  * 3.2), lse_p[b, j] = ln sum exp(target row / target_temperature).

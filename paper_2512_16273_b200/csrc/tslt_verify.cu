@@ -26,6 +26,11 @@
 namespace tslt {
 
 constexpr int kMaxChunks = 2048;   // chunk partials of one row must fit the resolver's shared memory
+// A residual mass at or below this is taken as zero: p is known to the accuracy of the row's fp32
+// normaliser (a few 1e-7 relative), so a residual sum max(0, p - q~) this small is rounding noise of
+// a draft that equals the target on its support.  Exact arithmetic gives 0 there, and the verifier
+// then samples the unmodified p (the fall-back the method's degenerate case takes).
+constexpr double kMinResidualMass = 4.0e-7;
 constexpr int kMaxTreeNodes = 1024;
 
 struct VerifyParams {
@@ -196,7 +201,7 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
     consumer_sync();
     block_inclusive_scan(A.chunkR, nch, tid, sh->scratch);
     const double Z = A.chunkR[nch - 1];
-    if (!(Z > 0.0)) {
+    if (!(Z > kMinResidualMass)) {
         consumer_sync();
         return -1;
     }
@@ -230,6 +235,10 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
     consumer_sync();
     block_inclusive_scan(cumr, ne, tid, sh->scratch);
     const double Rc2 = cumr[ne - 1];
+    if (!(Rc2 > 0.0)) {  // the chunk's mass was rounding noise of the corrections: nothing to sample here
+        consumer_sync();
+        return -1;
+    }
     int pos = frac < 1.5 ? first_greater(cumr, ne, frac * Rc2) : ne;
     if (pos >= ne) {
         pos = ne - 1;
@@ -442,7 +451,7 @@ __device__ int resolve_tree_node(const VerifyParams& p, int b, int node, const f
             zs += d > 0.0 ? d : 0.0;
         }
         const double Z = block_sum(zs, tid, sh->scratch) + c_out * out_mass;
-        if (Z > 0.0) {
+        if (Z > kMinResidualMass) {
             for (int i = tid; i < n; i += kBlockThreads) {
                 const double d = A.s_a[i] - A.s_q[i];
                 A.s_a[i] = d > 0.0 ? d / Z : 0.0;

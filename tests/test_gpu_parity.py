@@ -214,6 +214,29 @@ def test_verify_edge_tokens_and_uniforms():
     assert ref["accepted_len"][2] == 0 and ref["accept_prob"][2, 0] == 0.0
 
 
+def test_degenerate_residual_takes_the_same_fallback():
+    """p = q~ on S and -inf elsewhere, drafted token outside S: the rejection leaves no residual mass.
+    The oracle then samples the unmodified p (flag DEGEN); the kernel must land on the same token."""
+    V, k, B = 5000, 3, 4
+    S = np.array([11, 2047, 4999], np.int32)
+    lg = np.array([0.5, 1.25, -0.75], np.float32)
+    zp = torch.full((B, 2, V), -float("inf"))
+    zp[:, 0, torch.from_numpy(S.astype(np.int64))] = torch.from_numpy(lg)
+    zp[:, 1] = torch.randn(V, generator=torch.Generator().manual_seed(1))
+    idx = np.tile(S, (B, 1, 1)); logit = np.tile(lg, (B, 1, 1)); count = np.full((B, 1), k, np.int32)
+    tok = np.full((B, 1), 7, np.int32)  # not in S, target logit -inf
+    ua = np.zeros((B, 1), np.float32)
+    us = np.array([0.0, 0.3, 0.55, 0.999], np.float32)
+    ref = oracle.verify(zp, idx, logit, count, tok, 1.0, 1.0, ua, us)
+    assert (ref["flags"] & oracle.FLAG_DEGEN).all() and (ref["accepted_len"] == 0).all()
+    gpu = tslt.verify(zp.cuda(), torch.from_numpy(idx).cuda(), torch.from_numpy(logit).cuda(), torch.from_numpy(count).cuda(),
+                      torch.from_numpy(tok).cuda(), 1.0, 1.0, torch.from_numpy(ua).cuda(), torch.from_numpy(us).cuda())
+    torch.cuda.synchronize()
+    inp = dict(zp=zp, idx=idx, logit=logit, count=count, token=tok, Tq=1.0, Tp=1.0, ua=ua, us=us)
+    compare_verify(gpu, ref, "degenerate residual", inputs=inp)
+    assert np.array_equal(to_np(gpu["out_token"]), ref["out_token"])
+
+
 def test_identical_models_accept_everything():
     B, gamma, V = 4, 5, 30000
     zq, _ = small_logits(B, gamma, V, torch.bfloat16, seed=12)
