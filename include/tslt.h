@@ -262,6 +262,32 @@ int tslt_pack_payload(const int* idx, const float* logit, const int* count, int 
 int tslt_unpack_payload(const unsigned int* payload, int rows, int k, int V, int prob_format,
                         int* idx, float* logit, int* count, int* device_flag, void* stream);
 
+/*
+ * Truncation diagnostics on pairs of (draft, target) rows: what Section 5's top-K mass and acceptance
+ * figures plot, and what Theorem 1 (Section 3.2) and Theorem 2 (Section 4.3) bound.  For row r, with
+ * q = softmax(draft_logits[r] / draft_temperature), p = softmax(target_logits[r] / target_temperature):
+ *   beta_j[r, j-1]  = beta^(j) = sum_v min(q, p^(j)), the acceptance rate of the j-th candidate, where
+ *                     p^(1) = p and p^(j+1) = norm(max(0, p^(j) - q)) (the residual update of Algorithm 5);
+ *                     beta^(1) is the acceptance-rate lemma's sum min(q, p) = 1 - TV(q, p);
+ *   z_j[r, j-1]     = Z^(j+1) = sum_v max(0, p^(j) - q), the normaliser of that update (= 1 - beta^(j));
+ *   theta[r]        = beta^(1) + sum_{i>=2} beta^(i) prod_{j<i} (1 - beta^(j)), the total acceptance;
+ *   and for every K = k_list[i] (top-K set of q in the order (logit descending, index ascending),
+ *   q^ = q / rho on it and 0 elsewhere: the truncation equation of Section 3.1):
+ *   rho[r, i]             = sum over the set of q (sigma = 1 - rho is the truncated mass of Theorem 1),
+ *   beta_hat_j[r, i, j-1] = the same chain with q^ in place of q,
+ *   theta_hat[r, i]       = its total acceptance.
+ * k_list is a HOST array of n_k (1..16) strictly ascending values, each <= min(V, TSLT_MAX_K);
+ * 1 <= num_candidates <= 8; a row with fewer finite logits than K uses them all.  The rows are
+ * streamed 2 + 2 * num_candidates times: a diagnostic, not a hot path.  Workspace from
+ * tslt_diagnostics_workspace_bytes(rows, V, largest K, num_candidates).  All outputs fp32, required.
+ */
+int tslt_diagnostics_workspace_bytes(int rows, int V, int k_max, int num_candidates, size_t* bytes);
+int tslt_diagnostics(const void* draft_logits, const void* target_logits, int dtype, int rows, int V,
+                     long long row_stride_elems, const int* k_list, int n_k, int num_candidates,
+                     float draft_temperature, float target_temperature, float* beta_j, float* z_j,
+                     float* theta, float* rho, float* beta_hat_j, float* theta_hat, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,8 @@ EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status", "tslt_
            "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
            "tslt_tree_verify_walk_workspace_bytes", "tslt_tree_verify_walk",
-           "tslt_payload_words", "tslt_pack_payload", "tslt_unpack_payload"]
+           "tslt_payload_words", "tslt_pack_payload", "tslt_unpack_payload",
+           "tslt_diagnostics_workspace_bytes", "tslt_diagnostics"]
 
 PROB_F32, PROB_BF16, PROB_F16 = 0, 1, 2
 
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
     L.tslt_tree_verify_walk_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_tree_verify_walk.restype = i
     L.tslt_tree_verify_walk.argtypes = L.tslt_tree_verify.argtypes
+    L.tslt_diagnostics_workspace_bytes.restype = i
+    L.tslt_diagnostics_workspace_bytes.argtypes = [i, i, i, i, psz]
+    L.tslt_diagnostics.restype = i
+    L.tslt_diagnostics.argtypes = [p, p, i, i, i, ll, p, i, i, f, f, p, p, p, p, p, p, p, sz, p]
     L.tslt_payload_words.restype = i
     L.tslt_payload_words.argtypes = [i, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.tslt_pack_payload.restype = i
@@ -447,4 +452,34 @@ def unpack_payload(payload: torch.Tensor, k: int, V: int, prob_format: int) -> d
          "flag": torch.zeros(1, dtype=torch.int32, device=dev)}
     _check(lib().tslt_unpack_payload(_ptr(payload), rows, k, V, prob_format, _ptr(o["idx"]), _ptr(o["logit"]),
                                      _ptr(o["count"]), _ptr(o["flag"]), _stream()), "tslt_unpack_payload")
+    return o
+
+
+def diagnostics(draft_logits: torch.Tensor, target_logits: torch.Tensor, k_list: Sequence[int], num_candidates: int,
+                draft_temperature: float = 1.0, target_temperature: float = 1.0) -> dict:
+    """tslt_diagnostics on paired rows [rows, V]: dict(beta_j, z_j [rows, c], theta [rows], rho, theta_hat
+    [rows, n_k], beta_hat_j [rows, n_k, c]), all fp32."""
+    if not draft_logits.is_cuda or not target_logits.is_cuda:
+        raise ValueError("logits must be CUDA tensors (libtslt has no CPU path)")
+    if draft_logits.shape != target_logits.shape or draft_logits.dtype != target_logits.dtype:
+        raise ValueError("draft and target logits must have the same shape and dtype")
+    rows, V, stride = _row_layout(draft_logits)
+    rows2, _, stride2 = _row_layout(target_logits)
+    if stride != stride2 or rows != rows2:
+        raise ValueError("draft and target logits must have the same row layout")
+    ks = np.ascontiguousarray(np.asarray(list(k_list), dtype=np.int32))
+    nk, c, dev = int(ks.size), int(num_candidates), draft_logits.device
+    o = {"beta_j": torch.empty(rows, c, device=dev), "z_j": torch.empty(rows, c, device=dev),
+         "theta": torch.empty(rows, device=dev), "rho": torch.empty(rows, nk, device=dev),
+         "beta_hat_j": torch.empty(rows, nk, c, device=dev), "theta_hat": torch.empty(rows, nk, device=dev)}
+    n = ctypes.c_size_t(0)
+    _check(lib().tslt_diagnostics_workspace_bytes(rows, V, int(ks.max()) if nk else 1, c, ctypes.byref(n)),
+           "tslt_diagnostics_workspace_bytes")
+    ws = torch.empty(max(int(n.value), 256), dtype=torch.uint8, device=dev)
+    rc = lib().tslt_diagnostics(_ptr(draft_logits), _ptr(target_logits), _dtype_code(draft_logits), rows, V, stride,
+                                ks.ctypes.data_as(ctypes.c_void_p), nk, c, draft_temperature, target_temperature,
+                                _ptr(o["beta_j"]), _ptr(o["z_j"]), _ptr(o["theta"]), _ptr(o["rho"]), _ptr(o["beta_hat_j"]),
+                                _ptr(o["theta_hat"]), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "tslt_diagnostics")
+    o["workspace"] = ws
     return o
