@@ -63,6 +63,9 @@ extern "C" {
 /* largest supported k (top-k size, or the candidate cap when top-p is on) */
 #define TSLT_MAX_K 1024
 
+/* most vocabulary shards one tslt_sparsify_merge takes; it also needs nshards * k <= 2048 */
+#define TSLT_MAX_SHARDS 16
+
 /* size of the scratch array built into the library for tslt_verify_static */
 #define TSLT_STATIC_SCRATCH_BYTES (8u << 20)
 
@@ -109,6 +112,42 @@ int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
                   int num_samples, const float* uniforms, int* idx, float* logit, int* count,
                   int* token, float* lse, float* mass, void* workspace, size_t workspace_bytes,
                   void* stream);
+
+/*
+ * tslt_sparsify over a vocabulary that is split across devices (tensor-parallel output
+ * projection): every shard runs the truncation on its own slice, and one small merge turns the
+ * shards' results into exactly what tslt_sparsify gives on the whole row.  It rests on two facts:
+ * the k best tokens of the row (logit descending, index ascending) are among the k best of
+ * their own shards, and the row's normaliser is the sum of the shards' (Section 3.1's truncation
+ * equation needs nothing else of the row).
+ *
+ * tslt_sparsify_shard: tslt_sparsify on the shard's [rows, V_shard] logits with top_p = 1 and no
+ * samples.  idx holds indices LOCAL to the shard (ascending, -1 padded), logit the stored logits,
+ * count the number kept (min(k, finite logits of the shard)), lse2 [rows] (fp64) the base-2 log of
+ * sum 2^(z * log2(e) / temperature) over the shard (-inf if it has no finite logit).  Requires
+ * 1 <= k <= min(V_shard, TSLT_MAX_K); workspace as tslt_sparsify_workspace_bytes(rows, V_shard,
+ * k, 0) says.
+ *
+ * tslt_sparsify_merge: part_idx / part_logit [nshards, rows, k], part_count / part_lse2 [nshards,
+ * rows] are the shards' outputs side by side in ascending vocabulary order (on several devices:
+ * after an all-gather of these 8 k + 12 bytes per shard and row; no logits cross the link);
+ * shard_offset is a HOST array of nshards token ids, strictly ascending, the global id of each
+ * shard's first logit.  dtype is the element type the shards read (it fixes which logit values
+ * can occur).  Outputs, top_p, temperature, num_samples and uniforms as in tslt_sparsify, for the
+ * whole-vocabulary row; a part_count outside [0, k] or a part_idx below zero is read as an empty
+ * entry.  Requires 1 <= nshards <= TSLT_MAX_SHARDS and nshards * k <= 2048
+ * (TSLT_ERR_UNSUPPORTED otherwise); workspace >= 256 bytes (the status word), 256-byte aligned.
+ */
+int tslt_sparsify_shard(const void* logits, int dtype, int rows, int V_shard,
+                        long long row_stride_elems, int k, float temperature, int* idx,
+                        float* logit, int* count, double* lse2, void* workspace,
+                        size_t workspace_bytes, void* stream);
+int tslt_sparsify_merge(int dtype, int rows, int nshards, const int* shard_offset, int k,
+                        const int* part_idx, const float* part_logit, const int* part_count,
+                        const double* part_lse2, float top_p, float temperature, int num_samples,
+                        const float* uniforms, int* idx, float* logit, int* count, int* token,
+                        float* lse, float* mass, void* workspace, size_t workspace_bytes,
+                        void* stream);
 
 /*
  * Verifier side, single candidate: speculative sampling against the sparse draft

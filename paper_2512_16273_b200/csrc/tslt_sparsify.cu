@@ -40,6 +40,8 @@ constexpr int kSparsifyStreamCtasPerSm = 5;  // 51 registers, no spills (6 CTAs 
 constexpr int kMaxGroups = 4096;          // group maxima the finish kernel bisects over
 constexpr int kMaxTileList = 4096;        // survivor tiles it can list
 constexpr int kSelBins = 1024;            // bins of the selection histogram
+constexpr int kMaxShards = TSLT_MAX_SHARDS;  // vocabulary shards one merge takes
+constexpr int kMaxMergeList = 2048;       // candidates the merge holds (nshards * k)
 constexpr uint32_t kLowestFinite16 = 0x0080u;   // key of -FLT_MAX >> 16
 constexpr uint32_t kHighestFinite16 = 0xff7fu;  // key of +FLT_MAX >> 16
 
@@ -69,6 +71,7 @@ struct SparsifyParams {
     int* token;
     float* lse;
     float* mass;
+    double* lse2;     // optional: the row's base-2 log-normaliser in fp64 (what a vocabulary shard hands to the merge)
     int nchunks;
     RowSplit split;
     int group_log2;   // tiles per group = 1 << group_log2
@@ -82,6 +85,13 @@ struct SparsifyParams {
     unsigned short* tile_max; // rows cut into segments: [rows, nchunks * 32], top 16 bits of each tile's largest logit, slot order
     uint32_t* row_list;       // whole-row CTAs: [rows, tile_cap] survivor tiles in address order
     int local_bound;          // 1: each row is one streaming CTA, which finds the bound and lists the survivors itself
+    // merge of vocabulary shards only: what the shards handed over, [nshards, rows, part_k] / [nshards, rows]
+    int nshards, part_k;
+    const int* part_idx;
+    const float* part_logit;
+    const int* part_count;
+    const double* part_lse2;
+    int shard_offset[kMaxShards];  // token index of each shard's first logit
 };
 
 // Tile a of a row is its bytes [64 a, 64 a + 64).  In the streaming kernel vector j * 32 + l of a
@@ -702,18 +712,275 @@ __device__ __forceinline__ int finite_key16(float z) {
     return (k16 >= kLowestFinite16 && k16 <= kHighestFinite16) ? (int)k16 : -1;
 }
 
+// The exact top-k of a candidate list held in shared memory in ascending token index (c_raw: raw
+// logit bits, c_idx: token indices, n_c <= 8 * NT entries): ties at the k-th logit go to the lower
+// index.  The winners are compacted in place, still in ascending index; returns how many there are.
+// All NT threads call it; hist holds kSelBins words (it doubles as the rank-counting keys).
+template <typename T, int NT>
+__device__ __forceinline__ int select_in_list(int k, uint32_t* c_raw, int* c_idx, int n_c, uint32_t* hist, FinishShared* sh, int tid) {
+    constexpr bool kBf16 = (Elt<T>::kBytes == 2);
+    constexpr int kHeld = 8;  // most list entries a thread owns
+    unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
+    int n = 0;
+    {
+        // the candidates sit in shared memory in index order; thread t owns entries [i0, i1)
+        const int ipt = (n_c + NT - 1) / NT;  // <= kHeld
+        const int i0 = min(n_c, tid * ipt), i1 = min(n_c, i0 + ipt);
+        uint32_t winmask = 0;  // bit j: entry i0 + j is a winner
+        if (n_c <= k) {
+            winmask = (i1 - i0) >= 32 ? 0xffffffffu : ((1u << (i1 - i0)) - 1u);
+        } else if (n_c <= kRankListMax) {
+            // few candidates: count each one's rank under (logit descending, index ascending)
+            for (int i = tid; i < n_c; i += NT)
+                rkeys[i] = ((unsigned long long)float_to_key(__uint_as_float(c_raw[i])) << 32) |
+                           (unsigned long long)(0xffffffffu - (uint32_t)c_idx[i]);
+            fsync<NT>();
+            for (int i = i0; i < i1; ++i) {
+                const unsigned long long mine = rkeys[i];
+                int r = 0;
+                for (int j = 0; j < n_c; ++j) r += rkeys[j] > mine ? 1 : 0;
+                if (r < k) winmask |= 1u << (i - i0);
+            }
+        } else {
+            // many candidates: the k-th largest 16-bit key by two histogram passes, (fp32 rows) the low
+            // 16 bits inside that key the same way; ties by position
+            int above = 0;
+            const uint32_t e16 = radix_kth16<NT>(k, [&](auto f) {
+                for (int i = i0; i < i1; ++i) f(float_to_key(__uint_as_float(c_raw[i])) >> 16);
+            }, hist, &sh->sel_bin, tid, &above);
+            int need = k - above;
+            uint32_t e32;
+            if (kBf16) {
+                e32 = (e16 << 16) | ((e16 & 0x8000u) ? 0u : 0xffffu);  // keys of bf16 values: the low half follows the sign
+            } else {
+                int above2 = 0;
+                const uint32_t low = radix_kth16<NT>(need, [&](auto f) {
+                    for (int i = i0; i < i1; ++i) {
+                        const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
+                        if ((kz >> 16) == e16) f(kz & 0xffffu);
+                    }
+                }, hist, &sh->sel_bin, tid, &above2);
+                e32 = (e16 << 16) | low;
+                need -= above2;
+            }
+            int c_eq = 0;
+            for (int i = i0; i < i1; ++i) c_eq += float_to_key(__uint_as_float(c_raw[i])) == e32 ? 1 : 0;
+            int tot_eq;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            int ties_left = max(0, min(c_eq, need - eq_before));
+            for (int i = i0; i < i1; ++i) {
+                const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
+                bool win = kz > e32;
+                if (kz == e32 && ties_left > 0) {
+                    win = true;
+                    --ties_left;
+                }
+                if (win) winmask |= 1u << (i - i0);
+            }
+        }
+        // compact the winners in place: every thread reads its own first, then all write
+        uint32_t my_raw[kHeld];
+        int my_idx[kHeld];
+        int my_wins = 0;
+#pragma unroll
+        for (int j = 0; j < kHeld; ++j)
+            if ((winmask >> j) & 1u) {
+                my_raw[my_wins] = c_raw[i0 + j];
+                my_idx[my_wins] = c_idx[i0 + j];
+                ++my_wins;
+            }
+        int wpos = block_exscan<NT>(my_wins, tid, sh->iscr, &n);
+#pragma unroll
+        for (int j = 0; j < kHeld; ++j)
+            if (j < my_wins) {
+                c_raw[wpos + j] = my_raw[j];
+                c_idx[wpos + j] = my_idx[j];
+            }
+        fsync<NT>();
+    }
+    return n;
+}
+
+// Steps 6 and 7 of the finish: the top-rho cut of the n winners (c_raw / c_idx, ascending index), the
+// renormalised truncated distribution and its CDF in fp64 (cum: >= k doubles), the samples by inverse
+// CDF and the row's outputs.  L2 is the base-2 log of the full-vocabulary normaliser.  All NT threads call it.
+template <typename T, int NT>
+__device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int row, int n, uint32_t* c_raw, int* c_idx,
+                                                 double L2, uint32_t* hist, double* cum, FinishShared* sh, int tid) {
+    constexpr bool kBf16 = (Elt<T>::kBytes == 2);
+    const int lane = tid & 31, k = p.k;
+    const int n0 = n;
+    uint32_t* win_raw = c_raw;
+    int* win_idx = c_idx;
+    const double cf = (double)p.c.f;  // the scale the streaming sum used: keeps q consistent with the normaliser
+    const double cd = p.c.d;
+    double mass = 0.0;
+    // ---- 6. top-rho cut ---------------------------------------------------------------------------------------
+    // The smallest n whose cumulative q, in the order (logit descending, index ascending), reaches
+    // top_p.  No sort: the key of the entry at which the cumulative crosses is the largest t with
+    // mass(key >= t) >= top_p, found bit by bit with one block reduction per bit; then the ties of
+    // that key, which all carry the same q, are counted off in index order.  Masses are summed as
+    // 2^-62 fixed point, so the sums do not depend on the order of the adds: deterministic.  (A
+    // histogram of mass per key byte needs 64-bit shared atomics on a handful of hot bins and was
+    // three times slower than the sort it replaced; the bisection is three times faster.)
+    if (n0 > 0 && p.top_p < 1.0f) {
+        constexpr double kFix = 4611686018427387904.0;  // 2^62
+        unsigned long long* mhist = reinterpret_cast<unsigned long long*>(hist);  // 256 bins
+        const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
+        const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
+        uint32_t kz[4];
+        unsigned long long qf[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            kz[j] = 0u;
+            qf[j] = 0ull;
+            if (i0 + j < i1) {
+                const float z = __uint_as_float(win_raw[i0 + j]);
+                kz[j] = float_to_key(z);
+                qf[j] = __double2ull_rn(fmin(exp2((double)z * cf - L2), 1.0) * kFix);
+            }
+        }
+        const unsigned long long target = __double2ull_rn((double)p.top_p * kFix);
+        // mass of the entries whose key is >= t, over the block (fixed point: any order gives the same sum)
+        auto mass_from = [&](uint32_t t, int slot) -> unsigned long long {
+            unsigned long long m = 0ull;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1 && kz[j] >= t) m += qf[j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+            if (lane == 0 && m) smem_add64(&mhist[slot], m);  // one add per warp: 4 or 8 in all
+            fsync<NT>();
+            return mhist[slot];
+        };
+        for (int i = tid; i < 40; i += NT) mhist[i] = 0ull;
+        if (tid == 0) sh->scratch[1] = 0.0;
+        fsync<NT>();
+        unsigned long long mass_above = 0ull;
+        uint32_t prefix = 0u;
+        bool crossed = mass_from(0u, 0) >= target;
+        if (!crossed) {
+            mass_above = mhist[0];  // the whole mass: the cumulative never reaches top_p, everything is kept
+        } else {
+            // the crossing key: the largest t with mass(key >= t) >= top_p, bit by bit
+            int slot = 1;
+            unsigned long long last_rejected = 0ull;
+#pragma unroll 1
+            for (int bit = 31; bit >= (kBf16 ? 16 : 0); --bit) {
+                const uint32_t cand = prefix | (1u << bit);
+                const unsigned long long m = mass_from(cand, slot++);
+                if (m >= target) prefix = cand;
+                else last_rejected = m;
+            }
+            mass_above = last_rejected;  // mass of the keys above the crossing key (the last candidate refused is that key + 1 ulp)
+        }
+        if (!crossed) {
+            mass = (double)mass_above / kFix;
+        } else {
+            // (keys of bf16 values: the low half follows the sign and was not searched)
+            const uint32_t ckey = kBf16 ? ((prefix & 0xffff0000u) | ((prefix & 0x80000000u) ? 0u : 0xffffu)) : prefix;
+            // the ties of the crossing key share one q: how many of them, in index order, it takes
+            int c_gt = 0, c_eq = 0;
+            unsigned long long qk = 0ull;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1) {
+                    c_gt += kz[j] > ckey ? 1 : 0;
+                    if (kz[j] == ckey) {
+                        ++c_eq;
+                        qk = qf[j];
+                    }
+                }
+            if (qk) sh->scratch[1] = __longlong_as_double((long long)qk);  // (every writer writes the same value)
+            int tot_eq, tot_keep;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            qk = (unsigned long long)__double_as_longlong(sh->scratch[1]);
+            const unsigned long long missing = target - mass_above;  // > 0: the bins above did not reach it
+            int need = qk ? (int)min((unsigned long long)tot_eq, (missing + qk - 1ull) / qk) : tot_eq;
+            if (need < 1) need = 1;
+            const int my_ties = max(0, min(c_eq, need - eq_before));
+            // keep the larger keys and the first `need` ties: read mine, then (after the scan's barriers) write
+            uint32_t keep_raw[4];
+            int keep_idx[4];
+            int kept = 0, ties_left = my_ties;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < i1) {
+                    bool keep = kz[j] > ckey;
+                    if (kz[j] == ckey && ties_left > 0) {
+                        keep = true;
+                        --ties_left;
+                    }
+                    if (keep) {
+                        keep_raw[kept] = win_raw[i0 + j];
+                        keep_idx[kept] = win_idx[i0 + j];
+                        ++kept;
+                    }
+                }
+            const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot_keep);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < kept) {
+                    win_raw[kp + j] = keep_raw[j];
+                    win_idx[kp + j] = keep_idx[j];
+                }
+            n = tot_keep;
+            mass = (double)(mass_above + (unsigned long long)need * qk) / kFix;
+            fsync<NT>();
+        }
+    }
+    // ---- 7. renormalised truncated distribution in fp64, CDF, samples, outputs ----------------------------
+    double my_max = -INFINITY;
+    for (int i = tid; i < n; i += NT) my_max = fmax(my_max, (double)__uint_as_float(win_raw[i]) * cd);
+    const double mS = block_max_f64<NT>(my_max, tid, sh->scratch);
+    double my_mass = 0.0;
+    for (int i = tid; i < n; i += NT) {
+        const double z = (double)__uint_as_float(win_raw[i]);
+        if (!(p.top_p < 1.0f)) my_mass += exp2(z * cf - L2);
+        cum[i] = exp2(z * cd - mS);
+    }
+    if (!(p.top_p < 1.0f)) mass = block_sum_f64<NT>(my_mass, tid, sh->scratch);
+    else fsync<NT>();
+    block_inclusive_scan_f64<NT>(cum, n, tid, sh->scratch);
+
+    int* o_idx = p.idx + (size_t)row * k;
+    float* o_logit = p.logit + (size_t)row * k;
+    for (int i = tid; i < k; i += NT) {
+        o_idx[i] = i < n ? win_idx[i] : -1;
+        o_logit[i] = i < n ? __uint_as_float(win_raw[i]) : -INFINITY;
+    }
+    if (tid == 0) {
+        p.count[row] = n;
+        if (p.lse) p.lse[row] = n0 > 0 ? (float)(L2 * 0.6931471805599453) : -INFINITY;
+        if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
+        if (p.lse2) p.lse2[row] = n0 > 0 ? L2 : -INFINITY;
+    }
+    const double W = n > 0 ? cum[n - 1] : 0.0;
+    for (int sidx = tid; sidx < p.num_samples; sidx += NT) {
+        int tok = -1;
+        if (n > 0) {
+            const float u = clamp_uniform(p.uniforms[(size_t)row * p.num_samples + sidx]);
+            int pos2 = first_greater(cum, n, (double)u * W);
+            if (pos2 >= n) {
+                pos2 = n - 1;
+                while (pos2 > 0 && !(cum[pos2] - cum[pos2 - 1] > 0.0)) --pos2;  // the last entry with positive mass
+            }
+            tok = win_idx[pos2];
+        }
+        p.token[(size_t)row * p.num_samples + sidx] = tok;
+    }
+}
+
 template <typename T, int NT>
 __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kernel(const SparsifyParams p) {
     constexpr int kPer = Elt<T>::kPerVec;
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
-    constexpr int kHeld = 8;  // most list entries a thread owns (cand_cap <= 8 * NT, see the plan)
     extern __shared__ __align__(128) unsigned char smem_raw[];
     FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
     static_assert(sizeof(FinishShared) <= kFinishHeaderBytes, "header");
     const int k = p.k;
     const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks, p.local_bound != 0);
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + L.hist);
-    unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
     uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + L.a);
     uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + L.b);
     double* cum = reinterpret_cast<double*>(tl);
@@ -1003,80 +1270,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     // ---- 5. the exact top-k (ties at the k-th logit to the lower index), left in ascending index ----------
     int n = 0;
     if (in_smem) {
-        // the candidates sit in shared memory in index order; thread t owns entries [i0, i1)
-        const int ipt = (n_c + NT - 1) / NT;  // <= kHeld
-        const int i0 = min(n_c, tid * ipt), i1 = min(n_c, i0 + ipt);
-        uint32_t winmask = 0;  // bit j: entry i0 + j is a winner
-        if (n_c <= k) {
-            winmask = (i1 - i0) >= 32 ? 0xffffffffu : ((1u << (i1 - i0)) - 1u);
-        } else if (n_c <= kRankListMax) {
-            // few candidates: count each one's rank under (logit descending, index ascending)
-            for (int i = tid; i < n_c; i += NT)
-                rkeys[i] = ((unsigned long long)float_to_key(__uint_as_float(c_raw[i])) << 32) |
-                           (unsigned long long)(0xffffffffu - (uint32_t)c_idx[i]);
-            fsync<NT>();
-            for (int i = i0; i < i1; ++i) {
-                const unsigned long long mine = rkeys[i];
-                int r = 0;
-                for (int j = 0; j < n_c; ++j) r += rkeys[j] > mine ? 1 : 0;
-                if (r < k) winmask |= 1u << (i - i0);
-            }
-        } else {
-            // many candidates: the k-th largest 16-bit key by two histogram passes, (fp32 rows) the low
-            // 16 bits inside that key the same way; ties by position
-            int above = 0;
-            const uint32_t e16 = radix_kth16<NT>(k, [&](auto f) {
-                for (int i = i0; i < i1; ++i) f(float_to_key(__uint_as_float(c_raw[i])) >> 16);
-            }, hist, &sh->sel_bin, tid, &above);
-            int need = k - above;
-            uint32_t e32;
-            if (kBf16) {
-                e32 = (e16 << 16) | ((e16 & 0x8000u) ? 0u : 0xffffu);  // keys of bf16 values: the low half follows the sign
-            } else {
-                int above2 = 0;
-                const uint32_t low = radix_kth16<NT>(need, [&](auto f) {
-                    for (int i = i0; i < i1; ++i) {
-                        const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
-                        if ((kz >> 16) == e16) f(kz & 0xffffu);
-                    }
-                }, hist, &sh->sel_bin, tid, &above2);
-                e32 = (e16 << 16) | low;
-                need -= above2;
-            }
-            int c_eq = 0;
-            for (int i = i0; i < i1; ++i) c_eq += float_to_key(__uint_as_float(c_raw[i])) == e32 ? 1 : 0;
-            int tot_eq;
-            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
-            int ties_left = max(0, min(c_eq, need - eq_before));
-            for (int i = i0; i < i1; ++i) {
-                const uint32_t kz = float_to_key(__uint_as_float(c_raw[i]));
-                bool win = kz > e32;
-                if (kz == e32 && ties_left > 0) {
-                    win = true;
-                    --ties_left;
-                }
-                if (win) winmask |= 1u << (i - i0);
-            }
-        }
-        // compact the winners in place: every thread reads its own first, then all write
-        uint32_t my_raw[kHeld];
-        int my_idx[kHeld];
-        int my_wins = 0;
-#pragma unroll
-        for (int j = 0; j < kHeld; ++j)
-            if ((winmask >> j) & 1u) {
-                my_raw[my_wins] = c_raw[i0 + j];
-                my_idx[my_wins] = c_idx[i0 + j];
-                ++my_wins;
-            }
-        int wpos = block_exscan<NT>(my_wins, tid, sh->iscr, &n);
-#pragma unroll
-        for (int j = 0; j < kHeld; ++j)
-            if (j < my_wins) {
-                c_raw[wpos + j] = my_raw[j];
-                c_idx[wpos + j] = my_idx[j];
-            }
-        fsync<NT>();
+        n = select_in_list<T, NT>(k, c_raw, c_idx, n_c, hist, sh, tid);
     } else if (max16 >= lo16) {
         // The survivors do not fit (thousands of tied tile maxima, or more candidates than the list
         // holds): the same selection over the survivors' vectors, or all of the row's, in global
@@ -1142,168 +1336,67 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
             fsync<NT>();
         }
     }
-    const int n0 = n;
-    uint32_t* win_raw = c_raw;
-    int* win_idx = c_idx;
-    const double cf = (double)p.c.f;  // the scale the streaming sum used: keeps q consistent with the normaliser
-    const double cd = p.c.d;
-    double mass = 0.0;
-    // ---- 6. top-rho cut ---------------------------------------------------------------------------------------
-    // The smallest n whose cumulative q, in the order (logit descending, index ascending), reaches
-    // top_p.  No sort: the key of the entry at which the cumulative crosses is the largest t with
-    // mass(key >= t) >= top_p, found bit by bit with one block reduction per bit; then the ties of
-    // that key, which all carry the same q, are counted off in index order.  Masses are summed as
-    // 2^-62 fixed point, so the sums do not depend on the order of the adds: deterministic.  (A
-    // histogram of mass per key byte needs 64-bit shared atomics on a handful of hot bins and was
-    // three times slower than the sort it replaced; the bisection is three times faster.)
-    if (n0 > 0 && p.top_p < 1.0f) {
-        constexpr double kFix = 4611686018427387904.0;  // 2^62
-        unsigned long long* mhist = reinterpret_cast<unsigned long long*>(hist);  // 256 bins
-        const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
-        const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
-        uint32_t kz[4];
-        unsigned long long qf[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            kz[j] = 0u;
-            qf[j] = 0ull;
-            if (i0 + j < i1) {
-                const float z = __uint_as_float(win_raw[i0 + j]);
-                kz[j] = float_to_key(z);
-                qf[j] = __double2ull_rn(fmin(exp2((double)z * cf - L2), 1.0) * kFix);
-            }
-        }
-        const unsigned long long target = __double2ull_rn((double)p.top_p * kFix);
-        // mass of the entries whose key is >= t, over the block (fixed point: any order gives the same sum)
-        auto mass_from = [&](uint32_t t, int slot) -> unsigned long long {
-            unsigned long long m = 0ull;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j < i1 && kz[j] >= t) m += qf[j];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
-            if (lane == 0 && m) smem_add64(&mhist[slot], m);  // one add per warp: 4 or 8 in all
-            fsync<NT>();
-            return mhist[slot];
-        };
-        for (int i = tid; i < 40; i += NT) mhist[i] = 0ull;
-        if (tid == 0) sh->scratch[1] = 0.0;
-        fsync<NT>();
-        unsigned long long mass_above = 0ull;
-        uint32_t prefix = 0u;
-        bool crossed = mass_from(0u, 0) >= target;
-        if (!crossed) {
-            mass_above = mhist[0];  // the whole mass: the cumulative never reaches top_p, everything is kept
-        } else {
-            // the crossing key: the largest t with mass(key >= t) >= top_p, bit by bit
-            int slot = 1;
-            unsigned long long last_rejected = 0ull;
-#pragma unroll 1
-            for (int bit = 31; bit >= (kBf16 ? 16 : 0); --bit) {
-                const uint32_t cand = prefix | (1u << bit);
-                const unsigned long long m = mass_from(cand, slot++);
-                if (m >= target) prefix = cand;
-                else last_rejected = m;
-            }
-            mass_above = last_rejected;  // mass of the keys above the crossing key (the last candidate refused is that key + 1 ulp)
-        }
-        if (!crossed) {
-            mass = (double)mass_above / kFix;
-        } else {
-            // (keys of bf16 values: the low half follows the sign and was not searched)
-            const uint32_t ckey = kBf16 ? ((prefix & 0xffff0000u) | ((prefix & 0x80000000u) ? 0u : 0xffffu)) : prefix;
-            // the ties of the crossing key share one q: how many of them, in index order, it takes
-            int c_gt = 0, c_eq = 0;
-            unsigned long long qk = 0ull;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j < i1) {
-                    c_gt += kz[j] > ckey ? 1 : 0;
-                    if (kz[j] == ckey) {
-                        ++c_eq;
-                        qk = qf[j];
-                    }
-                }
-            if (qk) sh->scratch[1] = __longlong_as_double((long long)qk);  // (every writer writes the same value)
-            int tot_eq, tot_keep;
-            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
-            qk = (unsigned long long)__double_as_longlong(sh->scratch[1]);
-            const unsigned long long missing = target - mass_above;  // > 0: the bins above did not reach it
-            int need = qk ? (int)min((unsigned long long)tot_eq, (missing + qk - 1ull) / qk) : tot_eq;
-            if (need < 1) need = 1;
-            const int my_ties = max(0, min(c_eq, need - eq_before));
-            // keep the larger keys and the first `need` ties: read mine, then (after the scan's barriers) write
-            uint32_t keep_raw[4];
-            int keep_idx[4];
-            int kept = 0, ties_left = my_ties;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j < i1) {
-                    bool keep = kz[j] > ckey;
-                    if (kz[j] == ckey && ties_left > 0) {
-                        keep = true;
-                        --ties_left;
-                    }
-                    if (keep) {
-                        keep_raw[kept] = win_raw[i0 + j];
-                        keep_idx[kept] = win_idx[i0 + j];
-                        ++kept;
-                    }
-                }
-            const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot_keep);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j < kept) {
-                    win_raw[kp + j] = keep_raw[j];
-                    win_idx[kp + j] = keep_idx[j];
-                }
-            n = tot_keep;
-            mass = (double)(mass_above + (unsigned long long)need * qk) / kFix;
-            fsync<NT>();
-        }
-    }
-    // ---- 7. renormalised truncated distribution in fp64, CDF, samples, outputs ----------------------------
-    double my_max = -INFINITY;
-    for (int i = tid; i < n; i += NT) my_max = fmax(my_max, (double)__uint_as_float(win_raw[i]) * cd);
-    const double mS = block_max_f64<NT>(my_max, tid, sh->scratch);
-    double my_mass = 0.0;
-    for (int i = tid; i < n; i += NT) {
-        const double z = (double)__uint_as_float(win_raw[i]);
-        if (!(p.top_p < 1.0f)) my_mass += exp2(z * cf - L2);
-        cum[i] = exp2(z * cd - mS);
-    }
-    if (!(p.top_p < 1.0f)) mass = block_sum_f64<NT>(my_mass, tid, sh->scratch);
-    else fsync<NT>();
-    block_inclusive_scan_f64<NT>(cum, n, tid, sh->scratch);
-
-    int* o_idx = p.idx + (size_t)row * k;
-    float* o_logit = p.logit + (size_t)row * k;
-    for (int i = tid; i < k; i += NT) {
-        o_idx[i] = i < n ? win_idx[i] : -1;
-        o_logit[i] = i < n ? __uint_as_float(win_raw[i]) : -INFINITY;
-    }
-    if (tid == 0) {
-        p.count[row] = n;
-        if (p.lse) p.lse[row] = n0 > 0 ? (float)(L2 * 0.6931471805599453) : -INFINITY;
-        if (p.mass) p.mass[row] = n0 > 0 ? (float)mass : 0.f;
-    }
-    const double W = n > 0 ? cum[n - 1] : 0.0;
-    for (int sidx = tid; sidx < p.num_samples; sidx += NT) {
-        int tok = -1;
-        if (n > 0) {
-            const float u = clamp_uniform(p.uniforms[(size_t)row * p.num_samples + sidx]);
-            int pos2 = first_greater(cum, n, (double)u * W);
-            if (pos2 >= n) {
-                pos2 = n - 1;
-                while (pos2 > 0 && !(cum[pos2] - cum[pos2 - 1] > 0.0)) --pos2;  // the last entry with positive mass
-            }
-            tok = win_idx[pos2];
-        }
-        p.token[(size_t)row * p.num_samples + sidx] = tok;
-    }
+    cut_sample_write<T, NT>(p, row, n, c_raw, c_idx, L2, hist, cum, sh, tid);
     // this kernel's completion must imply the streaming kernel's (what follows on the stream relies
     // on it): one CTA sees to that; the others leave and make room
     if (row == 0) wait_for_primary_kernel();
+}
+
+// ---- merge of vocabulary shards ------------------------------------------------------------------------
+// One CTA of 256 threads per row.  The shards' (index, logit) lists, each ascending in its own
+// indices, laid end to end in shard order are one candidate list in ascending token index: exactly
+// what the finish kernel's selection works on.  The row's normaliser is the sum of the shards'.
+constexpr int kMergeThreads = 256;
+template <typename T>
+__global__ void __launch_bounds__(kMergeThreads, 4) sparsify_merge_kernel(const SparsifyParams p) {
+    constexpr int NT = kMergeThreads;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
+    const int k = p.k;
+    const FinishLayout L = finish_layout(0, 0, p.cand_cap, k, 0, true);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + L.hist);
+    double* cum = reinterpret_cast<double*>(smem_raw + L.b);
+    uint32_t* c_raw = reinterpret_cast<uint32_t*>(smem_raw + L.c);
+    int* c_idx = reinterpret_cast<int*>(c_raw + p.cand_cap);
+    const int tid = threadIdx.x, lane = tid & 31, row = blockIdx.x, S = p.nshards;
+    if (row == 0 && tid == 0) *p.status = 0;  // this call's first (and only) kernel
+    if (tid < 32) {
+        // where each shard's entries go, and the row's log-normaliser
+        int cnt = 0;
+        double l2 = -INFINITY;
+        if (lane < S) {
+            cnt = p.part_count[(size_t)lane * p.rows + row];
+            cnt = cnt < 0 ? 0 : (cnt > p.part_k ? p.part_k : cnt);
+            l2 = p.part_lse2[(size_t)lane * p.rows + row];
+            if (!(l2 > -INFINITY) || !(l2 < INFINITY)) l2 = -INFINITY;  // an empty shard (or a NaN)
+        }
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane < S) sh->iscr[lane] = incl - cnt;
+        const double M = warp_max(l2);
+        const double sum = warp_sum(l2 > -INFINITY ? exp2(l2 - M) : 0.0);
+        if (lane == 31) sh->sel_total = incl;
+        if (lane == 0) sh->lrow = sum > 0.0 ? M + log2(sum) : -INFINITY;
+    }
+    fsync<NT>();
+    const int n_c = sh->sel_total;
+    const double L2 = sh->lrow;
+    for (int s = 0; s < S; ++s) {
+        const int base = sh->iscr[s];
+        const int cnt = (s + 1 < S ? sh->iscr[s + 1] : n_c) - base;
+        const size_t src = ((size_t)s * p.rows + row) * p.part_k;
+        for (int i = tid; i < cnt; i += NT) {
+            c_raw[base + i] = __float_as_uint(p.part_logit[src + i]);
+            c_idx[base + i] = p.part_idx[src + i] + p.shard_offset[s];
+        }
+    }
+    fsync<NT>();
+    const int n = select_in_list<T, NT>(k, c_raw, c_idx, n_c, hist, sh, tid);
+    cut_sample_write<T, NT>(p, row, n, c_raw, c_idx, L2, hist, cum, sh, tid);
 }
 
 }  // namespace tslt
@@ -1431,11 +1524,10 @@ extern "C" int tslt_set_ready_poll_limit(int polls) {
     return TSLT_OK;
 }
 
-extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
-                             long long row_stride_elems, int k, float top_p, float temperature,
-                             int num_samples, const float* uniforms, int* idx, float* logit, int* count,
-                             int* token, float* lse, float* mass, void* workspace, size_t workspace_bytes,
-                             void* stream) {
+static int sparsify_impl(const void* logits, int dtype, int B, int gamma, int V, long long row_stride_elems, int k,
+                         float top_p, float temperature, int num_samples, const float* uniforms, int* idx, float* logit,
+                         int* count, int* token, float* lse, float* mass, double* lse2, void* workspace,
+                         size_t workspace_bytes, void* stream) {
     if (dtype != TSLT_F32 && dtype != TSLT_BF16) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
     if (B < 0 || gamma < 0 || V <= 0 || k <= 0 || k > V || !(top_p > 0.0f) || !(temperature > 0.0f) ||
@@ -1463,7 +1555,8 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
     p.c = make_scale(temperature);
     p.num_samples = num_samples;
     p.uniforms = uniforms;
-    p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass;
+    p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass; p.lse2 = lse2;
+    p.nshards = 0; p.part_k = 0; p.part_idx = nullptr; p.part_logit = nullptr; p.part_count = nullptr; p.part_lse2 = nullptr;
     p.nchunks = pl.nchunks; p.split = pl.split;
     p.group_log2 = pl.group_log2; p.ngroups = pl.ngroups; p.tile_cap = pl.tile_cap; p.cand_cap = pl.cand_cap;
     p.poll_limit = g_sparsify_poll_limit;
@@ -1493,5 +1586,62 @@ extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, in
         !raise_smem_limit_once(fin, (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1), kFinishSmemLimit))
         return TSLT_ERR_CUDA;
     if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
+    return TSLT_OK;
+}
+
+extern "C" int tslt_sparsify(const void* logits, int dtype, int B, int gamma, int V,
+                             long long row_stride_elems, int k, float top_p, float temperature,
+                             int num_samples, const float* uniforms, int* idx, float* logit, int* count,
+                             int* token, float* lse, float* mass, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+    return sparsify_impl(logits, dtype, B, gamma, V, row_stride_elems, k, top_p, temperature, num_samples, uniforms, idx,
+                         logit, count, token, lse, mass, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" int tslt_sparsify_shard(const void* logits, int dtype, int rows, int V_shard, long long row_stride_elems, int k,
+                                   float temperature, int* idx, float* logit, int* count, double* lse2, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    if (rows > 0 && !lse2) return TSLT_ERR_INVALID_ARG;
+    return sparsify_impl(logits, dtype, rows, 1, V_shard, row_stride_elems, k, 1.0f, temperature, 0, nullptr, idx, logit,
+                         count, nullptr, nullptr, nullptr, lse2, workspace, workspace_bytes, stream);
+}
+
+extern "C" int tslt_sparsify_merge(int dtype, int rows, int nshards, const int* shard_offset, int k, const int* part_idx,
+                                   const float* part_logit, const int* part_count, const double* part_lse2, float top_p,
+                                   float temperature, int num_samples, const float* uniforms, int* idx, float* logit,
+                                   int* count, int* token, float* lse, float* mass, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    if (dtype != TSLT_F32 && dtype != TSLT_BF16) return TSLT_ERR_UNSUPPORTED;
+    if (rows < 0 || nshards < 1 || k <= 0 || !shard_offset || !(top_p > 0.0f) || !(temperature > 0.0f) ||
+        !isfinite(temperature) || num_samples < 0)
+        return TSLT_ERR_INVALID_ARG;
+    if (nshards > kMaxShards || k > TSLT_MAX_K || (long long)nshards * k > kMaxMergeList) return TSLT_ERR_UNSUPPORTED;
+    if (shard_offset[0] < 0) return TSLT_ERR_INVALID_ARG;
+    for (int s = 1; s < nshards; ++s)
+        if (shard_offset[s] <= shard_offset[s - 1]) return TSLT_ERR_INVALID_ARG;
+    if (rows > 0x7fffffff / 64) return TSLT_ERR_UNSUPPORTED;
+    if (rows == 0) return TSLT_OK;
+    if (!part_idx || !part_logit || !part_count || !part_lse2 || !idx || !logit || !count || !workspace ||
+        (num_samples > 0 && (!uniforms || !token)))
+        return TSLT_ERR_INVALID_ARG;
+    if (((uintptr_t)workspace & 255)) return TSLT_ERR_INVALID_ARG;
+    if (workspace_bytes < (size_t)kWsHeaderBytes) return TSLT_ERR_WORKSPACE;
+
+    SparsifyParams p = {};
+    p.rows = rows; p.k = k;
+    p.top_p = top_p;
+    p.c = make_scale(temperature);
+    p.num_samples = num_samples;
+    p.uniforms = uniforms;
+    p.idx = idx; p.logit = logit; p.count = count; p.token = token; p.lse = lse; p.mass = mass; p.lse2 = nullptr;
+    p.cand_cap = nshards * k;
+    p.status = (int*)workspace;
+    p.nshards = nshards; p.part_k = k;
+    p.part_idx = part_idx; p.part_logit = part_logit; p.part_count = part_count; p.part_lse2 = part_lse2;
+    for (int s = 0; s < kMaxShards; ++s) p.shard_offset[s] = s < nshards ? shard_offset[s] : 0;
+    void (*kern)(const SparsifyParams) = dtype == TSLT_F32 ? sparsify_merge_kernel<float> : sparsify_merge_kernel<bf16_t>;
+    const size_t smem = finish_layout(0, 0, p.cand_cap, k, 0, true).total;  // at most 512 + 4096 + 8192 + 16384 bytes
+    kern<<<rows, kMergeThreads, smem, (cudaStream_t)stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }

@@ -24,7 +24,7 @@ F32, BF16 = 0, 1
 MAX_K = 1024
 
 EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status", "tslt_set_ready_poll_limit",
-           "tslt_sparsify_workspace_bytes", "tslt_sparsify",
+           "tslt_sparsify_workspace_bytes", "tslt_sparsify", "tslt_sparsify_shard", "tslt_sparsify_merge",
            "tslt_verify_workspace_bytes", "tslt_verify", "tslt_verify_static",
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
            "tslt_tree_verify_walk_workspace_bytes", "tslt_tree_verify_walk",
@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
     L.tslt_sparsify_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_sparsify.restype = i
     L.tslt_sparsify.argtypes = [p, i, i, i, i, ll, i, f, f, i, p, p, p, p, p, p, p, p, sz, p]
+    L.tslt_sparsify_shard.restype = i
+    L.tslt_sparsify_shard.argtypes = [p, i, i, i, ll, i, f, p, p, p, p, p, sz, p]
+    L.tslt_sparsify_merge.restype = i
+    L.tslt_sparsify_merge.argtypes = [i, i, i, ctypes.POINTER(i), i, p, p, p, p, f, f, i, p, p, p, p, p, p, p, p, sz, p]
     L.tslt_verify_workspace_bytes.restype = i
     L.tslt_verify_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_verify.restype = i
@@ -261,6 +265,122 @@ def sparsify(logits: torch.Tensor, k: int, top_p: float = 1.0, temperature: floa
                              ws.numel(), _stream())
     _check(rc, "tslt_sparsify")
     o["workspace"] = ws
+    return o
+
+
+MAX_SHARDS = 16
+
+
+def sparsify_shard(logits_shard: torch.Tensor, k: int, temperature: float = 1.0, *, out: Optional[dict] = None,
+                   ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_sparsify_shard on one vocabulary shard [rows, V_shard] (a column slice of a wider tensor
+    is fine if it starts on a 16-byte boundary).  Returns dict(idx, logit [rows, k], count [rows]
+    int32, lse2 [rows] fp64, workspace); idx is local to the shard."""
+    if not logits_shard.is_cuda:
+        raise ValueError("logits must be a CUDA tensor (libtslt has no CPU path)")
+    rows, V, stride = _row_layout(logits_shard)
+    dev = logits_shard.device
+    o = out if out is not None else {}
+    if "idx" not in o:
+        o["idx"] = torch.empty(rows, k, dtype=torch.int32, device=dev)
+        o["logit"] = torch.empty(rows, k, dtype=torch.float32, device=dev)
+        o["count"] = torch.empty(rows, dtype=torch.int32, device=dev)
+        o["lse2"] = torch.empty(rows, dtype=torch.float64, device=dev)
+    for name, dt, ne in (("idx", torch.int32, rows * k), ("logit", torch.float32, rows * k),
+                         ("count", torch.int32, rows), ("lse2", torch.float64, rows)):
+        _out(o, name, dt, ne)
+    if ws is None:
+        ws = workspace(sparsify_workspace_bytes(rows, V, k, 0), dev)
+    rc = lib().tslt_sparsify_shard(_ptr(logits_shard), _dtype_code(logits_shard), rows, V, stride, k, temperature,
+                                   _ptr(o["idx"]), _ptr(o["logit"]), _ptr(o["count"]), _ptr(o["lse2"]), _ptr(ws),
+                                   ws.numel(), _stream())
+    _check(rc, "tslt_sparsify_shard")
+    o["workspace"] = ws
+    return o
+
+
+def sparsify_merge(part_idx: torch.Tensor, part_logit: torch.Tensor, part_count: torch.Tensor,
+                   part_lse2: torch.Tensor, shard_offset: Sequence[int], dtype: torch.dtype, top_p: float = 1.0,
+                   temperature: float = 1.0, uniforms: Optional[torch.Tensor] = None, *, want_stats: bool = True,
+                   out: Optional[dict] = None, ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_sparsify_merge: part_idx / part_logit [nshards, rows, k], part_count (int32) / part_lse2
+    (fp64) [nshards, rows], as the shards wrote them; dtype = the logits' element type.  Returns what
+    sparsify() returns for the whole-vocabulary rows."""
+    _cuda(part_idx, "part_idx", torch.int32)
+    _cuda(part_logit, "part_logit", torch.float32)
+    _cuda(part_count, "part_count", torch.int32)
+    _cuda(part_lse2, "part_lse2", torch.float64)
+    if part_idx.dim() != 3 or part_idx.shape != part_logit.shape:
+        raise ValueError("part_idx and part_logit must be [nshards, rows, k]")
+    nshards, rows, k = part_idx.shape
+    if tuple(part_count.shape) != (nshards, rows) or tuple(part_lse2.shape) != (nshards, rows):
+        raise ValueError("part_count and part_lse2 must be [nshards, rows]")
+    if len(shard_offset) != nshards:
+        raise ValueError("one offset per shard")
+    dev = part_idx.device
+    ns = 0
+    if uniforms is not None:
+        _cuda(uniforms, "uniforms", torch.float32)
+        if rows and uniforms.numel() % rows:
+            raise ValueError("uniforms must be [rows, num_samples]")
+        ns = uniforms.numel() // rows if rows else 0
+    o = out if out is not None else {}
+    if "idx" not in o:
+        o["idx"] = torch.empty(rows, k, dtype=torch.int32, device=dev)
+        o["logit"] = torch.empty(rows, k, dtype=torch.float32, device=dev)
+        o["count"] = torch.empty(rows, dtype=torch.int32, device=dev)
+        o["token"] = torch.empty(rows, ns, dtype=torch.int32, device=dev)
+        if want_stats:
+            o["lse"] = torch.empty(rows, dtype=torch.float32, device=dev)
+            o["mass"] = torch.empty(rows, dtype=torch.float32, device=dev)
+    for name, dt, ne, req in (("idx", torch.int32, rows * k, True), ("logit", torch.float32, rows * k, True),
+                              ("count", torch.int32, rows, True), ("token", torch.int32, rows * ns, True),
+                              ("lse", torch.float32, rows, False), ("mass", torch.float32, rows, False)):
+        _out(o, name, dt, ne, req)
+    if ws is None:
+        ws = torch.empty(4096, dtype=torch.uint8, device=dev)
+    code = F32 if dtype == torch.float32 else BF16 if dtype == torch.bfloat16 else None
+    if code is None:
+        raise TsltError(ERR_UNSUPPORTED, "dtype %s" % dtype)
+    offs = (ctypes.c_int * nshards)(*[int(x) for x in shard_offset])
+    rc = lib().tslt_sparsify_merge(code, rows, nshards, offs, k, _ptr(part_idx), _ptr(part_logit), _ptr(part_count),
+                                   _ptr(part_lse2), top_p, temperature, ns, _ptr(uniforms), _ptr(o["idx"]),
+                                   _ptr(o["logit"]), _ptr(o["count"]), _ptr(o["token"]), _ptr(o.get("lse")),
+                                   _ptr(o.get("mass")), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "tslt_sparsify_merge")
+    o["workspace"] = ws
+    return o
+
+
+def sparsify_sharded(logits: torch.Tensor, shard_bounds: Sequence[int], k: int, top_p: float = 1.0,
+                     temperature: float = 1.0, uniforms: Optional[torch.Tensor] = None) -> dict:
+    """The two-stage path on ONE device: logits [rows, V] are cut at shard_bounds (ascending token
+    ids 0 = b_0 < b_1 < ... < b_n = V, each a multiple of 16 bytes' worth of elements), every slice
+    goes through sparsify_shard with its own workspace, and sparsify_merge joins them.  On several
+    devices each rank runs sparsify_shard on its slice and the parts are all-gathered before the
+    merge; the kernels are the same."""
+    if logits.dim() != 2:
+        raise ValueError("logits must be [rows, V]")
+    rows, V = logits.shape
+    b = [int(x) for x in shard_bounds]
+    if len(b) < 2 or b[0] != 0 or b[-1] != V or any(y <= x for x, y in zip(b, b[1:])):
+        raise ValueError("shard_bounds must ascend from 0 to V")
+    n = len(b) - 1
+    dev = logits.device
+    part = dict(idx=torch.empty(n, rows, k, dtype=torch.int32, device=dev),
+                logit=torch.empty(n, rows, k, dtype=torch.float32, device=dev),
+                count=torch.empty(n, rows, dtype=torch.int32, device=dev),
+                lse2=torch.empty(n, rows, dtype=torch.float64, device=dev))
+    spaces = []
+    for s in range(n):
+        sl = logits[:, b[s]:b[s + 1]]
+        ws = torch.empty(max(sparsify_workspace_bytes(rows, b[s + 1] - b[s], k, 0), 4096), dtype=torch.uint8, device=dev)
+        sparsify_shard(sl, k, temperature, out={name: part[name][s] for name in part}, ws=ws)
+        spaces.append(ws)
+    o = sparsify_merge(part["idx"], part["logit"], part["count"], part["lse2"], b[:-1], logits.dtype, top_p,
+                       temperature, uniforms)
+    o["parts"] = part
+    o["shard_workspaces"] = spaces
     return o
 
 
