@@ -557,7 +557,7 @@ __host__ __device__ inline int pow2_at_least(int n) {
 __host__ __device__ constexpr int finish_threads(int k) { return k <= 128 ? 128 : 256; }
 __host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
 constexpr int kFinishHeaderBytes = 512;
-constexpr int kRankListMax = 512;  // candidates up to which the k-th is found by counting ranks
+constexpr int kRankListMax = 160;  // candidates up to which the k-th is found by counting ranks (n * n / NT compares)
 
 // Dynamic shared memory of the finish kernel:
 //   header | histogram | region A | region B | region C | line maxima
@@ -1221,8 +1221,8 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
             }
         } else {
             // many vectors per thread: one pass; the first candidates a thread finds wait in a small
-            // stash while the prefix sum finds where they go.  Only if some thread found more than
-            // its stash holds are the vectors read a second time (from L2).
+            // stash while the prefix sum finds where they go.  A thread that found more than its
+            // stash holds reads its own vectors a second time (from L2).
             constexpr int kStash = 12;
             uint32_t st_raw[kStash];
             int st_idx[kStash];
@@ -1244,15 +1244,15 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
                     }
             });
             int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
-            const int over = __syncthreads_or(cnt > kStash ? 1 : 0);
             if (n_c <= p.cand_cap) {
                 in_smem = true;
-                if (!over) {
+                if (cnt <= kStash) {
                     for (int j = 0; j < cnt; ++j) {
                         c_raw[cpos + j] = st_raw[j];
                         c_idx[cpos + j] = st_idx[j];
                     }
                 } else {
+                    // (this thread alone reads its vectors again; they are in L2 now)
                     for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
 #pragma unroll
                         for (int e = 0; e < kPer; ++e)
