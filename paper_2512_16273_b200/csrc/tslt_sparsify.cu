@@ -36,7 +36,7 @@ namespace tslt {
 
 constexpr int kTilesPerChunk = 32;        // 64-byte tiles in a 2 KB chunk
 constexpr int kVecsPerTile = 4;           // 16-byte vectors in a tile
-constexpr int kSparsifyStreamCtasPerSm = 5;  // 51 registers, no spills (6 CTAs of 40 registers spill and run 8 % slower)
+constexpr int kSparsifyStreamCtasPerSm = 4;  // 64 registers: two chunks per warp in flight (5 CTAs with one chunk in flight: 1.5 % slower; 3 CTAs: 4 % slower)
 constexpr int kMaxGroups = 4096;          // group maxima the finish kernel bisects over
 constexpr int kMaxTileList = 4096;        // survivor tiles it can list
 constexpr int kSelBins = 1024;            // bins of the selection histogram
@@ -385,8 +385,11 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
     const float c = p.c.f;
     const unsigned char* lane_rowp = rowp + lane * kVecBytes;
     int ch = wk.chunk_begin + warp;
-    LaneTile<T> lt;
+    // two chunks per warp are in flight at any time (4 KB; 128 KB per SM with four CTAs): the loads of
+    // chunk ch + 16 are issued as soon as chunk ch has been consumed
+    LaneTile<T> lt, lt2;
     if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);  // in flight during the set-up below
+    if (ch + kWarps < wk.chunk_end) lt2.load_lane(lane_rowp, (ch + kWarps) * kVecsPerChunk, ext);
     // The segment's ready flag is cleared here, by the CTA that will set it, and the store is fenced
     // before the barrier after which this CTA lets the finish kernel be scheduled.  A finish CTA
     // runs only after every streaming CTA has passed that point, so it never sees a flag (or a
@@ -403,14 +406,18 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
     ls.reset();
     unsigned short* tmax = kLocal ? reinterpret_cast<unsigned short*>(stream_smem + kStreamHeaderBytes)
                                   : p.tile_max + (size_t)wk.row * p.nchunks * kTilesPerChunk;
-    while (ch < wk.chunk_end) {
-        const float lm = lt.reduce_max();
-        const uint2 q = QuadMax<T>::keys(lt);
+    auto consume = [&](LaneTile<T>& t) {
+        const float lm = t.reduce_max();
+        const uint2 q = QuadMax<T>::keys(t);
         if ((lane & 3) == 0) *reinterpret_cast<uint2*>(tmax + ch * kTilesPerChunk + lane) = q;  // slots (lane >> 2) * 4 ..+3
         ls.raise_to(lm, c);
-        lt.accumulate(ls, c);
+        t.accumulate(ls, c);
+        if (ch + 2 * kWarps < wk.chunk_end) t.load_lane(lane_rowp, (ch + 2 * kWarps) * kVecsPerChunk, ext);
         ch += kWarps;
-        if (ch < wk.chunk_end) lt.load_lane(lane_rowp, ch * kVecsPerChunk, ext);
+    };
+    while (ch < wk.chunk_end) {
+        consume(lt);
+        if (ch < wk.chunk_end) consume(lt2);
     }
     // hand-over: one (M, S) pair per warp
     const float Mw = warp_max(ls.M);
@@ -554,7 +561,7 @@ __host__ __device__ inline int pow2_at_least(int n) {
     while (p < n) p <<= 1;
     return p;
 }
-__host__ __device__ constexpr int finish_threads(int k) { return k <= 128 ? 128 : 256; }
+__host__ __device__ constexpr int finish_threads(int k) { return k <= 512 ? 128 : 256; }
 __host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
 constexpr int kFinishHeaderBytes = 512;
 constexpr int kRankListMax = 160;  // candidates up to which the k-th is found by counting ranks (n * n / NT compares)
@@ -719,7 +726,7 @@ __device__ __forceinline__ int finite_key16(float z) {
 template <typename T, int NT>
 __device__ __forceinline__ int select_in_list(int k, uint32_t* c_raw, int* c_idx, int n_c, uint32_t* hist, FinishShared* sh, int tid) {
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
-    constexpr int kHeld = 8;  // most list entries a thread owns
+    constexpr int kHeld = kMaxMergeList / NT;  // most list entries a thread owns (the lists hold 2048 at most)
     unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
     int n = 0;
     {
@@ -808,6 +815,7 @@ template <typename T, int NT>
 __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int row, int n, uint32_t* c_raw, int* c_idx,
                                                  double L2, uint32_t* hist, double* cum, FinishShared* sh, int tid) {
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
+    constexpr int kMine = TSLT_MAX_K / NT;  // most winners a thread owns in the top-rho cut
     const int lane = tid & 31, k = p.k;
     const int n0 = n;
     uint32_t* win_raw = c_raw;
@@ -826,12 +834,12 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
     if (n0 > 0 && p.top_p < 1.0f) {
         constexpr double kFix = 4611686018427387904.0;  // 2^62
         unsigned long long* mhist = reinterpret_cast<unsigned long long*>(hist);  // 256 bins
-        const int ipt = (n0 + NT - 1) / NT;  // <= 4 (n0 <= 1024 with 256 threads, <= NT otherwise)
+        const int ipt = (n0 + NT - 1) / NT;  // <= kMine
         const int i0 = min(n0, tid * ipt), i1 = min(n0, i0 + ipt);
-        uint32_t kz[4];
-        unsigned long long qf[4];
+        uint32_t kz[kMine];
+        unsigned long long qf[kMine];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kMine; ++j) {
             kz[j] = 0u;
             qf[j] = 0ull;
             if (i0 + j < i1) {
@@ -845,7 +853,7 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
         auto mass_from = [&](uint32_t t, int slot) -> unsigned long long {
             unsigned long long m = 0ull;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < kMine; ++j)
                 if (i0 + j < i1 && kz[j] >= t) m += qf[j];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
@@ -883,7 +891,7 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
             int c_gt = 0, c_eq = 0;
             unsigned long long qk = 0ull;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < kMine; ++j)
                 if (i0 + j < i1) {
                     c_gt += kz[j] > ckey ? 1 : 0;
                     if (kz[j] == ckey) {
@@ -900,11 +908,11 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
             if (need < 1) need = 1;
             const int my_ties = max(0, min(c_eq, need - eq_before));
             // keep the larger keys and the first `need` ties: read mine, then (after the scan's barriers) write
-            uint32_t keep_raw[4];
-            int keep_idx[4];
+            uint32_t keep_raw[kMine];
+            int keep_idx[kMine];
             int kept = 0, ties_left = my_ties;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < kMine; ++j)
                 if (i0 + j < i1) {
                     bool keep = kz[j] > ckey;
                     if (kz[j] == ckey && ties_left > 0) {
@@ -919,7 +927,7 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
                 }
             const int kp = block_exscan<NT>(kept, tid, sh->iscr, &tot_keep);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < kMine; ++j)
                 if (j < kept) {
                     win_raw[kp + j] = keep_raw[j];
                     win_idx[kp + j] = keep_idx[j];
