@@ -979,15 +979,211 @@ __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int ro
     }
 }
 
+// Step 4 of the finish: the finite logits of the survivor tiles (tl: n_surv tile numbers in address
+// order) at or above the bound go to the candidate list in shared memory, in ascending token index.
+// Returns how many there are, or -1 if they do not fit cand_cap (nothing usable is written then).
 template <typename T, int NT>
-__global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kernel(const SparsifyParams p) {
+__device__ __forceinline__ int gather_candidates(const unsigned char* rowp, const RowExtent& ext, int V, const uint32_t* tl,
+                                                 int n_surv, int lo16, int cand_cap, uint32_t* c_raw, int* c_idx,
+                                                 FinishShared* sh, int tid) {
     constexpr int kPer = Elt<T>::kPerVec;
+    // the vectors this thread works on: a contiguous run of the survivors' vectors, or of the row's
+    const uint32_t* units = tl;
+    const int n_units = tl ? n_surv * kVecsPerTile : (V + kPer - 1) / kPer;
+    const int upt = (n_units + NT - 1) / NT;
+    const int u0 = min(n_units, tid * upt), u1 = min(n_units, u0 + upt);
+    const float lo_f = key_to_float((uint32_t)lo16 << 16);  // the smallest float whose 16-bit key is lo16
+    auto is_candidate = [lo_f](float z) { return z >= lo_f && z <= 3.4028234e38f; };
+    bool in_smem = false;
+    int n_c = 0;
+    {
+        constexpr int kRegVecs = 4;
+        if (upt <= kRegVecs) {
+            // few vectors per thread (small k): one trip to memory, the vectors wait in registers
+            // while the prefix sum finds where their candidates go
+            uint4 d[kRegVecs];
+            int vi[kRegVecs];
+#pragma unroll
+            for (int j = 0; j < kRegVecs; ++j) {
+                const int u = u0 + j;
+                vi[j] = u < u1 ? (int)(tl[u >> 2] * (uint32_t)kVecsPerTile) + (u & 3) : -1;
+                if (vi[j] >= 0 && vi[j] < ext.nvec_full) d[j] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[j]);
+            }
+            int cnt = 0;
+#pragma unroll
+            for (int j = 0; j < kRegVecs; ++j) {
+                if (vi[j] < 0) continue;
+                float z[kPer];
+                if (vi[j] < ext.nvec_full) {
+                    unpack_vec<T>(d[j], z);
+                } else {  // the row's ragged last vector: fetched element by element, kept in the same form
+                    load_row_vector<T>(rowp, vi[j], ext, V, z);
+                    d[j] = pack_vec<T>(z);
+                }
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
+            }
+            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+            if (n_c <= cand_cap) {
+                in_smem = true;
+#pragma unroll
+                for (int j = 0; j < kRegVecs; ++j) {
+                    if (vi[j] < 0) continue;
+                    float z[kPer];
+                    unpack_vec<T>(d[j], z);
+#pragma unroll
+                    for (int e = 0; e < kPer; ++e)
+                        if (is_candidate(z[e])) {
+                            c_raw[cpos] = __float_as_uint(z[e]);
+                            c_idx[cpos] = vi[j] * kPer + e;
+                            ++cpos;
+                        }
+                }
+                fsync<NT>();
+            }
+        } else {
+            // many vectors per thread: one pass; the first candidates a thread finds wait in a small
+            // stash while the prefix sum finds where they go.  A thread that found more than its
+            // stash holds reads its own vectors a second time (from L2).
+            constexpr int kStash = 12;
+            uint32_t st_raw[kStash];
+            int st_idx[kStash];
+            int cnt = 0;
+            // every tile of this thread is asked of L2 first, so that the batches of loads below (six
+            // vectors in flight per thread) do not each pay a trip to HBM
+            for (int u = u0; u < u1; ++u)
+                if (u == u0 || (u & 3) == 0)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + (size_t)tl[u >> 2] * (kVecsPerTile * kVecBytes)));
+            for_my_vectors<T>(rowp, ext, V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e)
+                    if (is_candidate(z[e])) {
+                        if (cnt < kStash) {
+                            st_raw[cnt] = __float_as_uint(z[e]);
+                            st_idx[cnt] = vi * kPer + e;
+                        }
+                        ++cnt;
+                    }
+            });
+            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
+            if (n_c <= cand_cap) {
+                in_smem = true;
+                if (cnt <= kStash) {
+                    for (int j = 0; j < cnt; ++j) {
+                        c_raw[cpos + j] = st_raw[j];
+                        c_idx[cpos + j] = st_idx[j];
+                    }
+                } else {
+                    // (this thread alone reads its vectors again; they are in L2 now)
+                    for_my_vectors<T>(rowp, ext, V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+                        for (int e = 0; e < kPer; ++e)
+                            if (is_candidate(z[e])) {
+                                c_raw[cpos] = __float_as_uint(z[e]);
+                                c_idx[cpos] = vi * kPer + e;
+                                ++cpos;
+                            }
+                    });
+                }
+                fsync<NT>();
+            }
+        }
+    }
+    return in_smem ? n_c : -1;
+}
+
+// The rare rows whose survivors or candidates do not fit their lists (thousands of tied tile maxima;
+// k close to V): the same selection over the survivors' vectors (tl), or all of the row's (tl ==
+// nullptr), in global memory: a histogram for the 16-bit key (fp32 rows: another for the low 16 bits), a
+// count and a collecting pass.  The winners go to c_raw / c_idx in ascending index; returns how many.
+// hist: kSelBins words.  Kept out of line: it is several times the code of the common path.
+template <typename T, int NT>
+__device__ __noinline__ int select_from_global(const unsigned char* rowp, const RowExtent ext, int V, const uint32_t* tl,
+                                               int n_surv, int lo16, int max16, int k, uint32_t* c_raw, int* c_idx,
+                                               uint32_t* hist, FinishShared* sh, int tid) {
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
+    constexpr int kPer = Elt<T>::kPerVec;
+    // the vectors this thread works on: a contiguous run of the survivors' vectors, or of the row's
+    const uint32_t* units = tl;
+    const int n_units = tl ? n_surv * kVecsPerTile : (V + kPer - 1) / kPer;
+    const int upt = (n_units + NT - 1) / NT;
+    const int u0 = min(n_units, tid * upt), u1 = min(n_units, u0 + upt);
+    const float lo_f = key_to_float((uint32_t)lo16 << 16);  // the smallest float whose 16-bit key is lo16
+    auto is_candidate = [lo_f](float z) { return z >= lo_f && z <= 3.4028234e38f; };
+    int n = 0;
+        // The survivors do not fit (thousands of tied tile maxima, or more candidates than the list
+        // holds): the same selection over the survivors' vectors, or all of the row's, in global
+        // memory: a histogram for the 16-bit key (fp32 rows: another for the low 16 bits), a count
+        // and a collecting pass.
+        auto key16_of = [](float z) -> int { return finite_key16(z); };
+        hist_select<T, NT>(rowp, ext, V, units, u0, u1, key16_of, lo16, max16, k, sh, hist, tid);
+        const int e16 = sh->sel_bin, above = sh->sel_above, total = sh->sel_total;
+        fsync<NT>();
+        uint32_t e32 = 0;   // key of the k-th largest logit (0: fewer than k finite logits, all of them win)
+        int need_ties = 0;  // how many logits equal to it are winners (the lowest indices)
+        if (e16 >= 0) {
+            if (kBf16) {
+                e32 = ((uint32_t)e16 << 16) | ((e16 & 0x8000) ? 0u : 0xffffu);
+                need_ties = k - above;
+            } else {
+                const uint32_t hi_bits = (uint32_t)e16;
+                auto low16_of = [hi_bits](float z) -> int {
+                    const uint32_t kz = float_to_key(z);
+                    return (kz >> 16) == hi_bits ? (int)(kz & 0xffffu) : -1;
+                };
+                hist_select<T, NT>(rowp, ext, V, units, u0, u1, low16_of, 0, 0xffff, k - above, sh, hist, tid);
+                const int low = sh->sel_bin, above2 = sh->sel_above;
+                fsync<NT>();
+                e32 = (hi_bits << 16) | (uint32_t)low;
+                need_ties = k - above - above2;
+            }
+        }
+        if (total > 0) {
+            int c_gt = 0, c_eq = 0;
+            for_my_vectors<T>(rowp, ext, V, units, u0, u1, [&](const float(&z)[kPer], int) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    if (!is_candidate(z[e])) continue;
+                    const uint32_t kz = float_to_key(z[e]);
+                    c_gt += kz > e32 ? 1 : 0;
+                    c_eq += kz == e32 ? 1 : 0;
+                }
+            });
+            int tot_eq, tot_w;
+            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
+            const int my_ties = max(0, min(c_eq, need_ties - eq_before));
+            int wpos = block_exscan<NT>(c_gt + my_ties, tid, sh->iscr, &tot_w);
+            int ties_left = my_ties;
+            for_my_vectors<T>(rowp, ext, V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) {
+                    if (!is_candidate(z[e])) continue;
+                    const uint32_t kz = float_to_key(z[e]);
+                    bool win = kz > e32;
+                    if (kz == e32 && ties_left > 0) {
+                        win = true;
+                        --ties_left;
+                    }
+                    if (win && wpos < k) {
+                        c_raw[wpos] = __float_as_uint(z[e]);
+                        c_idx[wpos] = vi * kPer + e;
+                        ++wpos;
+                    }
+                }
+            });
+            n = min(tot_w, k);
+            fsync<NT>();
+        }
+    return n;
+}
+
+template <typename T, int NT, bool kLocal>
+__global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kernel(const SparsifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     FinishShared* sh = reinterpret_cast<FinishShared*>(smem_raw);
     static_assert(sizeof(FinishShared) <= kFinishHeaderBytes, "header");
     const int k = p.k;
-    const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks, p.local_bound != 0);
+    const FinishLayout L = finish_layout(p.ngroups, p.tile_cap, p.cand_cap, k, p.nchunks, kLocal);
     uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw + L.hist);
     uint32_t* gm = reinterpret_cast<uint32_t*>(smem_raw + L.a);
     uint32_t* tl = reinterpret_cast<uint32_t*>(smem_raw + L.b);
@@ -1004,7 +1200,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) sh->gmax = 0;
     const int glog = p.group_log2, ngroups = p.ngroups;
-    if (glog > 5 && !p.local_bound)
+    if (glog > 5 && !kLocal)
         for (int i = tid; i < ngroups; i += NT) gm[i] = 0u;
     // ---- wait for the row's segments --------------------------------------------------------------
     // Nothing the streaming kernel wrote is read before this point.  The row's own segments being
@@ -1053,7 +1249,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     }
     int lo16, max16, n_surv;
     bool listed;
-    if (p.local_bound) {
+    if (kLocal) {
         // ---- 1-3 done by the row's streaming CTA: its bound, its survivor list ------------------------------
         const SegStat* st = p.seg_stats + row;
         const int n_list = __ldcg(&st->n_list);
@@ -1170,179 +1366,13 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         fsync<NT>();
     }
     const double L2 = sh->lrow;
-    // the vectors this thread works on from here: a contiguous run of the survivors' vectors, or of the row's
-    const uint32_t* units = listed ? tl : nullptr;
-    const int n_units = listed ? n_surv * kVecsPerTile : (p.V + kPer - 1) / kPer;
-    const int upt = (n_units + NT - 1) / NT;
-    const int u0 = min(n_units, tid * upt), u1 = min(n_units, u0 + upt);
+    // ---- 4. candidates in shared memory, 5. the exact top-k (ties to the lower index), ascending index ----
     if (!listed) lo16 = (int)kLowestFinite16;
-    const float lo_f = key_to_float((uint32_t)lo16 << 16);  // the smallest float whose 16-bit key is lo16
-    auto is_candidate = [lo_f](float z) { return z >= lo_f && z <= 3.4028234e38f; };
-
-    // ---- 4. candidates: the finite logits of the survivors at or above the bound, in index order --------
-    bool in_smem = false;
-    int n_c = 0;
-    if (listed && max16 >= lo16) {
-        constexpr int kRegVecs = 4;
-        if (upt <= kRegVecs) {
-            // few vectors per thread (small k): one trip to memory, the vectors wait in registers
-            // while the prefix sum finds where their candidates go
-            uint4 d[kRegVecs];
-            int vi[kRegVecs];
-#pragma unroll
-            for (int j = 0; j < kRegVecs; ++j) {
-                const int u = u0 + j;
-                vi[j] = u < u1 ? (int)(tl[u >> 2] * (uint32_t)kVecsPerTile) + (u & 3) : -1;
-                if (vi[j] >= 0 && vi[j] < ext.nvec_full) d[j] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[j]);
-            }
-            int cnt = 0;
-#pragma unroll
-            for (int j = 0; j < kRegVecs; ++j) {
-                if (vi[j] < 0) continue;
-                float z[kPer];
-                if (vi[j] < ext.nvec_full) {
-                    unpack_vec<T>(d[j], z);
-                } else {  // the row's ragged last vector: fetched element by element, kept in the same form
-                    load_row_vector<T>(rowp, vi[j], ext, p.V, z);
-                    d[j] = pack_vec<T>(z);
-                }
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
-            }
-            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
-            if (n_c <= p.cand_cap) {
-                in_smem = true;
-#pragma unroll
-                for (int j = 0; j < kRegVecs; ++j) {
-                    if (vi[j] < 0) continue;
-                    float z[kPer];
-                    unpack_vec<T>(d[j], z);
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e)
-                        if (is_candidate(z[e])) {
-                            c_raw[cpos] = __float_as_uint(z[e]);
-                            c_idx[cpos] = vi[j] * kPer + e;
-                            ++cpos;
-                        }
-                }
-                fsync<NT>();
-            }
-        } else {
-            // many vectors per thread: one pass; the first candidates a thread finds wait in a small
-            // stash while the prefix sum finds where they go.  A thread that found more than its
-            // stash holds reads its own vectors a second time (from L2).
-            constexpr int kStash = 12;
-            uint32_t st_raw[kStash];
-            int st_idx[kStash];
-            int cnt = 0;
-            // every tile of this thread is asked of L2 first, so that the batches of loads below (six
-            // vectors in flight per thread) do not each pay a trip to HBM
-            for (int u = u0; u < u1; ++u)
-                if (u == u0 || (u & 3) == 0)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + (size_t)tl[u >> 2] * (kVecsPerTile * kVecBytes)));
-            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
-#pragma unroll
-                for (int e = 0; e < kPer; ++e)
-                    if (is_candidate(z[e])) {
-                        if (cnt < kStash) {
-                            st_raw[cnt] = __float_as_uint(z[e]);
-                            st_idx[cnt] = vi * kPer + e;
-                        }
-                        ++cnt;
-                    }
-            });
-            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
-            if (n_c <= p.cand_cap) {
-                in_smem = true;
-                if (cnt <= kStash) {
-                    for (int j = 0; j < cnt; ++j) {
-                        c_raw[cpos + j] = st_raw[j];
-                        c_idx[cpos + j] = st_idx[j];
-                    }
-                } else {
-                    // (this thread alone reads its vectors again; they are in L2 now)
-                    for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
-#pragma unroll
-                        for (int e = 0; e < kPer; ++e)
-                            if (is_candidate(z[e])) {
-                                c_raw[cpos] = __float_as_uint(z[e]);
-                                c_idx[cpos] = vi * kPer + e;
-                                ++cpos;
-                            }
-                    });
-                }
-                fsync<NT>();
-            }
-        }
-    }
-    // ---- 5. the exact top-k (ties at the k-th logit to the lower index), left in ascending index ----------
     int n = 0;
-    if (in_smem) {
-        n = select_in_list<T, NT>(k, c_raw, c_idx, n_c, hist, sh, tid);
-    } else if (max16 >= lo16) {
-        // The survivors do not fit (thousands of tied tile maxima, or more candidates than the list
-        // holds): the same selection over the survivors' vectors, or all of the row's, in global
-        // memory: a histogram for the 16-bit key (fp32 rows: another for the low 16 bits), a count
-        // and a collecting pass.
-        auto key16_of = [](float z) -> int { return finite_key16(z); };
-        hist_select<T, NT>(rowp, ext, p.V, units, u0, u1, key16_of, lo16, max16, k, sh, hist, tid);
-        const int e16 = sh->sel_bin, above = sh->sel_above, total = sh->sel_total;
-        fsync<NT>();
-        uint32_t e32 = 0;   // key of the k-th largest logit (0: fewer than k finite logits, all of them win)
-        int need_ties = 0;  // how many logits equal to it are winners (the lowest indices)
-        if (e16 >= 0) {
-            if (kBf16) {
-                e32 = ((uint32_t)e16 << 16) | ((e16 & 0x8000) ? 0u : 0xffffu);
-                need_ties = k - above;
-            } else {
-                const uint32_t hi_bits = (uint32_t)e16;
-                auto low16_of = [hi_bits](float z) -> int {
-                    const uint32_t kz = float_to_key(z);
-                    return (kz >> 16) == hi_bits ? (int)(kz & 0xffffu) : -1;
-                };
-                hist_select<T, NT>(rowp, ext, p.V, units, u0, u1, low16_of, 0, 0xffff, k - above, sh, hist, tid);
-                const int low = sh->sel_bin, above2 = sh->sel_above;
-                fsync<NT>();
-                e32 = (hi_bits << 16) | (uint32_t)low;
-                need_ties = k - above - above2;
-            }
-        }
-        if (total > 0) {
-            int c_gt = 0, c_eq = 0;
-            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int) {
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) {
-                    if (!is_candidate(z[e])) continue;
-                    const uint32_t kz = float_to_key(z[e]);
-                    c_gt += kz > e32 ? 1 : 0;
-                    c_eq += kz == e32 ? 1 : 0;
-                }
-            });
-            int tot_eq, tot_w;
-            const int eq_before = block_exscan<NT>(c_eq, tid, sh->iscr, &tot_eq);
-            const int my_ties = max(0, min(c_eq, need_ties - eq_before));
-            int wpos = block_exscan<NT>(c_gt + my_ties, tid, sh->iscr, &tot_w);
-            int ties_left = my_ties;
-            for_my_vectors<T>(rowp, ext, p.V, units, u0, u1, [&](const float(&z)[kPer], int vi) {
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) {
-                    if (!is_candidate(z[e])) continue;
-                    const uint32_t kz = float_to_key(z[e]);
-                    bool win = kz > e32;
-                    if (kz == e32 && ties_left > 0) {
-                        win = true;
-                        --ties_left;
-                    }
-                    if (win && wpos < k) {
-                        c_raw[wpos] = __float_as_uint(z[e]);
-                        c_idx[wpos] = vi * kPer + e;
-                        ++wpos;
-                    }
-                }
-            });
-            n = min(tot_w, k);
-            fsync<NT>();
-        }
+    if (max16 >= lo16) {
+        const int n_c = listed ? gather_candidates<T, NT>(rowp, ext, p.V, tl, n_surv, lo16, p.cand_cap, c_raw, c_idx, sh, tid) : -1;
+        if (n_c >= 0) n = select_in_list<T, NT>(k, c_raw, c_idx, n_c, hist, sh, tid);
+        else n = select_from_global<T, NT>(rowp, ext, p.V, listed ? tl : nullptr, n_surv, lo16, max16, k, c_raw, c_idx, hist, sh, tid);
     }
     cut_sample_write<T, NT>(p, row, n, c_raw, c_idx, L2, hist, cum, sh, tid);
     // this kernel's completion must imply the streaming kernel's (what follows on the stream relies
@@ -1582,17 +1612,22 @@ static int sparsify_impl(const void* logits, int dtype, int B, int gamma, int V,
     else strm = dtype == TSLT_F32 ? sparsify_stream_kernel<float, false> : sparsify_stream_kernel<bf16_t, false>;
     const int strm_slot = (pl.local_bound ? 2 : 0) + (dtype == TSLT_F32 ? 0 : 1);
     if (!prefer_shared_carveout_once(strm, strm_slot)) return TSLT_ERR_CUDA;
-    if (pl.stream_smem > 48 * 1024 && !raise_smem_limit_once(strm, 4 + strm_slot, kStreamSmemLimit)) return TSLT_ERR_CUDA;
+    if (pl.stream_smem > 48 * 1024 && !raise_smem_limit_once(strm, 8 + strm_slot, kStreamSmemLimit)) return TSLT_ERR_CUDA;
     strm<<<pl.split.grid, kBlockThreads, pl.stream_smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     void (*fin)(const SparsifyParams);
-    if (pl.fin_threads == 128) fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 128> : sparsify_finish_kernel<bf16_t, 128>;
-    else fin = dtype == TSLT_F32 ? sparsify_finish_kernel<float, 256> : sparsify_finish_kernel<bf16_t, 256>;
-    if (!prefer_shared_carveout_once(fin, 4 + (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1))) return TSLT_ERR_CUDA;
+    const bool f32 = dtype == TSLT_F32, small = pl.fin_threads == 128;
+    if (pl.local_bound) {
+        if (small) fin = f32 ? sparsify_finish_kernel<float, 128, true> : sparsify_finish_kernel<bf16_t, 128, true>;
+        else fin = f32 ? sparsify_finish_kernel<float, 256, true> : sparsify_finish_kernel<bf16_t, 256, true>;
+    } else {
+        if (small) fin = f32 ? sparsify_finish_kernel<float, 128, false> : sparsify_finish_kernel<bf16_t, 128, false>;
+        else fin = f32 ? sparsify_finish_kernel<float, 256, false> : sparsify_finish_kernel<bf16_t, 256, false>;
+    }
+    const int fin_slot = (small ? 0 : 2) + (f32 ? 0 : 1) + (pl.local_bound ? 4 : 0);
+    if (!prefer_shared_carveout_once(fin, 4 + fin_slot)) return TSLT_ERR_CUDA;
     if (pl.fin_smem > kFinishSmemLimit) return TSLT_ERR_UNSUPPORTED;  // (rows of tens of millions of logits: the line maxima no longer fit)
-    if (pl.fin_smem > 48 * 1024 &&
-        !raise_smem_limit_once(fin, (pl.fin_threads == 128 ? 0 : 2) + (dtype == TSLT_F32 ? 0 : 1), kFinishSmemLimit))
-        return TSLT_ERR_CUDA;
+    if (pl.fin_smem > 48 * 1024 && !raise_smem_limit_once(fin, fin_slot, kFinishSmemLimit)) return TSLT_ERR_CUDA;
     if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }
