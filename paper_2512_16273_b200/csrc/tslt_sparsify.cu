@@ -562,7 +562,8 @@ __host__ __device__ inline int pow2_at_least(int n) {
     return p;
 }
 __host__ __device__ constexpr int finish_threads(int k) { return k <= 512 ? 128 : 256; }
-__host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : 4; }
+__host__ __device__ constexpr int finish_resident(int nt) { return nt == 128 ? 8 : (nt == 256 ? 4 : 2); }
+constexpr int kSegmentFinishThreads = 256;
 constexpr int kFinishHeaderBytes = 512;
 constexpr int kRankListMax = 160;  // candidates up to which the k-th is found by counting ranks (n * n / NT compares)
 
@@ -1503,6 +1504,8 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     pl.split.grid = rows * pl.split.nseg;
     pl.stream_smem = stream_smem_bytes(pl.nchunks, pl.ngroups);
     pl.local_bound = pl.split.nseg == 1 && pl.stream_smem <= kStreamSmemLimit;
+    // rows cut into segments are few: a finish CTA has its SM to itself and the row's latency is what counts
+    if (!pl.local_bound) pl.fin_threads = kSegmentFinishThreads;
     if (!pl.local_bound) pl.stream_smem = 0;
     pl.fin_smem = finish_layout(pl.ngroups, pl.tile_cap, pl.cand_cap, k, pl.nchunks, pl.local_bound).total;
     size_t off = kWsHeaderBytes;
@@ -1621,8 +1624,7 @@ static int sparsify_impl(const void* logits, int dtype, int B, int gamma, int V,
         if (small) fin = f32 ? sparsify_finish_kernel<float, 128, true> : sparsify_finish_kernel<bf16_t, 128, true>;
         else fin = f32 ? sparsify_finish_kernel<float, 256, true> : sparsify_finish_kernel<bf16_t, 256, true>;
     } else {
-        if (small) fin = f32 ? sparsify_finish_kernel<float, 128, false> : sparsify_finish_kernel<bf16_t, 128, false>;
-        else fin = f32 ? sparsify_finish_kernel<float, 256, false> : sparsify_finish_kernel<bf16_t, 256, false>;
+        fin = f32 ? sparsify_finish_kernel<float, kSegmentFinishThreads, false> : sparsify_finish_kernel<bf16_t, kSegmentFinishThreads, false>;
     }
     const int fin_slot = (small ? 0 : 2) + (f32 ? 0 : 1) + (pl.local_bound ? 4 : 0);
     if (!prefer_shared_carveout_once(fin, 4 + fin_slot)) return TSLT_ERR_CUDA;
