@@ -3,30 +3,38 @@
 //
 // Streaming kernel.  One CTA reads one segment of one logits row from HBM exactly once, with
 // 16-byte loads that go straight to registers (each warp instruction covers 512 contiguous
-// bytes).  It keeps two things: each lane's online (max, sum) for the softmax normaliser, and,
-// for every 64-byte tile of the row (32 bf16 or 16 fp32 logits), the top 16 bits of the tile's
-// largest logit, written to the workspace (2 bytes per 64 read).  Nothing in it depends on k or
-// top_p: there is no threshold, no histogram, no shared memory and no barrier in the loop, so it
-// runs at the occupancy and speed of a plain streaming reduction.
+// bytes; two 2 KB chunks per warp are in flight).  It keeps two things: each lane's online
+// (max, sum) for the softmax normaliser, and, for every 64-byte tile of the row (32 bf16 or 16 fp32
+// logits), the top 16 bits of the tile's largest logit.  Nothing in the loop depends on k or top_p:
+// no threshold, no histogram, no barrier, so it runs at the speed of a plain streaming reduction.
+//   - Batches that fill the machine: one CTA per row.  The tile maxima stay in shared memory and, at
+//     the end of the row, the CTA itself takes the tiles in groups so that there are two to four
+//     times k groups, finds the k-th largest group maximum (a lower bound on the k-th largest logit:
+//     each of the k groups at or above it holds a logit at or above it) and lists the tiles at or
+//     above that bound in address order ("survivors": about 1.2 k of them).  Only the list goes to
+//     the workspace.
+//   - Smaller batches: rows are cut into segments so that every CTA slot has work; the tile maxima
+//     go to the workspace (2 bytes per 64 read) and the finish kernel, which sees the whole row,
+//     finds the bound and the survivors.
 //
 // Finish kernel (launched with programmatic stream serialization; a CTA starts on its row as soon
-// as the row's segments have been handed over).  One CTA of 64 to 256 threads per row:
-//   1. a lower bound on the k-th largest logit from the TILE maxima: tiles are taken in groups so
-//      that there are two to four times k groups, and the k-th largest group maximum is found by
-//      bisection on its bits (each of the k groups at or above it holds a logit at or above it);
-//   2. the tiles at or above that bound are listed in address order ("survivors": about 1.2 k of
-//      them) and read back from global memory: 64 bytes each, some k * 64 bytes of the row's V * e;
-//   3. their logits at or above the bound (the candidates, a little more than k) go to shared memory
+// as the row's segments have been handed over).  One CTA of 128 or 256 threads per row:
+//   1. the survivors are read back from global memory: 64 bytes each, some k * 64 bytes of the
+//      row's V * e;
+//   2. their logits at or above the bound (the candidates, a little more than k) go to shared memory
 //      in index order, by prefix sums over the survivors;
-//   4. the exact k-th largest among them: by counting ranks while they are few, else by bisection on
-//      the 16-bit key between the bound and the row maximum (fp32 rows: once more on the low 16
-//      bits); ties at the k-th logit go to the lower index; the winners are compacted in place and
-//      so come out in ascending token index without any sort;
-//   5. the top-rho cut (a sort of the at most k winners by logit, an fp64 cumulative), the
+//   3. the exact k-th largest among them: by counting ranks while they are few, else by a two-pass
+//      256-bin radix select on the 16-bit key (fp32 rows: once more on the low 16 bits); ties at the
+//      k-th logit go to the lower index; the winners are compacted in place and so come out in
+//      ascending token index without any sort;
+//   4. the top-rho cut (a bitwise descent on the crossing key over fixed-point masses, no sort), the
 //      renormalised distribution and its CDF in fp64, the samples by inverse CDF, the outputs.
 // A row whose survivors or candidates do not fit their lists (thousands of tied maxima: constant
 // rows, rows sorted by value; k close to V) runs the selection over the survivors' vectors, or all
 // of the row's, in global memory instead: a histogram select and two more passes, slower, exact.
+//
+// Vocabulary shards: tslt_sparsify_shard is the same pair of kernels on a slice of the vocabulary;
+// sparsify_merge_kernel joins the shards' lists with steps 3 and 4 of the finish kernel.
 #include <math.h>
 
 #include "tslt_common.cuh"
