@@ -56,6 +56,7 @@ extern "C" {
 
 /* bits of the device status word (tslt_workspace_status) */
 #define TSLT_STATUS_WAIT_FELL_BACK 1 /* a bounded device-side wait ran out and took its fall-back; results are valid */
+#define TSLT_STATUS_BAD_RECORD 2     /* a packed draft record had a count word outside [0, k]; that row was read as empty */
 
 #define TSLT_F32 0
 #define TSLT_BF16 1
@@ -300,6 +301,30 @@ int tslt_pack_payload(const int* idx, const float* logit, const int* count, int 
                       int prob_format, unsigned int* payload, long long* payload_bits, void* stream);
 int tslt_unpack_payload(const unsigned int* payload, int rows, int k, int V, int prob_format,
                         int* idx, float* logit, int* count, int* device_flag, void* stream);
+
+/*
+ * The verifiers reading the uplink records directly (Section 3, Solution 1: what arrives at the
+ * verifier IS the packed payload; unpacking it to arrays first costs a kernel and a round trip of
+ * 8 k bytes per row).  tslt_verify_packed is tslt_verify, and tslt_tree_verify_packed is
+ * tslt_tree_verify (walk = 0) or tslt_tree_verify_walk (walk != 0), with `payload` [draft rows,
+ * tslt_payload_words(k, V, prob_format)] in place of draft_idx / draft_logit / draft_count: record r
+ * is draft row r, exactly as tslt_pack_payload writes it.  Same outputs, workspace sizes and limits
+ * as the unpacked calls, bit for bit equal to them on the unpacked arrays.  A record whose count
+ * word is outside [0, k] is read as an empty row and sets TSLT_STATUS_BAD_RECORD in the status word.
+ */
+int tslt_verify_packed(const void* target_logits, int dtype, int B, int gamma, int V,
+                       long long row_stride_elems, int k, const unsigned int* payload, int prob_format,
+                       const int* draft_token, float draft_temperature, float target_temperature,
+                       const float* u_accept, const float* u_sample, int* accepted_len, int* out_token,
+                       float* accept_prob, float* beta_hat, float* lse_p, void* workspace,
+                       size_t workspace_bytes, void* stream);
+int tslt_tree_verify_packed(int walk, const void* target_logits, int dtype, int B, int N, int V,
+                            long long row_stride_elems, const int* parent, const int* node_draft_row,
+                            int M, int k, const int* node_token, const unsigned int* payload,
+                            int prob_format, float draft_temperature, float target_temperature,
+                            const float* u_accept, const float* u_sample, int max_depth,
+                            int* accepted_path, int* accepted_len, int* out_token, void* workspace,
+                            size_t workspace_bytes, void* stream);
 
 /*
  * Truncation diagnostics on pairs of (draft, target) rows: what Section 5's top-K mass and acceptance

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtslt.so")
 SOURCES = ["tslt_api.cu", "tslt_sparsify.cu", "tslt_verify.cu", "tslt_payload.cu", "tslt_diagnostics.cu"]
-HEADERS = ["tslt_common.cuh", "tslt_rowmath.cuh"]
+HEADERS = ["tslt_common.cuh", "tslt_rowmath.cuh", "tslt_payload.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -2,22 +2,11 @@
 // the bit widths; the record layout is stated in include/tslt.h).  Two small kernels, one CTA per
 // row: the work is a few hundred entries per row, so the only things that matter are coalesced
 // record traffic and not serialising the threads of a row on shared words.
-#include <cuda_fp16.h>
-#include <cuda_runtime.h>
-#include <stdint.h>
-
-#include "../../include/tslt.h"
+#include "tslt_payload.cuh"
 
 namespace tslt {
 
 constexpr int kPayloadThreads = 128;
-
-__host__ __device__ inline int index_bits_of(int V) {
-    int b = 0;
-    while (b < 31 && (1ll << b) < (long long)V) ++b;
-    return b;
-}
-__host__ __device__ inline int prob_bits_of(int fmt) { return fmt == TSLT_PROB_F32 ? 32 : 16; }
 
 // fp32 -> bf16 bit pattern, round to nearest even; inf stays inf, NaN stays NaN.
 __device__ __forceinline__ uint32_t bf16_pattern(float x) {
@@ -34,12 +23,6 @@ __device__ __forceinline__ uint32_t value_pattern(float x, int fmt) {
     if (fmt == TSLT_PROB_BF16) return bf16_pattern(x);
     return (uint32_t)__half_as_ushort(__float2half_rn(x));
 }
-__device__ __forceinline__ float pattern_value(uint32_t p, int fmt) {
-    if (fmt == TSLT_PROB_F32) return __uint_as_float(p);
-    if (fmt == TSLT_PROB_BF16) return __uint_as_float(p << 16);
-    return __half2float(__ushort_as_half((unsigned short)p));
-}
-
 // One CTA per row.  The record is assembled in shared memory: an entry of w <= 63 bits touches at
 // most three words, each through atomicOr (neighbouring entries share words), then the record goes
 // out with coalesced stores.
@@ -91,31 +74,17 @@ __global__ void __launch_bounds__(kPayloadThreads) unpack_payload_kernel(const u
         n = 0;
     }
     const int w = bi + bp;
-    const unsigned long long idx_mask = (1ull << bi) - 1ull, val_mask = bp == 32 ? 0xffffffffull : 0xffffull;
     for (int e = tid; e < k; e += kPayloadThreads) {
         int i_out = -1;
         float z_out = -INFINITY;
         if (e < n) {
-            const long long pos = (long long)e * w;
-            const int word = 1 + (int)(pos >> 5), sh = (int)(pos & 31);
-            const unsigned long long lo = rec[word], mid = rec[word + 1], hi = rec[word + 2];
-            unsigned long long entry = (lo | (mid << 32)) >> sh;
-            if (sh) entry |= hi << (64 - sh);
-            i_out = (int)(entry & idx_mask);
-            z_out = pattern_value((uint32_t)((entry >> bi) & val_mask), fmt);
+            const int word = 1 + (int)(((long long)e * w) >> 5);
+            decode_entry(rec[word], rec[word + 1], rec[word + 2], e, bi, bp, fmt, &i_out, &z_out);
         }
         idx[(size_t)row * k + e] = i_out;
         logit[(size_t)row * k + e] = z_out;
     }
     if (tid == 0) count[row] = n;
-}
-
-static bool payload_shape(int k, int V, int fmt, int* bi, int* bp, int* words) {
-    if (fmt != TSLT_PROB_F32 && fmt != TSLT_PROB_BF16 && fmt != TSLT_PROB_F16) return false;
-    *bi = index_bits_of(V);
-    *bp = prob_bits_of(fmt);
-    *words = 1 + (int)(((long long)k * (*bi + *bp) + 31) / 32);
-    return true;
 }
 
 }  // namespace tslt

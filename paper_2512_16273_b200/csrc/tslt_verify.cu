@@ -21,6 +21,7 @@
 #include <vector>
 
 #include "tslt_common.cuh"
+#include "tslt_payload.cuh"
 #include "tslt_rowmath.cuh"
 
 namespace tslt {
@@ -43,6 +44,9 @@ struct VerifyParams {
     const int* draft_idx;
     const float* draft_logit;
     const int* draft_count;
+    // the drafts as packed uplink records instead (draft_idx == nullptr): [draft rows, pay_words]
+    const uint32_t* payload;
+    int pay_words, pay_bi, pay_bp, pay_fmt;
     // sequence mode
     int gamma;
     const int* draft_token;
@@ -124,6 +128,37 @@ __device__ __forceinline__ double row_log2_norm(const float2* part, int nchunks,
     return s > 0.0 ? mx + log2(s) : -INFINITY;
 }
 
+// The transmitted pairs of a draft row, from the unpacked arrays or straight from the packed record.
+// A record whose count word is not in [0, k] was not written by this library: the row reads as empty
+// and TSLT_STATUS_BAD_RECORD is set in the status word.
+__device__ __forceinline__ int draft_len(const VerifyParams& p, size_t draft_row) {
+    int n;
+    if (p.payload) {
+        n = (int)__ldg(p.payload + draft_row * (size_t)p.pay_words);
+        if (n < 0 || n > p.k) {
+            atomicOr(p.status, TSLT_STATUS_BAD_RECORD);
+            n = 0;
+        }
+    } else {
+        n = p.draft_count[draft_row];
+        n = n < 0 ? 0 : (n > p.k ? p.k : n);
+    }
+    return n;
+}
+__device__ __forceinline__ void draft_entry(const VerifyParams& p, size_t draft_row, int i, int* idx, float* logit) {
+    if (p.payload) {
+        const uint32_t* rec = p.payload + draft_row * (size_t)p.pay_words;
+        const int word = 1 + (int)(((long long)i * (p.pay_bi + p.pay_bp)) >> 5);
+        const unsigned long long lo = __ldg(rec + word);
+        const unsigned long long mid = word + 1 < p.pay_words ? __ldg(rec + word + 1) : 0u;
+        const unsigned long long hi = word + 2 < p.pay_words ? __ldg(rec + word + 2) : 0u;
+        decode_entry(lo, mid, hi, i, p.pay_bi, p.pay_bp, p.pay_fmt, idx, logit);
+    } else {
+        *idx = p.draft_idx[draft_row * (size_t)p.k + i];
+        *logit = p.draft_logit[draft_row * (size_t)p.k + i];
+    }
+}
+
 // p(v) of a streamed row.  cs is the scale AS THE STREAMING PASS USED IT (the fp32 rounding of
 // log2(e) / T, widened): the row's log-normaliser L2 was accumulated with it, and only the same
 // scale in the numerator makes a common offset of the logits cancel exactly.
@@ -138,14 +173,13 @@ __device__ __forceinline__ double token_prob(const unsigned char* rowp, int v, i
 // Rebuild q~ from the transmitted pairs of one draft row into s_idx / s_q; returns n.
 __device__ __forceinline__ int load_draft(const VerifyParams& p, size_t draft_row, const ResolverArrays& A,
                                           int tid, double* scratch) {
-    int n = p.draft_count[draft_row];
-    n = n < 0 ? 0 : (n > p.k ? p.k : n);
-    const int* di = p.draft_idx + draft_row * (size_t)p.k;
-    const float* dl = p.draft_logit + draft_row * (size_t)p.k;
+    const int n = draft_len(p, draft_row);
     double mx = -INFINITY;
     for (int i = tid; i < n; i += kBlockThreads) {
-        A.s_idx[i] = di[i];
-        const float l = dl[i];
+        int v;
+        float l;
+        draft_entry(p, draft_row, i, &v, &l);
+        A.s_idx[i] = v;
         const bool fin = fabsf(l) <= 3.4028234e38f;
         const double y = fin ? (double)l * p.cq.d : -INFINITY;
         A.s_q[i] = y;
@@ -276,23 +310,24 @@ __device__ __forceinline__ double row_log2_norm_warp(const float2* part, int nch
 template <typename T>
 __device__ __forceinline__ double position_accept_prob(const VerifyParams& p, size_t draft_row, const unsigned char* rowp,
                                                        double L2, int lane, double* beta_hat_out) {
-    int n = p.draft_count[draft_row];
-    n = n < 0 ? 0 : (n > p.k ? p.k : n);
-    const int* di = p.draft_idx + draft_row * (size_t)p.k;
-    const float* dl = p.draft_logit + draft_row * (size_t)p.k;
+    const int n = draft_len(p, draft_row);
     const int x = p.draft_token[draft_row];
     double mx = -INFINITY;
     for (int i = lane; i < n; i += 32) {
-        const float l = dl[i];
+        int v;
+        float l;
+        draft_entry(p, draft_row, i, &v, &l);
         if (fabsf(l) <= 3.4028234e38f) mx = fmax(mx, (double)l * p.cq.d);
     }
     mx = warp_max(mx);
     double w = 0.0, ex = 0.0;
     for (int i = lane; i < n; i += 32) {
-        const float l = dl[i];
+        int v;
+        float l;
+        draft_entry(p, draft_row, i, &v, &l);
         const double e = fabsf(l) <= 3.4028234e38f ? exp2((double)l * p.cq.d - mx) : 0.0;
         w += e;
-        if (di[i] == x) ex = e;
+        if (v == x) ex = e;
     }
     const double W = warp_sum(w);
     ex = warp_max(ex);  // the pairs are distinct: at most one lane found x
@@ -300,9 +335,11 @@ __device__ __forceinline__ double position_accept_prob(const VerifyParams& p, si
     if (beta_hat_out) {
         double bh = 0.0;
         for (int i = lane; i < n; i += 32) {
-            const float l = dl[i];
+            int v;
+            float l;
+            draft_entry(p, draft_row, i, &v, &l);
             const double e = fabsf(l) <= 3.4028234e38f ? exp2((double)l * p.cq.d - mx) : 0.0;
-            bh += fmin(token_prob<T>(rowp, di[i], p.V, (double)p.cp.f, L2), W > 0.0 ? e / W : 0.0);
+            bh += fmin(token_prob<T>(rowp, v, p.V, (double)p.cp.f, L2), W > 0.0 ? e / W : 0.0);
         }
         *beta_hat_out = warp_sum(bh);
     }
@@ -326,9 +363,14 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
             // what the acceptance test will read after the log-normaliser is asked for now: the
             // position's transmitted pairs and the target logit of its drafted token
             const size_t dr = (size_t)b * gamma + j;
-            for (int o = lane * 32; o < p.k; o += 32 * 32) {
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_logit + dr * (size_t)p.k + o));
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_idx + dr * (size_t)p.k + o));
+            if (p.payload) {
+                for (int o = lane * 32; o < p.pay_words; o += 32 * 32)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.payload + dr * (size_t)p.pay_words + o));
+            } else {
+                for (int o = lane * 32; o < p.k; o += 32 * 32) {
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_logit + dr * (size_t)p.k + o));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.draft_idx + dr * (size_t)p.k + o));
+                }
             }
             if (lane == 0) {
                 const int x = p.draft_token[dr];
@@ -732,19 +774,23 @@ extern "C" int tslt_verify_workspace_bytes(int B, int gamma, int V, int k, size_
     return TSLT_OK;
 }
 
-extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,
-                           long long row_stride_elems, int k, const int* draft_idx, const float* draft_logit,
-                           const int* draft_count, const int* draft_token, float draft_temperature,
-                           float target_temperature, const float* u_accept, const float* u_sample,
-                           int* accepted_len, int* out_token, float* accept_prob, float* beta_hat,
-                           float* lse_p, void* workspace, size_t workspace_bytes, void* stream) {
+// The drafts come either as the arrays tslt_sparsify writes (payload == nullptr) or as packed records.
+static int verify_impl(const void* target_logits, int dtype, int B, int gamma, int V, long long row_stride_elems, int k,
+                       const int* draft_idx, const float* draft_logit, const int* draft_count,
+                       const unsigned int* payload, int prob_format, const int* draft_token, float draft_temperature,
+                       float target_temperature, const float* u_accept, const float* u_sample, int* accepted_len,
+                       int* out_token, float* accept_prob, float* beta_hat, float* lse_p, void* workspace,
+                       size_t workspace_bytes, void* stream) {
     if (B < 0 || gamma < 0) return TSLT_ERR_INVALID_ARG;
+    int bi = 0, bp = 0, words = 0;
+    if (payload && (V <= 0 || k <= 0 || k > TSLT_MAX_K || !payload_shape(k, V, prob_format, &bi, &bp, &words)))
+        return V <= 0 || k <= 0 ? TSLT_ERR_INVALID_ARG : TSLT_ERR_UNSUPPORTED;
     if (B == 0) return TSLT_OK;
     int rc = check_common(target_logits, dtype, V, row_stride_elems, k, draft_temperature, target_temperature,
                           workspace);
     if (rc != TSLT_OK) return rc;
     if (!u_sample || !accepted_len || !out_token ||
-        (gamma > 0 && (!draft_idx || !draft_logit || !draft_count || !draft_token || !u_accept)))
+        (gamma > 0 && ((!payload && (!draft_idx || !draft_logit || !draft_count)) || !draft_token || !u_accept)))
         return TSLT_ERR_INVALID_ARG;
     if ((long long)B * (gamma + 1) > 0x7fffffffLL / 16 || gamma >= 1024) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
@@ -758,6 +804,7 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
+    p.payload = payload; p.pay_words = words; p.pay_bi = bi; p.pay_bp = bp; p.pay_fmt = prob_format;
     p.gamma = gamma; p.draft_token = draft_token; p.u_accept = u_accept; p.u_sample = u_sample;
     p.accepted_len = accepted_len; p.out_token = out_token;
     p.accept_prob = accept_prob; p.beta_hat = beta_hat; p.lse_p = lse_p;
@@ -765,6 +812,31 @@ extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamm
     p.status = (int*)ws;
     p.partials = (float2*)(ws + pl.ws_partials_off);
     return launch_verify<false>(p, pl, dtype, (cudaStream_t)stream);
+}
+
+extern "C" int tslt_verify(const void* target_logits, int dtype, int B, int gamma, int V,
+                           long long row_stride_elems, int k, const int* draft_idx, const float* draft_logit,
+                           const int* draft_count, const int* draft_token, float draft_temperature,
+                           float target_temperature, const float* u_accept, const float* u_sample,
+                           int* accepted_len, int* out_token, float* accept_prob, float* beta_hat,
+                           float* lse_p, void* workspace, size_t workspace_bytes, void* stream) {
+    return verify_impl(target_logits, dtype, B, gamma, V, row_stride_elems, k, draft_idx, draft_logit, draft_count, nullptr,
+                       0, draft_token, draft_temperature, target_temperature, u_accept, u_sample, accepted_len, out_token,
+                       accept_prob, beta_hat, lse_p, workspace, workspace_bytes, stream);
+}
+
+extern "C" int tslt_verify_packed(const void* target_logits, int dtype, int B, int gamma, int V,
+                                  long long row_stride_elems, int k, const unsigned int* payload, int prob_format,
+                                  const int* draft_token, float draft_temperature, float target_temperature,
+                                  const float* u_accept, const float* u_sample, int* accepted_len, int* out_token,
+                                  float* accept_prob, float* beta_hat, float* lse_p, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+    if (B > 0 && gamma > 0 && !payload) return TSLT_ERR_INVALID_ARG;
+    static const unsigned int kNoRecords = 0;  // gamma == 0: nothing is read, but the packed path is still taken
+    return verify_impl(target_logits, dtype, B, gamma, V, row_stride_elems, k, nullptr, nullptr, nullptr,
+                       payload ? payload : &kNoRecords, prob_format, draft_token, draft_temperature, target_temperature,
+                       u_accept, u_sample, accepted_len, out_token, accept_prob, beta_hat, lse_p, workspace,
+                       workspace_bytes, stream);
 }
 
 // ---- tslt_verify_static: the same verification with the scratch memory built into the library ----
@@ -839,10 +911,14 @@ extern "C" int tslt_tree_verify_walk_workspace_bytes(int B, int N, int V, int k,
 static int tree_verify_impl(bool walk, const void* target_logits, int dtype, int B, int N, int V,
                             long long row_stride_elems, const int* parent, const int* node_draft_row, int M, int k,
                             const int* node_token, const int* draft_idx, const float* draft_logit,
-                            const int* draft_count, float draft_temperature, float target_temperature,
+                            const int* draft_count, const unsigned int* payload, int prob_format,
+                            float draft_temperature, float target_temperature,
                             const float* u_accept, const float* u_sample, int max_depth, int* accepted_path,
                             int* accepted_len, int* out_token, void* workspace, size_t workspace_bytes, void* stream) {
     if (B < 0 || N <= 0 || M < 0 || max_depth < 0 || !parent || !node_draft_row) return TSLT_ERR_INVALID_ARG;
+    int bi = 0, bp = 0, words = 0;
+    if (payload && (V <= 0 || k <= 0 || k > TSLT_MAX_K || !payload_shape(k, V, prob_format, &bi, &bp, &words)))
+        return V <= 0 || k <= 0 ? TSLT_ERR_INVALID_ARG : TSLT_ERR_UNSUPPORTED;
     if (N > kMaxTreeNodes) return TSLT_ERR_UNSUPPORTED;
     std::vector<int> meta;
     const int depth = build_tree_meta(N, M, parent, node_draft_row, meta);  // tree structure, checked on the host
@@ -852,7 +928,7 @@ static int tree_verify_impl(bool walk, const void* target_logits, int dtype, int
                           workspace);
     if (rc != TSLT_OK) return rc;
     if (!u_sample || !accepted_len || !out_token || (max_depth > 0 && !accepted_path) ||
-        (N > 1 && (!node_token || !u_accept)) || (M > 0 && (!draft_idx || !draft_logit || !draft_count)))
+        (N > 1 && (!node_token || !u_accept)) || (M > 0 && !payload && (!draft_idx || !draft_logit || !draft_count)))
         return TSLT_ERR_INVALID_ARG;
     if ((long long)B * N > 0x7fffffffLL / 64) return TSLT_ERR_UNSUPPORTED;
     const int eb = dtype == TSLT_F32 ? 4 : 2;
@@ -869,6 +945,7 @@ static int tree_verify_impl(bool walk, const void* target_logits, int dtype, int
     p.cp = make_scale(target_temperature);
     p.cq = make_scale(draft_temperature);
     p.draft_idx = draft_idx; p.draft_logit = draft_logit; p.draft_count = draft_count;
+    p.payload = payload; p.pay_words = words; p.pay_bi = bi; p.pay_bp = bp; p.pay_fmt = prob_format;
     p.u_accept = u_accept; p.u_sample = u_sample;
     p.accepted_len = accepted_len; p.out_token = out_token;
     p.N = N; p.M = M; p.max_depth = max_depth;
@@ -904,7 +981,7 @@ extern "C" int tslt_tree_verify(const void* target_logits, int dtype, int B, int
                                 int max_depth, int* accepted_path, int* accepted_len, int* out_token,
                                 void* workspace, size_t workspace_bytes, void* stream) {
     return tree_verify_impl(false, target_logits, dtype, B, N, V, row_stride_elems, parent, node_draft_row, M, k,
-                            node_token, draft_idx, draft_logit, draft_count, draft_temperature, target_temperature,
+                            node_token, draft_idx, draft_logit, draft_count, nullptr, 0, draft_temperature, target_temperature,
                             u_accept, u_sample, max_depth, accepted_path, accepted_len, out_token, workspace,
                             workspace_bytes, stream);
 }
@@ -917,7 +994,22 @@ extern "C" int tslt_tree_verify_walk(const void* target_logits, int dtype, int B
                                      int max_depth, int* accepted_path, int* accepted_len, int* out_token,
                                      void* workspace, size_t workspace_bytes, void* stream) {
     return tree_verify_impl(true, target_logits, dtype, B, N, V, row_stride_elems, parent, node_draft_row, M, k,
-                            node_token, draft_idx, draft_logit, draft_count, draft_temperature, target_temperature,
+                            node_token, draft_idx, draft_logit, draft_count, nullptr, 0, draft_temperature, target_temperature,
                             u_accept, u_sample, max_depth, accepted_path, accepted_len, out_token, workspace,
                             workspace_bytes, stream);
+}
+
+extern "C" int tslt_tree_verify_packed(int walk, const void* target_logits, int dtype, int B, int N, int V,
+                                       long long row_stride_elems, const int* parent, const int* node_draft_row,
+                                       int M, int k, const int* node_token, const unsigned int* payload,
+                                       int prob_format, float draft_temperature, float target_temperature,
+                                       const float* u_accept, const float* u_sample, int max_depth,
+                                       int* accepted_path, int* accepted_len, int* out_token, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+    if (B > 0 && M > 0 && !payload) return TSLT_ERR_INVALID_ARG;
+    static const unsigned int kNoRecords = 0;  // M == 0: nothing is read, but the packed path is still taken
+    return tree_verify_impl(walk != 0, target_logits, dtype, B, N, V, row_stride_elems, parent, node_draft_row, M, k,
+                            node_token, nullptr, nullptr, nullptr, payload ? payload : &kNoRecords, prob_format,
+                            draft_temperature, target_temperature, u_accept, u_sample, max_depth, accepted_path,
+                            accepted_len, out_token, workspace, workspace_bytes, stream);
 }

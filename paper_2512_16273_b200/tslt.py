@@ -29,6 +29,7 @@ EXPORTS = ["tslt_version", "tslt_status_string", "tslt_workspace_status", "tslt_
            "tslt_tree_verify_workspace_bytes", "tslt_tree_verify",
            "tslt_tree_verify_walk_workspace_bytes", "tslt_tree_verify_walk",
            "tslt_payload_words", "tslt_pack_payload", "tslt_unpack_payload",
+           "tslt_verify_packed", "tslt_tree_verify_packed",
            "tslt_diagnostics_workspace_bytes", "tslt_diagnostics"]
 
 PROB_F32, PROB_BF16, PROB_F16 = 0, 1, 2
@@ -89,6 +90,10 @@ def lib() -> ctypes.CDLL:
     L.tslt_diagnostics_workspace_bytes.argtypes = [i, i, i, i, psz]
     L.tslt_diagnostics.restype = i
     L.tslt_diagnostics.argtypes = [p, p, i, i, i, ll, p, i, i, f, f, p, p, p, p, p, p, p, sz, p]
+    L.tslt_verify_packed.restype = i
+    L.tslt_verify_packed.argtypes = [p, i, i, i, i, ll, i, p, i, p, f, f, p, p, p, p, p, p, p, p, sz, p]
+    L.tslt_tree_verify_packed.restype = i
+    L.tslt_tree_verify_packed.argtypes = [i, p, i, i, i, i, ll, p, p, i, i, p, p, i, f, f, p, p, i, p, p, p, p, sz, p]
     L.tslt_payload_words.restype = i
     L.tslt_payload_words.argtypes = [i, i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
     L.tslt_pack_payload.restype = i
@@ -218,6 +223,7 @@ def workspace_status(ws: torch.Tensor) -> int:
 
 
 STATUS_WAIT_FELL_BACK = 1
+STATUS_BAD_RECORD = 2
 
 
 def set_ready_poll_limit(polls: int) -> None:
@@ -530,6 +536,95 @@ def tree_verify(target_logits: torch.Tensor, parent: Sequence[int], node_draft_r
                                 max_depth, _ptr(o["accepted_path"]), _ptr(o["accepted_len"]),
                                 _ptr(o["out_token"]), _ptr(ws), ws.numel(), _stream())
     _check(rc, "tslt_tree_verify_walk" if walk else "tslt_tree_verify")
+    o["workspace"] = ws
+    return o
+
+
+def verify_packed(target_logits: torch.Tensor, payload: torch.Tensor, prob_format: int, k: int,
+                  draft_token: torch.Tensor, draft_temperature: float, target_temperature: float,
+                  u_accept: torch.Tensor, u_sample: torch.Tensor, *, want_diag: bool = True,
+                  out: Optional[dict] = None, ws: Optional[torch.Tensor] = None) -> dict:
+    """tslt_verify_packed: tslt_verify on the uplink records themselves.  payload [B*gamma, words] int32
+    as pack_payload writes it (words = payload_words(k, V, prob_format)[0]).  Returns what verify() returns."""
+    if not target_logits.is_cuda:
+        raise ValueError("target_logits must be a CUDA tensor (libtslt has no CPU path)")
+    if target_logits.dim() != 3:
+        raise ValueError("target_logits must be [B, gamma+1, V]")
+    B, g1, V = target_logits.shape
+    _, _, stride = _row_layout(target_logits)
+    gamma = g1 - 1
+    dev = target_logits.device
+    words, _ = payload_words(k, V, prob_format)
+    _cuda(payload, "payload", torch.int32)
+    _cuda(draft_token, "draft_token", torch.int32)
+    _cuda(u_accept, "u_accept", torch.float32)
+    _cuda(u_sample, "u_sample", torch.float32)
+    if payload.numel() != B * gamma * words or draft_token.numel() != B * gamma or \
+            u_accept.numel() != B * gamma or u_sample.numel() != B:
+        raise ValueError("payload / token / uniform shapes do not match target_logits")
+    o = out if out is not None else {}
+    if "accepted_len" not in o:
+        o["accepted_len"] = torch.empty(B, dtype=torch.int32, device=dev)
+        o["out_token"] = torch.empty(B, dtype=torch.int32, device=dev)
+        if want_diag:
+            o["accept_prob"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
+            o["beta_hat"] = torch.empty(B, gamma, dtype=torch.float32, device=dev)
+            o["lse_p"] = torch.empty(B, gamma + 1, dtype=torch.float32, device=dev)
+    _check_verify_outputs(o, B, gamma)
+    if ws is None:
+        ws = workspace(verify_workspace_bytes(B, gamma, V, k), dev)
+    rc = lib().tslt_verify_packed(_ptr(target_logits), _dtype_code(target_logits), B, gamma, V, stride, k,
+                                  _ptr(payload), prob_format, _ptr(draft_token), draft_temperature, target_temperature,
+                                  _ptr(u_accept), _ptr(u_sample), _ptr(o["accepted_len"]), _ptr(o["out_token"]),
+                                  _ptr(o.get("accept_prob")), _ptr(o.get("beta_hat")), _ptr(o.get("lse_p")), _ptr(ws),
+                                  ws.numel(), _stream())
+    _check(rc, "tslt_verify_packed")
+    o["workspace"] = ws
+    return o
+
+
+def tree_verify_packed(target_logits: torch.Tensor, parent: Sequence[int], node_draft_row: Sequence[int],
+                       node_token: torch.Tensor, payload: torch.Tensor, prob_format: int, k: int,
+                       draft_temperature: float, target_temperature: float, u_accept: torch.Tensor,
+                       u_sample: torch.Tensor, max_depth: int, *, out: Optional[dict] = None,
+                       ws: Optional[torch.Tensor] = None, walk: bool = False) -> dict:
+    """tslt_tree_verify_packed: tree_verify() with the drafts as uplink records, payload [B*M, words]."""
+    if not target_logits.is_cuda:
+        raise ValueError("target_logits must be a CUDA tensor (libtslt has no CPU path)")
+    if target_logits.dim() != 3:
+        raise ValueError("target_logits must be [B, N, V]")
+    B, N, V = target_logits.shape
+    _, _, stride = _row_layout(target_logits)
+    par = np.ascontiguousarray(np.asarray(parent, dtype=np.int32))
+    ndr = np.ascontiguousarray(np.asarray(node_draft_row, dtype=np.int32))
+    if par.shape != (N,) or ndr.shape != (N,):
+        raise ValueError("parent and node_draft_row must have N entries")
+    M = int((ndr >= 0).sum())
+    dev = target_logits.device
+    words, _ = payload_words(k, V, prob_format)
+    for name, t, dt in (("node_token", node_token, torch.int32), ("payload", payload, torch.int32),
+                        ("u_accept", u_accept, torch.float32), ("u_sample", u_sample, torch.float32)):
+        _cuda(t, name, dt)
+    if node_token.numel() != B * N or u_accept.numel() != B * N or u_sample.numel() != B * N or \
+            payload.numel() != B * M * words:
+        raise ValueError("tree tensors do not match target_logits / the tree shape")
+    o = out if out is not None else {}
+    if "accepted_len" not in o:
+        o["accepted_path"] = torch.empty(B, max_depth, dtype=torch.int32, device=dev)
+        o["accepted_len"] = torch.empty(B, dtype=torch.int32, device=dev)
+        o["out_token"] = torch.empty(B, dtype=torch.int32, device=dev)
+    for name, dt, ne in (("accepted_path", torch.int32, B * max_depth), ("accepted_len", torch.int32, B),
+                         ("out_token", torch.int32, B)):
+        _out(o, name, dt, ne)
+    if ws is None:
+        ws = workspace((tree_verify_walk_workspace_bytes if walk else tree_verify_workspace_bytes)(B, N, V, k), dev)
+    rc = lib().tslt_tree_verify_packed(1 if walk else 0, _ptr(target_logits), _dtype_code(target_logits), B, N, V, stride,
+                                       par.ctypes.data_as(ctypes.c_void_p), ndr.ctypes.data_as(ctypes.c_void_p), M, k,
+                                       _ptr(node_token), _ptr(payload), prob_format, draft_temperature,
+                                       target_temperature, _ptr(u_accept), _ptr(u_sample), max_depth,
+                                       _ptr(o["accepted_path"]), _ptr(o["accepted_len"]), _ptr(o["out_token"]), _ptr(ws),
+                                       ws.numel(), _stream())
+    _check(rc, "tslt_tree_verify_packed")
     o["workspace"] = ws
     return o
 
