@@ -69,7 +69,7 @@ def kernel_source_digest() -> str:
     while the kernels are the ones that were captured."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2512_16273_b200", "csrc")
-    for name in ("tslt_common.cuh", "tslt_rowmath.cuh", "tslt_sparsify.cu", "tslt_verify.cu"):  # the timed kernels
+    for name in ("tslt_common.cuh", "tslt_rowmath.cuh", "tslt_payload.cuh", "tslt_sparsify.cu", "tslt_verify.cu"):  # the timed kernels
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
