@@ -677,3 +677,33 @@ def test_degenerate_residual_falls_back_to_the_target():
     o = oracle.verify(zp, idx, logit, count, np.array([[3]], np.int32), 1.0, 1.0,
                       np.array([[0.5]], np.float32), np.array([0.5], np.float32))
     assert o["accepted_len"][0] == 1 and not (o["flags"][0] & oracle.FLAG_DEGEN)
+
+
+def test_truncation_of_a_row_from_its_vocabulary_shards():
+    """What the sharded two-stage form rests on, checked on the oracle alone: the k best tokens of a row
+    (logit descending, index ascending) are among the k best of their own shards, and the row's
+    normaliser is the sum of the shards' (Section 3.1's truncation equation needs nothing else of the
+    row).  Shards are ragged; one holds fewer than k finite logits, one holds ties that straddle the cut."""
+    rng = np.random.default_rng(12)
+    V, k, T = 3000, 40, 0.8
+    z = rng.normal(size=(3, V)).astype(np.float32) * 2.0
+    z[0, 1000:1990] = -np.inf            # a shard with 10 finite logits
+    z[1, 2100:2160] = z[1].max() + 1.0   # 60 ties at the top, all in the last shard: the cut falls among them
+    bounds = [0, 7, 1000, 2000, V]
+    u = np.zeros((3, 1), np.float32)
+    whole = oracle.sparsify(z, k, 1.0, T, u)
+    cand_idx, cand_logit, lses = [], [], []
+    for a, b in zip(bounds, bounds[1:]):
+        part = oracle.sparsify(np.ascontiguousarray(z[:, a:b]), min(k, b - a), 1.0, T, u)
+        cand_idx.append(np.where(part["idx"] >= 0, part["idx"] + a, -1))
+        cand_logit.append(part["logit"])
+        lses.append(part["lse"])
+    ci, cl = np.concatenate(cand_idx, 1), np.concatenate(cand_logit, 1)
+    for r in range(3):
+        keep = ci[r] >= 0
+        order = np.lexsort((ci[r][keep], -cl[r][keep].astype(np.float64)))[:k]
+        merged = np.sort(ci[r][keep][order])
+        n = int(whole["count"][r])
+        assert np.array_equal(merged[:n], whole["idx"][r, :n]) and len(merged) == n
+    lse = scipy.special.logsumexp(np.stack(lses, 1), axis=1)
+    assert np.allclose(lse, whole["lse"], rtol=1e-12, atol=1e-12)
