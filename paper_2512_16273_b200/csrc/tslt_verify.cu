@@ -284,19 +284,37 @@ __device__ __forceinline__ int sample_full_vocab(const VerifyParams& p, const un
 
 // One warp: base-2 log-normaliser of a row from its chunk partials (warp shuffles only).
 __device__ __forceinline__ double row_log2_norm_warp(const float2* part, int nchunks, int lane) {
-    double mx = -INFINITY;
-    for (int c = lane; c < nchunks; c += 32) {
-        const float2 ms = __ldcg(&part[c]);
-        if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
-    }
-    mx = warp_max(mx);
     // fp64 is scarce (two warp instructions per clock per SM): the per-chunk factors 2^(M_c - M)
     // are taken in fp32 (the exponents are differences of nearby chunk maxima, so the 1-ulp factor
     // errors are ~1e-7 with random sign over hundreds of chunks); the sum is kept in fp64
-    double s = 0.0;
-    for (int c = lane; c < nchunks; c += 32) {
-        const float2 ms = __ldcg(&part[c]);
-        if (ms.y > 0.f) s += (double)(ms.y * exp2f((float)((double)ms.x - mx)));
+    constexpr int kHold = 8;  // pairs a lane keeps in registers: rows of up to 256 chunks (512 KB) take one trip to memory
+    double mx = -INFINITY, s = 0.0;
+    if (nchunks <= 32 * kHold) {
+        float2 ms[kHold];
+#pragma unroll
+        for (int j = 0; j < kHold; ++j) {
+            const int c = lane + 32 * j;
+            ms[j] = c < nchunks ? __ldcg(&part[c]) : make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < kHold; ++j)
+            if (ms[j].y > 0.f) mx = fmax(mx, (double)ms[j].x);
+        mx = warp_max(mx);
+#pragma unroll
+        for (int j = 0; j < kHold; ++j)
+            if (ms[j].y > 0.f) s += (double)(ms[j].y * exp2f((float)((double)ms[j].x - mx)));
+    } else {
+#pragma unroll 4
+        for (int c = lane; c < nchunks; c += 32) {
+            const float2 ms = __ldcg(&part[c]);
+            if (ms.y > 0.f) mx = fmax(mx, (double)ms.x);
+        }
+        mx = warp_max(mx);
+#pragma unroll 4
+        for (int c = lane; c < nchunks; c += 32) {
+            const float2 ms = __ldcg(&part[c]);
+            if (ms.y > 0.f) s += (double)(ms.y * exp2f((float)((double)ms.x - mx)));
+        }
     }
     s = warp_sum(s);
     double L2 = -INFINITY;
@@ -305,13 +323,60 @@ __device__ __forceinline__ double row_log2_norm_warp(const float2* part, int nch
 }
 
 // One warp: acceptance probability min(1, p(x) / q~(x)) of one position, and (if wanted) the
-// truncated acceptance rate sum_S min(p, q~).  q~ is rebuilt from the transmitted pairs in
-// passes over global memory (at most 8 KB, cache resident); nothing is staged.
+// truncated acceptance rate sum_S min(p, q~).  q~ is rebuilt from the transmitted pairs: up to 256
+// pairs wait in registers (one trip to memory for them, one for the target logits at their tokens);
+// more are read in passes over global memory (at most 8 KB, cache resident).
 template <typename T>
 __device__ __forceinline__ double position_accept_prob(const VerifyParams& p, size_t draft_row, const unsigned char* rowp,
                                                        double L2, int lane, double* beta_hat_out) {
     const int n = draft_len(p, draft_row);
     const int x = p.draft_token[draft_row];
+    constexpr int kHold = 8;  // pairs a lane keeps in registers: up to 256 pairs take one trip to memory
+    if (n <= 32 * kHold) {
+        const double cs = (double)p.cp.f;
+        int v[kHold];
+        float l[kHold], zt[kHold];
+#pragma unroll
+        for (int j = 0; j < kHold; ++j) {
+            const int i = lane + 32 * j;
+            v[j] = -1;
+            l[j] = -INFINITY;
+            if (i < n) draft_entry(p, draft_row, i, &v[j], &l[j]);
+        }
+        const float zx = (x >= 0 && x < p.V) ? Elt<T>::load(rowp, x) : -INFINITY;  // asked for before the pairs are used
+        if (beta_hat_out) {
+#pragma unroll
+            for (int j = 0; j < kHold; ++j) zt[j] = (v[j] >= 0 && v[j] < p.V) ? Elt<T>::load(rowp, v[j]) : -INFINITY;
+        }
+        double mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < kHold; ++j)
+            if (fabsf(l[j]) <= 3.4028234e38f) mx = fmax(mx, (double)l[j] * p.cq.d);
+        mx = warp_max(mx);
+        double e[kHold], w = 0.0, ex = 0.0;
+#pragma unroll
+        for (int j = 0; j < kHold; ++j) {
+            e[j] = fabsf(l[j]) <= 3.4028234e38f ? exp2((double)l[j] * p.cq.d - mx) : 0.0;
+            w += e[j];
+            if (lane + 32 * j < n && v[j] == x) ex = e[j];
+        }
+        const double W = warp_sum(w);
+        ex = warp_max(ex);  // the pairs are distinct: at most one lane found x
+        const double qx = W > 0.0 ? ex / W : 0.0;
+        const bool row_ok = L2 > -INFINITY;
+        if (beta_hat_out) {
+            double bh = 0.0;
+#pragma unroll
+            for (int j = 0; j < kHold; ++j) {
+                const double pv = (row_ok && fabsf(zt[j]) <= 3.4028234e38f) ? exp2((double)zt[j] * cs - L2) : 0.0;
+                if (lane + 32 * j < n) bh += fmin(pv, W > 0.0 ? e[j] / W : 0.0);
+            }
+            *beta_hat_out = warp_sum(bh);
+        }
+        const double px = (row_ok && fabsf(zx) <= 3.4028234e38f) ? exp2((double)zx * cs - L2) : 0.0;
+        return accept_probability(px, qx);
+    }
+    // more pairs than a lane holds: passes over the pairs (cache resident after the first)
     double mx = -INFINITY;
     for (int i = lane; i < n; i += 32) {
         int v;
