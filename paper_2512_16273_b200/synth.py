@@ -59,6 +59,11 @@ def uniforms(shape: Sequence[int], seed: int, tensor_id: int, device="cpu") -> t
                       dtype=torch.float32)
 
 
+def draft_rows(rows: int, V: int, dtype: torch.dtype, seed: int, device="cpu") -> torch.Tensor:
+    """Draft logits [rows, V] alone (the rows sequence_logits would draw as its draft)."""
+    return _zipf_rows(rows, V, _gen(seed, TID_DRAFT, device), device).to(dtype).contiguous()
+
+
 def sequence_logits(B: int, gamma: int, V: int, dtype: torch.dtype, sigma_t: float,
                     seed: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
     """Draft logits [B, gamma, V] and target logits [B, gamma+1, V] for single-candidate TSLT.

@@ -66,6 +66,47 @@ def test_many_rows_take_the_two_launch_verifier():
     assert ref["accepted_len"].max() >= 1
 
 
+def sparsify_only_case(z_cpu, k, top_p, T, seed, ns, what):
+    rows, V = z_cpu.shape
+    u = synth.uniforms((rows, ns), seed, synth.TID_U_DRAFT)
+    ref = oracle_sparsify_parallel(z_cpu, k, top_p, T, u.numpy())
+    got = tslt.sparsify(to_gpu_rows(z_cpu), k, top_p, T, u.cuda())
+    torch.cuda.synchronize()
+    assert tslt.workspace_status(got["workspace"]) == 0
+    return compare_sparsify(got, ref, what, logits=z_cpu, uniforms=u, T=T)
+
+
+def test_long_rows_in_both_forms():
+    """Rows several times the benchmark's.  600 rows of 600 000 bf16 logits fill the machine, so each row
+    is one streaming CTA whose tile maxima (37 KB) no longer fit one line per thread and whose groups span
+    several lines; 3 rows of 3 000 000 logits are cut into 64 segments each, with thousands of groups at
+    k = 1024 and groups of 2048 tiles at k = 16."""
+    z = synth.draft_rows(600, 600000, torch.bfloat16, 41, "cuda").cpu()  # (drawn on the GPU: 360 M logits)
+    sparsify_only_case(z, 64, 1.0, 1.0, 41, 1, "600 x 600000 k=64")
+    sparsify_only_case(z, 1024, 0.95, 0.8, 42, 2, "600 x 600000 top-p cap 1024")
+    del z
+    z = synth.draft_rows(3, 3000000, torch.bfloat16, 43, "cuda").cpu()
+    sparsify_only_case(z, 1024, 1.0, 1.0, 43, 1, "3 x 3000000 k=1024")
+    sparsify_only_case(z, 16, 0.9, 1.0, 44, 3, "3 x 3000000 k=16 top-p")
+    zf = synth.draft_rows(2, 1500000, torch.float32, 45, "cuda").cpu()
+    sparsify_only_case(zf, 320, 1.0, 1.0, 45, 1, "2 x 1500000 fp32 k=320")
+
+
+def test_verify_longest_rows():
+    """The verifier's row limit (4 MiB per row: 2 097 152 bf16 logits, 2048 chunk partials per row) and an
+    fp32 row of 586 chunks: more partials than a lane keeps in registers."""
+    zq, zp = small_logits(2, 2, 2097152, torch.bfloat16, seed=51)
+    run_sequence_case(zq, zp, 64, 1.0, 1.0, seed=51, what="V=2097152 bf16")
+    zq, zp = small_logits(3, 3, 300000, torch.float32, seed=52)
+    run_sequence_case(zq, zp, 300, 0.95, 0.9, seed=52, num_samples=2, what="V=300000 fp32")
+    z = torch.zeros(1, 2, 2097160, dtype=torch.bfloat16, device="cuda")  # one vector beyond the limit
+    d = tslt.sparsify(z[:, :1].reshape(1, -1), 4, 1.0, 1.0, torch.zeros(1, 1, device="cuda"))
+    with pytest.raises(tslt.TsltError) as e:
+        tslt.verify(z, d["idx"].view(1, 1, 4), d["logit"].view(1, 1, 4), d["count"].view(1, 1), d["token"].view(1, 1), 1.0, 1.0,
+                    torch.zeros(1, 1, device="cuda"), torch.zeros(1, device="cuda"))
+    assert e.value.status == tslt.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("kk,top_p", synth.CONFIGS[4]["sweep"])
 def test_config4_full_size_every_row_against_oracle(kk, top_p):
     """The benchmark workload at full size (B = 256, gamma = 8, V = 256000, bf16: 2048 draft rows and
