@@ -454,6 +454,24 @@ def time_small_configs(tslt, dev, peak):
             assert tslt.workspace_status(ws_s) == 0 and tslt.workspace_status(ws_v) == 0
             res["tslt_sparsify"] = entry(us_s, sparsify_bytes(B * gamma, V, eb, k), B * gamma, peak)
             res["tslt_verify"] = entry(us_v, verify_bytes(B, gamma + 1, B * gamma, V, eb, k), B * (gamma + 1), peak)
+            # the verifier on the uplink records themselves against unpacking them first (same verdicts)
+            fmt = tslt.PROB_BF16 if cfg["dtype"] == "bf16" else tslt.PROB_F32
+            wire = tslt.pack_payload(s_out["idx"], s_out["logit"], s_out["count"], V, fmt)["payload"]
+            p_out = {n: torch.empty_like(t) for n, t in v_out.items()}
+            us_p = time_rotating(lambda i: tslt.verify_packed(zp_all[i], wire, fmt, k, s_out["token"], T, T, ua, us,
+                                                              out=p_out, ws=ws_v), cp)
+
+            d = tslt.unpack_payload(wire, k, V, fmt)
+
+            def unpack_then_verify(i):
+                tslt.unpack_payload(wire, k, V, fmt, out=d)
+                tslt.verify(zp_all[i], d["idx"], d["logit"], d["count"], s_out["token"], T, T, ua, us, out=v_out, ws=ws_v)
+            us_u = time_rotating(unpack_then_verify, cp)
+            torch.cuda.synchronize()
+            assert all(torch.equal(p_out[n], v_out[n]) for n in ("accepted_len", "out_token")), "packed verifier disagrees"
+            res["tslt_verify_packed"] = entry(us_p, verify_bytes(B, gamma + 1, B * gamma, V, eb, k), B * (gamma + 1), peak)
+            res["tslt_unpack_payload+tslt_verify"] = entry(us_u, verify_bytes(B, gamma + 1, B * gamma, V, eb, k),
+                                                           B * (gamma + 1), peak)
             res["input_copies"] = {"draft": cq, "target": cp}
             del zq_all, zp_all
         else:

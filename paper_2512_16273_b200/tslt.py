@@ -652,19 +652,23 @@ def pack_payload(idx: torch.Tensor, logit: torch.Tensor, count: torch.Tensor, V:
     return {"payload": payload, "bits": bits}
 
 
-def unpack_payload(payload: torch.Tensor, k: int, V: int, prob_format: int) -> dict:
+def unpack_payload(payload: torch.Tensor, k: int, V: int, prob_format: int, *, out: Optional[dict] = None) -> dict:
     """tslt_unpack_payload: records [rows, words] -> dict(idx, logit [rows, k], count [rows], flag [1])
-    in the form verify / tree_verify take."""
+    in the form verify / tree_verify take.  `out` reuses buffers of an earlier call (its flag is sticky)."""
     _cuda(payload, "payload", torch.int32)
     words, _ = payload_words(k, V, prob_format)
     if payload.dim() != 2 or payload.shape[1] != words:
         raise ValueError("payload must be [rows, %d] for this k, V and format" % words)
     rows = payload.shape[0]
     dev = payload.device
-    o = {"idx": torch.empty(rows, k, dtype=torch.int32, device=dev),
-         "logit": torch.empty(rows, k, dtype=torch.float32, device=dev),
-         "count": torch.empty(rows, dtype=torch.int32, device=dev),
-         "flag": torch.zeros(1, dtype=torch.int32, device=dev)}
+    o = out if out is not None else {
+        "idx": torch.empty(rows, k, dtype=torch.int32, device=dev),
+        "logit": torch.empty(rows, k, dtype=torch.float32, device=dev),
+        "count": torch.empty(rows, dtype=torch.int32, device=dev),
+        "flag": torch.zeros(1, dtype=torch.int32, device=dev)}
+    for name, dt, ne in (("idx", torch.int32, rows * k), ("logit", torch.float32, rows * k), ("count", torch.int32, rows),
+                         ("flag", torch.int32, 1)):
+        _out(o, name, dt, ne)
     _check(lib().tslt_unpack_payload(_ptr(payload), rows, k, V, prob_format, _ptr(o["idx"]), _ptr(o["logit"]),
                                      _ptr(o["count"]), _ptr(o["flag"]), _stream()), "tslt_unpack_payload")
     return o
