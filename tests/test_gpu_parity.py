@@ -92,6 +92,14 @@ def test_long_rows_in_both_forms():
     sparsify_only_case(zf, 320, 1.0, 1.0, 45, 1, "2 x 1500000 fp32 k=320")
 
 
+@pytest.mark.parametrize("rows", [591, 592, 593, 1184])
+def test_row_counts_around_the_machine_size(rows):
+    """One row fewer than the streaming kernel's CTA slots (rows cut in two), exactly as many and one more
+    (one CTA per row), and two full waves."""
+    z = synth.draft_rows(rows, 20011, torch.bfloat16, rows, "cpu")
+    sparsify_only_case(z, 32, 0.9, 1.0, rows, 1, "rows=%d" % rows)
+
+
 def test_verify_longest_rows():
     """The verifier's row limit (4 MiB per row: 2 097 152 bf16 logits, 2048 chunk partials per row) and an
     fp32 row of 586 chunks: more partials than a lane keeps in registers."""
