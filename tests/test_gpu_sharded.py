@@ -88,3 +88,27 @@ def test_merge_rejects_what_it_cannot_hold():
     with pytest.raises(tslt.TsltError) as e:
         tslt.sparsify_merge(part["idx"][:2], part["logit"][:2], part["count"][:2], part["lse2"][:2], [10, 10], torch.float32)
     assert e.value.status == tslt.ERR_INVALID_ARG  # offsets must ascend
+
+
+def test_vocab_parallel_glue_on_one_rank():
+    """The glue with the library's own kernels and NCCL, as far as one GPU goes: a process group of one
+    rank, whose single slice is the whole vocabulary; same outputs as tslt_sparsify."""
+    import torch.distributed as dist
+    from paper_2512_16273_b200 import vocab_parallel
+    created = False
+    if not dist.is_initialized():
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29877", rank=0, world_size=1)
+        created = True
+    try:
+        V, k = 20016, 64
+        z = synth.draft_rows(6, V, torch.bfloat16, 8, "cuda")
+        u = synth.uniforms((6, 2), 8, 11, "cuda")
+        got = vocab_parallel.sparsify_vocab_parallel(z, 0, k, 0.95, 0.8, u)
+        want = tslt.sparsify(z, k, 0.95, 0.8, u)
+        torch.cuda.synchronize()
+        for name in ("idx", "logit", "count", "token"):
+            assert to_np(got[name]).tobytes() == to_np(want[name]).tobytes(), name
+        assert np.allclose(to_np(got["lse"]), to_np(want["lse"]), rtol=1e-6, atol=1e-6)
+    finally:
+        if created:
+            dist.destroy_process_group()
