@@ -1006,60 +1006,16 @@ __device__ __forceinline__ int gather_candidates(const unsigned char* rowp, cons
     bool in_smem = false;
     int n_c = 0;
     {
-        constexpr int kRegVecs = 4;
-        if (upt <= kRegVecs) {
-            // few vectors per thread (small k): one trip to memory, the vectors wait in registers
-            // while the prefix sum finds where their candidates go
-            uint4 d[kRegVecs];
-            int vi[kRegVecs];
-#pragma unroll
-            for (int j = 0; j < kRegVecs; ++j) {
-                const int u = u0 + j;
-                vi[j] = u < u1 ? (int)(tl[u >> 2] * (uint32_t)kVecsPerTile) + (u & 3) : -1;
-                if (vi[j] >= 0 && vi[j] < ext.nvec_full) d[j] = __ldcg(reinterpret_cast<const uint4*>(rowp) + vi[j]);
-            }
-            int cnt = 0;
-#pragma unroll
-            for (int j = 0; j < kRegVecs; ++j) {
-                if (vi[j] < 0) continue;
-                float z[kPer];
-                if (vi[j] < ext.nvec_full) {
-                    unpack_vec<T>(d[j], z);
-                } else {  // the row's ragged last vector: fetched element by element, kept in the same form
-                    load_row_vector<T>(rowp, vi[j], ext, V, z);
-                    d[j] = pack_vec<T>(z);
-                }
-#pragma unroll
-                for (int e = 0; e < kPer; ++e) cnt += is_candidate(z[e]) ? 1 : 0;
-            }
-            int cpos = block_exscan<NT>(cnt, tid, sh->iscr, &n_c);
-            if (n_c <= cand_cap) {
-                in_smem = true;
-#pragma unroll
-                for (int j = 0; j < kRegVecs; ++j) {
-                    if (vi[j] < 0) continue;
-                    float z[kPer];
-                    unpack_vec<T>(d[j], z);
-#pragma unroll
-                    for (int e = 0; e < kPer; ++e)
-                        if (is_candidate(z[e])) {
-                            c_raw[cpos] = __float_as_uint(z[e]);
-                            c_idx[cpos] = vi[j] * kPer + e;
-                            ++cpos;
-                        }
-                }
-                fsync<NT>();
-            }
-        } else {
-            // many vectors per thread: one pass; the first candidates a thread finds wait in a small
+        {
+            // one pass over the thread's vectors; the first candidates it finds wait in a small
             // stash while the prefix sum finds where they go.  A thread that found more than its
             // stash holds reads its own vectors a second time (from L2).
             constexpr int kStash = 12;
             uint32_t st_raw[kStash];
             int st_idx[kStash];
             int cnt = 0;
-            // every tile of this thread is asked of L2 first, so that the batches of loads below (six
-            // vectors in flight per thread) do not each pay a trip to HBM
+            // every tile of this thread is asked of L2 first, so that the loads below (two vectors in
+            // flight per thread) do not each pay a trip to HBM
             for (int u = u0; u < u1; ++u)
                 if (u == u0 || (u & 3) == 0)
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + (size_t)tl[u >> 2] * (kVecsPerTile * kVecBytes)));
