@@ -158,6 +158,25 @@ inline cudaError_t launch_dependent(void (*kernel)(const Params), unsigned grid,
     return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
+// ---- optional time stamps (build with -DTSLT_STAMPS; see paper_2512_16273_b200/timeline.py) -----------------
+// Thread 0 of a CTA writes %globaltimer into stamps[cta * kStampSlots + slot]: where the microseconds of a
+// call go, phase by phase.  The array is per translation unit; each .cu file that stamps exports a reader.
+// In the ordinary build the macro is empty and nothing of this exists.
+#ifdef TSLT_STAMPS
+constexpr int kStampCtas = 16384, kStampSlots = 8;
+static __device__ unsigned long long g_stamps[kStampCtas * kStampSlots];
+__device__ __forceinline__ void stamp_now(int cta, int slot) {
+    if (threadIdx.x == 0 && cta < kStampCtas) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        g_stamps[cta * kStampSlots + slot] = t;
+    }
+}
+#define TSLT_STAMP(cta, slot) stamp_now((cta), (slot))
+#else
+#define TSLT_STAMP(cta, slot) do { } while (0)
+#endif
+
 // ---- small math --------------------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

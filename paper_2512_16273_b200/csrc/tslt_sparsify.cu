@@ -387,6 +387,7 @@ template <typename T, bool kLocal>
 __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) sparsify_stream_kernel(const SparsifyParams p) {
     extern __shared__ __align__(16) unsigned char stream_smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    TSLT_STAMP(blockIdx.x, 0);
     const RowWork wk = locate_work(p.split, blockIdx.x, p.nchunks);
     const unsigned char* rowp = p.logits + (long long)wk.row * p.row_stride_bytes;
     const RowExtent ext = row_extent<T>(p.V);
@@ -427,6 +428,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
         consume(lt);
         if (ch < wk.chunk_end) consume(lt2);
     }
+    TSLT_STAMP(blockIdx.x, 1);
     // hand-over: one (M, S) pair per warp
     const float Mw = warp_max(ls.M);
     const double Sw = warp_sum(ls.total_f64() * exp2((double)ls.M - (double)Mw));
@@ -555,6 +557,7 @@ __global__ void __launch_bounds__(kBlockThreads, kSparsifyStreamCtasPerSm) spars
     }
     __syncthreads();  // every warp's part of the hand-over is written
     if (tid == 0) publish_row_ready(&p.seg_ready[blockIdx.x]);
+    TSLT_STAMP(blockIdx.x, 2);
 }
 
 // ---- finish kernel ---------------------------------------------------------------------------------
@@ -1161,6 +1164,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
     const int nseg = p.split.nseg, nchunks = p.nchunks;
     const unsigned char* rowp = p.logits + (long long)row * p.row_stride_bytes;
     const RowExtent ext = row_extent<T>(p.V);
+    TSLT_STAMP(row, 3);
     if (tid == 0 && p.num_samples > 0)  // the uniforms are needed last: ask for their cache line now
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p.uniforms + (size_t)row * p.num_samples));
     if (tid == 0) sh->gmax = 0;
@@ -1183,6 +1187,7 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         wait_for_primary_kernel();
     }
     fsync<NT>();
+    TSLT_STAMP(row, 4);
     // ---- the row's log-normaliser, by one warp (fp64 is scarce) -------------------------------------
     if (warp == 1) {
         // every (max, sum) pair is asked for before any is used: one trip to memory
@@ -1330,16 +1335,20 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         }
         fsync<NT>();
     }
+    TSLT_STAMP(row, 5);
     const double L2 = sh->lrow;
     // ---- 4. candidates in shared memory, 5. the exact top-k (ties to the lower index), ascending index ----
     if (!listed) lo16 = (int)kLowestFinite16;
     int n = 0;
     if (max16 >= lo16) {
         const int n_c = listed ? gather_candidates<T, NT>(rowp, ext, p.V, tl, n_surv, lo16, p.cand_cap, c_raw, c_idx, sh, tid) : -1;
+        TSLT_STAMP(row, 6);
         if (n_c >= 0) n = select_in_list<T, NT>(k, c_raw, c_idx, n_c, hist, sh, tid);
         else n = select_from_global<T, NT>(rowp, ext, p.V, listed ? tl : nullptr, n_surv, lo16, max16, k, c_raw, c_idx, hist, sh, tid);
     }
+    TSLT_STAMP(row, 7);
     cut_sample_write<T, NT>(p, row, n, c_raw, c_idx, L2, hist, cum, sh, tid);
+    TSLT_STAMP(row + kStampCtas / 2, 0);
     // this kernel's completion must imply the streaming kernel's (what follows on the stream relies
     // on it): one CTA sees to that; the others leave and make room
     if (row == 0) wait_for_primary_kernel();
@@ -1454,7 +1463,7 @@ static SparsifyPlan make_sparsify_plan(int rows, int V, int k, int elt_bytes) {
     // eight times the CTAs is the very end of the streaming kernel.)
     int nseg = 1;
     if (rows > 0 && rows < slots) {
-        nseg = (slots + rows - 1) / rows;
+        nseg = slots / rows;  // (one wave: a CTA that had to wait for a slot would double the streaming time)
         const int by_len = pl.nchunks / kWarps;
         if (nseg > by_len) nseg = by_len;
         if (nseg > 64) nseg = 64;
@@ -1654,3 +1663,13 @@ extern "C" int tslt_sparsify_merge(int dtype, int rows, int nshards, const int* 
     if (cudaGetLastError() != cudaSuccess) return TSLT_ERR_CUDA;
     return TSLT_OK;
 }
+
+#ifdef TSLT_STAMPS
+// Timeline build only: the stamps of the last tslt_sparsify call, [kStampCtas, kStampSlots] nanoseconds
+// (streaming CTA c: slots 0 start, 1 end of its loop, 2 handed over; finish CTA of row r: slots 3 enter,
+// 4 row ready, 5 hand-over read, 6 candidates gathered, 7 top-k selected, and slot 0 of entry r + kStampCtas / 2: done).
+extern "C" int tslt_debug_stamps_sparsify(void* host, size_t bytes) {
+    if (bytes > sizeof(unsigned long long) * kStampCtas * kStampSlots) return TSLT_ERR_INVALID_ARG;
+    return cudaMemcpyFromSymbol(host, g_stamps, bytes) == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+}
+#endif

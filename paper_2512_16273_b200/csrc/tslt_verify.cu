@@ -462,6 +462,7 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
         }
     }
     consumer_sync();
+    TSLT_STAMP(b, 2);
     // ---- the leading run of accepted positions (strict <) ---------------------------------------
     int a = 0;
     while (a < gamma && (double)clamp_uniform(p.u_accept[(size_t)b * gamma + a]) < aps[a]) ++a;
@@ -486,8 +487,10 @@ __device__ void resolve_sequence(const VerifyParams& p, int b, unsigned char* ar
         }
         consumer_sync();
     }
+    TSLT_STAMP(b, 3);
     const float u = p.u_sample[b];
     int tok = sample_full_vocab<T>(p, rowp, part, L2_stop, 1.0, n, A, u, tid, sh);
+    TSLT_STAMP(b, 4);
     if (tok < 0 && n > 0) tok = sample_full_vocab<T>(p, rowp, part, L2_stop, 1.0, 0, A, u, tid, sh);  // degenerate residual
     if (tid == 0) {
         p.accepted_len[b] = a;
@@ -640,7 +643,9 @@ __global__ void __launch_bounds__(kBlockThreads, 4) verify_resolve_kernel(const 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* arena = smem_raw;  // plain offsets only: keeps the shared address space
     VerifyShared* sh = reinterpret_cast<VerifyShared*>(arena + kVerifyArena);
+    TSLT_STAMP(blockIdx.x, 0);
     wait_for_primary_kernel();  // the partials come from the streaming kernel
+    TSLT_STAMP(blockIdx.x, 1);
     if (kTree) resolve_tree<T>(p, blockIdx.x, arena, sh, threadIdx.x);
     else resolve_sequence<T>(p, blockIdx.x, arena, sh, threadIdx.x);
 }
@@ -1078,3 +1083,13 @@ extern "C" int tslt_tree_verify_packed(int walk, const void* target_logits, int 
                             draft_temperature, target_temperature, u_accept, u_sample, max_depth, accepted_path,
                             accepted_len, out_token, workspace, workspace_bytes, stream);
 }
+
+#ifdef TSLT_STAMPS
+// Timeline build only: the stamps of the last tslt_verify call, [kStampCtas, kStampSlots] nanoseconds
+// (resolver CTA of sequence b: slots 0 enter, 1 streaming kernel done, 2 positions judged, 3 draft of the
+// stop position loaded, 4 correction token sampled).
+extern "C" int tslt_debug_stamps_verify(void* host, size_t bytes) {
+    if (bytes > sizeof(unsigned long long) * kStampCtas * kStampSlots) return TSLT_ERR_INVALID_ARG;
+    return cudaMemcpyFromSymbol(host, g_stamps, bytes) == cudaSuccess ? TSLT_OK : TSLT_ERR_CUDA;
+}
+#endif
