@@ -1236,39 +1236,14 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         const unsigned short* tmax = p.tile_max + (size_t)row * nchunks * kTilesPerChunk;
         const int cpt = (nchunks + NT - 1) / NT;
         const int ch0 = min(nchunks, tid * cpt), ch1 = min(nchunks, ch0 + cpt);
-        // up to kKeep lines stay in registers for step 3 (rows up to kKeep * NT chunks: 512 KB with
-        // 128 threads); longer rows read their lines again there
-        constexpr int kKeep = 2;
-        uint32_t kept[kKeep][16];
-        const bool keep_lines = cpt <= kKeep;
-    #pragma unroll
-        for (int j = 0; j < kKeep; ++j) {
-            const int ch = ch0 + j;
-            if (keep_lines && ch < ch1) {
-                load_line(tmax + ch * kTilesPerChunk, kept[j]);
-            } else {
-    #pragma unroll
-                for (int i = 0; i < 16; ++i) kept[j][i] = 0xff80ff80u;  // -inf: never a survivor
-            }
-        }
-        if (keep_lines) {
-    #pragma unroll
-            for (int j = 0; j < kKeep; ++j) {
-                const int ch = ch0 + j;
-                if (ch < ch1) {
-                    const uint32_t lm = line_group_maxima(kept[j], glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
-                    if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
-                    lmax[ch] = (unsigned short)lm;
-                }
-            }
-        } else {
-            for (int ch = ch0; ch < ch1; ++ch) {
-                uint32_t w[16];
-                load_line(tmax + ch * kTilesPerChunk, w);
-                const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
-                if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
-                lmax[ch] = (unsigned short)lm;
-            }
+        // (keeping a thread's lines in registers from here to step 3 saved one trip to L2 and cost 32
+        // registers across the whole finish: the chain was 4 us longer on the smallest batches)
+        for (int ch = ch0; ch < ch1; ++ch) {
+            uint32_t w[16];
+            load_line(tmax + ch * kTilesPerChunk, w);
+            const uint32_t lm = line_group_maxima(w, glog, gm + ((ch * kTilesPerChunk) >> (glog <= 5 ? glog : 5)));
+            if (glog > 5) smem_max(&gm[ch >> (glog - 5)], raw16_to_key16(lm));
+            lmax[ch] = (unsigned short)lm;
         }
         fsync<NT>();
         {
@@ -1291,45 +1266,24 @@ __global__ void __launch_bounds__(NT, finish_resident(NT)) sparsify_finish_kerne
         lo16 = max((int)bound, (int)kLowestFinite16);
         // ---- 3. survivor tiles (key >= bound), listed in address order -----------------------------------------
         int my_surv = 0;
-        uint32_t kept_mask[kKeep];
-        if (keep_lines) {
-    #pragma unroll
-            for (int j = 0; j < kKeep; ++j) {
-                kept_mask[j] = line_survivors(kept[j], (uint32_t)lo16);  // bit a: tile a of the chunk (none beyond the row)
-                my_surv += __popc(kept_mask[j]);
-            }
-        } else {
-            for (int ch = ch0; ch < ch1; ++ch) {
-                if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
-                uint32_t w[16];
-                load_line(tmax + ch * kTilesPerChunk, w);
-                my_surv += __popc(line_survivors(w, (uint32_t)lo16));
-            }
+        for (int ch = ch0; ch < ch1; ++ch) {
+            if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+            uint32_t w[16];
+            load_line(tmax + ch * kTilesPerChunk, w);
+            my_surv += __popc(line_survivors(w, (uint32_t)lo16));  // bit a: tile a of the chunk (none beyond the row)
         }
         int pos = block_exscan<NT>(my_surv, tid, sh->iscr, &n_surv);
         listed = n_surv <= p.tile_cap;
         if (listed) {
-            if (keep_lines) {
-    #pragma unroll
-                for (int j = 0; j < kKeep; ++j) {
-                    uint32_t m = kept_mask[j];
-                    while (m) {
-                        const int a = __ffs(m) - 1;
-                        m &= m - 1;
-                        tl[pos++] = (uint32_t)((ch0 + j) * kTilesPerChunk + a);
-                    }
-                }
-            } else {
-                for (int ch = ch0; ch < ch1; ++ch) {
-                    if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
-                    uint32_t w[16];
-                    load_line(tmax + ch * kTilesPerChunk, w);
-                    uint32_t m = line_survivors(w, (uint32_t)lo16);
-                    while (m) {
-                        const int a = __ffs(m) - 1;
-                        m &= m - 1;
-                        tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
-                    }
+            for (int ch = ch0; ch < ch1; ++ch) {
+                if (raw16_to_key16(lmax[ch]) < (uint32_t)lo16) continue;
+                uint32_t w[16];
+                load_line(tmax + ch * kTilesPerChunk, w);
+                uint32_t m = line_survivors(w, (uint32_t)lo16);
+                while (m) {
+                    const int a = __ffs(m) - 1;
+                    m &= m - 1;
+                    tl[pos++] = (uint32_t)(ch * kTilesPerChunk + a);
                 }
             }
         }
