@@ -50,6 +50,8 @@ constexpr int kMaxTileList = 4096;        // survivor tiles it can list
 constexpr int kSelBins = 1024;            // bins of the selection histogram
 constexpr int kMaxShards = TSLT_MAX_SHARDS;  // vocabulary shards one merge takes
 constexpr int kMaxMergeList = 2048;       // candidates the merge holds (nshards * k)
+constexpr int kListPerThread = 8;         // candidate list entries per thread of a finishing CTA: lists of at most 8 * NT
+constexpr int kWinnersPerThread = 4;      // winners per thread in the top-rho cut: k <= 4 * NT
 constexpr uint32_t kLowestFinite16 = 0x0080u;   // key of -FLT_MAX >> 16
 constexpr uint32_t kHighestFinite16 = 0xff7fu;  // key of +FLT_MAX >> 16
 
@@ -738,7 +740,7 @@ __device__ __forceinline__ int finite_key16(float z) {
 template <typename T, int NT>
 __device__ __forceinline__ int select_in_list(int k, uint32_t* c_raw, int* c_idx, int n_c, uint32_t* hist, FinishShared* sh, int tid) {
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
-    constexpr int kHeld = kMaxMergeList / NT;  // most list entries a thread owns (the lists hold 2048 at most)
+    constexpr int kHeld = kListPerThread;  // most list entries a thread owns (the host sees to it: lists of at most 8 * NT)
     unsigned long long* rkeys = reinterpret_cast<unsigned long long*>(hist);
     int n = 0;
     {
@@ -827,7 +829,7 @@ template <typename T, int NT>
 __device__ __forceinline__ void cut_sample_write(const SparsifyParams& p, int row, int n, uint32_t* c_raw, int* c_idx,
                                                  double L2, uint32_t* hist, double* cum, FinishShared* sh, int tid) {
     constexpr bool kBf16 = (Elt<T>::kBytes == 2);
-    constexpr int kMine = TSLT_MAX_K / NT;  // most winners a thread owns in the top-rho cut
+    constexpr int kMine = kWinnersPerThread;  // most winners a thread owns in the top-rho cut (k <= 4 * NT, host-checked)
     const int lane = tid & 31, k = p.k;
     const int n0 = n;
     uint32_t* win_raw = c_raw;
@@ -1555,6 +1557,7 @@ static int sparsify_impl(const void* logits, int dtype, int B, int gamma, int V,
     }
     const int fin_slot = (small ? 0 : 2) + (f32 ? 0 : 1) + (pl.local_bound ? 4 : 0);
     if (!prefer_shared_carveout_once(fin, 4 + fin_slot)) return TSLT_ERR_CUDA;
+    if (pl.cand_cap > kListPerThread * pl.fin_threads || k > kWinnersPerThread * pl.fin_threads) return TSLT_ERR_UNSUPPORTED;  // (cannot happen: see finish_threads)
     if (pl.fin_smem > kFinishSmemLimit) return TSLT_ERR_UNSUPPORTED;  // (rows of tens of millions of logits: the line maxima no longer fit)
     if (pl.fin_smem > 48 * 1024 && !raise_smem_limit_once(fin, fin_slot, kFinishSmemLimit)) return TSLT_ERR_CUDA;
     if (launch_dependent(fin, rows, pl.fin_threads, pl.fin_smem, st, p) != cudaSuccess) return TSLT_ERR_CUDA;
